@@ -1,0 +1,230 @@
+"""CPU oracle for the 4-bit training hot path.  TEST INFRASTRUCTURE ONLY.
+
+Thin numpy/ctypes front end over ``luq_oracle.c`` (plain scalar C, compiled with
+gcc) plus ``literal.py`` (a pure-Python, exact-rational transcription of the
+paper's two-stage quantizer used to pin the C code).  Nothing here is imported
+by the CUDA library or its Python binding; only tests, the smoke check and the
+benchmark's CPU-baseline leg may use it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "luq_oracle.c")
+_LIB = os.path.join(_HERE, "libluq_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+FLAG_NONFINITE = 1
+FLAG_RANGE = 2
+KMAX_DEFAULT = 4  # Eq. alpha with b = 3: alpha = max / 2^(2^(b-1)) = max / 16
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared", "-fPIC",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    with _lock:
+        if _lib is None:
+            build()
+            L = ctypes.CDLL(_LIB)
+            u8p, f32p, f64p = (ctypes.POINTER(ctypes.c_uint8), ctypes.POINTER(ctypes.c_float),
+                               ctypes.POINTER(ctypes.c_double))
+            u32p, i64p, intp = (ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ctypes.c_int64),
+                                ctypes.POINTER(ctypes.c_int))
+            sz, i64, dbl = ctypes.c_size_t, ctypes.c_int64, ctypes.c_double
+            L.oracle_philox_constants.argtypes = [u32p]
+            L.oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
+            L.oracle_random_word.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint64]
+            L.oracle_random_word.restype = ctypes.c_uint32
+            L.oracle_amax.argtypes = [f32p, sz, intp]
+            L.oracle_amax.restype = ctypes.c_float
+            L.oracle_quant_int4.argtypes = [f32p, sz, ctypes.c_float, u8p, intp]
+            L.oracle_quant_int4.restype = ctypes.c_float
+            L.oracle_luq_alpha.argtypes = [ctypes.c_float, ctypes.c_int]
+            L.oracle_luq_alpha.restype = ctypes.c_float
+            L.oracle_quant_luq.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, ctypes.c_uint64,
+                                           ctypes.c_int, u8p, intp]
+            L.oracle_quant_luq.restype = ctypes.c_float
+            L.oracle_luq_bins.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, f64p, f64p, u32p]
+            L.oracle_dequant.argtypes = [u8p, sz, dbl, ctypes.c_int, f64p]
+            L.oracle_gemm_fwd.argtypes = [u8p, dbl, u8p, dbl, i64, i64, i64, f64p]
+            L.oracle_gemm_bwd.argtypes = [u8p, dbl, ctypes.c_int, u8p, dbl, i64, i64, i64, f64p]
+            L.oracle_gemm_wgrad.argtypes = [u8p, dbl, ctypes.c_int, u8p, dbl, i64, i64, i64, f64p]
+            L.oracle_gemm_int64.argtypes = [ctypes.c_int, u8p, ctypes.c_int, u8p, i64, i64, i64, i64p]
+            L.oracle_gemm_entries.argtypes = [ctypes.c_int, u8p, dbl, ctypes.c_int, u8p, dbl,
+                                              i64, i64, i64, i64p, i64p, sz, f64p]
+            _lib = L
+    return _lib
+
+
+def _ptr(a: np.ndarray, ctype):
+    return a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+def widen(x: np.ndarray) -> np.ndarray:
+    """fp32 view of the input.  bf16 tensors travel as uint16 bit patterns and
+    are widened exactly (bits << 16); fp32 passes through."""
+    x = np.ascontiguousarray(x)
+    if x.dtype == np.uint16:
+        return (x.astype(np.uint32) << 16).view(np.float32)
+    if x.dtype != np.float32:
+        raise TypeError("oracle inputs are float32 or bf16-as-uint16")
+    return x
+
+
+def philox4x32_10(counter, key) -> np.ndarray:
+    c = np.asarray(counter, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, dtype=np.uint32)
+    lib().oracle_philox4x32_10(_ptr(c, ctypes.c_uint32), _ptr(k, ctypes.c_uint32), _ptr(out, ctypes.c_uint32))
+    return out
+
+
+def philox_constants() -> np.ndarray:
+    out = np.zeros(4, dtype=np.uint32)
+    lib().oracle_philox_constants(_ptr(out, ctypes.c_uint32))
+    return out
+
+
+def random_word(seed: int, sample: int, index: int) -> int:
+    return int(lib().oracle_random_word(seed & (2**64 - 1), sample, index))
+
+
+def amax(x: np.ndarray):
+    """max|x| over the whole tensor (Eq. alpha).  Returns (value, flags)."""
+    xf = widen(x).reshape(-1)
+    flags = ctypes.c_int(0)
+    v = lib().oracle_amax(_ptr(xf, ctypes.c_float), xf.size, ctypes.byref(flags))
+    return np.float32(v), flags.value
+
+
+def quant_int4(x: np.ndarray, clip):
+    """Q_INT with round-to-nearest (Sec. 3.3).  Returns (codes[n/2] uint8, scale, flags)."""
+    xf = widen(x).reshape(-1)
+    codes = np.zeros((xf.size + 1) // 2, dtype=np.uint8)
+    flags = ctypes.c_int(0)
+    s = lib().oracle_quant_int4(_ptr(xf, ctypes.c_float), xf.size, np.float32(clip),
+                                _ptr(codes, ctypes.c_uint8), ctypes.byref(flags))
+    return codes, np.float32(s), flags.value
+
+
+def luq_alpha(mx, kmax: int = KMAX_DEFAULT) -> np.float32:
+    return np.float32(lib().oracle_luq_alpha(np.float32(mx), kmax))
+
+
+def quant_luq(x: np.ndarray, mx, seed: int, n_samples: int = 1, kmax: int = KMAX_DEFAULT):
+    """LUQ = Q_alpha(T_alpha(x)) (Sec. 4).  Returns (codes[n_samples, n/2], alpha, flags)."""
+    xf = widen(x).reshape(-1)
+    plane = (xf.size + 1) // 2
+    codes = np.zeros((n_samples, plane), dtype=np.uint8)
+    flags = ctypes.c_int(0)
+    a = lib().oracle_quant_luq(_ptr(xf, ctypes.c_float), xf.size, np.float32(mx), kmax,
+                               seed & (2**64 - 1), n_samples, _ptr(codes, ctypes.c_uint8),
+                               ctypes.byref(flags))
+    return codes, np.float32(a), flags.value
+
+
+def luq_bins(x: np.ndarray, mx, kmax: int = KMAX_DEFAULT):
+    """Per element (lo, hi, thr): candidate levels in units of alpha and the
+    32-bit threshold; P(hi) = thr / 2^32."""
+    xf = widen(x).reshape(-1)
+    lo = np.zeros(xf.size, dtype=np.float64)
+    hi = np.zeros(xf.size, dtype=np.float64)
+    thr = np.zeros(xf.size, dtype=np.uint32)
+    lib().oracle_luq_bins(_ptr(xf, ctypes.c_float), xf.size, np.float32(mx), kmax,
+                          _ptr(lo, ctypes.c_double), _ptr(hi, ctypes.c_double), _ptr(thr, ctypes.c_uint32))
+    return lo, hi, thr
+
+
+def unpack(codes: np.ndarray, n: int) -> np.ndarray:
+    """Nibbles of a packed plane, element 2j low, 2j+1 high."""
+    codes = np.ascontiguousarray(codes).reshape(-1)
+    out = np.empty(codes.size * 2, dtype=np.uint8)
+    out[0::2] = codes & 0xF
+    out[1::2] = codes >> 4
+    return out[:n]
+
+
+def dequant(codes: np.ndarray, n: int, scale, kind: str) -> np.ndarray:
+    """Values of a packed plane in float64.  kind: 'int4' or 'luq'."""
+    codes = np.ascontiguousarray(codes).reshape(-1)
+    out = np.zeros(n, dtype=np.float64)
+    lib().oracle_dequant(_ptr(codes, ctypes.c_uint8), n, float(scale), 0 if kind == "int4" else 1,
+                         _ptr(out, ctypes.c_double))
+    return out
+
+
+def gemm_fwd(a_codes, sa, w_codes, sw, M, N, K) -> np.ndarray:
+    """Z = A_d . W_d^T in float64 (Eq. Forward)."""
+    a_codes = np.ascontiguousarray(a_codes).reshape(-1)
+    w_codes = np.ascontiguousarray(w_codes).reshape(-1)
+    Z = np.zeros((M, N), dtype=np.float64)
+    lib().oracle_gemm_fwd(_ptr(a_codes, ctypes.c_uint8), float(sa), _ptr(w_codes, ctypes.c_uint8), float(sw),
+                          M, N, K, _ptr(Z, ctypes.c_double))
+    return Z
+
+
+def gemm_bwd(g_codes, alpha, n_samples, w_codes, sw, M, N, K) -> np.ndarray:
+    """dA = mean_s(G_d,s) . W_d in float64 (Eq. Backward, SMP average of Sec. 5.1)."""
+    g_codes = np.ascontiguousarray(g_codes).reshape(-1)
+    w_codes = np.ascontiguousarray(w_codes).reshape(-1)
+    dA = np.zeros((M, K), dtype=np.float64)
+    lib().oracle_gemm_bwd(_ptr(g_codes, ctypes.c_uint8), float(alpha), n_samples,
+                          _ptr(w_codes, ctypes.c_uint8), float(sw), M, N, K, _ptr(dA, ctypes.c_double))
+    return dA
+
+
+def gemm_wgrad(g_codes, alpha, n_samples, a_codes, sa, M, N, K) -> np.ndarray:
+    """dW = mean_s(G_d,s)^T . A_d in float64 (Eq. Update, SMP average of Sec. 5.1)."""
+    g_codes = np.ascontiguousarray(g_codes).reshape(-1)
+    a_codes = np.ascontiguousarray(a_codes).reshape(-1)
+    dW = np.zeros((N, K), dtype=np.float64)
+    lib().oracle_gemm_wgrad(_ptr(g_codes, ctypes.c_uint8), float(alpha), n_samples,
+                            _ptr(a_codes, ctypes.c_uint8), float(sa), M, N, K, _ptr(dW, ctypes.c_double))
+    return dW
+
+
+def gemm_int64(which: str, x_codes, n_samples, y_codes, M, N, K) -> np.ndarray:
+    """Integer-code products summed in int64 (Appendix A.1 scale factoring)."""
+    w = {"fwd": 0, "bwd": 1, "wgrad": 2}[which]
+    shape = {"fwd": (M, N), "bwd": (M, K), "wgrad": (N, K)}[which]
+    x_codes = np.ascontiguousarray(x_codes).reshape(-1)
+    y_codes = np.ascontiguousarray(y_codes).reshape(-1)
+    out = np.zeros(shape, dtype=np.int64)
+    lib().oracle_gemm_int64(w, _ptr(x_codes, ctypes.c_uint8), n_samples, _ptr(y_codes, ctypes.c_uint8),
+                            M, N, K, _ptr(out, ctypes.c_int64))
+    return out
+
+
+def gemm_entries(which: str, x_codes, sx, n_samples, y_codes, sy, M, N, K, rows, cols) -> np.ndarray:
+    """Selected entries of one of the three products, each computed on its own."""
+    w = {"fwd": 0, "bwd": 1, "wgrad": 2}[which]
+    x_codes = np.ascontiguousarray(x_codes).reshape(-1)
+    y_codes = np.ascontiguousarray(y_codes).reshape(-1)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    out = np.zeros(rows.size, dtype=np.float64)
+    lib().oracle_gemm_entries(w, _ptr(x_codes, ctypes.c_uint8), float(sx), n_samples,
+                              _ptr(y_codes, ctypes.c_uint8), float(sy), M, N, K,
+                              _ptr(rows, ctypes.c_int64), _ptr(cols, ctypes.c_int64), rows.size,
+                              _ptr(out, ctypes.c_double))
+    return out
+
+
+def host_threads() -> int:
+    """Threads the OpenMP loops of the C oracle will use."""
+    return int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))

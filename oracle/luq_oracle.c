@@ -1,0 +1,372 @@
+/*
+ * CPU oracle for the 4-bit training hot path (LUQ paper).  TEST INFRASTRUCTURE ONLY.
+ *
+ * Plain, slow, scalar C.  It shares no code, table or constant with the CUDA
+ * library; only tests, the smoke check and the benchmark's cpu_baseline leg may
+ * call it.  Every function names the passage of the paper it follows.
+ *
+ * Conventions (row-major everywhere):
+ *   activations A[M x K], weights W[N x K], pre-activation gradient G[M x N]
+ *   forward  Z  = A . W^T   [M x N]      (Eq. "Forward")
+ *   backward dA = G . W     [M x K]      (Eq. "Backward")
+ *   update   dW = G^T . A   [N x K]      (Eq. "Update")
+ *   packed codes: two 4-bit codes per byte along the contiguous dimension,
+ *   element 2j in the low nibble and element 2j+1 in the high nibble.
+ *
+ * Parity pins (see tests marked "not gpu"): grid membership, fixed points,
+ * exact expectation, the literal two-draw transcription of T_alpha / Q_alpha,
+ * the paper's worked values, Table 1 closed forms, brute force GEMMs, and the
+ * Philox constants / stream (cuRAND header constants on the CPU, the cuRAND
+ * device generator on a GPU box).  The raw Philox stream is "parity unpinned"
+ * on a box without cuRAND's header: any fixed bijective stream satisfies the paper.
+ *
+ * Build: gcc -O2 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_FLAG_NONFINITE 1
+#define ORACLE_FLAG_RANGE 2
+
+static uint32_t bits_of(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+static float float_of(uint32_t u) { float f; memcpy(&f, &u, 4); return f; }
+
+/* ------------------------------------------------------------------------ */
+/* Philox4x32-10 (Salmon et al., SC'11).  The paper is silent on the random  */
+/* source (Sec. 4, Appendix A.5); the build's reading fixes this generator.  */
+/* ------------------------------------------------------------------------ */
+static const uint32_t PHILOX_MUL_A = 0xD2511F53u;  /* multiplies counter word 0 */
+static const uint32_t PHILOX_MUL_B = 0xCD9E8D57u;  /* multiplies counter word 2 */
+static const uint32_t PHILOX_WEYL_0 = 0x9E3779B9u; /* floor(2^32 (golden ratio - 1)) */
+static const uint32_t PHILOX_WEYL_1 = 0xBB67AE85u; /* floor(2^32 (sqrt 3 - 1)) */
+
+void oracle_philox_constants(uint32_t out[4]) {
+  out[0] = PHILOX_MUL_A; out[1] = PHILOX_MUL_B; out[2] = PHILOX_WEYL_0; out[3] = PHILOX_WEYL_1;
+}
+
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    uint64_t p0 = (uint64_t)PHILOX_MUL_A * c0;
+    uint64_t p1 = (uint64_t)PHILOX_MUL_B * c2;
+    uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    uint32_t n1 = (uint32_t)p1;
+    uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    uint32_t n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += PHILOX_WEYL_0; k1 += PHILOX_WEYL_1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The 32-bit word that decides element `index` of sample `sample`:
+ * key = seed + sample (64 bit, wrapping), counter = index / 4, word index % 4. */
+uint32_t oracle_random_word(uint64_t seed, uint32_t sample, uint64_t index) {
+  uint64_t s = seed + (uint64_t)sample;
+  uint64_t block = index >> 2;
+  uint32_t ctr[4] = {(uint32_t)block, (uint32_t)(block >> 32), 0u, 0u};
+  uint32_t key[2] = {(uint32_t)s, (uint32_t)(s >> 32)};
+  uint32_t w[4];
+  oracle_philox4x32_10(ctr, key, w);
+  return w[index & 3];
+}
+
+/* ------------------------------------------------------------------------ */
+/* max|x| of a tensor (Sec. 4 "Above FP maximum", Eq. alpha: max(|x|)).       */
+/* flags gets ORACLE_FLAG_NONFINITE if any element is NaN or Inf.            */
+/* ------------------------------------------------------------------------ */
+float oracle_amax(const float* x, size_t n, int* flags) {
+  float m = 0.0f;
+  int bad = 0;
+  for (size_t i = 0; i < n; ++i) {
+    float a = fabsf(x[i]);
+    if (!(a <= 3.402823466e38f)) bad = 1; /* NaN or Inf */
+    else if (a > m) m = a;
+  }
+  if (flags) *flags = bad ? ORACLE_FLAG_NONFINITE : 0;
+  return m;
+}
+
+static int scale_usable(float c, int* flags) {
+  /* A clip / max that is zero, non-finite or outside [2^-100, 2^100] produces
+   * all-zero codes and a zero scale (build's convention; the paper is silent). */
+  if (flags) *flags = 0;
+  if (c == 0.0f) return 0;
+  if (!(c <= 3.402823466e38f) || c < 0.0f) { if (flags) *flags = ORACLE_FLAG_NONFINITE; return 0; }
+  if (c < 0x1p-100f || c > 0x1p100f) { if (flags) *flags = ORACLE_FLAG_RANGE; return 0; }
+  return 1;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Q_INT: INT4 round-to-nearest (Sec. 3.3: RDN for weights and activations;  */
+/* Appendix A.1: one high-precision scale per tensor).  Signed symmetric      */
+/* grid -7..7, step s = clip/7, ties to even, two's-complement nibble.        */
+/* ------------------------------------------------------------------------ */
+float oracle_quant_int4(const float* x, size_t n, float clip, uint8_t* codes, int* flags) {
+  if (!scale_usable(clip, flags)) { memset(codes, 0, (n + 1) / 2); return 0.0f; }
+  float s = clip / 7.0f;
+  float inv = 7.0f / clip;
+  memset(codes, 0, (n + 1) / 2);
+  for (size_t i = 0; i < n; ++i) {
+    float y = x[i] * inv;
+    float r = rintf(y); /* default rounding mode: nearest, ties to even */
+    if (r > 7.0f) r = 7.0f;
+    if (r < -7.0f) r = -7.0f;
+    if (r != r) r = 0.0f; /* NaN element (only with a caller-supplied clip) -> 0 */
+    int q = (int)r;
+    uint8_t nib = (uint8_t)(q & 0xF);
+    codes[i >> 1] |= (uint8_t)(nib << ((i & 1) * 4));
+  }
+  return s;
+}
+
+int oracle_int4_value(uint8_t nibble) { /* two's complement 4 bit */
+  int v = nibble & 0xF;
+  return v >= 8 ? v - 16 : v;
+}
+
+/* ------------------------------------------------------------------------ */
+/* LUQ = Q_alpha(T_alpha(x)) (Sec. 4).                                        */
+/*   alpha = max|x| / 2^kmax            (Eq. alpha; the paper prints 2^(2^(b-1)) */
+/*                                       with b = 3, i.e. kmax = 4)           */
+/*   |x| <  alpha : sign*alpha w.p. |x|/alpha, else 0   (Eq. StochasticPruning) */
+/*   2^(n-1) alpha <= |x| < 2^n alpha : up w.p. (|x| - 2^(n-1) alpha)/(2^(n-1) alpha) */
+/*                                                      (Eq. unbiasedFpQ)     */
+/* One random word decides both stages: T_alpha outputs 0, +-alpha or an     */
+/* untouched in-range value and Q_alpha is deterministic on 0 and +-alpha.   */
+/* t = |x|/alpha in IEEE binary32.  For t >= 1 the mantissa field of t is the */
+/* up-probability times 2^23 and its exponent is the lower level's index.    */
+/* Code c: 0 -> 0, c >= 1 -> alpha * 2^(c-1); nibble = sign<<3 | c, zero is 0x0. */
+/* ------------------------------------------------------------------------ */
+typedef struct { uint32_t lo_code; uint32_t threshold; } luq_bin;
+
+static luq_bin luq_bin_of(float a, float alpha, int kmax) {
+  luq_bin b;
+  float t = a / alpha; /* IEEE-754 binary32 division, round to nearest even */
+  if (t < 1.0f) {
+    b.lo_code = 0;
+    b.threshold = (uint32_t)(t * 4294967296.0f); /* exact scaling, truncation */
+  } else {
+    uint32_t u = bits_of(t);
+    int e = (int)((u >> 23) & 0xFF) - 127;
+    if (e >= kmax) { /* at or above the top level (or NaN/Inf): top code, no draw */
+      b.lo_code = (uint32_t)(kmax + 1);
+      b.threshold = 0;
+    } else {
+      b.lo_code = (uint32_t)(1 + e);
+      b.threshold = (u & 0x7FFFFFu) << 9;
+    }
+  }
+  return b;
+}
+
+float oracle_luq_alpha(float mx, int kmax) { return ldexpf(mx, -kmax); }
+
+/* codes: n_samples planes of (n+1)/2 bytes each, sample-major. Returns alpha. */
+float oracle_quant_luq(const float* x, size_t n, float mx, int kmax, uint64_t seed,
+                       int n_samples, uint8_t* codes, int* flags) {
+  size_t plane = (n + 1) / 2;
+  memset(codes, 0, plane * (size_t)n_samples);
+  if (!scale_usable(mx, flags)) return 0.0f;
+  float alpha = oracle_luq_alpha(mx, kmax);
+  for (int s = 0; s < n_samples; ++s) {
+    uint8_t* out = codes + plane * (size_t)s;
+    for (size_t i = 0; i < n; ++i) {
+      float a = fabsf(x[i]);
+      uint32_t sign = bits_of(x[i]) >> 31;
+      luq_bin b = luq_bin_of(a, alpha, kmax);
+      uint32_t r = oracle_random_word(seed, (uint32_t)s, (uint64_t)i);
+      uint32_t c = b.lo_code + (r < b.threshold ? 1u : 0u);
+      uint8_t nib = c ? (uint8_t)((sign << 3) | c) : 0;
+      out[i >> 1] |= (uint8_t)(nib << ((i & 1) * 4));
+    }
+  }
+  return alpha;
+}
+
+/* Exact-expectation helper (test only): per element the two candidate levels
+ * (as multiples of alpha: 0, 1, 2, 4, ...) and the 32-bit threshold, so that
+ * E[Q(x)] = alpha*(lo + (hi-lo)*thr/2^32) can be evaluated without sampling. */
+void oracle_luq_bins(const float* x, size_t n, float mx, int kmax,
+                     double* lo, double* hi, uint32_t* thr) {
+  float alpha = oracle_luq_alpha(mx, kmax);
+  for (size_t i = 0; i < n; ++i) {
+    luq_bin b = luq_bin_of(fabsf(x[i]), alpha, kmax);
+    uint32_t c = b.lo_code;
+    lo[i] = c ? ldexp(1.0, (int)c - 1) : 0.0;
+    hi[i] = ((int)c >= kmax + 1) ? lo[i] : ldexp(1.0, (int)c);
+    thr[i] = b.threshold;
+  }
+}
+
+double oracle_luq_value(uint8_t nibble) { /* in units of alpha */
+  int c = nibble & 7;
+  if (c == 0) return 0.0;
+  double v = ldexp(1.0, c - 1);
+  return (nibble & 8) ? -v : v;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Dequantise and multiply: the plain definition (Appendix A.1: the scale is  */
+/* a single high-precision factor, all MACs act on the low-precision values). */
+/* kind: 0 = INT4 codes (value q*scale), 1 = LUQ codes (value +-scale*2^(c-1)) */
+/* ------------------------------------------------------------------------ */
+static double code_value(const uint8_t* codes, size_t idx, int kind) {
+  uint8_t nib = (codes[idx >> 1] >> ((idx & 1) * 4)) & 0xF;
+  return kind ? oracle_luq_value(nib) : (double)oracle_int4_value(nib);
+}
+
+void oracle_dequant(const uint8_t* codes, size_t n, double scale, int kind, double* out) {
+  for (size_t i = 0; i < n; ++i) out[i] = scale * code_value(codes, i, kind);
+}
+
+/* Z[M x N] = A_d . W_d^T with A_d = dequant(A codes [M x K]), W_d = dequant(W codes [N x K]) */
+void oracle_gemm_fwd(const uint8_t* a_codes, double sa, const uint8_t* w_codes, double sw,
+                     int64_t M, int64_t N, int64_t K, double* Z) {
+  double* Ad = (double*)malloc(sizeof(double) * (size_t)(M * K));
+  double* Wd = (double*)malloc(sizeof(double) * (size_t)(N * K));
+  oracle_dequant(a_codes, (size_t)(M * K), sa, 0, Ad);
+  oracle_dequant(w_codes, (size_t)(N * K), sw, 0, Wd);
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n) {
+      double acc = 0.0;
+      for (int64_t k = 0; k < K; ++k) acc += Ad[m * K + k] * Wd[n * K + k];
+      Z[m * N + n] = acc;
+    }
+  free(Ad); free(Wd);
+}
+
+/* mean over samples of dequant(G codes, plane s) -> Gd[M x N] */
+static double* mean_gradient(const uint8_t* g_codes, double alpha, int n_samples,
+                             int64_t M, int64_t N) {
+  size_t n = (size_t)(M * N), plane = (n + 1) / 2;
+  double* Gd = (double*)calloc(n, sizeof(double));
+  for (int s = 0; s < n_samples; ++s)
+    for (size_t i = 0; i < n; ++i) Gd[i] += alpha * code_value(g_codes + plane * (size_t)s, i, 1);
+  for (size_t i = 0; i < n; ++i) Gd[i] /= (double)n_samples;
+  return Gd;
+}
+
+/* dA[M x K] = mean_s(G_d,s) . W_d   (SMP, Sec. 5.1: average of the samples) */
+void oracle_gemm_bwd(const uint8_t* g_codes, double alpha, int n_samples,
+                     const uint8_t* w_codes, double sw,
+                     int64_t M, int64_t N, int64_t K, double* dA) {
+  double* Gd = mean_gradient(g_codes, alpha, n_samples, M, N);
+  double* Wd = (double*)malloc(sizeof(double) * (size_t)(N * K));
+  oracle_dequant(w_codes, (size_t)(N * K), sw, 0, Wd);
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t k = 0; k < K; ++k) {
+      double acc = 0.0;
+      for (int64_t n = 0; n < N; ++n) acc += Gd[m * N + n] * Wd[n * K + k];
+      dA[m * K + k] = acc;
+    }
+  free(Gd); free(Wd);
+}
+
+/* dW[N x K] = mean_s(G_d,s)^T . A_d */
+void oracle_gemm_wgrad(const uint8_t* g_codes, double alpha, int n_samples,
+                       const uint8_t* a_codes, double sa,
+                       int64_t M, int64_t N, int64_t K, double* dW) {
+  double* Gd = mean_gradient(g_codes, alpha, n_samples, M, N);
+  double* Ad = (double*)malloc(sizeof(double) * (size_t)(M * K));
+  oracle_dequant(a_codes, (size_t)(M * K), sa, 0, Ad);
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t k = 0; k < K; ++k) {
+      double acc = 0.0;
+      for (int64_t m = 0; m < M; ++m) acc += Gd[m * N + n] * Ad[m * K + k];
+      dW[n * K + k] = acc;
+    }
+  free(Gd); free(Ad);
+}
+
+/* Second, independent form (Appendix A.1 scale factoring): integer codes are
+ * multiplied and summed in int64, the scale product is applied once.
+ * which: 0 fwd, 1 bwd, 2 wgrad.  out gets the integer sums (not yet scaled,
+ * summed over the n_samples planes). */
+void oracle_gemm_int64(int which, const uint8_t* x_codes, int n_samples, const uint8_t* y_codes,
+                       int64_t M, int64_t N, int64_t K, int64_t* out) {
+  if (which == 0) {
+    for (int64_t m = 0; m < M; ++m)
+      for (int64_t n = 0; n < N; ++n) {
+        int64_t acc = 0;
+        for (int64_t k = 0; k < K; ++k)
+          acc += (int64_t)code_value(x_codes, (size_t)(m * K + k), 0) *
+                 (int64_t)code_value(y_codes, (size_t)(n * K + k), 0);
+        out[m * N + n] = acc;
+      }
+    return;
+  }
+  size_t plane = ((size_t)(M * N) + 1) / 2;
+  if (which == 1) {
+    for (int64_t m = 0; m < M; ++m)
+      for (int64_t k = 0; k < K; ++k) {
+        int64_t acc = 0;
+        for (int s = 0; s < n_samples; ++s)
+          for (int64_t n = 0; n < N; ++n)
+            acc += (int64_t)code_value(x_codes + plane * (size_t)s, (size_t)(m * N + n), 1) *
+                   (int64_t)code_value(y_codes, (size_t)(n * K + k), 0);
+        out[m * K + k] = acc;
+      }
+  } else {
+    for (int64_t n = 0; n < N; ++n)
+      for (int64_t k = 0; k < K; ++k) {
+        int64_t acc = 0;
+        for (int s = 0; s < n_samples; ++s)
+          for (int64_t m = 0; m < M; ++m)
+            acc += (int64_t)code_value(x_codes + plane * (size_t)s, (size_t)(m * N + n), 1) *
+                   (int64_t)code_value(y_codes, (size_t)(m * K + k), 0);
+        out[n * K + k] = acc;
+      }
+  }
+}
+
+/* Selected output entries of the three products at any size, computed one by
+ * one from the codes (same definition as above: dequantise, multiply, add in
+ * double).  which: 0 fwd (r=m, c=n), 1 bwd (r=m, c=k), 2 wgrad (r=n, c=k). */
+void oracle_gemm_entries(int which, const uint8_t* x_codes, double sx, int n_samples,
+                         const uint8_t* y_codes, double sy,
+                         int64_t M, int64_t N, int64_t K,
+                         const int64_t* rows, const int64_t* cols, size_t count, double* out) {
+  size_t plane = ((size_t)(M * N) + 1) / 2;
+#pragma omp parallel for schedule(dynamic, 4)
+  for (size_t e = 0; e < count; ++e) {
+    int64_t r = rows[e], c = cols[e];
+    double acc = 0.0;
+    if (which == 0) {
+      for (int64_t k = 0; k < K; ++k)
+        acc += (sx * code_value(x_codes, (size_t)(r * K + k), 0)) *
+               (sy * code_value(y_codes, (size_t)(c * K + k), 0));
+    } else if (which == 1) {
+      for (int64_t n = 0; n < N; ++n) {
+        double g = 0.0;
+        for (int s = 0; s < n_samples; ++s)
+          g += sx * code_value(x_codes + plane * (size_t)s, (size_t)(r * N + n), 1);
+        acc += (g / (double)n_samples) * (sy * code_value(y_codes, (size_t)(n * K + c), 0));
+      }
+    } else {
+      for (int64_t m = 0; m < M; ++m) {
+        double g = 0.0;
+        for (int s = 0; s < n_samples; ++s)
+          g += sx * code_value(x_codes + plane * (size_t)s, (size_t)(m * N + r), 1);
+        acc += (g / (double)n_samples) * (sy * code_value(y_codes, (size_t)(m * K + c), 0));
+      }
+    }
+    out[e] = acc;
+  }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Deterministic rounding rules used as pins (Table 1, Sec. 3.1).            */
+/* ------------------------------------------------------------------------ */
+double oracle_round_nearest_in_bin(double x, double l, double u) { return (x - l <= u - x) ? l : u; }
+
+/* exported for the bit-level tests */
+uint32_t oracle_float_bits(float f) { return bits_of(f); }
+float oracle_bits_float(uint32_t u) { return float_of(u); }
