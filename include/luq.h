@@ -1,0 +1,142 @@
+/*
+ * luq.h - C ABI of the B200 (sm_100a) 4-bit training hot path.
+ *
+ * The library implements the quantize-then-multiply pipeline of "Accurate
+ * Neural Training with 4-bit Matrix Multiplications at Standard Formats":
+ * per-tensor max, INT4 round-to-nearest quantization of weights/activations,
+ * LUQ (logarithmic unbiased quantization) of neural gradients to the FP4
+ * [sign,exp,mantissa] = [1,3,0] grid, and the three training GEMMs.
+ *
+ * Conventions
+ *   - Row-major tensors.  A layer has activations A[M x K], weights W[N x K],
+ *     pre-activation gradient G[M x N].
+ *       forward   Z  = A . W^T  [M x N]
+ *       backward  dA = G . W    [M x K]
+ *       update    dW = G^T . A  [N x K]
+ *   - Packed codes: two 4-bit codes per byte along the contiguous dimension,
+ *     element 2j in the low nibble, element 2j+1 in the high nibble.
+ *       INT4 : two's-complement integer q in [-7, 7]; value q * scale.
+ *       LUQ  : bit 3 = sign, bits 0..2 = c; c = 0 is zero (always nibble 0x0),
+ *              c >= 1 is alpha * 2^(c-1).  With the compiled level count
+ *              (luq_kmax() = 4) the codes 0..5 occur.
+ *   - Every pointer named d_* is a DEVICE pointer owned by the caller and must
+ *     be 16-byte aligned.  Scalars (max, scales) stay in device memory so a
+ *     whole step needs no host synchronisation.
+ *   - Every call is asynchronous on `stream` (a cudaStream_t passed as void*;
+ *     NULL = the default stream) and returns 0 on success or a negative
+ *     LUQ_ERR_* code.  Nothing throws, aborts or traps the device.
+ *   - Conditions found on the device set bits in a status word read with
+ *     luq_status(): outputs stay defined (zero codes and a zero scale for a
+ *     non-finite or out-of-range max; unspecified values after a TIMEOUT).
+ *   - A context serves one stream at a time; calls that overlap on the GPU
+ *     through the same context race on its workspace.
+ */
+#ifndef LUQ_H_
+#define LUQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* element types of the high-precision inputs */
+#define LUQ_F32 0
+#define LUQ_BF16 1
+
+/* return codes */
+#define LUQ_OK 0
+#define LUQ_ERR_ARG (-1)         /* null/misaligned pointer, bad size, bad n_samples */
+#define LUQ_ERR_CUDA (-2)        /* a CUDA runtime/driver call failed */
+#define LUQ_ERR_UNSUPPORTED (-3) /* device is not sm_100, or option unknown */
+#define LUQ_ERR_WORKSPACE (-4)   /* problem needs more split workspace than the context holds */
+
+/* device status bits (luq_status) */
+#define LUQ_STATUS_NONFINITE 1 /* a max / clip was Inf or NaN: zero codes, zero scale */
+#define LUQ_STATUS_RANGE 2     /* a non-zero max / clip outside [2^-100, 2^100]: zero codes, zero scale */
+#define LUQ_STATUS_TIMEOUT 4   /* a bounded wait inside a kernel expired; outputs unspecified */
+
+/* options for luq_set_option */
+#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands (default); 1: kind::i8 on int8 operands */
+#define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
+
+#define LUQ_MAX_SAMPLES 8
+
+typedef struct luq_ctx luq_ctx;
+
+/* Creates a context on `device`: a device status word and the split workspace
+ * (16 MiB) used by GEMMs whose output has too few tiles to fill the GPU.
+ * Allocates device memory; call outside stream capture. */
+int luq_create(luq_ctx** out, int device);
+int luq_destroy(luq_ctx* ctx);
+int luq_set_option(luq_ctx* ctx, int option, int value);
+
+/* Number of binades between the underflow threshold and the tensor maximum:
+ * alpha = max|x| / 2^kmax.  The paper's Eq. (alpha) prints 2^(2^(b-1)) with
+ * b = 3, i.e. kmax = 4. */
+int luq_kmax(void);
+
+/* max_i |x_i| of a tensor of n elements (Sec. 4, "Above FP maximum": the top
+ * level is the tensor maximum, Eq. alpha).  d_amax receives one float.  If any
+ * element is Inf/NaN the result is Inf/NaN and LUQ_STATUS_NONFINITE is set. */
+int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, void* stream);
+
+/* Q_INT, INT4 round-to-nearest (Sec. 3.3: RDN for weights and activations in
+ * all phases; Appendix A.1: one high-precision scale per tensor).
+ *   scale = clip / 7, q = clamp(rint(x * (7 / clip)), -7, 7), ties to even.
+ * d_clip is usually the tensor max from luq_amax; any caller clip is allowed.
+ * rows*cols must be even.  d_codes: rows*cols/2 bytes.  d_scale: one float. */
+int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
+                   const float* d_clip, uint8_t* d_codes, float* d_scale, void* stream);
+
+/* Q_FP = LUQ (Sec. 4): alpha = max / 2^kmax (Eq. alpha); |x| < alpha becomes
+ * sign*alpha with probability |x|/alpha, else 0 (Eq. StochasticPruning);
+ * in-range values round stochastically between the two enclosing powers of two
+ * (Eq. unbiasedFpQ).  t = |x|/alpha is an IEEE binary32 quotient; one 32-bit
+ * Philox4x32-10 word per element and sample decides: key = seed + sample,
+ * counter = index/4, word = index%4 (index = flat row-major element index).
+ * SMP (Sec. 5.1): n_samples independent draws, written as n_samples planes of
+ * rows*cols/2 bytes, sample-major.  d_amax usually comes from luq_amax; a
+ * smaller value clips to the top level.  d_alpha receives alpha. */
+int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
+                   const float* d_amax, uint64_t seed, int n_samples,
+                   uint8_t* d_codes, float* d_alpha, void* stream);
+
+/* Forward GEMM (Eq. Forward; scale factoring of Appendix A.1):
+ *   Z[m,n] = (sa*sw) * sum_k qA[m,k] * qW[n,k]        fp32 accumulate, fp32 out.
+ * a_codes [M x K/2], w_codes [N x K/2].  K must be a multiple of 32. */
+int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa,
+                 const uint8_t* d_w_codes, const float* d_sw,
+                 float* d_z, int64_t M, int64_t N, int64_t K, void* stream);
+
+/* Backward GEMM (Eq. Backward), SMP average fused (Sec. 5.1):
+ *   dA[m,k] = (alpha*sw/n_samples) * sum_s sum_n qG_s[m,n] * qW[n,k].
+ * g_codes: n_samples planes [M x N/2]; w_codes [N x K/2].
+ * N and K must be multiples of 32. */
+int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
+                 const uint8_t* d_w_codes, const float* d_sw,
+                 float* d_da, int64_t M, int64_t N, int64_t K, void* stream);
+
+/* Update GEMM (Eq. Update), SMP average fused (Sec. 5.1):
+ *   dW[n,k] = (alpha*sa/n_samples) * sum_s sum_m qG_s[m,n] * qA[m,k].
+ * g_codes: n_samples planes [M x N/2]; a_codes [M x K/2].
+ * N and K must be multiples of 32.  Uses the context's split workspace when
+ * the output has few tiles (contraction over M is split across CTAs). */
+int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
+                   const uint8_t* d_a_codes, const float* d_sa,
+                   float* d_dw, int64_t M, int64_t N, int64_t K, void* stream);
+
+/* Synchronises `stream`, returns the device status bits in *host_flags and
+ * clears them. */
+int luq_status(luq_ctx* ctx, void* stream, int* host_flags);
+
+/* Number of kernels this library has launched through `ctx` so far. */
+int64_t luq_launch_count(luq_ctx* ctx);
+
+const char* luq_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LUQ_H_ */

@@ -16,9 +16,10 @@
  * Parity pins (see tests marked "not gpu"): grid membership, fixed points,
  * exact expectation, the literal two-draw transcription of T_alpha / Q_alpha,
  * the paper's worked values, Table 1 closed forms, brute force GEMMs, and the
- * Philox constants / stream (cuRAND header constants on the CPU, the cuRAND
- * device generator on a GPU box).  The raw Philox stream is "parity unpinned"
- * on a box without cuRAND's header: any fixed bijective stream satisfies the paper.
+ * Philox constants and stream (cuRAND's header constants and cuRAND's own block
+ * function compiled for the host).  On a machine without the CUDA toolkit the
+ * raw Philox stream is "parity unpinned": any fixed bijective stream satisfies
+ * the paper, which names no generator.
  *
  * Build: gcc -O2 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
  */

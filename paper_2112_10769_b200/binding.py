@@ -1,0 +1,166 @@
+"""ctypes binding of the C-ABI library declared in ``include/luq.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of
+``libluq_b200.so``.  PyTorch supplies device memory and the current stream.
+There is no fallback: if the library has not been built (``python -m
+paper_2112_10769_b200.build``) or no sm_100 GPU is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libluq_b200.so")
+
+LUQ_F32, LUQ_BF16 = 0, 1
+STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT = 1, 2, 4
+OPT_MMA_KIND, OPT_SPLITS = 1, 2
+ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
+
+SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
+           "luq_quant_grad", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_status",
+           "luq_launch_count", "luq_strerror")
+
+_lib = None
+
+
+class LuqError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {load().luq_strerror(code).decode()} ({code})")
+
+
+def load() -> ctypes.CDLL:
+    """Loads the compiled library; raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2112_10769_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, i64, u64 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int64, ctypes.c_uint64
+        L.luq_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+        L.luq_destroy.argtypes = [vp]
+        L.luq_set_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+        L.luq_kmax.argtypes = []
+        L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
+        L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp]
+        L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp]
+        L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_gemm_wgrad.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int)]
+        L.luq_launch_count.argtypes = [vp]
+        L.luq_launch_count.restype = i64
+        L.luq_strerror.argtypes = [ctypes.c_int]
+        L.luq_strerror.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return LUQ_F32
+    if t.dtype == torch.bfloat16:
+        return LUQ_BF16
+    raise TypeError("inputs are float32 or bfloat16")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise LuqError(rc, what)
+
+
+class Context:
+    """Owns one luq_ctx (status word + split workspace) on a device."""
+
+    def __init__(self, device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: this library has no CPU path")
+        self.device = device
+        h = ctypes.c_void_p()
+        _check(load().luq_create(ctypes.byref(h), device), "luq_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load().luq_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_option(self, option: int, value: int):
+        _check(load().luq_set_option(self.handle, option, value), "luq_set_option")
+
+    @property
+    def launches(self) -> int:
+        return int(load().luq_launch_count(self.handle))
+
+    # ---- the path ----------------------------------------------------------
+    def amax(self, x: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+        out = torch.empty(1, dtype=torch.float32, device=x.device) if out is None else out
+        _check(load().luq_amax(self.handle, x.data_ptr(), _dtype_code(x), x.numel(), out.data_ptr(), _stream()),
+               "luq_amax")
+        return out
+
+    def quant_int4(self, x: torch.Tensor, clip: torch.Tensor, codes: torch.Tensor | None = None,
+                   scale: torch.Tensor | None = None):
+        rows, cols = (x.shape[0], x.numel() // max(x.shape[0], 1)) if x.dim() > 1 else (1, x.numel())
+        codes = torch.empty(x.numel() // 2, dtype=torch.uint8, device=x.device) if codes is None else codes
+        scale = torch.empty(1, dtype=torch.float32, device=x.device) if scale is None else scale
+        _check(load().luq_quant_int4(self.handle, x.data_ptr(), _dtype_code(x), rows, cols, clip.data_ptr(),
+                                     codes.data_ptr(), scale.data_ptr(), _stream()), "luq_quant_int4")
+        return codes, scale
+
+    def quant_grad(self, g: torch.Tensor, amax: torch.Tensor, seed: int, n_samples: int = 1,
+                   codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None):
+        rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
+        if codes is None:
+            codes = torch.empty((n_samples, g.numel() // 2), dtype=torch.uint8, device=g.device)
+        alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
+        _check(load().luq_quant_grad(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
+                                     seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
+                                     _stream()), "luq_quant_grad")
+        return codes, alpha
+
+    def gemm_fwd(self, a_codes, sa, w_codes, sw, M: int, N: int, K: int, out: torch.Tensor | None = None):
+        out = torch.empty((M, N), dtype=torch.float32, device=a_codes.device) if out is None else out
+        _check(load().luq_gemm_fwd(self.handle, a_codes.data_ptr(), sa.data_ptr(), w_codes.data_ptr(),
+                                   sw.data_ptr(), out.data_ptr(), M, N, K, _stream()), "luq_gemm_fwd")
+        return out
+
+    def gemm_bwd(self, g_codes, alpha, n_samples: int, w_codes, sw, M: int, N: int, K: int,
+                 out: torch.Tensor | None = None):
+        out = torch.empty((M, K), dtype=torch.float32, device=g_codes.device) if out is None else out
+        _check(load().luq_gemm_bwd(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
+                                   w_codes.data_ptr(), sw.data_ptr(), out.data_ptr(), M, N, K, _stream()),
+               "luq_gemm_bwd")
+        return out
+
+    def gemm_wgrad(self, g_codes, alpha, n_samples: int, a_codes, sa, M: int, N: int, K: int,
+                   out: torch.Tensor | None = None):
+        out = torch.empty((N, K), dtype=torch.float32, device=g_codes.device) if out is None else out
+        _check(load().luq_gemm_wgrad(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
+                                     a_codes.data_ptr(), sa.data_ptr(), out.data_ptr(), M, N, K, _stream()),
+               "luq_gemm_wgrad")
+        return out
+
+    def status(self) -> int:
+        """Synchronises the current stream; returns and clears the device status bits."""
+        flags = ctypes.c_int(0)
+        _check(load().luq_status(self.handle, _stream(), ctypes.byref(flags)), "luq_status")
+        return flags.value
+
+
+def kmax() -> int:
+    return int(load().luq_kmax())

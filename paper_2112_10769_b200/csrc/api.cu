@@ -1,0 +1,222 @@
+// C ABI of the library (declared in luq.h): argument checks, context, launches.
+#include <new>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr size_t kWorkspaceBytes = 16u << 20;
+constexpr int kMaxTickets = 1024;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+int cuda_rc(int e) { return e == 0 ? LUQ_OK : (e < 0 ? e : LUQ_ERR_CUDA); }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+int luq_kmax(void) { return LUQ_KMAX; }
+
+const char* luq_strerror(int code) {
+  switch (code) {
+    case LUQ_OK: return "ok";
+    case LUQ_ERR_ARG: return "invalid argument (null or misaligned pointer, bad size or sample count)";
+    case LUQ_ERR_CUDA: return "a CUDA call failed";
+    case LUQ_ERR_UNSUPPORTED: return "unsupported device or option";
+    case LUQ_ERR_WORKSPACE: return "split workspace too small for this problem";
+    default: return "unknown error";
+  }
+}
+
+int luq_create(luq_ctx** out, int device) {
+  if (!out) return LUQ_ERR_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return LUQ_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return LUQ_ERR_CUDA;
+  if (prop.major != 10) return LUQ_ERR_UNSUPPORTED;  // the kernels are sm_100a only
+  DeviceGuard guard(device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  luq_ctx* c = new (std::nothrow) luq_ctx();
+  if (!c) return LUQ_ERR_CUDA;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  c->mma_kind = 0;
+  c->forced_splits = 0;
+  c->launches = 0;
+  c->workspace_bytes = kWorkspaceBytes;
+  c->max_tickets = kMaxTickets;
+  c->d_status = nullptr; c->d_workspace = nullptr; c->d_tickets = nullptr; c->encode_tiled = nullptr;
+  bool ok = cudaMalloc(&c->d_status, sizeof(unsigned int)) == cudaSuccess &&
+            cudaMalloc(&c->d_workspace, kWorkspaceBytes) == cudaSuccess &&
+            cudaMalloc(&c->d_tickets, kMaxTickets * sizeof(unsigned int)) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_status, 0, sizeof(unsigned int)) == cudaSuccess &&
+       cudaMemset(c->d_workspace, 0, kWorkspaceBytes) == cudaSuccess &&
+       cudaMemset(c->d_tickets, 0, kMaxTickets * sizeof(unsigned int)) == cudaSuccess;
+  if (ok) {
+    cudaDriverEntryPointQueryResult q;
+    ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) == cudaSuccess &&
+         q == cudaDriverEntryPointSuccess && c->encode_tiled != nullptr;
+  }
+  if (!ok) { luq_destroy(c); return LUQ_ERR_CUDA; }
+  *out = c;
+  return LUQ_OK;
+}
+
+int luq_destroy(luq_ctx* ctx) {
+  if (!ctx) return LUQ_OK;
+  DeviceGuard guard(ctx->device);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->d_workspace) cudaFree(ctx->d_workspace);
+  if (ctx->d_tickets) cudaFree(ctx->d_tickets);
+  delete ctx;
+  return LUQ_OK;
+}
+
+int luq_set_option(luq_ctx* ctx, int option, int value) {
+  if (!ctx) return LUQ_ERR_ARG;
+  switch (option) {
+    case LUQ_OPT_MMA_KIND:
+      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      ctx->mma_kind = value;
+      return LUQ_OK;
+    case LUQ_OPT_SPLITS:
+      if (value < 0 || value > 1024) return LUQ_ERR_ARG;
+      ctx->forced_splits = value;
+      return LUQ_OK;
+    default:
+      return LUQ_ERR_UNSUPPORTED;
+  }
+}
+
+int64_t luq_launch_count(luq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, void* stream) {
+  if (!ctx || !d_amax || (n && !d_x) || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  if (!aligned16(d_x) || (reinterpret_cast<uintptr_t>(d_amax) & 3u)) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_amax(ctx, d_x, dtype, n, d_amax, as_stream(stream)));
+}
+
+int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, const float* d_clip,
+                   uint8_t* d_codes, float* d_scale, void* stream) {
+  if (!ctx || !d_clip || !d_scale || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  const size_t n = rows * cols;
+  if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
+  if (n & 1u) return LUQ_ERR_ARG;
+  if (n && (!d_x || !d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_codes)) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, d_clip, d_codes, d_scale, as_stream(stream)));
+}
+
+int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
+                   uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, void* stream) {
+  if (!ctx || !d_amax || !d_alpha || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  if (n_samples < 1 || n_samples > LUQ_MAX_SAMPLES) return LUQ_ERR_ARG;
+  const size_t n = rows * cols;
+  if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
+  if (n & 1u) return LUQ_ERR_ARG;
+  if (n && (!d_g || !d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_g) || !aligned16(d_codes)) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_grad(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes, d_alpha,
+                                       as_stream(stream)));
+}
+
+static int gemm_common(luq_ctx* ctx, const uint8_t* x, const float* sx, const uint8_t* y, const float* sy,
+                       float* out, int64_t M, int64_t N, int64_t K, int n_samples) {
+  if (!ctx || !sx || !sy) return LUQ_ERR_ARG;
+  if (M < 0 || N < 0 || K < 0 || M > (1ll << 31) || N > (1ll << 31) || K > (1ll << 31)) return LUQ_ERR_ARG;
+  if (n_samples < 1 || n_samples > LUQ_MAX_SAMPLES) return LUQ_ERR_ARG;
+  if (M && N && K && (!x || !y || !out)) return LUQ_ERR_ARG;
+  if (!aligned16(x) || !aligned16(y) || !aligned16(out)) return LUQ_ERR_ARG;
+  return LUQ_OK;
+}
+
+int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, const uint8_t* d_w_codes,
+                 const float* d_sw, float* d_z, int64_t M, int64_t N, int64_t K, void* stream) {
+  int rc = gemm_common(ctx, d_a_codes, d_sa, d_w_codes, d_sw, d_z, M, N, K, 1);
+  if (rc) return rc;
+  if (K % 32 || N % 4) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  luq_gemm_args a{};
+  a.a_codes = d_a_codes; a.a_kind = 0; a.a_mn = 0; a.n_samples = 1;
+  a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 0;
+  a.d_scale_a = d_sa; a.d_scale_b = d_sw; a.d_out = d_z; a.Mo = M; a.No = N; a.Kc = K;
+  a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
+  a.d_tickets = ctx->d_tickets; a.max_tickets = ctx->max_tickets; a.allow_split = 1;
+  return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
+}
+
+int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
+                 const uint8_t* d_w_codes, const float* d_sw, float* d_da, int64_t M, int64_t N, int64_t K,
+                 void* stream) {
+  int rc = gemm_common(ctx, d_g_codes, d_alpha, d_w_codes, d_sw, d_da, M, N, K, n_samples);
+  if (rc) return rc;
+  if (N % 32 || K % 32) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  luq_gemm_args a{};
+  a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 0; a.n_samples = n_samples;   // G[M x N]: contraction n contiguous
+  a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 1;                            // W[N x K]: rows are the contraction
+  a.d_scale_a = d_alpha; a.d_scale_b = d_sw; a.d_out = d_da; a.Mo = M; a.No = K; a.Kc = N;
+  a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
+  a.d_tickets = ctx->d_tickets; a.max_tickets = ctx->max_tickets; a.allow_split = 1;
+  return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
+}
+
+int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
+                   const uint8_t* d_a_codes, const float* d_sa, float* d_dw, int64_t M, int64_t N, int64_t K,
+                   void* stream) {
+  int rc = gemm_common(ctx, d_g_codes, d_alpha, d_a_codes, d_sa, d_dw, M, N, K, n_samples);
+  if (rc) return rc;
+  if (N % 32 || K % 32) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  luq_gemm_args a{};
+  a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 1; a.n_samples = n_samples;   // G[M x N]: rows are the contraction
+  a.b_codes = d_a_codes; a.b_kind = 0; a.b_mn = 1;                            // A[M x K]: rows are the contraction
+  a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.Mo = N; a.No = K; a.Kc = M;
+  a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
+  a.d_tickets = ctx->d_tickets; a.max_tickets = ctx->max_tickets; a.allow_split = 1;
+  return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
+}
+
+int luq_status(luq_ctx* ctx, void* stream, int* host_flags) {
+  if (!ctx || !host_flags) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  cudaStream_t st = as_stream(stream);
+  unsigned int flags = 0;
+  if (cudaMemcpyAsync(&flags, ctx->d_status, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return LUQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LUQ_ERR_CUDA;
+  if (flags) {
+    if (cudaMemsetAsync(ctx->d_status, 0, sizeof(unsigned int), st) != cudaSuccess) return LUQ_ERR_CUDA;
+    if (flags & LUQ_STATUS_TIMEOUT) {  // an aborted split GEMM may have left partial sums behind
+      cudaMemsetAsync(ctx->d_workspace, 0, ctx->workspace_bytes, st);
+      cudaMemsetAsync(ctx->d_tickets, 0, ctx->max_tickets * sizeof(unsigned int), st);
+    }
+    if (cudaStreamSynchronize(st) != cudaSuccess) return LUQ_ERR_CUDA;
+  }
+  *host_flags = static_cast<int>(flags);
+  return LUQ_OK;
+}
+
+}  // extern "C"

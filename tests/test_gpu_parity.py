@@ -1,0 +1,297 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI.
+
+Codes must match bit for bit; GEMM outputs within 1e-5 relative (products and
+sums are exact integers, only the two scale roundings of the epilogue differ
+from the float64 oracle) and exact zeros must be exact zeros.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2112_10769_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    assert c.status() == 0
+    c.close()
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    if a.dtype == np.uint16:  # bf16 bit patterns
+        return torch.from_numpy(a.view(np.int16).copy()).cuda().view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def scalar(v) -> torch.Tensor:
+    return torch.tensor([v], dtype=torch.float32, device="cuda")
+
+
+def assert_gemm_close(got: np.ndarray, ref: np.ndarray):
+    got = got.astype(np.float64)
+    zero = ref == 0
+    assert (got[zero] == 0).all(), "entries that are exactly zero in the oracle must be exactly zero"
+    nz = ~zero
+    if nz.any():
+        rel = np.abs(got[nz] - ref[nz]) / np.abs(ref[nz])
+        assert rel.max() <= RTOL, f"max relative error {rel.max():.3e}"
+        assert np.abs(got - ref).max() <= RTOL * np.abs(ref).max()
+
+
+# ------------------------------------------------------------------ amax ----
+
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 1023, 4096, 65537, (1 << 20) + 6, 5_000_011])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_amax_matches_oracle(ctx, n, dtype):
+    x = inputs.lognormal_gradient((n,), -10.0, 3.0, 0.2, 1000 + n)
+    if dtype == "bf16":
+        x = inputs.to_bf16_bits(x)
+    want, fl = oracle.amax(x)
+    got = ctx.amax(to_dev(x)).cpu().numpy()[0]
+    assert fl == 0 and got == want and got.dtype == np.float32
+    assert ctx.status() == 0
+
+
+def test_amax_zero_empty_and_nonfinite(ctx):
+    assert ctx.amax(torch.zeros(1000, device="cuda")).item() == 0.0
+    assert ctx.amax(torch.zeros(0, device="cuda")).item() == 0.0
+    assert ctx.status() == 0
+    for bad in (float("inf"), float("-inf"), float("nan")):
+        x = torch.randn(100000, device="cuda")
+        x[77777] = bad
+        got = ctx.amax(x).item()
+        assert not np.isfinite(got)
+        assert ctx.status() == binding.STATUS_NONFINITE
+        assert ctx.status() == 0  # reading clears
+
+
+# ------------------------------------------------------------------ INT4 ----
+
+@pytest.mark.parametrize("n", [2, 6, 8, 10, 1000, 4098, 65536, (1 << 20) + 2, 3_000_004])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_quant_int4_bit_exact(ctx, n, dtype):
+    x = inputs.normal((n,), 1.0, 2000 + n, relu=(n % 4 == 0))
+    if dtype == "bf16":
+        x = inputs.to_bf16_bits(x)
+    clip, _ = oracle.amax(x)
+    want, s_want, fl = oracle.quant_int4(x, clip)
+    xd = to_dev(x)
+    codes, scale = ctx.quant_int4(xd, ctx.amax(xd))
+    assert fl == 0 and scale.item() == s_want
+    np.testing.assert_array_equal(codes.cpu().numpy(), want)
+    assert ctx.status() == 0
+
+
+def test_quant_int4_caller_clip_ties_and_specials(ctx):
+    x = np.array([0.5, 1.5, 2.5, 3.5, -0.5, -1.5, -2.5, 6.5, 100.0, -100.0, 7.49, 7.51, 0.0, -0.0, np.nan, np.inf,
+                  -np.inf, 1e-30], dtype=np.float32)
+    want, s_want, _ = oracle.quant_int4(x, np.float32(7.0))
+    codes, scale = ctx.quant_int4(to_dev(x), scalar(7.0))
+    np.testing.assert_array_equal(codes.cpu().numpy(), want)
+    assert scale.item() == s_want == 1.0
+    # window of consecutive floats around a rounding boundary
+    clip = np.float32(3.0)
+    start = np.array([2.5 * 3.0 / 7.0], dtype=np.float32).view(np.uint32)[0]
+    x = (np.arange(-2000, 2000, dtype=np.int64) + int(start)).astype(np.uint32).view(np.float32)
+    want, _, _ = oracle.quant_int4(x, clip)
+    codes, _ = ctx.quant_int4(to_dev(x), scalar(3.0))
+    np.testing.assert_array_equal(codes.cpu().numpy(), want)
+
+
+def test_quant_zero_and_unusable_scale(ctx):
+    x = torch.randn(4096, device="cuda")
+    for clip, flag in ((0.0, 0), (float("inf"), binding.STATUS_NONFINITE), (float("nan"), binding.STATUS_NONFINITE),
+                       (2.0 ** -120, binding.STATUS_RANGE), (2.0 ** 110, binding.STATUS_RANGE)):
+        codes, scale = ctx.quant_int4(x, scalar(clip))
+        assert scale.item() == 0 and not codes.any().item()
+        assert ctx.status() == flag
+        codes, alpha = ctx.quant_grad(x, scalar(clip), seed=1, n_samples=2)
+        assert alpha.item() == 0 and not codes.any().item()
+        assert ctx.status() == flag
+    z = torch.zeros(4096, device="cuda")
+    codes, alpha = ctx.quant_grad(z, ctx.amax(z), seed=1)
+    assert alpha.item() == 0 and not codes.any().item() and ctx.status() == 0
+
+
+def test_argument_errors(ctx):
+    x = torch.randn(64, device="cuda")
+    with pytest.raises(binding.LuqError):
+        ctx.quant_grad(x, scalar(1.0), seed=0, n_samples=0)
+    with pytest.raises(binding.LuqError):
+        ctx.quant_grad(x, scalar(1.0), seed=0, n_samples=9)
+    with pytest.raises(binding.LuqError):
+        ctx.quant_int4(x[:63], scalar(1.0))          # odd element count
+    with pytest.raises(binding.LuqError):
+        ctx.quant_int4(x[1:33], scalar(1.0))         # misaligned pointer
+    c = torch.zeros(64 * 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.LuqError):
+        ctx.gemm_fwd(c, scalar(1.0), c, scalar(1.0), 64, 32, 16)   # K not a multiple of 32
+
+
+# ------------------------------------------------------------------- LUQ ----
+
+def luq_inputs(n, seed):
+    x = inputs.log_uniform_magnitudes(n, -30, 3, seed)
+    mx = np.abs(x).max()
+    al = mx / 16
+    special = [0.0, -0.0, mx, -mx, al, -al, 2 * al, 4 * al, 8 * al, 1e-38, -1e-45, al * (1 - 2 ** -24), al * (1 + 2 ** -23)]
+    k = min(len(special), n)
+    x[:k] = np.array(special[:k], dtype=np.float32)
+    if n > 20:
+        x[20] = np.float32(mx)
+    return x
+
+
+@pytest.mark.parametrize("n", [2, 6, 8, 10, 1000, 4098, 65536, (1 << 20) + 2, 3_000_004])
+@pytest.mark.parametrize("dtype,ns", [("f32", 1), ("f32", 2), ("bf16", 1), ("bf16", 3)])
+def test_quant_grad_bit_exact(ctx, n, dtype, ns):
+    x = luq_inputs(n, 3000 + n)
+    if dtype == "bf16":
+        x = inputs.to_bf16_bits(x)
+    mx, _ = oracle.amax(x)
+    seed = 12345 + n
+    want, a_want, fl = oracle.quant_luq(x, mx, seed, ns)
+    xd = to_dev(x)
+    codes, alpha = ctx.quant_grad(xd, ctx.amax(xd), seed, ns)
+    assert fl == 0 and alpha.item() == a_want
+    np.testing.assert_array_equal(codes.cpu().numpy().reshape(ns, -1), want)
+    assert ctx.status() == 0
+
+
+def test_quant_grad_seed_semantics_and_clipping(ctx):
+    x = luq_inputs(50000, 9)
+    xd = to_dev(x)
+    mx = ctx.amax(xd)
+    big = (1 << 63) + 12345678901234
+    for seed in (0, 1, 2 ** 32 - 1, 2 ** 32, big):
+        want, _, _ = oracle.quant_luq(x, mx.item(), seed, 2)
+        codes, _ = ctx.quant_grad(xd, mx, seed, 2)
+        np.testing.assert_array_equal(codes.cpu().numpy(), want)
+    # sample s of seed equals sample 0 of seed + s
+    c2, _ = ctx.quant_grad(xd, mx, 40, 3)
+    c0, _ = ctx.quant_grad(xd, mx, 42, 1)
+    assert torch.equal(c2[2], c0[0])
+    # a caller max below the true one clips to the top level
+    small = scalar(float(mx.item()) / 64)
+    want, a_want, _ = oracle.quant_luq(x, small.item(), 5, 1)
+    codes, alpha = ctx.quant_grad(xd, small, 5, 1)
+    np.testing.assert_array_equal(codes.cpu().numpy(), want)
+    assert alpha.item() == a_want
+    # many scales: on-grid inputs are fixed points for every seed
+    rng = np.random.default_rng(3)
+    for mxv in np.exp2(rng.uniform(-20, 20, 40)).astype(np.float32):
+        al = np.float32(mxv) / np.float32(16)
+        grid = np.array([al * 2 ** k for k in range(5)] * 8, dtype=np.float32)
+        want, _, _ = oracle.quant_luq(grid, mxv, 7, 1)
+        codes, _ = ctx.quant_grad(to_dev(grid), scalar(float(mxv)), 7, 1)
+        np.testing.assert_array_equal(codes.cpu().numpy(), want)
+        assert list(oracle.unpack(want[0], 5)) == [1, 2, 3, 4, 5]
+
+
+# ------------------------------------------------------------------ GEMMs ----
+
+def run_layer(ctx, A, W, G, seed, ns):
+    """Whole path on the GPU; returns device tensors and the oracle's codes."""
+    M, K = A.shape
+    N = W.shape[0]
+    Ad, Wd, Gd = to_dev(A), to_dev(W), to_dev(G)
+    ca, sa = ctx.quant_int4(Ad, ctx.amax(Ad))
+    cw, sw = ctx.quant_int4(Wd, ctx.amax(Wd))
+    cg, al = ctx.quant_grad(Gd, ctx.amax(Gd), seed, ns)
+    Z = ctx.gemm_fwd(ca, sa, cw, sw, M, N, K)
+    dA = ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K)
+    dW = ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K)
+    oa, osa, _ = oracle.quant_int4(A, oracle.amax(A)[0])
+    ow, osw, _ = oracle.quant_int4(W, oracle.amax(W)[0])
+    og, oal, _ = oracle.quant_luq(G, oracle.amax(G)[0], seed, ns)
+    np.testing.assert_array_equal(ca.cpu().numpy(), oa)
+    np.testing.assert_array_equal(cw.cpu().numpy(), ow)
+    np.testing.assert_array_equal(cg.cpu().numpy().reshape(ns, -1), og)
+    assert (sa.item(), sw.item(), al.item()) == (osa, osw, oal)
+    return (Z, dA, dW), (oa, osa), (ow, osw), (og, oal)
+
+
+SHAPES = [
+    (128, 128, 256, 1),    # one tile, one contraction block
+    (256, 256, 256, 1),    # config 1 shape
+    (300, 160, 96, 1),     # ragged in every dimension
+    (130, 416, 544, 2),    # several tiles with tails, two samples
+    (1000, 32, 32, 1),     # minimum contraction
+    (64, 1024, 288, 3),    # three samples
+]
+
+
+@pytest.mark.parametrize("mma_kind", [0, 1])
+@pytest.mark.parametrize("M,K,N,ns", SHAPES)
+def test_three_gemms_match_oracle(ctx, M, K, N, ns, mma_kind):
+    ctx.set_option(binding.OPT_MMA_KIND, mma_kind)
+    try:
+        A, W, G = inputs.small_layer(M, K, N, 500 + M + K)
+        (Z, dA, dW), (oa, osa), (ow, osw), (og, oal) = run_layer(ctx, A, W, G, seed=M, ns=ns)
+        assert ctx.status() == 0
+        assert_gemm_close(Z.cpu().numpy(), oracle.gemm_fwd(oa, osa, ow, osw, M, N, K))
+        assert_gemm_close(dA.cpu().numpy(), oracle.gemm_bwd(og, oal, ns, ow, osw, M, N, K))
+        assert_gemm_close(dW.cpu().numpy(), oracle.gemm_wgrad(og, oal, ns, oa, osa, M, N, K))
+    finally:
+        ctx.set_option(binding.OPT_MMA_KIND, 0)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 5])
+def test_wgrad_contraction_split(ctx, splits):
+    """The update GEMM contracts over the batch; splitting that contraction over
+    CTAs must not change the result."""
+    M, K, N = 2500, 160, 96
+    A, W, G = inputs.small_layer(M, K, N, 77)
+    ctx.set_option(binding.OPT_SPLITS, splits)
+    try:
+        for _ in range(2):  # twice: the workspace must be left clean
+            (Z, dA, dW), (oa, osa), (ow, osw), (og, oal) = run_layer(ctx, A, W, G, seed=3, ns=2)
+            assert ctx.status() == 0
+            assert_gemm_close(dW.cpu().numpy(), oracle.gemm_wgrad(og, oal, 2, oa, osa, M, N, K))
+            assert_gemm_close(dA.cpu().numpy(), oracle.gemm_bwd(og, oal, 2, ow, osw, M, N, K))
+            assert_gemm_close(Z.cpu().numpy(), oracle.gemm_fwd(oa, osa, ow, osw, M, N, K))
+    finally:
+        ctx.set_option(binding.OPT_SPLITS, 0)
+
+
+def test_config1_whole_step(ctx):
+    cfg = inputs.CONFIGS["cfg1"]
+    A, W, G = inputs.layer_inputs(cfg)
+    (Z, dA, dW), (oa, osa), (ow, osw), (og, oal) = run_layer(ctx, A, W, G, cfg.luq_seed, cfg.n_samples)
+    M, K, N = cfg.M, cfg.K, cfg.N
+    assert_gemm_close(Z.cpu().numpy(), oracle.gemm_fwd(oa, osa, ow, osw, M, N, K))
+    assert_gemm_close(dA.cpu().numpy(), oracle.gemm_bwd(og, oal, 1, ow, osw, M, N, K))
+    assert_gemm_close(dW.cpu().numpy(), oracle.gemm_wgrad(og, oal, 1, oa, osa, M, N, K))
+    assert ctx.status() == 0
+
+
+def test_gemm_large_integer_sums_are_exact(ctx):
+    """Worst-case operands (every code at its extreme) over a long contraction:
+    the accumulator must hold every integer partial sum exactly."""
+    M, N, K = 128, 256, 4096
+    a = torch.full((M, K // 2), 0x77, dtype=torch.uint8, device="cuda")     # all +7
+    w = torch.full((N, K // 2), 0x77, dtype=torch.uint8, device="cuda")
+    w[1::2] = 0x99                                                           # odd rows all -7
+    for kind in (0, 1):
+        ctx.set_option(binding.OPT_MMA_KIND, kind)
+        Z = ctx.gemm_fwd(a, scalar(1.0), w, scalar(1.0), M, N, K).cpu().numpy()
+        assert (Z[:, 0::2] == 49 * K).all() and (Z[:, 1::2] == -49 * K).all()
+        # sums that need all 24 bits: 49*K + small odd corrections
+        a2 = a.clone()
+        a2[:, 0] = 0x71                                                     # first element +1 instead of +7
+        Z = ctx.gemm_fwd(a2, scalar(1.0), w, scalar(1.0), M, N, K).cpu().numpy()
+        assert (Z[:, 0::2] == 49 * K - 42).all()
+        # gradient levels up to 16 times weights up to 7 over the whole contraction
+        g = torch.full((M, K // 2), 0x55, dtype=torch.uint8, device="cuda")  # all +16 (code 5)
+        wk = torch.full((K, N // 2), 0x77, dtype=torch.uint8, device="cuda")
+        dA = ctx.gemm_bwd(g, scalar(1.0), 1, wk, scalar(1.0), M, K, N).cpu().numpy()
+        assert (dA == 16 * 7 * K).all()
+    ctx.set_option(binding.OPT_MMA_KIND, 0)
+    assert ctx.status() == 0

@@ -531,3 +531,27 @@ def test_integer_partial_sums_fit_fp32():
     worst_bwd = 7 * 2 ** kmax * 4096 * 1
     worst_wgrad = 7 * 2 ** kmax * 50176 * 2
     assert max(worst_fwd, worst_bwd, worst_wgrad) < 2 ** 24
+
+
+def test_philox_stream_matches_curand_host_function(tmp_path):
+    """The generator equals NVIDIA's own Philox4x32-10 block function, compiled
+    for the host from the cuRAND header (an implementation independent of the oracle)."""
+    import ctypes
+    import shutil
+    import subprocess
+    if shutil.which("nvcc") is None:
+        pytest.skip("nvcc not on this machine")
+    src = os.path.join(os.path.dirname(__file__), "curand_philox_host.cu")
+    so = str(tmp_path / "libcurand_philox_host.so")
+    subprocess.run(["nvcc", "-Wno-deprecated-gpu-targets", "-shared", "-Xcompiler", "-fPIC", "-o", so, src], check=True)
+    L = ctypes.CDLL(so)
+    u32p = ctypes.POINTER(ctypes.c_uint32)
+    rng = np.random.default_rng(1)
+    cases = [(np.zeros(4, np.uint32), np.zeros(2, np.uint32)),
+             (np.full(4, 0xFFFFFFFF, np.uint32), np.full(2, 0xFFFFFFFF, np.uint32))]
+    cases += [(rng.integers(0, 2 ** 32, 4, dtype=np.uint32), rng.integers(0, 2 ** 32, 2, dtype=np.uint32))
+              for _ in range(200)]
+    for c, k in cases:
+        out = np.zeros(4, dtype=np.uint32)
+        L.curand_philox_block(c.ctypes.data_as(u32p), k.ctypes.data_as(u32p), out.ctypes.data_as(u32p))
+        np.testing.assert_array_equal(out, oracle.philox4x32_10(c, k))
