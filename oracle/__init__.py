@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
             L.oracle_quant_luq.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, ctypes.c_uint64,
                                            ctypes.c_int, u8p, intp]
             L.oracle_quant_luq.restype = ctypes.c_float
+            L.oracle_quant_luq_window.argtypes = [f32p, sz, ctypes.c_uint64, ctypes.c_float, ctypes.c_int,
+                                                  ctypes.c_uint64, ctypes.c_int, u8p, intp]
+            L.oracle_quant_luq_window.restype = ctypes.c_float
             L.oracle_luq_bins.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, f64p, f64p, u32p]
             L.oracle_dequant.argtypes = [u8p, sz, dbl, ctypes.c_int, f64p]
             L.oracle_gemm_fwd.argtypes = [u8p, dbl, u8p, dbl, i64, i64, i64, f64p]
@@ -126,15 +129,17 @@ def luq_alpha(mx, kmax: int = KMAX_DEFAULT) -> np.float32:
     return np.float32(lib().oracle_luq_alpha(np.float32(mx), kmax))
 
 
-def quant_luq(x: np.ndarray, mx, seed: int, n_samples: int = 1, kmax: int = KMAX_DEFAULT):
-    """LUQ = Q_alpha(T_alpha(x)) (Sec. 4).  Returns (codes[n_samples, n/2], alpha, flags)."""
+def quant_luq(x: np.ndarray, mx, seed: int, n_samples: int = 1, kmax: int = KMAX_DEFAULT,
+              first_index: int = 0):
+    """LUQ = Q_alpha(T_alpha(x)) (Sec. 4).  Returns (codes[n_samples, n/2], alpha, flags).
+    `first_index` (even) is the position of x[0] inside the full tensor."""
     xf = widen(x).reshape(-1)
     plane = (xf.size + 1) // 2
     codes = np.zeros((n_samples, plane), dtype=np.uint8)
     flags = ctypes.c_int(0)
-    a = lib().oracle_quant_luq(_ptr(xf, ctypes.c_float), xf.size, np.float32(mx), kmax,
-                               seed & (2**64 - 1), n_samples, _ptr(codes, ctypes.c_uint8),
-                               ctypes.byref(flags))
+    a = lib().oracle_quant_luq_window(_ptr(xf, ctypes.c_float), xf.size, first_index, np.float32(mx), kmax,
+                                      seed & (2**64 - 1), n_samples, _ptr(codes, ctypes.c_uint8),
+                                      ctypes.byref(flags))
     return codes, np.float32(a), flags.value
 
 

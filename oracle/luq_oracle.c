@@ -167,9 +167,20 @@ static luq_bin luq_bin_of(float a, float alpha, int kmax) {
 
 float oracle_luq_alpha(float mx, int kmax) { return ldexpf(mx, -kmax); }
 
-/* codes: n_samples planes of (n+1)/2 bytes each, sample-major. Returns alpha. */
+/* codes: n_samples planes of (n+1)/2 bytes each, sample-major. Returns alpha.
+ * x[0] is element `first_index` (even) of the full tensor: the random word of an
+ * element depends on its index in the whole tensor, so a window can be checked
+ * without quantizing everything before it. */
+float oracle_quant_luq_window(const float* x, size_t n, uint64_t first_index, float mx, int kmax,
+                              uint64_t seed, int n_samples, uint8_t* codes, int* flags);
+
 float oracle_quant_luq(const float* x, size_t n, float mx, int kmax, uint64_t seed,
                        int n_samples, uint8_t* codes, int* flags) {
+  return oracle_quant_luq_window(x, n, 0, mx, kmax, seed, n_samples, codes, flags);
+}
+
+float oracle_quant_luq_window(const float* x, size_t n, uint64_t first_index, float mx, int kmax,
+                              uint64_t seed, int n_samples, uint8_t* codes, int* flags) {
   size_t plane = (n + 1) / 2;
   memset(codes, 0, plane * (size_t)n_samples);
   if (!scale_usable(mx, flags)) return 0.0f;
@@ -180,7 +191,7 @@ float oracle_quant_luq(const float* x, size_t n, float mx, int kmax, uint64_t se
       float a = fabsf(x[i]);
       uint32_t sign = bits_of(x[i]) >> 31;
       luq_bin b = luq_bin_of(a, alpha, kmax);
-      uint32_t r = oracle_random_word(seed, (uint32_t)s, (uint64_t)i);
+      uint32_t r = oracle_random_word(seed, (uint32_t)s, first_index + (uint64_t)i);
       uint32_t c = b.lo_code + (r < b.threshold ? 1u : 0u);
       uint8_t nib = c ? (uint8_t)((sign << 3) | c) : 0;
       out[i >> 1] |= (uint8_t)(nib << ((i & 1) * 4));

@@ -1,0 +1,135 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+Codes are compared bit for bit over the whole tensors (the scalar oracle still
+finishes in seconds); GEMM outputs are compared on sampled entries that the
+oracle computes one by one from the codes.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2112_10769_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    assert c.status() == 0
+    c.close()
+
+
+def to_dev(a):
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(a).cuda()
+
+
+def sample_entries(rows, cols, count, seed):
+    rng = np.random.default_rng(seed)
+    r = rng.integers(0, rows, count)
+    c = rng.integers(0, cols, count)
+    # always include the corners and the last tile's edge
+    r[:4] = [0, rows - 1, 0, rows - 1]
+    c[:4] = [0, cols - 1, cols - 1, 0]
+    return r.astype(np.int64), c.astype(np.int64)
+
+
+def check_entries(got, ref):
+    got = got.astype(np.float64)
+    floor = 1e-12 * max(np.abs(ref).max(), 1e-300)
+    assert (got[ref == 0] == 0).all()
+    assert (np.abs(got - ref) <= RTOL * np.abs(ref) + floor).all()
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg5"])
+def test_layer_configs_full_size(ctx, name):
+    cfg = inputs.CONFIGS[name]
+    M, K, N, ns, seed = cfg.M, cfg.K, cfg.N, cfg.n_samples, cfg.luq_seed
+    A, W, G = inputs.layer_inputs(cfg)
+    Ad, Wd, Gd = to_dev(A), to_dev(W), to_dev(G)
+    mA, mW, mG = ctx.amax(Ad), ctx.amax(Wd), ctx.amax(Gd)
+    ca, sa = ctx.quant_int4(Ad, mA)
+    cw, sw = ctx.quant_int4(Wd, mW)
+    cg, al = ctx.quant_grad(Gd, mG, seed, ns)
+    Z = ctx.gemm_fwd(ca, sa, cw, sw, M, N, K)
+    dA = ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K)
+    dW = ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K)
+    assert ctx.status() == 0
+
+    # maxima, scales and every code, bit for bit
+    oA, oW, oG = oracle.amax(A)[0], oracle.amax(W)[0], oracle.amax(G)[0]
+    assert (mA.item(), mW.item(), mG.item()) == (oA, oW, oG)
+    oa, osa, _ = oracle.quant_int4(A, oA)
+    ow, osw, _ = oracle.quant_int4(W, oW)
+    og, oal, _ = oracle.quant_luq(G, oG, seed, ns)
+    assert (sa.item(), sw.item(), al.item()) == (osa, osw, oal)
+    assert np.array_equal(ca.cpu().numpy(), oa)
+    assert np.array_equal(cw.cpu().numpy(), ow)
+    assert np.array_equal(cg.cpu().numpy().reshape(ns, -1), og)
+
+    # sampled GEMM outputs
+    r, c = sample_entries(M, N, 300, 1)
+    check_entries(Z[torch.from_numpy(r).cuda(), torch.from_numpy(c).cuda()].cpu().numpy(),
+                  oracle.gemm_entries("fwd", oa, osa, 1, ow, osw, M, N, K, r, c))
+    r, c = sample_entries(M, K, 300, 2)
+    check_entries(dA[torch.from_numpy(r).cuda(), torch.from_numpy(c).cuda()].cpu().numpy(),
+                  oracle.gemm_entries("bwd", og, oal, ns, ow, osw, M, N, K, r, c))
+    r, c = sample_entries(N, K, 300, 3)
+    check_entries(dW[torch.from_numpy(r).cuda(), torch.from_numpy(c).cuda()].cpu().numpy(),
+                  oracle.gemm_entries("wgrad", og, oal, ns, oa, osa, M, N, K, r, c))
+
+    # properties that hold at any size: two samples are two single-sample runs
+    if ns == 2:
+        c0, _ = ctx.quant_grad(Gd, mG, seed, 1)
+        c1, _ = ctx.quant_grad(Gd, mG, seed + 1, 1)
+        assert torch.equal(c0[0], cg[0]) and torch.equal(c1[0], cg[1])
+        w0 = ctx.gemm_wgrad(c0, al, 1, ca, sa, M, N, K)
+        w1 = ctx.gemm_wgrad(c1, al, 1, ca, sa, M, N, K)
+        mean = (w0.double() + w1.double()) / 2
+        assert torch.allclose(dW.double(), mean, rtol=1e-6, atol=1e-12 * float(mean.abs().max()))
+    assert ctx.status() == 0
+
+
+@pytest.mark.parametrize("exponent", [20, 22, 24, 26])
+@pytest.mark.parametrize("ns", [1, 2])
+def test_quantizer_sweep_sizes(ctx, exponent, ns):
+    x = inputs.sweep_tensor(exponent)
+    xd = to_dev(x)
+    mx = ctx.amax(xd)
+    codes, alpha = ctx.quant_grad(xd, mx, 0, ns)
+    omx, _ = oracle.amax(x)
+    want, oal, _ = oracle.quant_luq(x, omx, 0, ns)
+    assert mx.item() == omx and alpha.item() == oal
+    assert np.array_equal(codes.cpu().numpy(), want)
+    assert ctx.status() == 0
+
+
+def test_quantizer_sweep_largest_size_windows(ctx):
+    """2^30 elements (4 GiB of input): the maximum is checked against numpy, codes
+    on windows at the start, across the 2^32-byte boundary and at the end."""
+    e = inputs.SWEEP_EXPONENTS[-1]
+    n = 1 << e
+    x = inputs.sweep_tensor(e)
+    xd = to_dev(x)
+    mx = ctx.amax(xd)
+    omx = np.abs(x).max()
+    assert mx.item() == omx
+    codes, alpha = ctx.quant_grad(xd, mx, 0, 2)
+    assert alpha.item() == oracle.luq_alpha(omx)
+    win = 1 << 18
+    for first in (0, n // 2 - win // 2, n - win, 123456 * 8):
+        want, _, _ = oracle.quant_luq(x[first:first + win], omx, 0, 2, first_index=first)
+        got = codes[:, first // 2:(first + win) // 2].cpu().numpy()
+        assert np.array_equal(got, want)
+    # whole-tensor property: no code above the top level kmax + 1 anywhere
+    for s in range(2):
+        plane = codes[s]
+        assert int(((plane & 7) > 5).sum().item()) == 0 and int((((plane >> 4) & 7) > 5).sum().item()) == 0
+    assert ctx.status() == 0
+    del xd, codes
+    torch.cuda.empty_cache()

@@ -555,3 +555,11 @@ def test_philox_stream_matches_curand_host_function(tmp_path):
         out = np.zeros(4, dtype=np.uint32)
         L.curand_philox_block(c.ctypes.data_as(u32p), k.ctypes.data_as(u32p), out.ctypes.data_as(u32p))
         np.testing.assert_array_equal(out, oracle.philox4x32_10(c, k))
+
+
+def test_luq_window_equals_slice_of_full_tensor():
+    x = luq_test_tensor(seed=91, n=5000)
+    mx, _ = oracle.amax(x)
+    full, _, _ = oracle.quant_luq(x, mx, seed=5, n_samples=2)
+    win, _, _ = oracle.quant_luq(x[1000:3000], mx, seed=5, n_samples=2, first_index=1000)
+    np.testing.assert_array_equal(win, full[:, 500:1500])
