@@ -20,7 +20,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -67,41 +66,46 @@ def algorithmic(cfg, ns):
 
 
 class ClockSampler(threading.Thread):
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock, power and throttle reasons (NVML) while the timed region runs."""
 
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.index = index
         self.samples = []
         self.stop_flag = threading.Event()
+        self.error = None
 
     def run(self):
-        while not self.stop_flag.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
-                parts = [p.strip() for p in out.strip().split(",")]
-                if len(parts) >= 8:
-                    self.samples.append(parts)
-            except Exception:
-                pass
-            self.stop_flag.wait(0.1)
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_sm = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            while not self.stop_flag.is_set():
+                sm = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+                pw = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+                try:
+                    rs = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    rs = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                self.samples.append((sm, pw, rs))
+                self.stop_flag.wait(0.01)
+        except Exception as e:  # pragma: no cover
+            self.error = repr(e)
 
     def summary(self):
         if not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
-        sm = sorted(float(s[0]) for s in self.samples)
-        reasons = set()
-        for s in self.samples:
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), s[4:8]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.samples[0][1]),
-                "power_w_max": max(float(s[2]) for s in self.samples), "samples": len(self.samples),
-                "reasons": sorted(reasons)}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable: %s" % self.error]}
+        import pynvml as nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        sm = sorted(s[0] for s in self.samples)
+        reasons = sorted(n for n, bit in names.items() if any(s[2] & bit for s in self.samples))
+        return {"sm_mhz": float(sm[len(sm) // 2]), "sm_min_mhz": float(sm[0]), "sm_max_mhz": float(self.max_sm),
+                "power_w_max": round(max(s[1] for s in self.samples), 1), "samples": len(self.samples),
+                "reasons": reasons}
 
 
 def gpu_physical_index(local: int) -> int:
@@ -116,12 +120,12 @@ def gpu_physical_index(local: int) -> int:
 
 # ---------------------------------------------------------------- CPU oracle --
 
-def oracle_sample(cfg, rows: int, ns: int):
+def oracle_sample(cfg, rows: int, ns: int, tensors=None):
     """The oracle, as it stands, on the first `rows` rows of the workload's batch
     dimension.  Returns (seconds, useful flops, threads)."""
     import oracle
     from paper_2112_10769_b200 import inputs
-    A, W, G = inputs.layer_inputs(cfg, rows=rows)
+    A, W, G = tensors if tensors is not None else inputs.layer_inputs(cfg, rows=rows)
     M, K, N = A.shape[0], cfg.K, cfg.N
     oracle.build()
     t0 = time.perf_counter()
@@ -141,13 +145,14 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2112_10769_b200 import inputs
-    cfg = inputs.CONFIGS[WORKLOAD]
-    rows = 512
+    cfg = inputs.CONFIGS[args.workload]
+    rows = min(512, cfg.M)  # about a quarter of a second per step on eight cores
+    tensors = inputs.layer_inputs(cfg, rows=rows)
     for _ in range(args.warmup):
-        oracle_sample(cfg, 128, cfg.n_samples)
+        oracle_sample(cfg, rows, cfg.n_samples, tensors)
     times, flops, threads = [], 0.0, 1
     for _ in range(args.steps):
-        dt, flops, threads = oracle_sample(cfg, rows, cfg.n_samples)
+        dt, flops, threads = oracle_sample(cfg, rows, cfg.n_samples, tensors)
         times.append(dt)
     mean = sum(times) / len(times)
     value = flops / mean / 1e12
@@ -155,9 +160,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: M=50176 K=2304 N=256 fp32, first {rows} rows of the batch per step"},
+        "config": {"workload": f"{args.workload}: M={cfg.M} K={cfg.K} N={cfg.N} {cfg.dtype}, first {rows} rows of the batch per step"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                         "sample": f"first {rows} of 50176 batch rows, all nine stages"},
+                         "sample": f"first {rows} of {cfg.M} batch rows, all nine stages"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -185,12 +190,20 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    cfg = inputs.CONFIGS[WORKLOAD]
+    cfg = inputs.CONFIGS[args.workload]
+    if args.rows:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, M=min(cfg.M, args.rows))
     M, K, N, ns, seed = cfg.M, cfg.K, cfg.N, cfg.n_samples, cfg.luq_seed
     A_h, W_h, G_h = inputs.layer_inputs(cfg)
+    if cfg.dtype == "bf16":
+        A_h, W_h, G_h = (t.view(np.int16) for t in (A_h, W_h, G_h))
     pin = lambda a: torch.from_numpy(a).pin_memory()  # noqa: E731
     A_p, W_p, G_p = pin(A_h), pin(W_h), pin(G_h)
     A, W, G = A_p.cuda(), W_p.cuda(), G_p.cuda()
+    if cfg.dtype == "bf16":
+        A, W, G = (t.view(torch.bfloat16) for t in (A, W, G))
+        A_p, W_p, G_p = (t.view(torch.bfloat16) for t in (A_p, W_p, G_p))
     ctx = binding.Context(local)
     dev = A.device
     f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)  # noqa: E731
@@ -270,31 +283,34 @@ def run_ours(args):
                 "peak_source": f"{peaks['source']}" + (" hbm copy" if d["bound"] == "hbm" else " bf16 sustained x2 (fp8)")}
 
     # ---- end to end: host buffers in, host buffers out, through the same calls
+    e2e = None
+    cpu_baseline = None
+
     def e2e_step():
         A.copy_(A_p, non_blocking=True); W.copy_(W_p, non_blocking=True); G.copy_(G_p, non_blocking=True)
         step()
         Z_p.copy_(Z, non_blocking=True); dA_p.copy_(dA, non_blocking=True); dW_p.copy_(dW, non_blocking=True)
-    e2e_steps = max(2, min(args.steps, 5))
-    e2e_step()
-    barrier()
-    t0.record()
-    for _ in range(e2e_steps):
+    if not args.kernel_only:
+        e2e_steps = max(2, min(args.steps, 5))
         e2e_step()
-    t1.record()
-    barrier()
-    e2e_ms = t0.elapsed_time(t1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    h2d = A_p.numel() * 4 + W_p.numel() * 4 + G_p.numel() * 4
-    d2h = Z_p.numel() * 4 + dA_p.numel() * 4 + dW_p.numel() * 4
-    e2e = {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        barrier()
+        t0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        t1.record()
+        barrier()
+        e2e_ms = t0.elapsed_time(t1) / e2e_steps
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        h2d = sum(t.numel() * t.element_size() for t in (A_p, W_p, G_p))
+        d2h = sum(t.numel() * t.element_size() for t in (Z_p, dA_p, dW_p))
+        e2e = {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
-    cpu_baseline = None
-    if rank == 0 and world == 1:
-        rows = 512
+    if rank == 0 and world == 1 and not args.kernel_only:
+        rows = min(2048, M)
         dt, fl, threads = oracle_sample(cfg, rows, ns)
         cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": f"first {rows} of {M} batch rows, all nine stages, {dt:.2f} s"}
@@ -304,10 +320,10 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "e4m3 operands, f32 accumulate", "data": "synthetic",
-            "config": {"workload": f"{WORKLOAD}: ResNet-50 3x3 conv as im2col GEMM, M={M} K={K} N={N}, fp32 inputs, "
+            "config": {"workload": f"{args.workload}: M={M} K={K} N={N}, {cfg.dtype} inputs, "
                                    f"LUQ seed {seed}, {ns} sample(s)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                       "l2": "inputs (462 MB activations) larger than the 126 MB L2; no explicit flush"},
+                       "l2": "inputs (%d MB of activations per step) against a 126 MB L2; no explicit flush" % (A.numel() * A.element_size() >> 20)},
             "luq_quantizer_gbs": kernels["quant_grad_G"]["gbs"],
             "amax_plus_luq_gbs": round((alg["amax_G"][0] + alg["quant_grad_G"][0]) /
                                        ((per_kernel_ms["amax_G"] + per_kernel_ms["quant_grad_G"]) * 1e-3) / 1e9, 1),
@@ -323,9 +339,13 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD, choices=["cfg1", "cfg2", "cfg3", "cfg5"],
+                    help="layer shape; the headline number is cfg2")
+    ap.add_argument("--rows", type=int, default=None, help="truncate the batch dimension M (small profiling runs)")
+    ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
