@@ -205,6 +205,8 @@ def run_ours(args):
         A, W, G = (t.view(torch.bfloat16) for t in (A, W, G))
         A_p, W_p, G_p = (t.view(torch.bfloat16) for t in (A_p, W_p, G_p))
     ctx = binding.Context(local)
+    if args.mma_kind is not None:
+        ctx.set_option(binding.OPT_MMA_KIND, args.mma_kind)
     dev = A.device
     f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)  # noqa: E731
     u8 = lambda *s: torch.empty(s, dtype=torch.uint8, device=dev)  # noqa: E731
@@ -346,6 +348,8 @@ def main():
                     help="layer shape; the headline number is cfg2")
     ap.add_argument("--rows", type=int, default=None, help="truncate the batch dimension M (small profiling runs)")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs")
+    ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1],
+                    help="tensor-core operand type: 0 e4m3 (kind::f8f6f4), 1 int8 (kind::i8); default: the library's")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

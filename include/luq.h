@@ -58,7 +58,7 @@ extern "C" {
 #define LUQ_STATUS_TIMEOUT 4   /* a bounded wait inside a kernel expired; outputs unspecified */
 
 /* options for luq_set_option */
-#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands (default); 1: kind::i8 on int8 operands */
+#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands; 1: kind::i8 on int8 operands */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
 
 #define LUQ_MAX_SAMPLES 8
@@ -66,7 +66,7 @@ extern "C" {
 typedef struct luq_ctx luq_ctx;
 
 /* Creates a context on `device`: a device status word and the split workspace
- * (16 MiB) used by GEMMs whose output has too few tiles to fill the GPU.
+ * (32 MiB) used by GEMMs whose output has too few tiles to fill the GPU.
  * Allocates device memory; call outside stream capture. */
 int luq_create(luq_ctx** out, int device);
 int luq_destroy(luq_ctx* ctx);
@@ -102,6 +102,13 @@ int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t
 int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
                    const float* d_amax, uint64_t seed, int n_samples,
                    uint8_t* d_codes, float* d_alpha, void* stream);
+
+/* Diagnostic for the division-free quotient inside luq_quant_grad (reading of
+ * Eq. StochasticPruning / Eq. unbiasedFpQ: the probabilities are functions of
+ * t = |x| / alpha): writes, for n fp32 elements, the value t the quantizer forms
+ * with alpha = *d_amax / 2^kmax, before its clamp to the top level.  It must
+ * equal the IEEE binary32 quotient wherever that quotient is a normal number. */
+int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream);
 
 /* Forward GEMM (Eq. Forward; scale factoring of Appendix A.1):
  *   Z[m,n] = (sa*sw) * sum_k qA[m,k] * qW[n,k]        fp32 accumulate, fp32 out.

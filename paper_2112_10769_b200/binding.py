@@ -21,7 +21,7 @@ OPT_MMA_KIND, OPT_SPLITS = 1, 2
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_quant_grad", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_status",
+           "luq_quant_grad", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_status",
            "luq_launch_count", "luq_strerror")
 
 _lib = None
@@ -48,6 +48,7 @@ def load() -> ctypes.CDLL:
         L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
         L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp]
         L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp]
+        L.luq_debug_quotient.argtypes = [vp, vp, sz, vp, vp, vp]
         L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_wgrad.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
@@ -132,6 +133,12 @@ class Context:
                                      seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
                                      _stream()), "luq_quant_grad")
         return codes, alpha
+
+    def debug_quotient(self, x: torch.Tensor, amax: torch.Tensor) -> torch.Tensor:
+        out = torch.empty_like(x, dtype=torch.float32)
+        _check(load().luq_debug_quotient(self.handle, x.data_ptr(), x.numel(), amax.data_ptr(), out.data_ptr(),
+                                         _stream()), "luq_debug_quotient")
+        return out
 
     def gemm_fwd(self, a_codes, sa, w_codes, sw, M: int, N: int, K: int, out: torch.Tensor | None = None):
         out = torch.empty((M, N), dtype=torch.float32, device=a_codes.device) if out is None else out

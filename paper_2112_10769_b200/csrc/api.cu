@@ -5,8 +5,7 @@
 
 namespace {
 
-constexpr size_t kWorkspaceBytes = 16u << 20;
-constexpr int kMaxTickets = 1024;
+constexpr size_t kWorkspaceBytes = 32u << 20;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
@@ -57,14 +56,10 @@ int luq_create(luq_ctx** out, int device) {
   c->forced_splits = 0;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;
-  c->max_tickets = kMaxTickets;
-  c->d_status = nullptr; c->d_workspace = nullptr; c->d_tickets = nullptr; c->encode_tiled = nullptr;
+  c->d_status = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
   bool ok = cudaMalloc(&c->d_status, sizeof(unsigned int)) == cudaSuccess &&
-            cudaMalloc(&c->d_workspace, kWorkspaceBytes) == cudaSuccess &&
-            cudaMalloc(&c->d_tickets, kMaxTickets * sizeof(unsigned int)) == cudaSuccess;
-  ok = ok && cudaMemset(c->d_status, 0, sizeof(unsigned int)) == cudaSuccess &&
-       cudaMemset(c->d_workspace, 0, kWorkspaceBytes) == cudaSuccess &&
-       cudaMemset(c->d_tickets, 0, kMaxTickets * sizeof(unsigned int)) == cudaSuccess;
+            cudaMalloc(&c->d_workspace, kWorkspaceBytes) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_status, 0, sizeof(unsigned int)) == cudaSuccess;
   if (ok) {
     cudaDriverEntryPointQueryResult q;
     ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) == cudaSuccess &&
@@ -80,7 +75,6 @@ int luq_destroy(luq_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->d_workspace) cudaFree(ctx->d_workspace);
-  if (ctx->d_tickets) cudaFree(ctx->d_tickets);
   delete ctx;
   return LUQ_OK;
 }
@@ -139,6 +133,13 @@ int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t
                                        as_stream(stream)));
 }
 
+int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream) {
+  if (!ctx || !d_amax || (n && (!d_x || !d_t))) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_debug_quotient(ctx, d_x, n, d_amax, d_t, as_stream(stream)));
+}
+
 static int gemm_common(luq_ctx* ctx, const uint8_t* x, const float* sx, const uint8_t* y, const float* sy,
                        float* out, int64_t M, int64_t N, int64_t K, int n_samples) {
   if (!ctx || !sx || !sy) return LUQ_ERR_ARG;
@@ -161,7 +162,7 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, cons
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 0;
   a.d_scale_a = d_sa; a.d_scale_b = d_sw; a.d_out = d_z; a.Mo = M; a.No = N; a.Kc = K;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
-  a.d_tickets = ctx->d_tickets; a.max_tickets = ctx->max_tickets; a.allow_split = 1;
+  a.allow_split = 1;
   return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
 }
 
@@ -178,7 +179,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 1;                            // W[N x K]: rows are the contraction
   a.d_scale_a = d_alpha; a.d_scale_b = d_sw; a.d_out = d_da; a.Mo = M; a.No = K; a.Kc = N;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
-  a.d_tickets = ctx->d_tickets; a.max_tickets = ctx->max_tickets; a.allow_split = 1;
+  a.allow_split = 1;
   return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
 }
 
@@ -195,7 +196,7 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
   a.b_codes = d_a_codes; a.b_kind = 0; a.b_mn = 1;                            // A[M x K]: rows are the contraction
   a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.Mo = N; a.No = K; a.Kc = M;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
-  a.d_tickets = ctx->d_tickets; a.max_tickets = ctx->max_tickets; a.allow_split = 1;
+  a.allow_split = 1;
   return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
 }
 
@@ -209,10 +210,6 @@ int luq_status(luq_ctx* ctx, void* stream, int* host_flags) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return LUQ_ERR_CUDA;
   if (flags) {
     if (cudaMemsetAsync(ctx->d_status, 0, sizeof(unsigned int), st) != cudaSuccess) return LUQ_ERR_CUDA;
-    if (flags & LUQ_STATUS_TIMEOUT) {  // an aborted split GEMM may have left partial sums behind
-      cudaMemsetAsync(ctx->d_workspace, 0, ctx->workspace_bytes, st);
-      cudaMemsetAsync(ctx->d_tickets, 0, ctx->max_tickets * sizeof(unsigned int), st);
-    }
     if (cudaStreamSynchronize(st) != cudaSuccess) return LUQ_ERR_CUDA;
   }
   *host_flags = static_cast<int>(flags);

@@ -12,10 +12,8 @@ struct luq_ctx {
   int device;
   int sm_count;
   unsigned int* d_status;   // device status word (LUQ_STATUS_* bits)
-  float* d_workspace;       // split-contraction partial sums
+  float* d_workspace;       // split-contraction partial tiles
   size_t workspace_bytes;
-  unsigned int* d_tickets;  // one arrival counter per output tile
-  int max_tickets;
   int mma_kind;             // 0 f8f6f4/e4m3, 1 i8
   int forced_splits;        // 0 = automatic
   int64_t launches;
@@ -29,6 +27,9 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
 int luq_launch_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
                           uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, cudaStream_t st);
 
+int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,
+                              cudaStream_t st);
+
 // One GEMM  D[Mo x No] = scale * sum_s sum_k opA_s[mo,k] * opB[no,k].
 //   a_mn / b_mn: operand is stored contraction-major (rows = k) instead of
 //   k-contiguous (rows = mo / no).  a_kind / b_kind: 0 INT4 codes, 1 LUQ codes.
@@ -37,8 +38,7 @@ struct luq_gemm_args {
   const uint8_t* b_codes; int b_kind; int b_mn;
   const float* d_scale_a; const float* d_scale_b;
   float* d_out; int64_t Mo, No, Kc;
-  float* d_workspace; size_t workspace_bytes;   // split partial sums (caller-chosen memory)
-  unsigned int* d_tickets; int max_tickets;
+  float* d_workspace; size_t workspace_bytes;   // split partial tiles (caller-chosen memory)
   int allow_split;
 };
 int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st);
@@ -116,6 +116,21 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
+}
+
+// store of a shared-memory box to global memory through a tensor map (clipped at the tensor's edges)
+__device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until at most N of this thread's bulk groups still read their shared-memory source
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N> __device__ __forceinline__ void bulk_wait() {
+  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 
 // ---- tcgen05 / tensor memory ---------------------------------------------------

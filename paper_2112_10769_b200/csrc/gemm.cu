@@ -7,14 +7,23 @@
 // ("K-major": rows are mo / no) or contraction-major ("MN-major": rows are k).
 //
 // One persistent CTA per SM, warp-specialised:
-//   warp 0      TMA producer: packed 128-row x 64-byte slabs -> shared memory ring
-//   warps 6-13  converters: nibble -> 8-bit operand (16-entry byte table through
-//               PRMT), written in the 128-byte-swizzled layout the tensor core reads
-//   warp 1      one thread issues tcgen05.mma (128 x 256 x 32 per instruction),
-//               accumulators live in tensor memory, two buffers of 256 columns
-//   warps 2-5   epilogue: tcgen05.ld -> scale -> global store (or split reduction)
+//   warp 0       TMA producer: packed 128-row x 64-byte slabs -> shared memory ring
+//   warps 6-21   converters: nibble -> 8-bit operand, written in the 128-byte
+//                swizzled layout the tensor core reads
+//   warp 1       one thread issues tcgen05.mma (128 x 256 x 32 per instruction),
+//                accumulators live in tensor memory, two buffers of 256 columns
+//   warps 2-5    epilogue: tcgen05.ld -> scale -> swizzled staging -> TMA store
 // Every slab, in either orientation, is 128 rows x 64 packed bytes and expands to
 // 128 rows x 128 bytes; only the matrix descriptor differs between orientations.
+//
+// Operand bytes.  kind::f8f6f4: e4m3 through a 16-entry byte table (PRMT).
+// kind::i8: LUQ levels +-2^(c-1) through the table; INT4 integers without a
+// table - the two's-complement nibble moved to the high half of a byte is the
+// int8 value 16*q, and the epilogue divides by 16 per INT4 operand (exact).
+//
+// Few output tiles (the update GEMM): the contraction is split over CTAs, each
+// stores its partial tile to a workspace and a second kernel adds them in a fixed
+// order (deterministic; no atomics).
 // All waits are bounded; on expiry the CTA flags LUQ_STATUS_TIMEOUT, drains its
 // copies, frees its tensor memory and returns.
 #include <cuda.h>
@@ -36,32 +45,34 @@ constexpr int kPackedStage = kSlabs * kPackedSlab;
 constexpr int kExpandedStage = kSlabs * kExpandedSlab;
 constexpr int kPackedStages = 4;
 constexpr int kExpandedStages = 2;
-constexpr int kConvWarps = 8;
+constexpr int kConvWarps = 16;
+constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kFirstEpiWarp = 2;
 constexpr int kFirstConvWarp = 6;
 constexpr int kThreads = 32 * (kFirstConvWarp + kConvWarps);
 constexpr int kTmemCols = 2 * BN;
 constexpr int kTileFloats = BM * BN;
+constexpr int kStageBox = 32 * 32 * 4;           // one 32 x 32 fp32 store box
+
+static_assert(kSlabs * 512 % kConvThreads == 0, "converter tasks must divide evenly");
 
 struct SmemLayout {
   static constexpr int expanded = 0;
   static constexpr int packed = expanded + kExpandedStages * kExpandedStage;
-  static constexpr int barriers = packed + kPackedStages * kPackedStage;
+  static constexpr int staging = packed + kPackedStages * kPackedStage;  // 4 warps x 2 boxes
+  static constexpr int barriers = staging + 4 * 2 * kStageBox;
   // barrier order: pk_full[PS] pk_empty[PS] ex_full[ES] ex_empty[ES] acc_full[2] acc_empty[2]
   static constexpr int num_barriers = 2 * kPackedStages + 2 * kExpandedStages + 4;
   static constexpr int tmem_slot = barriers + 8 * num_barriers;
   static constexpr int abort_flag = tmem_slot + 4;
-  static constexpr int last_flag = abort_flag + 4;
-  static constexpr int total = last_flag + 4;
+  static constexpr int total = abort_flag + 4;
 };
 constexpr int kSmemBytes = SmemLayout::total + 1024;  // slack to align the base to 1024 bytes
+static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
 struct GemmParams {
   const float* scale_a;
   const float* scale_b;
-  float* out;
-  float* workspace;
-  unsigned int* tickets;
   unsigned int* status;
   long long Mo, No, Kc;
   int n_samples;
@@ -69,12 +80,12 @@ struct GemmParams {
   int num_kb;          // contraction blocks per sample plane
   int splits;          // contraction splits per tile
   int iters_per_split;
-  float inv_samples;
+  float post_scale;    // 1/n_samples times the power of two that undoes the int8 operand scaling
   uint4 lut_a, lut_b;  // nibble -> operand byte
 };
 
-// eight nibbles of `w` -> eight operand bytes
-__device__ __forceinline__ void expand8(uint32_t w, const uint4& lut, uint32_t& lo, uint32_t& hi) {
+// eight nibbles of `w` -> eight operand bytes through a 16-entry table
+__device__ __forceinline__ void expand8_lut(uint32_t w, const uint4& lut, uint32_t& lo, uint32_t& hi) {
   const uint32_t sel0 = w & 0x7777u;
   const uint32_t sel1 = (w >> 16) & 0x7777u;
   const uint32_t pick0 = 0x3210u | ((w >> 1) & 0x4444u);
@@ -82,11 +93,25 @@ __device__ __forceinline__ void expand8(uint32_t w, const uint4& lut, uint32_t& 
   lo = __byte_perm(__byte_perm(lut.x, lut.y, sel0), __byte_perm(lut.z, lut.w, sel0), pick0);
   hi = __byte_perm(__byte_perm(lut.x, lut.y, sel1), __byte_perm(lut.z, lut.w, sel1), pick1);
 }
+// eight two's-complement nibbles -> eight int8 values 16*q.  PERMUTED keeps the
+// even elements in `lo` and the odd ones in `hi` (a fixed permutation of the
+// contraction index, legal when both operands of the product apply it).
+template <bool PERMUTED>
+__device__ __forceinline__ void expand8_int4_x16(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  const uint32_t even = (w << 4) & 0xF0F0F0F0u;
+  const uint32_t odd = w & 0xF0F0F0F0u;
+  if constexpr (PERMUTED) { lo = even; hi = odd; }
+  else { lo = __byte_perm(even, odd, 0x5140); hi = __byte_perm(even, odd, 0x7362); }
+}
 
-template <int KIND, bool A_MN, bool B_MN>
+// KIND 0 f8f6f4 / 1 i8; A_MN, B_MN operand orientation; A_LUQ: A holds LUQ codes (B is always INT4)
+template <int KIND, bool A_MN, bool B_MN, bool A_LUQ>
 __global__ void __launch_bounds__(kThreads, 1)
 luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                const GemmParams p) {
+                const __grid_constant__ CUtensorMap tm_out, const GemmParams p) {
+  // with int8 operands and both INT4 operands k-contiguous the expansion may permute k
+  constexpr bool kPermuteK = KIND == 1 && !A_MN && !B_MN && !A_LUQ;
+
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -101,7 +126,6 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kPackedStages + 2 * kExpandedStages + 2 + b); };
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + SmemLayout::tmem_slot);
   volatile uint32_t* const abort_flag = reinterpret_cast<volatile uint32_t*>(gen + SmemLayout::abort_flag);
-  volatile uint32_t* const last_flag = reinterpret_cast<volatile uint32_t*>(gen + SmemLayout::last_flag);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -111,11 +135,10 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     for (int s = 0; s < kExpandedStages; ++s) { mbar_init(ex_full(s), kConvWarps); mbar_init(ex_empty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     *abort_flag = 0;
-    *last_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
-  if (warp == 0 && lane == 0) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_b); }
+  if (warp == 0 && lane == 0) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_b); tma_prefetch_desc(&tm_out); }
   if (warp == 1) {  // this warp owns the tensor-memory allocation
     tmem_alloc(base + SmemLayout::tmem_slot, kTmemCols);
     tmem_relinquish();
@@ -210,85 +233,63 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   } else if (warp < kFirstConvWarp) {
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;  // tensor-memory lanes this warp may read
-    const int row_in_tile = quarter * 32 + lane;
-    const float scale = (__ldg(p.scale_a) * __ldg(p.scale_b)) * p.inv_samples;
-    uint32_t tile_it = 0;
+    const float scale = p.splits == 1 ? (__ldg(p.scale_a) * __ldg(p.scale_b)) * p.post_scale : 1.0f;
+    const uint32_t stage0 = base + SmemLayout::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
+    uint8_t* const stage0_gen = gen + SmemLayout::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
+    const int sw = lane & 7;
+    uint32_t tile_it = 0, box_it = 0;
     bool ok = true;
     for (int u = blockIdx.x; ok && u < units; u += gridDim.x, ++tile_it) {
       int tile, it_begin, it_end;
       unit_range(u, tile, it_begin, it_end);
-      const long long m0 = static_cast<long long>(tile % p.tiles_m) * BM;
-      const long long n0 = static_cast<long long>(tile / p.tiles_m) * BN;
+      // a split stores its whole partial tile at row u*128 of the workspace
+      const long long row0 = (p.splits == 1 ? static_cast<long long>(tile % p.tiles_m) * BM
+                                            : static_cast<long long>(u) * BM) + quarter * 32;
+      const long long col_base = p.splits == 1 ? static_cast<long long>(tile / p.tiles_m) * BN : 0;
+      const long long row_limit = p.splits == 1 ? p.Mo : static_cast<long long>(units) * BM;
+      const long long col_limit = p.splits == 1 ? p.No : BN;
       const uint32_t buf = tile_it & 1u;
-      const long long row = m0 + row_in_tile;
-      float* const ws_row = p.workspace + static_cast<size_t>(tile) * kTileFloats + row_in_tile * BN;
-      // a warp whose wait expired still takes part in the block barriers below
-      const bool have = mbar_wait(acc_full(buf), (tile_it >> 1) & 1u, abort_flag);
-      if (have) {
-        tc_fence_after();
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+      if (!mbar_wait(acc_full(buf), (tile_it >> 1) & 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld_32x32(taddr + c * 32, r);
-          tmem_ld_wait();
-          float v[32];
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + c * 32, r);
+        tmem_ld_wait();
+        const long long col0 = col_base + c * 32;
+        if (row0 < row_limit && col0 < col_limit) {   // warp-uniform
+          const uint32_t b = box_it & 1u;
+          ++box_it;
+          if (lane == 0) bulk_wait_read<1>();          // the store that last read this box is done
+          __syncwarp();
+          uint8_t* const rowp = stage0_gen + b * kStageBox + lane * 128;
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            v[j] = KIND == 0 ? __uint_as_float(r[j]) : static_cast<float>(static_cast<int>(r[j]));
-          const long long col = n0 + c * 32;
-          if (p.splits == 1) {
-            if (row < p.Mo && col < p.No) {
-              float4* dst = reinterpret_cast<float4*>(p.out + row * p.No + col);
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                dst[j] = make_float4(v[4 * j] * scale, v[4 * j + 1] * scale, v[4 * j + 2] * scale, v[4 * j + 3] * scale);
+          for (int j = 0; j < 8; ++j) {
+            float4 v;
+            if constexpr (KIND == 0) {
+              v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                              __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+            } else {
+              v = make_float4(static_cast<float>(static_cast<int>(r[4 * j])), static_cast<float>(static_cast<int>(r[4 * j + 1])),
+                              static_cast<float>(static_cast<int>(r[4 * j + 2])), static_cast<float>(static_cast<int>(r[4 * j + 3])));
             }
-          } else {
-            // partial sums are integers below 2^24: float atomics add them exactly in any order
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              if (v[4 * j] != 0.0f || v[4 * j + 1] != 0.0f || v[4 * j + 2] != 0.0f || v[4 * j + 3] != 0.0f)
-                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(ws_row + c * 32 + 4 * j),
-                             "f"(v[4 * j]), "f"(v[4 * j + 1]), "f"(v[4 * j + 2]), "f"(v[4 * j + 3]) : "memory");
-            }
+            v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
+            *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tm_out, stage0 + b * kStageBox, static_cast<int>(col0), static_cast<int>(row0));
+            bulk_commit();
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty(buf));
       }
-
-      if (p.splits > 1) {
-        // the last CTA to finish a tile scales the sums and writes the result
-        __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (warp == kFirstEpiWarp && lane == 0) {
-          const unsigned int prev = atomicAdd(p.tickets + tile, 1u);
-          *last_flag = (prev == static_cast<unsigned int>(p.splits - 1)) ? 1u : 0u;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        const bool last = *last_flag != 0;
-        const bool aborted = *abort_flag != 0;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (last) {
-          __threadfence();
-          for (int c = 0; c < BN / 4; ++c) {
-            float4 v = __ldcg(reinterpret_cast<const float4*>(ws_row) + c);
-            __stcg(reinterpret_cast<float4*>(ws_row) + c, make_float4(0.f, 0.f, 0.f, 0.f));
-            const long long col = n0 + c * 4;
-            if (row < p.Mo && col < p.No) {
-              v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
-              *reinterpret_cast<float4*>(p.out + row * p.No + col) = v;
-            }
-          }
-          if (warp == kFirstEpiWarp && lane == 0) p.tickets[tile] = 0u;
-        }
-        if (aborted) ok = false;
-      } else if (!have) {
-        ok = false;
-      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(buf));
     }
+    if (lane == 0) bulk_wait<0>();   // all stores of this warp are complete before the CTA exits
   } else {
     // -------------------------------------------------------------- converters
     const int ctid = threadIdx.x - kFirstConvWarp * 32;
@@ -304,24 +305,35 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (!mbar_wait(ex_empty(es), ((it / kExpandedStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         const uint8_t* src = gen + SmemLayout::packed + ps * kPackedStage;
         uint8_t* dst = gen + SmemLayout::expanded + es * kExpandedStage;
+        uint4 w[kSlabs * 512 / kConvThreads];
 #pragma unroll
-        for (int j = 0; j < kSlabs * 512 / (kConvWarps * 32); ++j) {
-          const int id = ctid + j * (kConvWarps * 32);
-          const int slab = id >> 9;
+        for (int j = 0; j < kSlabs * 512 / kConvThreads; ++j)
+          w[j] = *reinterpret_cast<const uint4*>(src + (ctid + j * kConvThreads) * 16);
+#pragma unroll
+        for (int j = 0; j < kSlabs * 512 / kConvThreads; ++j) {
+          const int id = ctid + j * kConvThreads;
+          const int slab = id >> 9;           // compile-time per j
           const int idx = id & 511;
           const int row = idx >> 2;
           const int q = idx & 3;
-          const uint4 w = *reinterpret_cast<const uint4*>(src + slab * kPackedSlab + idx * 16);
-          const uint4 lut = slab == 0 ? p.lut_a : p.lut_b;
           uint4 o0, o1;
-          expand8(w.x, lut, o0.x, o0.y);
-          expand8(w.y, lut, o0.z, o0.w);
-          expand8(w.z, lut, o1.x, o1.y);
-          expand8(w.w, lut, o1.z, o1.w);
+          const bool is_a = slab == 0;
+          if (KIND == 1 && !(is_a && A_LUQ)) {
+            expand8_int4_x16<kPermuteK>(w[j].x, o0.x, o0.y);
+            expand8_int4_x16<kPermuteK>(w[j].y, o0.z, o0.w);
+            expand8_int4_x16<kPermuteK>(w[j].z, o1.x, o1.y);
+            expand8_int4_x16<kPermuteK>(w[j].w, o1.z, o1.w);
+          } else {
+            const uint4 lut = is_a ? p.lut_a : p.lut_b;
+            expand8_lut(w[j].x, lut, o0.x, o0.y);
+            expand8_lut(w[j].y, lut, o0.z, o0.w);
+            expand8_lut(w[j].z, lut, o1.x, o1.y);
+            expand8_lut(w[j].w, lut, o1.z, o1.w);
+          }
           uint8_t* drow = dst + slab * kExpandedSlab + row * 128;
-          const int sw = row & 7;
-          *reinterpret_cast<uint4*>(drow + (((2 * q) ^ sw) << 4)) = o0;
-          *reinterpret_cast<uint4*>(drow + (((2 * q + 1) ^ sw) << 4)) = o1;
+          const int swz = row & 7;
+          *reinterpret_cast<uint4*>(drow + (((2 * q) ^ swz) << 4)) = o0;
+          *reinterpret_cast<uint4*>(drow + (((2 * q + 1) ^ swz) << 4)) = o1;
         }
         fence_proxy_async();   // make the generic-proxy writes visible to the tensor core
         __syncwarp();
@@ -337,6 +349,33 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Sums the partial tiles of a split contraction in a fixed order, applies the
+// scales and writes the output.  One thread per float4 of a tile.
+__global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restrict__ ws, float* __restrict__ out,
+                                                           const float* __restrict__ scale_a,
+                                                           const float* __restrict__ scale_b, float post_scale,
+                                                           int tiles, int tiles_m, int splits, long long Mo,
+                                                           long long No) {
+  const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<long long>(tiles) * (kTileFloats / 4)) return;
+  const int tile = static_cast<int>(idx / (kTileFloats / 4));
+  const int rem = static_cast<int>(idx % (kTileFloats / 4));
+  const int r = rem / (BN / 4), c4 = rem % (BN / 4);
+  const float4* src = reinterpret_cast<const float4*>(ws) + (static_cast<size_t>(tile) * splits) * (kTileFloats / 4) + rem;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < splits; ++s) {
+    const float4 v = __ldcg(src + static_cast<size_t>(s) * (kTileFloats / 4));
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
+  const long long row = static_cast<long long>(tile % tiles_m) * BM + r;
+  const long long col = static_cast<long long>(tile / tiles_m) * BN + c4 * 4;
+  if (row < Mo && col < No) {
+    const float scale = (__ldg(scale_a) * __ldg(scale_b)) * post_scale;
+    acc.x *= scale; acc.y *= scale; acc.z *= scale; acc.w *= scale;
+    *reinterpret_cast<float4*>(out + row * No + col) = acc;
   }
 }
 
@@ -373,8 +412,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 // packed-code tensor: `planes` x `rows` x `pitch` bytes, box = 1 x 128 rows x 64 bytes
-int encode_map(void* fn, CUtensorMap* map, const uint8_t* ptr, uint64_t pitch, uint64_t rows, uint64_t planes,
-               bool three_d) {
+int encode_codes_map(void* fn, CUtensorMap* map, const uint8_t* ptr, uint64_t pitch, uint64_t rows, uint64_t planes,
+                     bool three_d) {
   const cuuint64_t dims[3] = {pitch, rows, planes};
   const cuuint64_t strides[2] = {pitch, pitch * rows};
   const cuuint32_t box[3] = {64, 128, 1};
@@ -385,13 +424,25 @@ int encode_map(void* fn, CUtensorMap* map, const uint8_t* ptr, uint64_t pitch, u
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : 1;
 }
+// fp32 output (or workspace) tensor rows x cols, box = 32 rows x 32 columns, 128-byte swizzle in shared memory
+int encode_out_map(void* fn, CUtensorMap* map, float* ptr, uint64_t rows, uint64_t cols) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * sizeof(float)};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+      map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : 1;
+}
 
-template <int KIND, bool A_MN, bool B_MN>
-int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int grid, cudaStream_t st) {
-  auto kernel = luq_gemm_kernel<KIND, A_MN, B_MN>;
+template <int KIND, bool A_MN, bool B_MN, bool A_LUQ>
+int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmParams& p, int grid,
+           cudaStream_t st) {
+  auto kernel = luq_gemm_kernel<KIND, A_MN, B_MN, A_LUQ>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return static_cast<int>(e);
-  kernel<<<grid, kThreads, kSmemBytes, st>>>(ta, tb, p);
+  kernel<<<grid, kThreads, kSmemBytes, st>>>(ta, tb, to, p);
   return static_cast<int>(cudaGetLastError());
 }
 
@@ -400,16 +451,25 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, in
 int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
   if (a.Mo <= 0 || a.No <= 0 || a.Kc <= 0) return 0;
   GemmParams p{};
-  p.scale_a = a.d_scale_a; p.scale_b = a.d_scale_b; p.out = a.d_out;
-  p.workspace = a.d_workspace; p.tickets = a.d_tickets; p.status = ctx->d_status;
+  p.scale_a = a.d_scale_a; p.scale_b = a.d_scale_b; p.status = ctx->d_status;
   p.Mo = a.Mo; p.No = a.No; p.Kc = a.Kc;
   p.n_samples = a.n_samples;
   p.tiles_m = static_cast<int>((a.Mo + BM - 1) / BM);
   p.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
   p.num_kb = static_cast<int>((a.Kc + BK - 1) / BK);
-  p.inv_samples = 1.0f / static_cast<float>(a.n_samples);
   p.lut_a = make_lut(ctx->mma_kind, a.a_kind);
   p.lut_b = make_lut(ctx->mma_kind, a.b_kind);
+  // int8 operands carry INT4 integers as 16*q: undo with an exact power of two
+  float pow2 = 1.0f;
+  long long worst = 1;   // largest |operand product| as fed to the tensor core
+  if (ctx->mma_kind == 1) {
+    const int a_mag = a.a_kind == 0 ? 7 * 16 : 64, b_mag = a.b_kind == 0 ? 7 * 16 : 64;
+    if (a.a_kind == 0) pow2 *= 1.0f / 16.0f;
+    if (a.b_kind == 0) pow2 *= 1.0f / 16.0f;
+    worst = static_cast<long long>(a_mag) * b_mag;
+    if (worst * a.Kc * a.n_samples >= (1ll << 31)) return LUQ_ERR_ARG;  // the int32 accumulator could wrap
+  }
+  p.post_scale = (1.0f / static_cast<float>(a.n_samples)) * pow2;
 
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const int total_iters = p.n_samples * p.num_kb;
@@ -421,37 +481,51 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
     if (splits > total_iters) splits = total_iters;
     if (splits < 1) splits = 1;
   }
-  if (splits > 1) {
-    const size_t need = static_cast<size_t>(tiles) * kTileFloats * sizeof(float);
-    if (a.d_workspace == nullptr || need > a.workspace_bytes || tiles > a.max_tickets) {
-      if (ctx->forced_splits > 0) return LUQ_ERR_WORKSPACE;
-      splits = 1;
-    }
-  }
   p.iters_per_split = (total_iters + splits - 1) / splits;
   p.splits = (total_iters + p.iters_per_split - 1) / p.iters_per_split;  // no empty split
+  const long long units = tiles * p.splits;
+  if (p.splits > 1) {
+    const size_t need = static_cast<size_t>(units) * kTileFloats * sizeof(float);
+    if (a.d_workspace == nullptr || need > a.workspace_bytes) {
+      if (ctx->forced_splits > 0) return LUQ_ERR_WORKSPACE;
+      p.splits = 1;
+      p.iters_per_split = total_iters;
+    }
+  }
+  const long long units_final = tiles * p.splits;
 
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, to;
   int bad = 0;
-  if (a.a_mn) bad |= encode_map(ctx->encode_tiled, &ta, a.a_codes, a.Mo / 2, a.Kc, a.n_samples, true);
-  else bad |= encode_map(ctx->encode_tiled, &ta, a.a_codes, a.Kc / 2, a.Mo, a.n_samples, true);
-  if (a.b_mn) bad |= encode_map(ctx->encode_tiled, &tb, a.b_codes, a.No / 2, a.Kc, 1, false);
-  else bad |= encode_map(ctx->encode_tiled, &tb, a.b_codes, a.Kc / 2, a.No, 1, false);
+  if (a.a_mn) bad |= encode_codes_map(ctx->encode_tiled, &ta, a.a_codes, a.Mo / 2, a.Kc, a.n_samples, true);
+  else bad |= encode_codes_map(ctx->encode_tiled, &ta, a.a_codes, a.Kc / 2, a.Mo, a.n_samples, true);
+  if (a.b_mn) bad |= encode_codes_map(ctx->encode_tiled, &tb, a.b_codes, a.No / 2, a.Kc, 1, false);
+  else bad |= encode_codes_map(ctx->encode_tiled, &tb, a.b_codes, a.Kc / 2, a.No, 1, false);
+  if (p.splits > 1) bad |= encode_out_map(ctx->encode_tiled, &to, a.d_workspace, units_final * BM, BN);
+  else bad |= encode_out_map(ctx->encode_tiled, &to, a.d_out, a.Mo, a.No);
   if (bad) return LUQ_ERR_CUDA;
 
-  const long long units = tiles * p.splits;
-  const int grid = static_cast<int>(units < ctx->sm_count ? units : ctx->sm_count);
+  const int grid = static_cast<int>(units_final < ctx->sm_count ? units_final : ctx->sm_count);
   int rc;
   const int sel = (ctx->mma_kind ? 4 : 0) | (a.a_mn ? 2 : 0) | (a.b_mn ? 1 : 0);
+  if (a.b_kind != 0 || (a.a_kind == 1) != (sel & 3 ? true : false)) return LUQ_ERR_UNSUPPORTED;
   switch (sel) {
-    case 0: rc = launch<0, false, false>(ta, tb, p, grid, st); break;
-    case 1: rc = launch<0, false, true>(ta, tb, p, grid, st); break;
-    case 3: rc = launch<0, true, true>(ta, tb, p, grid, st); break;
-    case 4: rc = launch<1, false, false>(ta, tb, p, grid, st); break;
-    case 5: rc = launch<1, false, true>(ta, tb, p, grid, st); break;
-    case 7: rc = launch<1, true, true>(ta, tb, p, grid, st); break;
+    case 0: rc = launch<0, false, false, false>(ta, tb, to, p, grid, st); break;
+    case 1: rc = launch<0, false, true, true>(ta, tb, to, p, grid, st); break;
+    case 3: rc = launch<0, true, true, true>(ta, tb, to, p, grid, st); break;
+    case 4: rc = launch<1, false, false, false>(ta, tb, to, p, grid, st); break;
+    case 5: rc = launch<1, false, true, true>(ta, tb, to, p, grid, st); break;
+    case 7: rc = launch<1, true, true, true>(ta, tb, to, p, grid, st); break;
     default: return LUQ_ERR_UNSUPPORTED;
   }
-  if (rc == 0) ctx->launches += 1;
+  if (rc != 0) return rc;
+  ctx->launches += 1;
+  if (p.splits > 1) {
+    const long long work = tiles * (kTileFloats / 4);
+    split_reduce_kernel<<<static_cast<int>((work + 255) / 256), 256, 0, st>>>(
+        a.d_workspace, a.d_out, a.d_scale_a, a.d_scale_b, p.post_scale, static_cast<int>(tiles), p.tiles_m, p.splits,
+        a.Mo, a.No);
+    rc = static_cast<int>(cudaGetLastError());
+    if (rc == 0) ctx->launches += 1;
+  }
   return rc;
 }

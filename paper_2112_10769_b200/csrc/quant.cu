@@ -6,7 +6,7 @@
 // pieces, so every load instruction of a warp covers 512 contiguous bytes and
 // the packed codes leave as contiguous 64- or 128-byte warp stores.  Grids are
 // sized to the number of CTAs the GPU holds at once (SM count x occupancy) and
-// walk the tensor with a grid-stride loop, several loads in flight per thread.
+// walk the tensor in contiguous 16 KB tiles, several loads in flight per thread.
 //
 // Compile this file without FMA contraction and with IEEE division: code
 // decisions must be bit-identical to a scalar IEEE implementation.
@@ -16,6 +16,9 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kUnroll = 4;  // independent 16-byte loads in flight per thread
+// A block walks the tensor in contiguous tiles of kThreads * kUnroll pieces (16 KB):
+// the loads a thread has in flight are 4 KB apart, inside one DRAM page neighbourhood.
+constexpr int kTileItems = kThreads * kUnroll;
 
 // zero, non-finite or far-out-of-range max: every code is zero, the scale is zero
 __device__ __forceinline__ bool scale_usable(float c, unsigned int* status) {
@@ -71,11 +74,15 @@ template <bool BF16> struct Item {
 // Inf/NaN pattern is larger than every finite one: one unsigned max does both
 // the reduction and the non-finite detection.  Warp shuffle reduction (redux),
 // then one shared-memory step per block, then one atomicMax per block.
+constexpr int kAmaxUnroll = 4;
+constexpr int kAmaxCtasPerSm = 8;
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__ x, size_t n,
                                                         unsigned int* __restrict__ out_bits,
                                                         unsigned int* __restrict__ status) {
   constexpr int kElems = Item<BF16>::kElems;
+  constexpr int kUnroll = kAmaxUnroll;
+  constexpr int kTileItems = kThreads * kUnroll;
   const size_t items = n / kElems;
   const uint4* p = reinterpret_cast<const uint4*>(x);
   uint32_t m = 0;
@@ -92,16 +99,17 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
       m = max(m, u.z & 0x7FFFFFFFu); m = max(m, u.w & 0x7FFFFFFFu);
     }
   };
-  const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
-  size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x;
-  for (; i + (kUnroll - 1) * stride < items; i += kUnroll * stride) {
+  const size_t full_tiles = items / kTileItems;
+  for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {
+    const uint4* q = p + t * kTileItems + threadIdx.x;
     uint4 u[kUnroll];
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i + j * stride);
+    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(q + j * kThreads);
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) fold(u[j]);
   }
-  for (; i < items; i += stride) fold(__ldg(p + i));
+  if (blockIdx.x == gridDim.x - 1)   // pieces after the last full tile
+    for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) fold(__ldg(p + i));
   // ragged tail: fewer elements than one piece
   if (blockIdx.x == 0 && threadIdx.x < n - items * kElems)
     m = max(m, __float_as_uint(Item<BF16>::load1(x, items * kElems + threadIdx.x)) & 0x7FFFFFFFu);
@@ -121,12 +129,14 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
 }
 
 // ------------------------------------------------------------------ INT4 ----
+// clamp, then add 1.5 * 2^23: the sum's low mantissa bits hold the integer rounded to
+// nearest-even, already in two's complement (clamping before rounding equals clamping
+// after it: the bounds are integers and rounding is monotone)
 __device__ __forceinline__ uint32_t int4_code(float x, float inv) {
   const float y = x * inv;
-  float r = rintf(y);                 // nearest, ties to even
-  r = fminf(fmaxf(r, -7.0f), 7.0f);
-  if (y != y) r = 0.0f;               // NaN element -> 0
-  return static_cast<uint32_t>(static_cast<int>(r)) & 0xFu;
+  const float c = fminf(fmaxf(y, -7.0f), 7.0f);
+  const uint32_t code = __float_as_uint(c + 12582912.0f) & 0xFu;
+  return (y == y) ? code : 0u;        // NaN element -> 0
 }
 
 template <bool BF16>
@@ -153,16 +163,20 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
     for (int j = 0; j < kElems; ++j) word |= int4_code(v[j], inv) << (4 * j);
     return word;
   };
-  const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
-  size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x;
-  for (; i + (kUnroll - 1) * stride < items; i += kUnroll * stride) {
+  // The tensor was just read front to back by the max reduction; its tail is what the
+  // L2 still holds, so this pass walks the tiles from the back.
+  const size_t full_tiles = items / kTileItems;
+  for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {
+    const size_t i0 = (full_tiles - 1 - t) * kTileItems + threadIdx.x;
     uint4 u[kUnroll];
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i + j * stride);
+    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i0 + j * kThreads);
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) Item<BF16>::store(codes, i + j * stride, encode(u[j]), true);
+    for (int j = 0; j < kUnroll; ++j) Item<BF16>::store(codes, i0 + j * kThreads, encode(u[j]), true);
   }
-  for (; i < items; i += stride) Item<BF16>::store(codes, i, encode(__ldg(p + i)), true);
+  if (blockIdx.x == gridDim.x - 1)
+    for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads)
+      Item<BF16>::store(codes, i, encode(__ldg(p + i)), true);
   if (first) {  // tail: fewer elements than one piece, two per byte
     for (size_t e = items * kElems; e < n; e += 2) {
       const uint32_t lo = ok ? int4_code(Item<BF16>::load1(x, e), inv) : 0u;
@@ -174,24 +188,23 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
 
 // ------------------------------------------------------------------- LUQ ----
 // Philox4x32-10: counter-based generator, ten rounds of two 32x32->64 multiplies
-// with a Weyl key schedule.  The key is the same for the whole tensor, so the
-// round keys are loop-invariant.
+// with a Weyl key schedule.  The key is the same for the whole tensor: the host
+// expands it into the ten round keys of every sample and passes them as kernel
+// parameters, so a round is two wide multiplies and two three-input XORs.
 struct PhiloxKeys { uint32_t k0[10]; uint32_t k1[10]; };
+struct PhiloxKeySet { PhiloxKeys s[LUQ_MAX_SAMPLES]; };
 
-__device__ __forceinline__ PhiloxKeys philox_keys(uint64_t key) {
-  PhiloxKeys ks;
-  uint32_t a = static_cast<uint32_t>(key), b = static_cast<uint32_t>(key >> 32);
-#pragma unroll
-  for (int r = 0; r < 10; ++r) { ks.k0[r] = a; ks.k1[r] = b; a += 0x9E3779B9u; b += 0xBB67AE85u; }
-  return ks;
+__device__ __forceinline__ void mul_wide(uint32_t a, uint32_t b, uint32_t& lo, uint32_t& hi) {
+  asm("{\n\t.reg .b64 t;\n\tmul.wide.u32 t, %2, %3;\n\tmov.b64 {%0, %1}, t;\n\t}" : "=r"(lo), "=r"(hi) : "r"(a), "r"(b));
 }
 
 __device__ __forceinline__ uint4 philox_block(uint64_t block, const PhiloxKeys& ks) {
   uint32_t c0 = static_cast<uint32_t>(block), c1 = static_cast<uint32_t>(block >> 32), c2 = 0u, c3 = 0u;
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    uint32_t lo0, hi0, lo1, hi1;
+    mul_wide(0xD2511F53u, c0, lo0, hi0);
+    mul_wide(0xCD9E8D57u, c2, lo1, hi1);
     c0 = hi1 ^ c1 ^ ks.k0[r];
     c1 = lo1;
     c2 = hi0 ^ c3 ^ ks.k1[r];
@@ -200,59 +213,121 @@ __device__ __forceinline__ uint4 philox_block(uint64_t block, const PhiloxKeys& 
   return make_uint4(c0, c1, c2, c3);
 }
 
-// Per element: lower code and the 32-bit threshold of the up-decision.
-//   t = |x| / alpha (IEEE quotient).  t < 1: code 0, threshold trunc(t * 2^32)
-//   (prune-up probability |x|/alpha).  t >= 1: code 1 + exponent(t), threshold
-//   = mantissa field << 9 (up-probability (|x| - lo)/lo); at or above the top
-//   level the code is kmax + 1 with no draw.
-__device__ __forceinline__ void luq_bin(float x, float alpha, uint32_t& lo_code, uint32_t& thr) {
-  const float t = __fdiv_rn(fabsf(x), alpha);
+// The scale of one tensor, prepared once per thread.
+//   alpha = max / 2^kmax (exact).  The quotient t = |x| / alpha must be the IEEE
+//   round-to-nearest quotient.  With y = RN(1/alpha) (correctly rounded) it is
+//   obtained without a division: q0 = a*y is within 1.5 ulp, one residual
+//   correction makes it faithful, a second one (residual now exact) makes it
+//   correctly rounded (Markstein).  For a tiny max both operands are first scaled
+//   by 2^64 (exact) so that no residual that matters falls into the denormal range.
+struct LuqScale { float alpha_s, recip, pre; };
+
+__device__ __forceinline__ LuqScale luq_scale(float alpha) {
+  LuqScale sc;
+  sc.pre = alpha < 0x1p-44f ? 0x1p64f : 1.0f;
+  sc.alpha_s = alpha * sc.pre;
+  sc.recip = __frcp_rn(sc.alpha_s);
+  return sc;
+}
+
+__device__ __forceinline__ float luq_quotient_raw(float x, const LuqScale& sc) {
+  const float a = fabsf(x) * sc.pre;
+  const float q0 = a * sc.recip;
+  const float r0 = __fmaf_rn(-sc.alpha_s, q0, a);
+  const float q1 = __fmaf_rn(r0, sc.recip, q0);
+  const float r1 = __fmaf_rn(-sc.alpha_s, q1, a);
+  return __fmaf_rn(r1, sc.recip, q1);
+}
+__device__ __forceinline__ float luq_quotient(float x, const LuqScale& sc) {
+  // an overflowing or non-finite quotient turns into NaN above; both belong to the top level
+  return fminf(luq_quotient_raw(x, sc), static_cast<float>(1 << LUQ_KMAX));   // fminf(NaN, c) = c
+}
+
+// Per element: lower code and the 32-bit threshold of the up-decision, from the
+// bit fields of t (already clamped to 2^kmax).
+//   t >= 1: code 1 + exponent(t), threshold = mantissa << 9 (up-probability
+//           (|x| - lo)/lo); t = 2^kmax gives the top code with threshold 0.
+//   t <  1: code 0, threshold trunc(t * 2^32) (prune-up probability |x|/alpha),
+//           computed as (1.mantissa << 8) >> (126 - exponent field).
+__device__ __forceinline__ void luq_bin(float t, uint32_t& lo_code, uint32_t& thr) {
   const uint32_t u = __float_as_uint(t);
-  if (t < 1.0f) {
-    lo_code = 0;
-    thr = __float2uint_rz(t * 4294967296.0f);
-  } else {
-    const int e = static_cast<int>((u >> 23) & 0xFFu) - 127;
-    if (e >= LUQ_KMAX) { lo_code = LUQ_KMAX + 1; thr = 0; }
-    else { lo_code = 1 + e; thr = (u & 0x7FFFFFu) << 9; }
-  }
+  const int e = static_cast<int>(u >> 23);
+  const uint32_t thr_in = u << 9;
+  const uint32_t thr_under = __funnelshift_rc((u << 8) | 0x80000000u, 0u, static_cast<uint32_t>(126 - e));
+  thr = u >= 0x3F800000u ? thr_in : thr_under;
+  lo_code = static_cast<uint32_t>(max(e - 126, 0));
 }
 
-__device__ __forceinline__ uint32_t luq_nibble(uint32_t sign, uint32_t lo_code, uint32_t thr, uint32_t word) {
+__device__ __forceinline__ uint32_t luq_nibble(uint32_t xbits, uint32_t lo_code, uint32_t thr, uint32_t word) {
   const uint32_t c = lo_code + (word < thr ? 1u : 0u);
-  return c ? ((sign << 3) | c) : 0u;
+  return c ? (((xbits >> 28) & 8u) | c) : 0u;
 }
 
-template <bool BF16>
+// NS: number of samples known at compile time (1, 2) or 0 = read n_samples at run time
+template <bool BF16, int NS>
 __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restrict__ x, size_t n,
                                                              const float* __restrict__ d_amax,
-                                                             uint64_t seed, int n_samples,
+                                                             const __grid_constant__ PhiloxKeySet keys,
+                                                             int n_samples_rt,
                                                              uint8_t* __restrict__ codes,
                                                              float* __restrict__ d_alpha,
                                                              unsigned int* __restrict__ status) {
+  const int n_samples = NS > 0 ? NS : n_samples_rt;
   constexpr int kElems = Item<BF16>::kElems;
   const float mx = __ldg(d_amax);
   const bool first = blockIdx.x == 0 && threadIdx.x == 0;
   const bool ok = scale_usable(mx, first ? status : nullptr);
   const float alpha = ok ? mx * (1.0f / static_cast<float>(1 << LUQ_KMAX)) : 0.0f;  // exact scaling
   if (first) *d_alpha = alpha;
+  const LuqScale sc = luq_scale(ok ? alpha : 1.0f);
 
   const size_t plane = n / 2;
   const bool aligned = (plane % (kElems / 2)) == 0;  // planes start on a store boundary
   const size_t items = n / kElems;
   const uint4* p = reinterpret_cast<const uint4*>(x);
 
-  auto process = [&](size_t item, const uint4& u) {
+  // Neural gradients are heavy-tailed: almost every element lies below alpha, in
+  // the underflow bin, where the code is 0 or 1 and the threshold is trunc(t * 2^32).
+  // A warp whose elements all do takes the short route; |x| < alpha is equivalent
+  // to t < 1 (and false for NaN), so both routes give the same codes.
+  auto process = [&](size_t item, const uint4& u, bool whole_warp) {
     float v[kElems];
-    uint32_t lo_code[kElems], thr[kElems], sign[kElems];
     Item<BF16>::widen(u, v);
+    bool in_range = false;
 #pragma unroll
-    for (int j = 0; j < kElems; ++j) {
-      luq_bin(v[j], alpha, lo_code[j], thr[j]);
-      sign[j] = __float_as_uint(v[j]) >> 31;
+    for (int j = 0; j < kElems; ++j) in_range |= !(fabsf(v[j]) < alpha);
+    // the vote needs every lane of the warp here: only the full-tile loop qualifies
+    if (whole_warp && !__any_sync(0xFFFFFFFFu, in_range)) {
+      uint32_t thr[kElems], sn[kElems];
+#pragma unroll
+      for (int j = 0; j < kElems; ++j) {
+        thr[j] = __float2uint_rz(luq_quotient_raw(v[j], sc) * 4294967296.0f);
+        sn[j] = ((__float_as_uint(v[j]) >> 28) & 8u) | 1u;
+      }
+#pragma unroll
+      for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
+        if (NS == 0 && s >= n_samples) break;
+        const PhiloxKeys& ks = keys.s[s];
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < kElems / 4; ++b) {
+          const uint4 r = philox_block(item * (kElems / 4) + b, ks);
+          const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            word += (rw[j] < thr[4 * b + j] ? sn[4 * b + j] : 0u) << (4 * (4 * b + j));
+        }
+        Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
+      }
+      return;
     }
-    for (int s = 0; s < n_samples; ++s) {
-      const PhiloxKeys ks = philox_keys(seed + static_cast<uint64_t>(s));
+    uint32_t lo_code[kElems], thr[kElems];
+#pragma unroll
+    for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient(v[j], sc), lo_code[j], thr[j]);
+#pragma unroll
+    for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
+      if (NS == 0 && s >= n_samples) break;
+      const PhiloxKeys& ks = keys.s[s];
       uint32_t word = 0;
 #pragma unroll
       for (int b = 0; b < kElems / 4; ++b) {
@@ -260,28 +335,33 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
         const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-          word |= luq_nibble(sign[4 * b + j], lo_code[4 * b + j], thr[4 * b + j], rw[j]) << (4 * (4 * b + j));
+          word |= luq_nibble(__float_as_uint(v[4 * b + j]), lo_code[4 * b + j], thr[4 * b + j], rw[j])
+                  << (4 * (4 * b + j));
       }
       Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
     }
   };
 
-  const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
-  size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x;
+  const size_t full_tiles = items / kTileItems;
   if (ok) {
-    for (; i + stride < items; i += 2 * stride) {
-      const uint4 u0 = __ldg(p + i), u1 = __ldg(p + i + stride);
-      process(i, u0);
-      process(i + stride, u1);
+    for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {
+      const size_t i0 = t * kTileItems + threadIdx.x;
+      uint4 u[kUnroll];
+#pragma unroll
+      for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i0 + j * kThreads);
+#pragma unroll
+      for (int j = 0; j < kUnroll; ++j) process(i0 + j * kThreads, u[j], true);
     }
-    for (; i < items; i += stride) process(i, __ldg(p + i));
+    if (blockIdx.x == gridDim.x - 1)
+      for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) process(i, __ldg(p + i), false);
   } else {
-    for (; i < items; i += stride)
+    const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
+    for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < items; i += stride)
       for (int s = 0; s < n_samples; ++s) Item<BF16>::store(codes + plane * s, i, 0u, aligned || s == 0);
   }
   if (first) {  // tail: fewer elements than one piece, two per byte
     for (int s = 0; s < n_samples; ++s) {
-      const PhiloxKeys ks = philox_keys(seed + static_cast<uint64_t>(s));
+      const PhiloxKeys& ks = keys.s[s];
       for (size_t e = items * kElems; e < n; e += 2) {
         uint32_t nib[2] = {0u, 0u};
         for (int h = 0; h < 2; ++h) {
@@ -289,10 +369,10 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
           if (ok && idx < n) {
             const float xv = Item<BF16>::load1(x, idx);
             uint32_t lc, th;
-            luq_bin(xv, alpha, lc, th);
+            luq_bin(luq_quotient(xv, sc), lc, th);
             const uint4 r = philox_block(idx >> 2, ks);
             const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
-            nib[h] = luq_nibble(__float_as_uint(xv) >> 31, lc, th, rw[idx & 3]);
+            nib[h] = luq_nibble(__float_as_uint(xv), lc, th, rw[idx & 3]);
           }
         }
         codes[plane * s + (e >> 1)] = static_cast<uint8_t>(nib[0] | (nib[1] << 4));
@@ -301,16 +381,38 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
   }
 }
 
-// CTAs the GPU holds at once for `kernel`, capped by the work available
+// Diagnostic: the quotient t = |x| / alpha exactly as the quantizer forms it
+// (before the clamp to the top level), for comparison with an IEEE division.
+__global__ void __launch_bounds__(kThreads) luq_quotient_kernel(const float* __restrict__ x, size_t n,
+                                                                const float* __restrict__ d_amax,
+                                                                float* __restrict__ out) {
+  const float alpha = __ldg(d_amax) * (1.0f / static_cast<float>(1 << LUQ_KMAX));
+  const LuqScale sc = luq_scale(alpha);
+  const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < n; i += stride) {
+    const float a = fabsf(x[i]) * sc.pre;
+    const float q0 = a * sc.recip;
+    const float r0 = __fmaf_rn(-sc.alpha_s, q0, a);
+    const float q1 = __fmaf_rn(r0, sc.recip, q0);
+    const float r1 = __fmaf_rn(-sc.alpha_s, q1, a);
+    out[i] = __fmaf_rn(r1, sc.recip, q1);
+  }
+}
+
+// Grid for a kernel that walks `tiles` tiles: at most the CTAs the GPU holds at once
+// (optionally fewer per SM), and then the smallest grid with the same number of rounds,
+// so that every CTA gets the same share.
 template <typename K>
-int grid_for(const luq_ctx* ctx, K kernel, size_t thread_items) {
+int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 30) {
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1)
     per_sm = 1;
-  size_t want = (thread_items + kThreads - 1) / kThreads;
+  if (per_sm > max_per_sm) per_sm = max_per_sm;
   const size_t cap = static_cast<size_t>(ctx->sm_count) * per_sm;
-  if (want < 1) want = 1;
-  return static_cast<int>(want < cap ? want : cap);
+  if (tiles < 1) tiles = 1;
+  if (tiles <= cap) return static_cast<int>(tiles);
+  const size_t rounds = (tiles + cap - 1) / cap;
+  return static_cast<int>((tiles + rounds - 1) / rounds);
 }
 
 }  // namespace
@@ -320,10 +422,10 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
   if (e != cudaSuccess) return static_cast<int>(e);
   if (n == 0) return 0;
   if (dtype == LUQ_BF16) {
-    const int grid = grid_for(ctx, amax_kernel<true>, n / 8 / kUnroll + 1);
+    const int grid = grid_for(ctx, amax_kernel<true>, n / 8 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
     amax_kernel<true><<<grid, kThreads, 0, st>>>(d_x, n, reinterpret_cast<unsigned int*>(d_amax), ctx->d_status);
   } else {
-    const int grid = grid_for(ctx, amax_kernel<false>, n / 4 / kUnroll + 1);
+    const int grid = grid_for(ctx, amax_kernel<false>, n / 4 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
     amax_kernel<false><<<grid, kThreads, 0, st>>>(d_x, n, reinterpret_cast<unsigned int*>(d_amax), ctx->d_status);
   }
   ctx->launches += 1;
@@ -333,27 +435,55 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
 int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
                           uint8_t* d_codes, float* d_scale, cudaStream_t st) {
   if (dtype == LUQ_BF16) {
-    const int grid = grid_for(ctx, quant_int4_kernel<true>, n / 8 / kUnroll + 1);
+    const int grid = grid_for(ctx, quant_int4_kernel<true>, n / 8 / kTileItems + 1);
     quant_int4_kernel<true><<<grid, kThreads, 0, st>>>(d_x, n, d_clip, d_codes, d_scale, ctx->d_status);
   } else {
-    const int grid = grid_for(ctx, quant_int4_kernel<false>, n / 4 / kUnroll + 1);
+    const int grid = grid_for(ctx, quant_int4_kernel<false>, n / 4 / kTileItems + 1);
     quant_int4_kernel<false><<<grid, kThreads, 0, st>>>(d_x, n, d_clip, d_codes, d_scale, ctx->d_status);
   }
   ctx->launches += 1;
   return static_cast<int>(cudaGetLastError());
 }
 
+namespace {
+template <bool BF16>
+int launch_luq(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys, int n_samples,
+               uint8_t* d_codes, float* d_alpha, cudaStream_t st) {
+  const size_t thread_items = n / Item<BF16>::kElems / kTileItems + 1;
+  if (n_samples == 1) {
+    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 1>, thread_items);
+    quant_luq_kernel<BF16, 1><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 1, d_codes, d_alpha, ctx->d_status);
+  } else if (n_samples == 2) {
+    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 2>, thread_items);
+    quant_luq_kernel<BF16, 2><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 2, d_codes, d_alpha, ctx->d_status);
+  } else {
+    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 0>, thread_items);
+    quant_luq_kernel<BF16, 0><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, n_samples, d_codes, d_alpha,
+                                                        ctx->d_status);
+  }
+  return static_cast<int>(cudaGetLastError());
+}
+}  // namespace
+
 int luq_launch_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
                           uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, cudaStream_t st) {
-  if (dtype == LUQ_BF16) {
-    const int grid = grid_for(ctx, quant_luq_kernel<true>, n / 8 / 2 + 1);
-    quant_luq_kernel<true><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, seed, n_samples, d_codes, d_alpha,
-                                                      ctx->d_status);
-  } else {
-    const int grid = grid_for(ctx, quant_luq_kernel<false>, n / 4 / 2 + 1);
-    quant_luq_kernel<false><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, seed, n_samples, d_codes, d_alpha,
-                                                       ctx->d_status);
+  PhiloxKeySet keys{};
+  for (int s = 0; s < n_samples; ++s) {   // sample s is keyed by seed + s
+    const uint64_t key = seed + static_cast<uint64_t>(s);
+    uint32_t a = static_cast<uint32_t>(key), b = static_cast<uint32_t>(key >> 32);
+    for (int r = 0; r < 10; ++r) { keys.s[s].k0[r] = a; keys.s[s].k1[r] = b; a += 0x9E3779B9u; b += 0xBB67AE85u; }
   }
+  const int rc = dtype == LUQ_BF16 ? launch_luq<true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, st)
+                                   : launch_luq<false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, st);
+  ctx->launches += 1;
+  return rc;
+}
+
+int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,
+                              cudaStream_t st) {
+  if (n == 0) return 0;
+  const int grid = grid_for(ctx, luq_quotient_kernel, n / kThreads + 1);
+  luq_quotient_kernel<<<grid, kThreads, 0, st>>>(d_x, n, d_amax, d_t);
   ctx->launches += 1;
   return static_cast<int>(cudaGetLastError());
 }

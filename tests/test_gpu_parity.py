@@ -298,3 +298,37 @@ def test_gemm_large_integer_sums_are_exact(ctx):
         assert (dA == 16 * 7 * K).all()
     ctx.set_option(binding.OPT_MMA_KIND, 0)
     assert ctx.status() == 0
+
+
+def test_division_free_quotient_equals_ieee_division(ctx):
+    """The quantizer forms t = |x|/alpha with a reciprocal and two residual
+    corrections; it must be the IEEE round-to-nearest quotient for every scale,
+    including maxima near the ends of the accepted range [2^-100, 2^100]."""
+    rng = np.random.default_rng(123)
+    n = 1 << 21
+    exps = list(rng.uniform(-99, 99, 40)) + [-100, -99.5, -63, -44.2, -43.9, -40, 0, 40, 99.9]
+    total = 0
+    for ex in exps:
+        mx = np.float32(2.0 ** ex) * np.float32(rng.uniform(1.0, 1.9999))
+        if ex <= -100:
+            mx = np.float32(2.0 ** -100)
+        alpha = np.float32(mx) / np.float32(16)
+        # magnitudes from far below alpha up to a few times the maximum, plus values hugging the levels
+        t_target = np.exp2(rng.uniform(-45, 5.5, n))
+        x = (t_target * float(alpha)).astype(np.float32)
+        lv = (alpha * np.float32(2.0) ** rng.integers(0, 5, 4096)).astype(np.float32)
+        x[:4096] = lv
+        x[4096:8192] = np.nextafter(lv, np.float32(0))
+        x[8192:12288] = np.nextafter(lv, np.float32(np.inf))
+        x[12288:16384] = (lv * np.float32(1.5)).astype(np.float32)
+        x *= np.where(rng.random(n) < 0.5, -1, 1).astype(np.float32)
+        with np.errstate(over="ignore", under="ignore"):
+            ref = (np.abs(x) / alpha).astype(np.float32)
+        got = ctx.debug_quotient(to_dev(x), scalar(float(mx))).cpu().numpy()
+        check = (ref >= np.float32(2.0 ** -60)) & (ref <= np.float32(64.0))
+        np.testing.assert_array_equal(got[check].view(np.uint32), ref[check].view(np.uint32))
+        small = ref < np.float32(2.0 ** -60)
+        assert (got[small] < 2.0 ** -40).all()
+        total += int(check.sum())
+    assert total > 50_000_000
+    assert ctx.status() == 0
