@@ -321,7 +321,7 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "e4m3 operands, f32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "int8 operands, int32 accumulate" if (args.mma_kind in (None, 1)) else "e4m3 operands, f32 accumulate", "data": "synthetic",
             "config": {"workload": f"{args.workload}: M={M} K={K} N={N}, {cfg.dtype} inputs, "
                                    f"LUQ seed {seed}, {ns} sample(s)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",

@@ -58,7 +58,7 @@ extern "C" {
 #define LUQ_STATUS_TIMEOUT 4   /* a bounded wait inside a kernel expired; outputs unspecified */
 
 /* options for luq_set_option */
-#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands; 1: kind::i8 on int8 operands */
+#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands; 1: kind::i8 on int8 operands (default) */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
 
 #define LUQ_MAX_SAMPLES 8

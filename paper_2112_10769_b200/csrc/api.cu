@@ -52,7 +52,7 @@ int luq_create(luq_ctx** out, int device) {
   if (!c) return LUQ_ERR_CUDA;
   c->device = device;
   c->sm_count = prop.multiProcessorCount;
-  c->mma_kind = 0;
+  c->mma_kind = LUQ_DEFAULT_MMA_KIND;
   c->forced_splits = 0;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;

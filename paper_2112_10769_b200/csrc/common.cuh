@@ -7,6 +7,7 @@
 #include "luq.h"
 
 #define LUQ_KMAX 4  // alpha = max / 2^LUQ_KMAX (Eq. alpha with b = 3)
+#define LUQ_DEFAULT_MMA_KIND 1  // int8 operands (kind::i8): same tensor-core rate as e4m3, cheaper INT4 expansion
 
 struct luq_ctx {
   int device;

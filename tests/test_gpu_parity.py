@@ -243,7 +243,7 @@ def test_three_gemms_match_oracle(ctx, M, K, N, ns, mma_kind):
         assert_gemm_close(dA.cpu().numpy(), oracle.gemm_bwd(og, oal, ns, ow, osw, M, N, K))
         assert_gemm_close(dW.cpu().numpy(), oracle.gemm_wgrad(og, oal, ns, oa, osa, M, N, K))
     finally:
-        ctx.set_option(binding.OPT_MMA_KIND, 0)
+        ctx.set_option(binding.OPT_MMA_KIND, 1)
 
 
 @pytest.mark.parametrize("splits", [1, 2, 5])
@@ -296,7 +296,7 @@ def test_gemm_large_integer_sums_are_exact(ctx):
         wk = torch.full((K, N // 2), 0x77, dtype=torch.uint8, device="cuda")
         dA = ctx.gemm_bwd(g, scalar(1.0), 1, wk, scalar(1.0), M, K, N).cpu().numpy()
         assert (dA == 16 * 7 * K).all()
-    ctx.set_option(binding.OPT_MMA_KIND, 0)
+    ctx.set_option(binding.OPT_MMA_KIND, 1)
     assert ctx.status() == 0
 
 
