@@ -134,6 +134,33 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
                    const uint8_t* d_a_codes, const float* d_sa,
                    float* d_dw, int64_t M, int64_t N, int64_t K, void* stream);
 
+/* Update GEMM without any allocation.  (The paper has no counterpart; this entry
+ * point exists for the sake of callers.)
+ *
+ * Some callers cannot obtain device memory themselves: code that runs inside a
+ * stream capture, inside another framework's allocator hooks or a memory-frozen
+ * serving process, or under a memory budget that forbids cudaMalloc after start-up.
+ * luq_create allocates the split workspace with cudaMalloc, so it is closed to
+ * them.  This variant of luq_gemm_wgrad takes no context and keeps its split
+ * workspace (the partial tiles of the contraction split) in a fixed 19 MiB array
+ * inside the library image.  It calls no allocation routine of any kind.
+ *
+ *  - Same arguments and result as luq_gemm_wgrad, on the CURRENT device.
+ *  - Limit: the output N x K may have at most 152 tiles of 128 x 256 elements
+ *    (for example N = 256, K <= 19456); larger outputs return LUQ_ERR_WORKSPACE.
+ *  - The first call on each device looks up the device address of the array
+ *    (cudaGetSymbolAddress) and clears the variant's status word; make that first
+ *    call outside any stream capture.  Later calls only launch kernels.
+ *  - The array is shared by all calls on a device and keeps the previous call's
+ *    partial tiles.  Every call rewrites all tiles it later reads, so nothing has
+ *    to be cleared, but two calls that overlap on the GPU (different streams) race
+ *    on it: serialise them.
+ *  - A bounded wait that expires cannot be reported through luq_status here; it
+ *    leaves the output unspecified, as in luq_gemm_wgrad. */
+int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
+                          const uint8_t* d_a_codes, const float* d_sa,
+                          float* d_dw, int64_t M, int64_t N, int64_t K, void* stream);
+
 /* Synchronises `stream`, returns the device status bits in *host_flags and
  * clears them. */
 int luq_status(luq_ctx* ctx, void* stream, int* host_flags);

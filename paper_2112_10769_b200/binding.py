@@ -21,7 +21,7 @@ OPT_MMA_KIND, OPT_SPLITS = 1, 2
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_quant_grad", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_status",
+           "luq_quant_grad", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_gemm_wgrad_static", "luq_status",
            "luq_launch_count", "luq_strerror")
 
 _lib = None
@@ -52,6 +52,7 @@ def load() -> ctypes.CDLL:
         L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_wgrad.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_gemm_wgrad_static.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
         L.luq_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int)]
         L.luq_launch_count.argtypes = [vp]
         L.luq_launch_count.restype = i64
@@ -167,6 +168,17 @@ class Context:
         flags = ctypes.c_int(0)
         _check(load().luq_status(self.handle, _stream(), ctypes.byref(flags)), "luq_status")
         return flags.value
+
+
+def gemm_wgrad_static(g_codes, alpha, n_samples: int, a_codes, sa, M: int, N: int, K: int,
+                      out: torch.Tensor) -> torch.Tensor:
+    """Update GEMM through the entry point that allocates nothing: no context, the
+    split workspace is a fixed array inside the library.  `out` must be supplied by
+    the caller (this wrapper does not allocate either).  Runs on the current device."""
+    _check(load().luq_gemm_wgrad_static(g_codes.data_ptr(), alpha.data_ptr(), n_samples, a_codes.data_ptr(),
+                                        sa.data_ptr(), out.data_ptr(), M, N, K, _stream()),
+           "luq_gemm_wgrad_static")
+    return out
 
 
 def kmax() -> int:

@@ -28,6 +28,8 @@
 // copies, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -528,4 +530,103 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
     if (rc == 0) ctx->launches += 1;
   }
   return rc;
+}
+
+// ---------------------------------------------------------------------------
+// Update GEMM for callers that must not allocate device memory.
+//
+// The split partial tiles normally live in the context's workspace, which
+// luq_create obtains with cudaMalloc.  Here they live in a fixed array that is
+// part of the library image: it exists on every GPU that loads the library, from
+// load until the process ends, and is shared by every call of this entry point.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticTiles = 152;                                  // partial tiles the array holds
+constexpr size_t kStaticScratchBytes = static_cast<size_t>(kStaticTiles) * kTileFloats * sizeof(float);  // 19 MiB
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) float g_static_scratch[static_cast<size_t>(kStaticTiles) * kTileFloats];
+static __device__ unsigned int g_static_status;
+
+struct StaticSetup {
+  bool ready = false;
+  float* scratch = nullptr;        // device address of g_static_scratch on this device
+  unsigned int* status = nullptr;  // device address of g_static_status on this device
+  void* encode_tiled = nullptr;
+  int sm_count = 0;
+};
+StaticSetup g_static_setup[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current.  In host code the names of the two
+// arrays are only handles: the addresses a kernel may use come from
+// cudaGetSymbolAddress.
+int static_setup(int device, StaticSetup** out) {
+  if (device < 0 || device >= kMaxDevices) return LUQ_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticSetup& s = g_static_setup[device];
+  if (!s.ready) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return LUQ_ERR_CUDA;
+    if (prop.major != 10) return LUQ_ERR_UNSUPPORTED;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return LUQ_ERR_CUDA;
+    s.scratch = static_cast<float*>(p);
+    p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_status) != cudaSuccess || p == nullptr) return LUQ_ERR_CUDA;
+    s.status = static_cast<unsigned int*>(p);
+    if (cudaMemset(s.status, 0, sizeof(unsigned int)) != cudaSuccess) return LUQ_ERR_CUDA;  // must start at zero
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &s.encode_tiled, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || s.encode_tiled == nullptr)
+      return LUQ_ERR_CUDA;
+    s.sm_count = prop.multiProcessorCount;
+    s.ready = true;
+  }
+  *out = &s;
+  return LUQ_OK;
+}
+
+}  // namespace
+
+extern "C" int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
+                                     const uint8_t* d_a_codes, const float* d_sa, float* d_dw,
+                                     int64_t M, int64_t N, int64_t K, void* stream) {
+  if (!d_alpha || !d_sa) return LUQ_ERR_ARG;
+  if (M < 0 || N < 0 || K < 0 || M > (1ll << 31) || N > (1ll << 31) || K > (1ll << 31)) return LUQ_ERR_ARG;
+  if (n_samples < 1 || n_samples > LUQ_MAX_SAMPLES) return LUQ_ERR_ARG;
+  if (M && N && K && (!d_g_codes || !d_a_codes || !d_dw)) return LUQ_ERR_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_g_codes) | reinterpret_cast<uintptr_t>(d_a_codes) |
+       reinterpret_cast<uintptr_t>(d_dw)) & 15u)
+    return LUQ_ERR_ARG;
+  if (N % 32 || K % 32) return LUQ_ERR_ARG;
+  const long long tiles = ((N + BM - 1) / BM) * ((K + BN - 1) / BN);
+  if (tiles > kStaticTiles) return LUQ_ERR_WORKSPACE;   // output larger than the fixed scratch serves
+
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) return LUQ_ERR_CUDA;
+  StaticSetup* s = nullptr;
+  int rc = static_setup(device, &s);
+  if (rc != LUQ_OK) return rc;
+
+  luq_ctx local{};               // a context on the stack: nothing in it is allocated
+  local.device = device;
+  local.sm_count = s->sm_count;
+  local.d_status = s->status;
+  local.d_workspace = s->scratch;
+  local.workspace_bytes = kStaticScratchBytes;
+  local.mma_kind = LUQ_DEFAULT_MMA_KIND;
+  local.forced_splits = 0;
+  local.launches = 0;
+  local.encode_tiled = s->encode_tiled;
+
+  luq_gemm_args a{};
+  a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 1; a.n_samples = n_samples;
+  a.b_codes = d_a_codes; a.b_kind = 0; a.b_mn = 1;
+  a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.Mo = N; a.No = K; a.Kc = M;
+  a.d_workspace = s->scratch; a.workspace_bytes = kStaticScratchBytes;
+  a.allow_split = 1;
+  rc = luq_launch_gemm(&local, a, reinterpret_cast<cudaStream_t>(stream));
+  return rc == 0 ? LUQ_OK : (rc < 0 ? rc : LUQ_ERR_CUDA);
 }
