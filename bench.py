@@ -170,10 +170,54 @@ def run_reference(args):
 
 # ------------------------------------------------------------------ GPU arm --
 
+def run_sweep(args, binding, inputs, torch, local):
+    """Quantizer bandwidth sweep (config 4): amax + LUQ quantize-and-pack on 1-D fp32
+    gradient tensors of 2^20..2^30 elements, 1 and 2 samples.  GB/s = algorithmic bytes
+    (4 + 4 + 0.5 n_s per element: the tensor is read twice, codes written once) / time.
+    "cold": a 512 MB buffer is overwritten before every repetition (L2 flushed);
+    "warm": back-to-back repetitions."""
+    ctx = binding.Context(local)
+    peaks = load_peaks()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    rows = []
+    for e in inputs.SWEEP_EXPONENTS:
+        n = 1 << e
+        x = torch.from_numpy(inputs.sweep_tensor(e)).cuda()
+        mx, al = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
+        for ns in (1, 2):
+            codes = torch.empty((ns, n // 2), dtype=torch.uint8, device="cuda")
+            reps = 20 if e <= 26 else 5
+            res = {}
+            for mode in ("cold", "warm"):
+                times = {"amax": [], "quant": []}
+                for it in range(reps + 3):
+                    if mode == "cold":
+                        flush.fill_(it & 0xFF)
+                    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                    ev[0].record(); ctx.amax(x, mx); ev[1].record(); ctx.quant_grad(x, mx, 0, ns, codes, al); ev[2].record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        times["amax"].append(ev[0].elapsed_time(ev[1])); times["quant"].append(ev[1].elapsed_time(ev[2]))
+                med = {k: sorted(v)[len(v) // 2] for k, v in times.items()}
+                total = med["amax"] + med["quant"]
+                res[mode] = {"amax_us": round(med["amax"] * 1e3, 2), "quant_us": round(med["quant"] * 1e3, 2),
+                             "quant_gbs": round((4 + 0.5 * ns) * n / (med["quant"] * 1e-3) / 1e9, 1),
+                             "amax_plus_quant_gbs": round((8 + 0.5 * ns) * n / (total * 1e-3) / 1e9, 1),
+                             "frac_of_hbm_peak": round((8 + 0.5 * ns) * n / (total * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
+            rows.append({"elements": n, "n_samples": ns, **res})
+            del codes
+        del x
+        torch.cuda.empty_cache()
+    assert ctx.status() == 0
+    print(json.dumps({"metric": "luq_quantizer_hbm_gbs", "unit": "GB/s", "workload": "cfg4 sweep", "dtype": "f32",
+                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "rows": rows}))
+    ctx.close()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2112_10769_b200 import binding, inputs
+    from paper_2112_10769_b200 import binding, inputs, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -186,9 +230,12 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
+
+    if args.workload == "cfg4":
+        run_sweep(args, binding, inputs, torch, local)
+        return
 
     cfg = inputs.CONFIGS[args.workload]
     if args.rows:
@@ -252,10 +299,7 @@ def run_ours(args):
     sampler.stop_flag.set()
     total_ms = t0.elapsed_time(t1)
     launches = ctx.launches - launches0
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = replicas.max_over_ranks(total_ms, dev)
     assert ctx.status() == 0
     ms_per_step = total_ms / args.steps
     flops_step = 3 * 2.0 * M * N * K
@@ -302,10 +346,7 @@ def run_ours(args):
         t1.record()
         barrier()
         e2e_ms = t0.elapsed_time(t1) / e2e_steps
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks(e2e_ms, dev)
         h2d = sum(t.numel() * t.element_size() for t in (A_p, W_p, G_p))
         d2h = sum(t.numel() * t.element_size() for t in (Z_p, dA_p, dW_p))
         e2e = {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
@@ -344,8 +385,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=WORKLOAD, choices=["cfg1", "cfg2", "cfg3", "cfg5"],
-                    help="layer shape; the headline number is cfg2")
+    ap.add_argument("--workload", default=WORKLOAD, choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"],
+                    help="layer shape (the headline number is cfg2), or cfg4 = the quantizer bandwidth sweep")
     ap.add_argument("--rows", type=int, default=None, help="truncate the batch dimension M (small profiling runs)")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs")
     ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1],
