@@ -362,7 +362,7 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "int8 operands, int32 accumulate" if (args.mma_kind in (None, 1)) else "e4m3 operands, f32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": {None: "int8 or e4m3 operands per product, exact accumulate", 0: "e4m3 operands, f32 accumulate", 1: "int8 operands, int32 accumulate", 2: "int8 or e4m3 operands per product, exact accumulate"}[args.mma_kind], "data": "synthetic",
             "config": {"workload": f"{args.workload}: M={M} K={K} N={N}, {cfg.dtype} inputs, "
                                    f"LUQ seed {seed}, {ns} sample(s)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
@@ -389,8 +389,8 @@ def main():
                     help="layer shape (the headline number is cfg2), or cfg4 = the quantizer bandwidth sweep")
     ap.add_argument("--rows", type=int, default=None, help="truncate the batch dimension M (small profiling runs)")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs")
-    ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1],
-                    help="tensor-core operand type: 0 e4m3 (kind::f8f6f4), 1 int8 (kind::i8); default: the library's")
+    ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1, 2],
+                    help="tensor-core operand type: 0 e4m3 (kind::f8f6f4), 1 int8 (kind::i8), 2 per product; default: the library's")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -58,7 +58,9 @@ extern "C" {
 #define LUQ_STATUS_TIMEOUT 4   /* a bounded wait inside a kernel expired; outputs unspecified */
 
 /* options for luq_set_option */
-#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands; 1: kind::i8 on int8 operands (default) */
+#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands; 1: kind::i8 on int8 operands;
+                              2 (default): chosen per product - int8 where INT4 codes are expanded inside the
+                              kernel, e4m3 where both operands are pre-expanded planes */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
 
 #define LUQ_MAX_SAMPLES 8
@@ -66,7 +68,7 @@ extern "C" {
 typedef struct luq_ctx luq_ctx;
 
 /* Creates a context on `device`: a device status word and the split workspace
- * (32 MiB) used by GEMMs whose output has too few tiles to fill the GPU.
+ * (96 MiB: partial tiles of split contractions and 8-bit operand planes of the GEMMs).
  * Allocates device memory; call outside stream capture. */
 int luq_create(luq_ctx** out, int device);
 int luq_destroy(luq_ctx* ctx);

@@ -5,7 +5,7 @@
 
 namespace {
 
-constexpr size_t kWorkspaceBytes = 32u << 20;
+constexpr size_t kWorkspaceBytes = 96u << 20;  // 20 MiB of split partial tiles + 76 MiB of operand planes
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
@@ -83,7 +83,7 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
   if (!ctx) return LUQ_ERR_ARG;
   switch (option) {
     case LUQ_OPT_MMA_KIND:
-      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      if (value < 0 || value > 2) return LUQ_ERR_ARG;
       ctx->mma_kind = value;
       return LUQ_OK;
     case LUQ_OPT_SPLITS:

@@ -7,7 +7,7 @@
 #include "luq.h"
 
 #define LUQ_KMAX 4  // alpha = max / 2^LUQ_KMAX (Eq. alpha with b = 3)
-#define LUQ_DEFAULT_MMA_KIND 1  // int8 operands (kind::i8): same tensor-core rate as e4m3, cheaper INT4 expansion
+#define LUQ_DEFAULT_MMA_KIND 2  // chosen per product: int8 where INT4 codes are expanded in the kernel, else e4m3
 
 struct luq_ctx {
   int device;
@@ -15,7 +15,7 @@ struct luq_ctx {
   unsigned int* d_status;   // device status word (LUQ_STATUS_* bits)
   float* d_workspace;       // split-contraction partial tiles
   size_t workspace_bytes;
-  int mma_kind;             // 0 f8f6f4/e4m3, 1 i8
+  int mma_kind;             // 0 f8f6f4/e4m3, 1 i8, 2 chosen per product
   int forced_splits;        // 0 = automatic
   int64_t launches;
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved at create

@@ -7,14 +7,23 @@
 // ("K-major": rows are mo / no) or contraction-major ("MN-major": rows are k).
 //
 // One persistent CTA per SM, warp-specialised:
-//   warp 0       TMA producer: packed 128-row x 64-byte slabs -> shared memory ring
-//   warps 6-21   converters: nibble -> 8-bit operand, written in the 128-byte
-//                swizzled layout the tensor core reads
+//   warp 0       TMA producer for packed slabs (128 rows x 64 bytes) -> packed ring
+//   warp 6       TMA producer for operand planes (128 rows x 128 bytes, already
+//                8-bit, 128-byte swizzle) -> straight into the operand ring
+//   warps 7-22   converters: packed nibbles -> 8-bit operands, written in the
+//                128-byte swizzled layout the tensor core reads
 //   warp 1       one thread issues tcgen05.mma (128 x 256 x 32 per instruction),
 //                accumulators live in tensor memory, two buffers of 256 columns
 //   warps 2-5    epilogue: tcgen05.ld -> scale -> swizzled staging -> TMA store
-// Every slab, in either orientation, is 128 rows x 64 packed bytes and expands to
-// 128 rows x 128 bytes; only the matrix descriptor differs between orientations.
+// Every slab, in either orientation, expands to 128 rows x 128 bytes; only the
+// matrix descriptor differs between orientations.
+//
+// Shared-memory bandwidth bounds the in-kernel expansion (TMA write + converter
+// read + converter write + tensor-core read of every operand byte).  An operand
+// that many tiles re-read (the weights; the gradient in the backward and update
+// products) is therefore expanded once by a small kernel into an 8-bit "plane"
+// in the context workspace and fetched by TMA in its final layout; only operands
+// used by a single row or column of tiles are expanded inside the GEMM.
 //
 // Operand bytes.  kind::f8f6f4: e4m3 through a 16-entry byte table (PRMT).
 // kind::i8: LUQ levels +-2^(c-1) through the table; INT4 integers without a
@@ -43,34 +52,44 @@ constexpr int kSlabRows = 128;
 constexpr int kPackedSlab = kSlabRows * 64;      // bytes
 constexpr int kExpandedSlab = kSlabRows * 128;   // bytes
 constexpr int kSlabs = 1 + BN / 128;             // A, B0, B1
-constexpr int kPackedStage = kSlabs * kPackedSlab;
 constexpr int kExpandedStage = kSlabs * kExpandedSlab;
-constexpr int kPackedStages = 4;
-constexpr int kExpandedStages = 2;
-constexpr int kConvWarps = 16;
-constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kFirstEpiWarp = 2;
-constexpr int kFirstConvWarp = 6;
-constexpr int kThreads = 32 * (kFirstConvWarp + kConvWarps);
+constexpr int kPlaneWarp = 6;
+constexpr int kFirstConvWarp = 7;
 constexpr int kTmemCols = 2 * BN;
 constexpr int kTileFloats = BM * BN;
 constexpr int kStageBox = 32 * 32 * 4;           // one 32 x 32 fp32 store box
+constexpr int kMaxBarriers = 24;
 
-static_assert(kSlabs * 512 % kConvThreads == 0, "converter tasks must divide evenly");
-
-struct SmemLayout {
+// Ring depths and shared-memory map for one choice of "which operands arrive as planes".
+template <bool A_PLANE, bool B_PLANE>
+struct Cfg {
+  static constexpr int packed_slabs = (A_PLANE ? 0 : 1) + (B_PLANE ? 0 : BN / 128);
+  static constexpr int packed_stage = packed_slabs * kPackedSlab;
+  static constexpr int b_packed_off = A_PLANE ? 0 : kPackedSlab;        // first B slab inside a packed stage
+  static constexpr int ES = (A_PLANE && B_PLANE) ? 4 : ((A_PLANE || B_PLANE) ? 3 : 2);
+  static constexpr int PS = packed_slabs == 0 ? 0 : (packed_slabs == 2 ? 3 : 4);
+  static constexpr int plane_bytes = (A_PLANE ? kExpandedSlab : 0) + (B_PLANE ? (BN / 128) * kExpandedSlab : 0);
+  // sixteen converter warps when all three slabs are expanded here, eight otherwise; with the
+  // smaller CTA the register budget allows the epilogue to double-buffer its tensor-memory loads
+  static constexpr int conv_warps = packed_slabs == 3 ? 16 : 8;
+  static constexpr int conv_threads = conv_warps * 32;
+  static constexpr int threads = 32 * (kFirstConvWarp + conv_warps);
+  static constexpr bool epi_double = threads <= 512;
+  static constexpr int tasks_per_thread = packed_slabs * 512 / conv_threads;
+  // shared-memory offsets from the 1024-byte aligned base
   static constexpr int expanded = 0;
-  static constexpr int packed = expanded + kExpandedStages * kExpandedStage;
-  static constexpr int staging = packed + kPackedStages * kPackedStage;  // 4 warps x 2 boxes
+  static constexpr int packed = expanded + ES * kExpandedStage;
+  static constexpr int staging = packed + PS * packed_stage;             // 4 warps x 2 boxes
   static constexpr int barriers = staging + 4 * 2 * kStageBox;
-  // barrier order: pk_full[PS] pk_empty[PS] ex_full[ES] ex_empty[ES] acc_full[2] acc_empty[2]
-  static constexpr int num_barriers = 2 * kPackedStages + 2 * kExpandedStages + 4;
-  static constexpr int tmem_slot = barriers + 8 * num_barriers;
+  static constexpr int tmem_slot = barriers + 8 * kMaxBarriers;
   static constexpr int abort_flag = tmem_slot + 4;
   static constexpr int total = abort_flag + 4;
+  static constexpr int smem_bytes = total + 1024;                        // slack to align the base
+  static_assert(smem_bytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+  static_assert(2 * PS + 2 * ES + 4 <= kMaxBarriers, "barrier area too small");
+  static_assert(packed_slabs * 512 % conv_threads == 0, "converter tasks must divide evenly");
 };
-constexpr int kSmemBytes = SmemLayout::total + 1024;  // slack to align the base to 1024 bytes
-static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
 struct GemmParams {
   const float* scale_a;
@@ -105,36 +124,73 @@ __device__ __forceinline__ void expand8_int4_x16(uint32_t w, uint32_t& lo, uint3
   if constexpr (PERMUTED) { lo = even; hi = odd; }
   else { lo = __byte_perm(even, odd, 0x5140); hi = __byte_perm(even, odd, 0x7362); }
 }
+// 32 packed codes (16 bytes) -> 32 operand bytes in element order
+template <int KIND, bool LUQ_CODES, bool PERMUTED>
+__device__ __forceinline__ void expand32(const uint4& w, const uint4& lut, uint4& o0, uint4& o1) {
+  if constexpr (KIND == 1 && !LUQ_CODES) {
+    expand8_int4_x16<PERMUTED>(w.x, o0.x, o0.y);
+    expand8_int4_x16<PERMUTED>(w.y, o0.z, o0.w);
+    expand8_int4_x16<PERMUTED>(w.z, o1.x, o1.y);
+    expand8_int4_x16<PERMUTED>(w.w, o1.z, o1.w);
+  } else {
+    expand8_lut(w.x, lut, o0.x, o0.y);
+    expand8_lut(w.y, lut, o0.z, o0.w);
+    expand8_lut(w.z, lut, o1.x, o1.y);
+    expand8_lut(w.w, lut, o1.z, o1.w);
+  }
+}
 
-// KIND 0 f8f6f4 / 1 i8; A_MN, B_MN operand orientation; A_LUQ: A holds LUQ codes (B is always INT4)
-template <int KIND, bool A_MN, bool B_MN, bool A_LUQ>
-__global__ void __launch_bounds__(kThreads, 1)
+// Expands a whole packed tensor into an 8-bit operand plane (element order kept).
+template <int KIND, bool LUQ_CODES>
+__global__ void __launch_bounds__(256) expand_plane_kernel(const uint4* __restrict__ codes, uint4* __restrict__ plane,
+                                                           size_t pieces, uint4 lut) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < pieces; i += stride) {
+    uint4 o0, o1;
+    expand32<KIND, LUQ_CODES, false>(__ldg(codes + i), lut, o0, o1);
+    plane[2 * i] = o0;
+    plane[2 * i + 1] = o1;
+  }
+}
+
+// KIND 0 f8f6f4 / 1 i8; A_MN, B_MN operand orientation; A_LUQ: A holds LUQ codes (B is always
+// INT4); A_PLANE / B_PLANE: the operand arrives as an 8-bit plane instead of packed codes
+template <int KIND, bool A_MN, bool B_MN, bool A_LUQ, bool A_PLANE, bool B_PLANE>
+__global__ void __launch_bounds__((Cfg<A_PLANE, B_PLANE>::threads), 1)
 luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_out, const GemmParams p) {
-  // with int8 operands and both INT4 operands k-contiguous the expansion may permute k
-  constexpr bool kPermuteK = KIND == 1 && !A_MN && !B_MN && !A_LUQ;
+  using C = Cfg<A_PLANE, B_PLANE>;
+  constexpr int PS = C::PS, ES = C::ES;
+  constexpr int kConvWarps = C::conv_warps, kConvThreads = C::conv_threads;
+  constexpr bool kAnyPacked = C::packed_slabs > 0;
+  constexpr bool kAnyPlane = A_PLANE || B_PLANE;
+  // with int8 operands and both INT4 operands expanded here and k-contiguous, the expansion may permute k
+  constexpr bool kPermuteK = KIND == 1 && !A_MN && !B_MN && !A_LUQ && !A_PLANE && !B_PLANE;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* const gen = smem_raw + (base - raw);
 
-  const uint32_t bar0 = base + SmemLayout::barriers;
+  const uint32_t bar0 = base + C::barriers;
   auto pk_full = [&](int s) { return bar0 + 8u * s; };
-  auto pk_empty = [&](int s) { return bar0 + 8u * (kPackedStages + s); };
-  auto ex_full = [&](int s) { return bar0 + 8u * (2 * kPackedStages + s); };
-  auto ex_empty = [&](int s) { return bar0 + 8u * (2 * kPackedStages + kExpandedStages + s); };
-  auto acc_full = [&](int b) { return bar0 + 8u * (2 * kPackedStages + 2 * kExpandedStages + b); };
-  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kPackedStages + 2 * kExpandedStages + 2 + b); };
-  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + SmemLayout::tmem_slot);
-  volatile uint32_t* const abort_flag = reinterpret_cast<volatile uint32_t*>(gen + SmemLayout::abort_flag);
+  auto pk_empty = [&](int s) { return bar0 + 8u * (PS + s); };
+  auto ex_full = [&](int s) { return bar0 + 8u * (2 * PS + s); };
+  auto ex_empty = [&](int s) { return bar0 + 8u * (2 * PS + ES + s); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * PS + 2 * ES + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * PS + 2 * ES + 2 + b); };
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + C::tmem_slot);
+  volatile uint32_t* const abort_flag = reinterpret_cast<volatile uint32_t*>(gen + C::abort_flag);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kPackedStages; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kConvWarps); }
-    for (int s = 0; s < kExpandedStages; ++s) { mbar_init(ex_full(s), kConvWarps); mbar_init(ex_empty(s), 1); }
+    for (int s = 0; s < PS; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kConvWarps); }
+    for (int s = 0; s < ES; ++s) {
+      mbar_init(ex_full(s), (kAnyPacked ? kConvWarps : 0) + (kAnyPlane ? 1 : 0));
+      mbar_init(ex_empty(s), 1);
+    }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     *abort_flag = 0;
     fence_barrier_init();
@@ -142,7 +198,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   }
   if (warp == 0 && lane == 0) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_b); tma_prefetch_desc(&tm_out); }
   if (warp == 1) {  // this warp owns the tensor-memory allocation
-    tmem_alloc(base + SmemLayout::tmem_slot, kTmemCols);
+    tmem_alloc(base + C::tmem_slot, kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -161,8 +217,8 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   };
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- producer
-    if (lane == 0) {
+    // ------------------------------------------------- producer of packed slabs
+    if (kAnyPacked && lane == 0) {
       uint32_t it = 0;
       bool ok = true;
       for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
@@ -171,28 +227,72 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int m0 = (tile % p.tiles_m) * BM;
         const int n0 = (tile / p.tiles_m) * BN;
         for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
-          const int s = it % kPackedStages;
-          const uint32_t ph = (it / kPackedStages) & 1u;
+          const int s = it % (PS > 0 ? PS : 1);
+          const uint32_t ph = (it / (PS > 0 ? PS : 1)) & 1u;
           if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag)) { ok = false; break; }
           const int sample = k_it / p.num_kb;
           const int kb = k_it - sample * p.num_kb;
-          const uint32_t dst = base + SmemLayout::packed + s * kPackedStage;
-          mbar_arrive_expect_tx(pk_full(s), kPackedStage);
-          if constexpr (A_MN) tma_load_3d(dst, &tm_a, pk_full(s), m0 / 2, kb * BK, sample);
-          else tma_load_3d(dst, &tm_a, pk_full(s), kb * (BK / 2), m0, sample);
+          const uint32_t dst = base + C::packed + s * C::packed_stage;
+          mbar_arrive_expect_tx(pk_full(s), C::packed_stage);
+          if constexpr (!A_PLANE) {
+            if constexpr (A_MN) tma_load_3d(dst, &tm_a, pk_full(s), m0 / 2, kb * BK, sample);
+            else tma_load_3d(dst, &tm_a, pk_full(s), kb * (BK / 2), m0, sample);
+          }
+          if constexpr (!B_PLANE) {
 #pragma unroll
-          for (int j = 0; j < BN / 128; ++j) {
-            if constexpr (B_MN) tma_load_2d(dst + (1 + j) * kPackedSlab, &tm_b, pk_full(s), n0 / 2 + 64 * j, kb * BK);
-            else tma_load_2d(dst + (1 + j) * kPackedSlab, &tm_b, pk_full(s), kb * (BK / 2), n0 + 128 * j);
+            for (int j = 0; j < BN / 128; ++j) {
+              const uint32_t d = dst + C::b_packed_off + j * kPackedSlab;
+              if constexpr (B_MN) tma_load_2d(d, &tm_b, pk_full(s), n0 / 2 + 64 * j, kb * BK);
+              else tma_load_2d(d, &tm_b, pk_full(s), kb * (BK / 2), n0 + 128 * j);
+            }
           }
         }
       }
       // drain: every copy this thread issued must have landed before the CTA may exit
       const uint32_t issued = it;
-      for (int s = 0; s < kPackedStages; ++s) {
+      for (int s = 0; s < PS; ++s) {
         if (issued > static_cast<uint32_t>(s)) {
-          const uint32_t last = ((issued - 1 - s) / kPackedStages);  // last fill index of stage s
+          const uint32_t last = ((issued - 1 - s) / (PS > 0 ? PS : 1));  // last fill index of stage s
           mbar_wait(pk_full(s), last & 1u, abort_flag);
+        }
+      }
+    }
+  } else if (warp == kPlaneWarp) {
+    // ------------------------------------------------ producer of operand planes
+    if (kAnyPlane && lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
+        int tile, it_begin, it_end;
+        unit_range(u, tile, it_begin, it_end);
+        const int m0 = (tile % p.tiles_m) * BM;
+        const int n0 = (tile / p.tiles_m) * BN;
+        for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
+          const int s = it % ES;
+          if (!mbar_wait(ex_empty(s), ((it / ES) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          const int sample = k_it / p.num_kb;
+          const int kb = k_it - sample * p.num_kb;
+          const uint32_t dst = base + C::expanded + s * kExpandedStage;
+          mbar_arrive_expect_tx(ex_full(s), C::plane_bytes);
+          if constexpr (A_PLANE) {
+            if constexpr (A_MN) tma_load_3d(dst, &tm_a, ex_full(s), m0, kb * BK, sample);
+            else tma_load_3d(dst, &tm_a, ex_full(s), kb * BK, m0, sample);
+          }
+          if constexpr (B_PLANE) {
+#pragma unroll
+            for (int j = 0; j < BN / 128; ++j) {
+              const uint32_t d = dst + (1 + j) * kExpandedSlab;
+              if constexpr (B_MN) tma_load_2d(d, &tm_b, ex_full(s), n0 + 128 * j, kb * BK);
+              else tma_load_2d(d, &tm_b, ex_full(s), kb * BK, n0 + 128 * j);
+            }
+          }
+        }
+      }
+      const uint32_t issued = it;
+      for (int s = 0; s < ES; ++s) {
+        if (issued > static_cast<uint32_t>(s)) {
+          const uint32_t last = ((issued - 1 - s) / ES);
+          mbar_wait(ex_full(s), last & 1u, abort_flag);
         }
       }
     }
@@ -214,10 +314,10 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + buf * BN;
         for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
-          const int s = it % kExpandedStages;
-          if (!mbar_wait(ex_full(s), (it / kExpandedStages) & 1u, abort_flag)) { ok = false; break; }
+          const int s = it % ES;
+          if (!mbar_wait(ex_full(s), (it / ES) & 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_base = base + SmemLayout::expanded + s * kExpandedStage;
+          const uint32_t a_base = base + C::expanded + s * kExpandedStage;
           const uint32_t b_base = a_base + kExpandedSlab;
 #pragma unroll
           for (int kk = 0; kk < BK / 32; ++kk) {
@@ -232,12 +332,12 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (ok) tc_commit(acc_full(buf));
       }
     }
-  } else if (warp < kFirstConvWarp) {
+  } else if (warp < kPlaneWarp) {
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;  // tensor-memory lanes this warp may read
     const float scale = p.splits == 1 ? (__ldg(p.scale_a) * __ldg(p.scale_b)) * p.post_scale : 1.0f;
-    const uint32_t stage0 = base + SmemLayout::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
-    uint8_t* const stage0_gen = gen + SmemLayout::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
+    const uint32_t stage0 = base + C::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
+    uint8_t* const stage0_gen = gen + C::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
     const int sw = lane & 7;
     uint32_t tile_it = 0, box_it = 0;
     bool ok = true;
@@ -254,11 +354,8 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (!mbar_wait(acc_full(buf), (tile_it >> 1) & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld_32x32(taddr + c * 32, r);
-        tmem_ld_wait();
+      // scale one 32 x 32 block held in registers, stage it (swizzled) and hand it to the TMA store
+      auto emit = [&](const uint32_t (&r)[32], int c) {
         const long long col0 = col_base + c * 32;
         if (row0 < row_limit && col0 < col_limit) {   // warp-uniform
           const uint32_t b = box_it & 1u;
@@ -286,13 +383,36 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             bulk_commit();
           }
         }
+      };
+      if constexpr (C::epi_double) {
+        // two register sets: the tensor-memory load of the next block is in flight while this one is emitted
+        uint32_t r0[32], r1[32];
+        tmem_ld_32x32(taddr, r0);
+        tmem_ld_wait();
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; c += 2) {
+          tmem_ld_32x32(taddr + (c + 1) * 32, r1);
+          emit(r0, c);
+          tmem_ld_wait();
+          if (c + 2 < BN / 32) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
+          emit(r1, c + 1);
+          tmem_ld_wait();
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32(taddr + c * 32, r);
+          tmem_ld_wait();
+          emit(r, c);
+        }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty(buf));
     }
     if (lane == 0) bulk_wait<0>();   // all stores of this warp are complete before the CTA exits
-  } else {
+  } else if (kAnyPacked) {
     // -------------------------------------------------------------- converters
     const int ctid = threadIdx.x - kFirstConvWarp * 32;
     uint32_t it = 0;
@@ -301,37 +421,28 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       int tile, it_begin, it_end;
       unit_range(u, tile, it_begin, it_end);
       for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
-        const int ps = it % kPackedStages;
-        const int es = it % kExpandedStages;
-        if (!mbar_wait(pk_full(ps), (it / kPackedStages) & 1u, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(ex_empty(es), ((it / kExpandedStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-        const uint8_t* src = gen + SmemLayout::packed + ps * kPackedStage;
-        uint8_t* dst = gen + SmemLayout::expanded + es * kExpandedStage;
-        uint4 w[kSlabs * 512 / kConvThreads];
+        const int ps = it % (PS > 0 ? PS : 1);
+        const int es = it % ES;
+        if (!mbar_wait(pk_full(ps), (it / (PS > 0 ? PS : 1)) & 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(ex_empty(es), ((it / ES) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        const uint8_t* src = gen + C::packed + ps * C::packed_stage;
+        uint8_t* dst = gen + C::expanded + es * kExpandedStage;
+        constexpr int kTasks = C::tasks_per_thread > 0 ? C::tasks_per_thread : 1;
+        uint4 w[kTasks];
 #pragma unroll
-        for (int j = 0; j < kSlabs * 512 / kConvThreads; ++j)
+        for (int j = 0; j < C::tasks_per_thread; ++j)
           w[j] = *reinterpret_cast<const uint4*>(src + (ctid + j * kConvThreads) * 16);
 #pragma unroll
-        for (int j = 0; j < kSlabs * 512 / kConvThreads; ++j) {
+        for (int j = 0; j < C::tasks_per_thread; ++j) {
           const int id = ctid + j * kConvThreads;
-          const int slab = id >> 9;           // compile-time per j
+          const int pslab = id >> 9;                         // slab inside the packed stage, compile-time per j
+          const int slab = A_PLANE ? pslab + 1 : pslab;      // slab inside the operand stage (0 = A)
           const int idx = id & 511;
           const int row = idx >> 2;
           const int q = idx & 3;
           uint4 o0, o1;
-          const bool is_a = slab == 0;
-          if (KIND == 1 && !(is_a && A_LUQ)) {
-            expand8_int4_x16<kPermuteK>(w[j].x, o0.x, o0.y);
-            expand8_int4_x16<kPermuteK>(w[j].y, o0.z, o0.w);
-            expand8_int4_x16<kPermuteK>(w[j].z, o1.x, o1.y);
-            expand8_int4_x16<kPermuteK>(w[j].w, o1.z, o1.w);
-          } else {
-            const uint4 lut = is_a ? p.lut_a : p.lut_b;
-            expand8_lut(w[j].x, lut, o0.x, o0.y);
-            expand8_lut(w[j].y, lut, o0.z, o0.w);
-            expand8_lut(w[j].z, lut, o1.x, o1.y);
-            expand8_lut(w[j].w, lut, o1.z, o1.w);
-          }
+          if (slab == 0) expand32<KIND, A_LUQ, kPermuteK>(w[j], p.lut_a, o0, o1);
+          else expand32<KIND, false, kPermuteK>(w[j], p.lut_b, o0, o1);
           uint8_t* drow = dst + slab * kExpandedSlab + row * 128;
           const int swz = row & 7;
           *reinterpret_cast<uint4*>(drow + (((2 * q) ^ swz) << 4)) = o0;
@@ -413,17 +524,18 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// packed-code tensor: `planes` x `rows` x `pitch` bytes, box = 1 x 128 rows x 64 bytes
-int encode_codes_map(void* fn, CUtensorMap* map, const uint8_t* ptr, uint64_t pitch, uint64_t rows, uint64_t planes,
-                     bool three_d) {
+// byte tensor `planes` x `rows` x `pitch` bytes.  Packed codes: box 1 x 128 rows x 64 bytes, no
+// swizzle.  Operand planes: box 1 x 128 rows x 128 bytes, 128-byte swizzle (the tensor core's layout).
+int encode_bytes_map(void* fn, CUtensorMap* map, const uint8_t* ptr, uint64_t pitch, uint64_t rows, uint64_t planes,
+                     bool three_d, bool operand_plane) {
   const cuuint64_t dims[3] = {pitch, rows, planes};
   const cuuint64_t strides[2] = {pitch, pitch * rows};
-  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t box[3] = {operand_plane ? 128u : 64u, 128, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
       map, CU_TENSOR_MAP_DATA_TYPE_UINT8, three_d ? 3 : 2, const_cast<uint8_t*>(ptr), dims, strides, box, estr,
-      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      CU_TENSOR_MAP_INTERLEAVE_NONE, operand_plane ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : 1;
 }
 // fp32 output (or workspace) tensor rows x cols, box = 32 rows x 32 columns, 128-byte swizzle in shared memory
@@ -438,20 +550,48 @@ int encode_out_map(void* fn, CUtensorMap* map, float* ptr, uint64_t rows, uint64
   return r == CUDA_SUCCESS ? 0 : 1;
 }
 
-template <int KIND, bool A_MN, bool B_MN, bool A_LUQ>
+template <int KIND, bool A_MN, bool B_MN, bool A_LUQ, bool A_PLANE, bool B_PLANE>
 int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmParams& p, int grid,
            cudaStream_t st) {
-  auto kernel = luq_gemm_kernel<KIND, A_MN, B_MN, A_LUQ>;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  auto kernel = luq_gemm_kernel<KIND, A_MN, B_MN, A_LUQ, A_PLANE, B_PLANE>;
+  constexpr int smem = Cfg<A_PLANE, B_PLANE>::smem_bytes;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return static_cast<int>(e);
-  kernel<<<grid, kThreads, kSmemBytes, st>>>(ta, tb, to, p);
+  kernel<<<grid, Cfg<A_PLANE, B_PLANE>::threads, smem, st>>>(ta, tb, to, p);
   return static_cast<int>(cudaGetLastError());
 }
 
+template <int KIND, bool A_MN, bool B_MN, bool A_LUQ>
+int launch_planes(bool a_plane, bool b_plane, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
+                  const GemmParams& p, int grid, cudaStream_t st) {
+  if (a_plane && b_plane) return launch<KIND, A_MN, B_MN, A_LUQ, true, true>(ta, tb, to, p, grid, st);
+  if (a_plane) return launch<KIND, A_MN, B_MN, A_LUQ, true, false>(ta, tb, to, p, grid, st);
+  if (b_plane) return launch<KIND, A_MN, B_MN, A_LUQ, false, true>(ta, tb, to, p, grid, st);
+  return launch<KIND, A_MN, B_MN, A_LUQ, false, false>(ta, tb, to, p, grid, st);
+}
+
+template <int KIND>
+int launch_expand(bool luq_codes, const uint8_t* codes, uint8_t* plane, size_t packed_bytes, const uint4& lut, int sms,
+                  cudaStream_t st) {
+  const size_t pieces = packed_bytes / 16;
+  size_t blocks = (pieces + 255) / 256;
+  const size_t cap = static_cast<size_t>(sms) * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  if (luq_codes)
+    expand_plane_kernel<KIND, true><<<static_cast<int>(blocks), 256, 0, st>>>(
+        reinterpret_cast<const uint4*>(codes), reinterpret_cast<uint4*>(plane), pieces, lut);
+  else
+    expand_plane_kernel<KIND, false><<<static_cast<int>(blocks), 256, 0, st>>>(
+        reinterpret_cast<const uint4*>(codes), reinterpret_cast<uint4*>(plane), pieces, lut);
+  return static_cast<int>(cudaGetLastError());
+}
+
+constexpr size_t kSplitRegionBytes = 20u << 20;   // the first 20 MiB of a workspace hold split partial tiles
+
 }  // namespace
 
-int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
-  if (a.Mo <= 0 || a.No <= 0 || a.Kc <= 0) return 0;
+static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
   GemmParams p{};
   p.scale_a = a.d_scale_a; p.scale_b = a.d_scale_b; p.status = ctx->d_status;
   p.Mo = a.Mo; p.No = a.No; p.Kc = a.Kc;
@@ -459,20 +599,6 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
   p.tiles_m = static_cast<int>((a.Mo + BM - 1) / BM);
   p.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
   p.num_kb = static_cast<int>((a.Kc + BK - 1) / BK);
-  p.lut_a = make_lut(ctx->mma_kind, a.a_kind);
-  p.lut_b = make_lut(ctx->mma_kind, a.b_kind);
-  // int8 operands carry INT4 integers as 16*q: undo with an exact power of two
-  float pow2 = 1.0f;
-  long long worst = 1;   // largest |operand product| as fed to the tensor core
-  if (ctx->mma_kind == 1) {
-    const int a_mag = a.a_kind == 0 ? 7 * 16 : 64, b_mag = a.b_kind == 0 ? 7 * 16 : 64;
-    if (a.a_kind == 0) pow2 *= 1.0f / 16.0f;
-    if (a.b_kind == 0) pow2 *= 1.0f / 16.0f;
-    worst = static_cast<long long>(a_mag) * b_mag;
-    if (worst * a.Kc * a.n_samples >= (1ll << 31)) return LUQ_ERR_ARG;  // the int32 accumulator could wrap
-  }
-  p.post_scale = (1.0f / static_cast<float>(a.n_samples)) * pow2;
-
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const int total_iters = p.n_samples * p.num_kb;
   int splits = 1;
@@ -485,38 +611,96 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
   }
   p.iters_per_split = (total_iters + splits - 1) / splits;
   p.splits = (total_iters + p.iters_per_split - 1) / p.iters_per_split;  // no empty split
-  const long long units = tiles * p.splits;
+  const size_t split_region = a.workspace_bytes < kSplitRegionBytes ? a.workspace_bytes : kSplitRegionBytes;
   if (p.splits > 1) {
-    const size_t need = static_cast<size_t>(units) * kTileFloats * sizeof(float);
-    if (a.d_workspace == nullptr || need > a.workspace_bytes) {
+    const size_t need = static_cast<size_t>(tiles * p.splits) * kTileFloats * sizeof(float);
+    if (a.d_workspace == nullptr || need > split_region) {
       if (ctx->forced_splits > 0) return LUQ_ERR_WORKSPACE;
       p.splits = 1;
       p.iters_per_split = total_iters;
     }
   }
-  const long long units_final = tiles * p.splits;
+  const long long units = tiles * p.splits;
+
+  // Operand planes: an operand that at least two tiles re-read is expanded once, if the
+  // workspace behind the split region has room for it.  A product with a short contraction
+  // is bound by its output stream and hides the in-kernel expansion completely (measured:
+  // the backward product of the ResNet shape, 2 blocks per tile), so it keeps the codes.
+  const size_t a_plane_bytes = static_cast<size_t>(a.Mo) * a.Kc * a.n_samples;
+  const size_t b_plane_bytes = static_cast<size_t>(a.No) * a.Kc;
+  size_t plane_room = (a.d_workspace && a.workspace_bytes > kSplitRegionBytes) ? a.workspace_bytes - kSplitRegionBytes : 0;
+  uint8_t* plane_ptr = a.d_workspace ? reinterpret_cast<uint8_t*>(a.d_workspace) + kSplitRegionBytes : nullptr;
+  auto packed_ok = [](size_t bytes) { return bytes % 32 == 0; };   // whole 16-byte pieces of packed codes
+  bool b_plane = false, a_plane = false;
+  const bool long_contraction = total_iters >= 8;
+  uint8_t* b_plane_ptr = nullptr; uint8_t* a_plane_ptr = nullptr;
+  if (long_contraction && p.tiles_m >= 2 && packed_ok(b_plane_bytes) && b_plane_bytes <= plane_room) {
+    b_plane = true; b_plane_ptr = plane_ptr;
+    const size_t used = (b_plane_bytes + 1023) & ~static_cast<size_t>(1023);
+    plane_ptr += used; plane_room -= used <= plane_room ? used : plane_room;
+  }
+  if (long_contraction && p.tiles_n >= 2 && packed_ok(a_plane_bytes) && a_plane_bytes <= plane_room) {
+    a_plane = true; a_plane_ptr = plane_ptr;
+  }
+  // Operand type.  "Automatic" takes int8 whenever an INT4 operand is expanded inside the
+  // kernel (three instructions per eight codes instead of a table lookup) and e4m3 when both
+  // operands arrive as planes (fp32 accumulators spare the epilogue the int-to-float conversions).
+  if (ctx->mma_kind == 2) ctx->mma_kind = (a_plane && b_plane) ? 0 : 1;
+  p.lut_a = make_lut(ctx->mma_kind, a.a_kind);
+  p.lut_b = make_lut(ctx->mma_kind, a.b_kind);
+  // int8 operands carry INT4 integers as 16*q: undo with an exact power of two
+  float pow2 = 1.0f;
+  if (ctx->mma_kind == 1) {
+    const int a_mag = a.a_kind == 0 ? 7 * 16 : 64, b_mag = a.b_kind == 0 ? 7 * 16 : 64;
+    if (a.a_kind == 0) pow2 *= 1.0f / 16.0f;
+    if (a.b_kind == 0) pow2 *= 1.0f / 16.0f;
+    const long long worst = static_cast<long long>(a_mag) * b_mag;   // largest |operand product|
+    if (worst * a.Kc * a.n_samples >= (1ll << 31)) return LUQ_ERR_ARG;  // the int32 accumulator could wrap
+  }
+  p.post_scale = (1.0f / static_cast<float>(a.n_samples)) * pow2;
+
+  int rc = 0;
+  if (b_plane) {
+    rc = ctx->mma_kind ? launch_expand<1>(a.b_kind == 1, a.b_codes, b_plane_ptr, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st)
+                       : launch_expand<0>(a.b_kind == 1, a.b_codes, b_plane_ptr, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st);
+    if (rc != 0) return rc;
+    ctx->launches += 1;
+  }
+  if (a_plane) {
+    rc = ctx->mma_kind ? launch_expand<1>(a.a_kind == 1, a.a_codes, a_plane_ptr, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st)
+                       : launch_expand<0>(a.a_kind == 1, a.a_codes, a_plane_ptr, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st);
+    if (rc != 0) return rc;
+    ctx->launches += 1;
+  }
 
   CUtensorMap ta, tb, to;
   int bad = 0;
-  if (a.a_mn) bad |= encode_codes_map(ctx->encode_tiled, &ta, a.a_codes, a.Mo / 2, a.Kc, a.n_samples, true);
-  else bad |= encode_codes_map(ctx->encode_tiled, &ta, a.a_codes, a.Kc / 2, a.Mo, a.n_samples, true);
-  if (a.b_mn) bad |= encode_codes_map(ctx->encode_tiled, &tb, a.b_codes, a.No / 2, a.Kc, 1, false);
-  else bad |= encode_codes_map(ctx->encode_tiled, &tb, a.b_codes, a.Kc / 2, a.No, 1, false);
-  if (p.splits > 1) bad |= encode_out_map(ctx->encode_tiled, &to, a.d_workspace, units_final * BM, BN);
+  {
+    const uint8_t* ptr = a_plane ? a_plane_ptr : a.a_codes;
+    const uint64_t div = a_plane ? 1 : 2;   // bytes per row: elements (plane) or elements / 2 (codes)
+    if (a.a_mn) bad |= encode_bytes_map(ctx->encode_tiled, &ta, ptr, a.Mo / div, a.Kc, a.n_samples, true, a_plane);
+    else bad |= encode_bytes_map(ctx->encode_tiled, &ta, ptr, a.Kc / div, a.Mo, a.n_samples, true, a_plane);
+  }
+  {
+    const uint8_t* ptr = b_plane ? b_plane_ptr : a.b_codes;
+    const uint64_t div = b_plane ? 1 : 2;
+    if (a.b_mn) bad |= encode_bytes_map(ctx->encode_tiled, &tb, ptr, a.No / div, a.Kc, 1, false, b_plane);
+    else bad |= encode_bytes_map(ctx->encode_tiled, &tb, ptr, a.Kc / div, a.No, 1, false, b_plane);
+  }
+  if (p.splits > 1) bad |= encode_out_map(ctx->encode_tiled, &to, a.d_workspace, units * BM, BN);
   else bad |= encode_out_map(ctx->encode_tiled, &to, a.d_out, a.Mo, a.No);
   if (bad) return LUQ_ERR_CUDA;
 
-  const int grid = static_cast<int>(units_final < ctx->sm_count ? units_final : ctx->sm_count);
-  int rc;
+  const int grid = static_cast<int>(units < ctx->sm_count ? units : ctx->sm_count);
   const int sel = (ctx->mma_kind ? 4 : 0) | (a.a_mn ? 2 : 0) | (a.b_mn ? 1 : 0);
   if (a.b_kind != 0 || (a.a_kind == 1) != (sel & 3 ? true : false)) return LUQ_ERR_UNSUPPORTED;
   switch (sel) {
-    case 0: rc = launch<0, false, false, false>(ta, tb, to, p, grid, st); break;
-    case 1: rc = launch<0, false, true, true>(ta, tb, to, p, grid, st); break;
-    case 3: rc = launch<0, true, true, true>(ta, tb, to, p, grid, st); break;
-    case 4: rc = launch<1, false, false, false>(ta, tb, to, p, grid, st); break;
-    case 5: rc = launch<1, false, true, true>(ta, tb, to, p, grid, st); break;
-    case 7: rc = launch<1, true, true, true>(ta, tb, to, p, grid, st); break;
+    case 0: rc = launch_planes<0, false, false, false>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
+    case 1: rc = launch_planes<0, false, true, true>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
+    case 3: rc = launch_planes<0, true, true, true>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
+    case 4: rc = launch_planes<1, false, false, false>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
+    case 5: rc = launch_planes<1, false, true, true>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
+    case 7: rc = launch_planes<1, true, true, true>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
     default: return LUQ_ERR_UNSUPPORTED;
   }
   if (rc != 0) return rc;
@@ -531,6 +715,16 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st) {
   }
   return rc;
 }
+
+int luq_launch_gemm(luq_ctx* ctx_in, const luq_gemm_args& a, cudaStream_t st) {
+  if (a.Mo <= 0 || a.No <= 0 || a.Kc <= 0) return 0;
+  luq_ctx ctx_copy = *ctx_in;            // the operand type may be chosen per product below
+  luq_ctx* ctx = &ctx_copy;
+  const int rc_all = luq_launch_gemm_impl(ctx, a, st);
+  ctx_in->launches = ctx->launches;
+  return rc_all;
+}
+
 
 // ---------------------------------------------------------------------------
 // Update GEMM for callers that must not allocate device memory.

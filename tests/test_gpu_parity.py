@@ -231,7 +231,7 @@ SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("mma_kind", [0, 1])
+@pytest.mark.parametrize("mma_kind", [0, 1, 2])
 @pytest.mark.parametrize("M,K,N,ns", SHAPES)
 def test_three_gemms_match_oracle(ctx, M, K, N, ns, mma_kind):
     ctx.set_option(binding.OPT_MMA_KIND, mma_kind)
@@ -243,7 +243,7 @@ def test_three_gemms_match_oracle(ctx, M, K, N, ns, mma_kind):
         assert_gemm_close(dA.cpu().numpy(), oracle.gemm_bwd(og, oal, ns, ow, osw, M, N, K))
         assert_gemm_close(dW.cpu().numpy(), oracle.gemm_wgrad(og, oal, ns, oa, osa, M, N, K))
     finally:
-        ctx.set_option(binding.OPT_MMA_KIND, 1)
+        ctx.set_option(binding.OPT_MMA_KIND, 2)
 
 
 @pytest.mark.parametrize("splits", [1, 2, 5])
@@ -282,7 +282,7 @@ def test_gemm_large_integer_sums_are_exact(ctx):
     a = torch.full((M, K // 2), 0x77, dtype=torch.uint8, device="cuda")     # all +7
     w = torch.full((N, K // 2), 0x77, dtype=torch.uint8, device="cuda")
     w[1::2] = 0x99                                                           # odd rows all -7
-    for kind in (0, 1):
+    for kind in (0, 1, 2):
         ctx.set_option(binding.OPT_MMA_KIND, kind)
         Z = ctx.gemm_fwd(a, scalar(1.0), w, scalar(1.0), M, N, K).cpu().numpy()
         assert (Z[:, 0::2] == 49 * K).all() and (Z[:, 1::2] == -49 * K).all()
@@ -296,7 +296,7 @@ def test_gemm_large_integer_sums_are_exact(ctx):
         wk = torch.full((K, N // 2), 0x77, dtype=torch.uint8, device="cuda")
         dA = ctx.gemm_bwd(g, scalar(1.0), 1, wk, scalar(1.0), M, K, N).cpu().numpy()
         assert (dA == 16 * 7 * K).all()
-    ctx.set_option(binding.OPT_MMA_KIND, 1)
+    ctx.set_option(binding.OPT_MMA_KIND, 2)
     assert ctx.status() == 0
 
 
