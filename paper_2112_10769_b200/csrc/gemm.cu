@@ -219,37 +219,40 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   if (warp == 0) {
     // ------------------------------------------------- producer of packed slabs
     if (kAnyPacked && lane == 0) {
-      uint32_t it = 0;
+      // stage index and phase are counted, not divided: this loop is one thread's serial
+      // instruction stream and must stay well below the time of a stage
+      uint32_t issued = 0, stage = 0, phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
         int tile, it_begin, it_end;
         unit_range(u, tile, it_begin, it_end);
         const int m0 = (tile % p.tiles_m) * BM;
         const int n0 = (tile / p.tiles_m) * BN;
-        for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
-          const int s = it % (PS > 0 ? PS : 1);
-          const uint32_t ph = (it / (PS > 0 ? PS : 1)) & 1u;
-          if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const int sample = k_it / p.num_kb;
-          const int kb = k_it - sample * p.num_kb;
-          const uint32_t dst = base + C::packed + s * C::packed_stage;
-          mbar_arrive_expect_tx(pk_full(s), C::packed_stage);
+        int sample = it_begin / p.num_kb;
+        int kb = it_begin - sample * p.num_kb;
+        for (int k_it = it_begin; k_it < it_end; ++k_it) {
+          const uint32_t full = pk_full(stage);
+          if (!mbar_wait(pk_empty(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t dst = base + C::packed + stage * C::packed_stage;
+          mbar_arrive_expect_tx(full, C::packed_stage);
           if constexpr (!A_PLANE) {
-            if constexpr (A_MN) tma_load_3d(dst, &tm_a, pk_full(s), m0 / 2, kb * BK, sample);
-            else tma_load_3d(dst, &tm_a, pk_full(s), kb * (BK / 2), m0, sample);
+            if constexpr (A_MN) tma_load_3d(dst, &tm_a, full, m0 / 2, kb * BK, sample);
+            else tma_load_3d(dst, &tm_a, full, kb * (BK / 2), m0, sample);
           }
           if constexpr (!B_PLANE) {
 #pragma unroll
             for (int j = 0; j < BN / 128; ++j) {
               const uint32_t d = dst + C::b_packed_off + j * kPackedSlab;
-              if constexpr (B_MN) tma_load_2d(d, &tm_b, pk_full(s), n0 / 2 + 64 * j, kb * BK);
-              else tma_load_2d(d, &tm_b, pk_full(s), kb * (BK / 2), n0 + 128 * j);
+              if constexpr (B_MN) tma_load_2d(d, &tm_b, full, n0 / 2 + 64 * j, kb * BK);
+              else tma_load_2d(d, &tm_b, full, kb * (BK / 2), n0 + 128 * j);
             }
           }
+          ++issued;
+          if (++kb == p.num_kb) { kb = 0; ++sample; }
+          if (++stage == static_cast<uint32_t>(PS)) { stage = 0; phase ^= 1u; }
         }
       }
       // drain: every copy this thread issued must have landed before the CTA may exit
-      const uint32_t issued = it;
       for (int s = 0; s < PS; ++s) {
         if (issued > static_cast<uint32_t>(s)) {
           const uint32_t last = ((issued - 1 - s) / (PS > 0 ? PS : 1));  // last fill index of stage s
@@ -260,35 +263,37 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   } else if (warp == kPlaneWarp) {
     // ------------------------------------------------ producer of operand planes
     if (kAnyPlane && lane == 0) {
-      uint32_t it = 0;
+      uint32_t issued = 0, stage = 0, phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
         int tile, it_begin, it_end;
         unit_range(u, tile, it_begin, it_end);
         const int m0 = (tile % p.tiles_m) * BM;
         const int n0 = (tile / p.tiles_m) * BN;
-        for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
-          const int s = it % ES;
-          if (!mbar_wait(ex_empty(s), ((it / ES) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          const int sample = k_it / p.num_kb;
-          const int kb = k_it - sample * p.num_kb;
-          const uint32_t dst = base + C::expanded + s * kExpandedStage;
-          mbar_arrive_expect_tx(ex_full(s), C::plane_bytes);
+        int sample = it_begin / p.num_kb;
+        int kb = it_begin - sample * p.num_kb;
+        for (int k_it = it_begin; k_it < it_end; ++k_it) {
+          const uint32_t full = ex_full(stage);
+          if (!mbar_wait(ex_empty(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t dst = base + C::expanded + stage * kExpandedStage;
+          mbar_arrive_expect_tx(full, C::plane_bytes);
           if constexpr (A_PLANE) {
-            if constexpr (A_MN) tma_load_3d(dst, &tm_a, ex_full(s), m0, kb * BK, sample);
-            else tma_load_3d(dst, &tm_a, ex_full(s), kb * BK, m0, sample);
+            if constexpr (A_MN) tma_load_3d(dst, &tm_a, full, m0, kb * BK, sample);
+            else tma_load_3d(dst, &tm_a, full, kb * BK, m0, sample);
           }
           if constexpr (B_PLANE) {
 #pragma unroll
             for (int j = 0; j < BN / 128; ++j) {
               const uint32_t d = dst + (1 + j) * kExpandedSlab;
-              if constexpr (B_MN) tma_load_2d(d, &tm_b, ex_full(s), n0 + 128 * j, kb * BK);
-              else tma_load_2d(d, &tm_b, ex_full(s), kb * BK, n0 + 128 * j);
+              if constexpr (B_MN) tma_load_2d(d, &tm_b, full, n0 + 128 * j, kb * BK);
+              else tma_load_2d(d, &tm_b, full, kb * BK, n0 + 128 * j);
             }
           }
+          ++issued;
+          if (++kb == p.num_kb) { kb = 0; ++sample; }
+          if (++stage == static_cast<uint32_t>(ES)) { stage = 0; phase ^= 1u; }
         }
       }
-      const uint32_t issued = it;
       for (int s = 0; s < ES; ++s) {
         if (issued > static_cast<uint32_t>(s)) {
           const uint32_t last = ((issued - 1 - s) / ES);
@@ -304,7 +309,14 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                                  | ((KIND == 0 ? 0u : 1u) << 10)            // B: E4M3 / signed 8-bit
                                  | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16)
                                  | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
-      uint32_t it = 0, tile_it = 0;
+      // descriptors of stage 0; a stage or a 32-deep step further only moves the 14-bit
+      // address field (shared memory is below 256 KB, the field cannot carry out)
+      const uint32_t a0 = base + C::expanded, b0 = a0 + kExpandedSlab;
+      const uint64_t da0 = A_MN ? umma_desc_sw128(a0, kExpandedSlab, 1024) : umma_desc_sw128(a0, 16, 1024);
+      const uint64_t db0 = B_MN ? umma_desc_sw128(b0, kExpandedSlab, 1024) : umma_desc_sw128(b0, 16, 1024);
+      constexpr uint64_t kStepA = (A_MN ? 32 * 128 : 32) >> 4, kStepB = (B_MN ? 32 * 128 : 32) >> 4;
+      constexpr uint64_t kStageStep = kExpandedStage >> 4;
+      uint32_t stage = 0, phase = 0, tile_it = 0;
       bool ok = true;
       for (int u = blockIdx.x; ok && u < units; u += gridDim.x, ++tile_it) {
         int tile, it_begin, it_end;
@@ -313,21 +325,18 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (!mbar_wait(acc_empty(buf), ((tile_it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + buf * BN;
-        for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
-          const int s = it % ES;
-          if (!mbar_wait(ex_full(s), (it / ES) & 1u, abort_flag)) { ok = false; break; }
+        uint32_t accumulate = 0;
+        for (int k_it = it_begin; k_it < it_end; ++k_it) {
+          if (!mbar_wait(ex_full(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_base = base + C::expanded + s * kExpandedStage;
-          const uint32_t b_base = a_base + kExpandedSlab;
+          const uint64_t da = da0 + stage * kStageStep, db = db0 + stage * kStageStep;
 #pragma unroll
           for (int kk = 0; kk < BK / 32; ++kk) {
-            const uint64_t da = A_MN ? umma_desc_sw128(a_base + kk * 32 * 128, kExpandedSlab, 1024)
-                                     : umma_desc_sw128(a_base + kk * 32, 16, 1024);
-            const uint64_t db = B_MN ? umma_desc_sw128(b_base + kk * 32 * 128, kExpandedSlab, 1024)
-                                     : umma_desc_sw128(b_base + kk * 32, 16, 1024);
-            tc_mma<KIND>(tmem_d, da, db, idesc, (k_it > it_begin || kk > 0) ? 1u : 0u);
+            tc_mma<KIND>(tmem_d, da + kk * kStepA, db + kk * kStepB, idesc, accumulate);
+            accumulate = 1;
           }
-          tc_commit(ex_empty(s));
+          tc_commit(ex_empty(stage));
+          if (++stage == static_cast<uint32_t>(ES)) { stage = 0; phase ^= 1u; }
         }
         if (ok) tc_commit(acc_full(buf));
       }
@@ -415,16 +424,14 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   } else if (kAnyPacked) {
     // -------------------------------------------------------------- converters
     const int ctid = threadIdx.x - kFirstConvWarp * 32;
-    uint32_t it = 0;
+    uint32_t ps = 0, pphase = 0, es = 0, ephase = 0;
     bool ok = true;
     for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
       int tile, it_begin, it_end;
       unit_range(u, tile, it_begin, it_end);
-      for (int k_it = it_begin; k_it < it_end; ++k_it, ++it) {
-        const int ps = it % (PS > 0 ? PS : 1);
-        const int es = it % ES;
-        if (!mbar_wait(pk_full(ps), (it / (PS > 0 ? PS : 1)) & 1u, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(ex_empty(es), ((it / ES) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      for (int k_it = it_begin; k_it < it_end; ++k_it) {
+        if (!mbar_wait(pk_full(ps), pphase, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(ex_empty(es), ephase ^ 1u, abort_flag)) { ok = false; break; }
         const uint8_t* src = gen + C::packed + ps * C::packed_stage;
         uint8_t* dst = gen + C::expanded + es * kExpandedStage;
         constexpr int kTasks = C::tasks_per_thread > 0 ? C::tasks_per_thread : 1;
@@ -451,6 +458,8 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         fence_proxy_async();   // make the generic-proxy writes visible to the tensor core
         __syncwarp();
         if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive(ex_full(es)); }
+        if (++ps == static_cast<uint32_t>(PS > 0 ? PS : 1)) { ps = 0; pphase ^= 1u; }
+        if (++es == static_cast<uint32_t>(ES)) { es = 0; ephase ^= 1u; }
       }
     }
   }
