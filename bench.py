@@ -36,9 +36,11 @@ WORKLOAD = "cfg2"
 KERNELS = ("amax_A", "amax_W", "quant_int4_A", "quant_int4_W", "gemm_fwd",
            "amax_G", "quant_grad_G", "gemm_bwd", "gemm_wgrad")
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
-# summarised under profiles/ (None until a capture of that kernel exists).
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the cfg2 kernels, from the ncu
+# capture summarised in profiles/kernels_cfg2_full_size.md (other workloads: None).
+NCU_TRAFFIC_BYTES = {"amax_A": 466.7e6, "quant_int4_A": 511.9e6, "gemm_fwd": 65.1e6, "amax_G": 51.4e6,
+                     "quant_grad_G": 51.5e6, "gemm_bwd": 420.9e6, "gemm_wgrad": 75.7e6, "amax_W": 2.4e6,
+                     "quant_int4_W": 2.4e6}
 
 
 def load_peaks():
@@ -325,7 +327,9 @@ def run_ours(args):
     dominant = max(per_kernel_ms, key=per_kernel_ms.get)
     d = kernels[dominant]
     roofline = {"kernel": dominant, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
-                "frac": d["frac"], "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+                "frac": d["frac"],
+                "traffic": NCU_TRAFFIC_BYTES.get(dominant) if (args.workload == "cfg2" and not args.rows) else None,
+                "algorithmic_bytes": alg[dominant][0], "algorithmic_flops": alg[dominant][1],
                 "peak_source": f"{peaks['source']}" + (" hbm copy" if d["bound"] == "hbm" else " bf16 sustained x2 (fp8)")}
 
     # ---- end to end: host buffers in, host buffers out, through the same calls
