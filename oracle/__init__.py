@@ -62,6 +62,10 @@ def lib() -> ctypes.CDLL:
             L.oracle_quant_luq_window.argtypes = [f32p, sz, ctypes.c_uint64, ctypes.c_float, ctypes.c_int,
                                                   ctypes.c_uint64, ctypes.c_int, u8p, intp]
             L.oracle_quant_luq_window.restype = ctypes.c_float
+            L.oracle_pw2_ceil.argtypes = [ctypes.c_float]
+            L.oracle_pw2_ceil.restype = ctypes.c_float
+            L.oracle_hindsight_next.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float]
+            L.oracle_hindsight_next.restype = ctypes.c_float
             L.oracle_luq_bins.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, f64p, f64p, u32p]
             L.oracle_dequant.argtypes = [u8p, sz, dbl, ctypes.c_int, f64p]
             L.oracle_gemm_fwd.argtypes = [u8p, dbl, u8p, dbl, i64, i64, i64, f64p]
@@ -141,6 +145,31 @@ def quant_luq(x: np.ndarray, mx, seed: int, n_samples: int = 1, kmax: int = KMAX
                                       seed & (2**64 - 1), n_samples, _ptr(codes, ctypes.c_uint8),
                                       ctypes.byref(flags))
     return codes, np.float32(a), flags.value
+
+
+def pw2_ceil(mx) -> np.float32:
+    """2^ceil(log2 mx): the maximum rounded up to a power of two (Appendix A.7)."""
+    return np.float32(lib().oracle_pw2_ceil(np.float32(mx)))
+
+
+def quant_luq_pw2(x: np.ndarray, mx, seed: int, n_samples: int = 1, kmax: int = KMAX_DEFAULT):
+    """LUQ_PW2: the same quantizer with alpha = 2^ceil(log2 max) / 2^kmax."""
+    return quant_luq(x, pw2_ceil(mx), seed, n_samples, kmax)
+
+
+def hindsight_next(measured_max, m_hat, eta) -> np.float32:
+    """m_hat for the next step: (1 - eta) * max|x| of this step + eta * m_hat of this step."""
+    return np.float32(lib().oracle_hindsight_next(np.float32(measured_max), np.float32(m_hat), np.float32(eta)))
+
+
+def quant_luq_hindsight(x: np.ndarray, m_hat, eta, seed: int, n_samples: int = 1, pw2: bool = False,
+                        kmax: int = KMAX_DEFAULT):
+    """One hindsight step: quantize x with the estimate m_hat (not with its own maximum) and return
+    (codes, alpha, flags, measured max of x, m_hat for the next step)."""
+    mx_used = pw2_ceil(m_hat) if pw2 else np.float32(m_hat)
+    codes, alpha, flags = quant_luq(x, mx_used, seed, n_samples, kmax)
+    measured, mflags = amax(x)
+    return codes, alpha, flags | mflags, measured, hindsight_next(measured, m_hat, eta)
 
 
 def luq_bins(x: np.ndarray, mx, kmax: int = KMAX_DEFAULT):

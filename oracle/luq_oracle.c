@@ -200,6 +200,32 @@ float oracle_quant_luq_window(const float* x, size_t n, uint64_t first_index, fl
   return alpha;
 }
 
+/* ------------------------------------------------------------------------ */
+/* Power-of-two LUQ (Appendix A.7): alpha_PW2 = 2^ceil(log2 max|x|) / 2^kmax. */
+/* The maximum is rounded UP to a power of two (so nothing is clipped), the   */
+/* quantizer itself is unchanged; every level is then a power of two.         */
+/* ------------------------------------------------------------------------ */
+float oracle_pw2_ceil(float mx) {
+  if (!(mx > 0.0f) || !(mx <= 3.402823466e38f)) return mx; /* 0, NaN, Inf pass through */
+  int e;
+  float m = frexpf(mx, &e); /* mx = m * 2^e, m in [0.5, 1) */
+  return (m == 0.5f) ? mx : ldexpf(1.0f, e);
+}
+
+/* ------------------------------------------------------------------------ */
+/* In-hindsight maximum (Sec. 7 "Reducing the data movement", Appendix A.5.4): */
+/*   m_hat^t = (1 - eta) * max|x^(t-1)| + eta * m_hat^(t-1),  eta = 0.1 in the */
+/* paper's runs.  Tensor t is quantized with m_hat^t (values above it clip to  */
+/* the top level) while its own maximum is measured for step t+1.  Evaluated   */
+/* in binary32, each operation rounded once.                                   */
+/* ------------------------------------------------------------------------ */
+float oracle_hindsight_next(float measured_max, float m_hat, float eta) {
+  float keep = 1.0f - eta;
+  float a = keep * measured_max;
+  float b = eta * m_hat;
+  return a + b;
+}
+
 /* Exact-expectation helper (test only): per element the two candidate levels
  * (as multiples of alpha: 0, 1, 2, 4, ...) and the 32-bit threshold, so that
  * E[Q(x)] = alpha*(lo + (hi-lo)*thr/2^32) can be evaluated without sampling. */

@@ -563,3 +563,75 @@ def test_luq_window_equals_slice_of_full_tensor():
     full, _, _ = oracle.quant_luq(x, mx, seed=5, n_samples=2)
     win, _, _ = oracle.quant_luq(x[1000:3000], mx, seed=5, n_samples=2, first_index=1000)
     np.testing.assert_array_equal(win, full[:, 500:1500])
+
+
+# ------------------------------------------- power-of-two scale and hindsight ----
+
+def test_pw2_ceiling_of_the_maximum():
+    """alpha_PW2 = 2^ceil(log2 max) / 2^kmax (Appendix A.7): checked against exact rationals."""
+    rng = np.random.default_rng(12)
+    vals = list(np.exp2(rng.uniform(-90, 90, 500)).astype(np.float32)) + \
+        [np.float32(2.0 ** k) for k in range(-20, 21)] + [np.float32(1.0000001), np.float32(0.99999994)]
+    for v in vals:
+        p = float(oracle.pw2_ceil(v))
+        m, e = math.frexp(p)
+        assert m == 0.5                                   # a power of two
+        assert Fraction(p) >= Fraction(float(v)) and Fraction(p) < 2 * Fraction(float(v))
+        assert float(oracle.pw2_ceil(np.float32(p))) == p  # idempotent
+    assert oracle.pw2_ceil(0.0) == 0.0
+
+
+def test_pw2_luq_levels_are_powers_of_two_and_still_unbiased():
+    x = luq_test_tensor(seed=71, n=6000)
+    mx, _ = oracle.amax(x)
+    codes, alpha, fl = oracle.quant_luq_pw2(x, mx, seed=4)
+    assert fl == 0 and math.frexp(float(alpha))[0] == 0.5
+    assert float(alpha) * 16 >= float(mx) > float(alpha) * 8          # ceiling: no clipping, less than one binade of slack
+    val, c = decode_luq(codes[0], x.size, alpha)
+    assert all(math.frexp(abs(v))[0] == 0.5 for v in val[val != 0][:200])
+    p2 = oracle.pw2_ceil(mx)
+    lo, hi, thr = oracle.luq_bins(x, p2)
+    e = float(alpha) * (lo + (hi - lo) * thr.astype(np.float64) / 2.0 ** 32)
+    a = np.abs(x).astype(np.float64)
+    assert (np.abs(e - a) <= 2.0 ** -32 * float(alpha) + 1e-300).all()  # division by a power of two is exact
+    np.testing.assert_array_equal(codes, oracle.quant_luq(x, p2, seed=4)[0])
+
+
+def test_hindsight_recursion_closed_form_and_limits():
+    """m_hat^t - max = eta^t (m_hat^0 - max) for a constant maximum; eta = 0 copies the
+    previous maximum, eta = 1 never moves."""
+    mx, m0, eta = 3.0, 11.0, 0.1
+    m = np.float32(m0)
+    for t in range(1, 12):
+        m = oracle.hindsight_next(mx, m, eta)
+        want = mx + (eta ** t) * (m0 - mx)
+        assert abs(float(m) - want) <= 4e-7 * want
+    assert oracle.hindsight_next(2.5, 100.0, 0.0) == np.float32(2.5)
+    assert oracle.hindsight_next(2.5, 100.0, 1.0) == np.float32(100.0)
+    # one rounding per operation, in binary32
+    a = np.float32(np.float32(1.0) - np.float32(0.1)) * np.float32(0.7)
+    b = np.float32(0.1) * np.float32(0.3)
+    assert oracle.hindsight_next(0.7, 0.3, 0.1) == np.float32(np.float32(a) + np.float32(b))
+
+
+def test_hindsight_step_uses_the_estimate_and_clips_above_it():
+    x = luq_test_tensor(seed=81, n=4000)
+    true_max, _ = oracle.amax(x)
+    m_hat = np.float32(float(true_max) / 8)                 # stale, too small estimate
+    codes, alpha, fl, measured, nxt = oracle.quant_luq_hindsight(x, m_hat, 0.1, seed=9, n_samples=2)
+    assert fl == 0 and measured == true_max and float(alpha) * 16 == float(m_hat)
+    assert nxt == oracle.hindsight_next(true_max, m_hat, 0.1)
+    val, c = decode_luq(codes[0], x.size, alpha)
+    above = np.abs(x) >= m_hat
+    assert above.sum() > 0 and (np.abs(val[above]) == float(m_hat)).all() and (c[above] == 5).all()
+    np.testing.assert_array_equal(codes, oracle.quant_luq(x, m_hat, 9, 2)[0])
+    # an estimate at or above the maximum changes nothing but the scale: still unbiased
+    big = np.float32(float(true_max) * 1.7)
+    lo, hi, thr = oracle.luq_bins(x, big)
+    al = float(oracle.luq_alpha(big))
+    e = al * (lo + (hi - lo) * thr.astype(np.float64) / 2.0 ** 32)
+    a = np.abs(x).astype(np.float64)
+    assert (np.abs(e - a) <= 2.0 ** -23 * a + 2.0 ** -32 * al).all()
+    # with the power-of-two option the estimate is rounded up first
+    codes2, alpha2, _, _, nxt2 = oracle.quant_luq_hindsight(x, m_hat, 0.1, seed=9, pw2=True)
+    assert float(alpha2) * 16 == float(oracle.pw2_ceil(m_hat)) and nxt2 == nxt
