@@ -206,7 +206,26 @@ def run_sweep(args, binding, inputs, torch, local):
                              "quant_gbs": round((4 + 0.5 * ns) * n / (med["quant"] * 1e-3) / 1e9, 1),
                              "amax_plus_quant_gbs": round((8 + 0.5 * ns) * n / (total * 1e-3) / 1e9, 1),
                              "frac_of_hbm_peak": round((8 + 0.5 * ns) * n / (total * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
-            rows.append({"elements": n, "n_samples": ns, **res})
+            # the two variants the paper proposes against the max pass and the division:
+            # in-hindsight maximum (one pass over the tensor) and power-of-two scale
+            mh = mx.clone()
+            extra = {}
+            for name, fn, nbytes in (
+                    ("hindsight", lambda: ctx.quant_grad_hindsight(x, mh, 0.1, 0, ns, False, codes, al, mx), (4 + 0.5 * ns) * n),
+                    ("hindsight_pw2", lambda: ctx.quant_grad_hindsight(x, mh, 0.1, 0, ns, True, codes, al, mx), (4 + 0.5 * ns) * n),
+                    ("amax_plus_pw2", lambda: (ctx.amax(x, mx), ctx.quant_grad_pw2(x, mx, 0, ns, codes, al)), (8 + 0.5 * ns) * n)):
+                ts = []
+                for it in range(reps + 3):
+                    flush.fill_(it & 0xFF)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(); fn(); e1.record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                t = sorted(ts)[len(ts) // 2]
+                extra[name] = {"us": round(t * 1e3, 2), "gbs": round(nbytes / (t * 1e-3) / 1e9, 1),
+                               "frac_of_hbm_peak": round(nbytes / (t * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
+            rows.append({"elements": n, "n_samples": ns, **res, **extra})
             del codes
         del x
         torch.cuda.empty_cache()

@@ -105,6 +105,26 @@ int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t
                    const float* d_amax, uint64_t seed, int n_samples,
                    uint8_t* d_codes, float* d_alpha, void* stream);
 
+/* LUQ with a power-of-two scale (Appendix A.7, LUQ_PW2): as luq_quant_grad, but
+ * alpha = 2^ceil(log2 max) / 2^kmax - the maximum is rounded UP to a power of two,
+ * so nothing is clipped, every level is a power of two and |x| / alpha is an exact
+ * exponent shift.  d_alpha receives the power-of-two alpha. */
+int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
+                       const float* d_amax, uint64_t seed, int n_samples,
+                       uint8_t* d_codes, float* d_alpha, void* stream);
+
+/* LUQ with the in-hindsight maximum (Sec. 7 "Reducing the data movement", Appendix
+ * A.5.4): the tensor is quantized in ONE pass with the estimate *d_mhat made from
+ * earlier steps (values above it clip to the top level), its own max|x| is measured
+ * on the way into *d_measured_max, and the estimate for the next step replaces
+ * *d_mhat:   m_hat <- (1 - eta) * measured + eta * m_hat     (binary32, one
+ * rounding per operation; the paper uses eta = 0.1).  pw2 = 1 additionally rounds
+ * the estimate up to a power of two before use (LUQ_PW2 + Hindsight).  Initialise
+ * *d_mhat before the first step, e.g. with luq_amax.  0 <= eta <= 1. */
+int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
+                             float* d_mhat, float eta, int pw2, uint64_t seed, int n_samples,
+                             uint8_t* d_codes, float* d_alpha, float* d_measured_max, void* stream);
+
 /* Diagnostic for the division-free quotient inside luq_quant_grad (reading of
  * Eq. StochasticPruning / Eq. unbiasedFpQ: the probabilities are functions of
  * t = |x| / alpha): writes, for n fp32 elements, the value t the quantizer forms

@@ -21,7 +21,7 @@ OPT_MMA_KIND, OPT_SPLITS = 1, 2
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_quant_grad", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_gemm_wgrad_static", "luq_status",
+           "luq_quant_grad", "luq_quant_grad_pw2", "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_gemm_wgrad_static", "luq_status",
            "luq_launch_count", "luq_strerror")
 
 _lib = None
@@ -48,6 +48,9 @@ def load() -> ctypes.CDLL:
         L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
         L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp]
         L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp]
+        L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp]
+        L.luq_quant_grad_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, ctypes.c_int, u64,
+                                               ctypes.c_int, vp, vp, vp, vp]
         L.luq_debug_quotient.argtypes = [vp, vp, sz, vp, vp, vp]
         L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
@@ -134,6 +137,33 @@ class Context:
                                      seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
                                      _stream()), "luq_quant_grad")
         return codes, alpha
+
+    def quant_grad_pw2(self, g: torch.Tensor, amax: torch.Tensor, seed: int, n_samples: int = 1,
+                       codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None):
+        rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
+        if codes is None:
+            codes = torch.empty((n_samples, g.numel() // 2), dtype=torch.uint8, device=g.device)
+        alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
+        _check(load().luq_quant_grad_pw2(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
+                                         seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
+                                         _stream()), "luq_quant_grad_pw2")
+        return codes, alpha
+
+    def quant_grad_hindsight(self, g: torch.Tensor, m_hat: torch.Tensor, eta: float, seed: int, n_samples: int = 1,
+                             pw2: bool = False, codes: torch.Tensor | None = None,
+                             alpha: torch.Tensor | None = None, measured: torch.Tensor | None = None):
+        """One pass: quantize with the estimate in `m_hat`, measure this tensor's maximum into
+        `measured`, replace `m_hat` by the estimate for the next step."""
+        rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
+        if codes is None:
+            codes = torch.empty((n_samples, g.numel() // 2), dtype=torch.uint8, device=g.device)
+        alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
+        measured = torch.empty(1, dtype=torch.float32, device=g.device) if measured is None else measured
+        _check(load().luq_quant_grad_hindsight(self.handle, g.data_ptr(), _dtype_code(g), rows, cols,
+                                               m_hat.data_ptr(), eta, int(pw2), seed & (2 ** 64 - 1), n_samples,
+                                               codes.data_ptr(), alpha.data_ptr(), measured.data_ptr(), _stream()),
+               "luq_quant_grad_hindsight")
+        return codes, alpha, measured
 
     def debug_quotient(self, x: torch.Tensor, amax: torch.Tensor) -> torch.Tensor:
         out = torch.empty_like(x, dtype=torch.float32)

@@ -133,6 +133,47 @@ int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t
                                        as_stream(stream)));
 }
 
+static int quant_grad_args(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
+                           int n_samples, const uint8_t* d_codes, const float* d_alpha, size_t* n_out) {
+  if (!ctx || !d_amax || !d_alpha || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  if (n_samples < 1 || n_samples > LUQ_MAX_SAMPLES) return LUQ_ERR_ARG;
+  const size_t n = rows * cols;
+  if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
+  if (n & 1u) return LUQ_ERR_ARG;
+  if (n && (!d_g || !d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_g) || !aligned16(d_codes)) return LUQ_ERR_ARG;
+  *n_out = n;
+  return LUQ_OK;
+}
+
+int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
+                       uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, void* stream) {
+  size_t n = 0;
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, &n);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes, d_alpha, 1, nullptr,
+                                          as_stream(stream)));
+}
+
+int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, float* d_mhat,
+                             float eta, int pw2, uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha,
+                             float* d_measured_max, void* stream) {
+  size_t n = 0;
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_mhat, n_samples, d_codes, d_alpha, &n);
+  if (rc) return rc;
+  if (!d_measured_max || !(eta >= 0.0f && eta <= 1.0f) || (pw2 != 0 && pw2 != 1)) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  cudaStream_t st = as_stream(stream);
+  if (cudaMemsetAsync(d_measured_max, 0, sizeof(float), st) != cudaSuccess) return LUQ_ERR_CUDA;
+  int e = luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_mhat, seed, n_samples, d_codes, d_alpha, 2 | pw2,
+                                   d_measured_max, st);
+  if (e) return cuda_rc(e);
+  return cuda_rc(luq_launch_hindsight_update(ctx, d_mhat, d_measured_max, eta, st));
+}
+
 int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream) {
   if (!ctx || !d_amax || (n && (!d_x || !d_t))) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);

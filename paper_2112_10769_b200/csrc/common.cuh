@@ -28,6 +28,11 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
 int luq_launch_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
                           uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, cudaStream_t st);
 
+// flags: bit 0 = power-of-two scale, bit 1 = also reduce max|x| of this tensor into d_measured (pre-zeroed)
+int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
+                             int n_samples, uint8_t* d_codes, float* d_alpha, int flags, float* d_measured,
+                             cudaStream_t st);
+int luq_launch_hindsight_update(luq_ctx* ctx, float* d_mhat, const float* d_measured, float eta, cudaStream_t st);
 int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,
                               cudaStream_t st);
 

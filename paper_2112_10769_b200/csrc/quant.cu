@@ -230,7 +230,9 @@ __device__ __forceinline__ LuqScale luq_scale(float alpha) {
   return sc;
 }
 
+template <bool PW2 = false>
 __device__ __forceinline__ float luq_quotient_raw(float x, const LuqScale& sc) {
+  if constexpr (PW2) return fabsf(x) * sc.recip;   // alpha is a power of two: exact up to the final rounding
   const float a = fabsf(x) * sc.pre;
   const float q0 = a * sc.recip;
   const float r0 = __fmaf_rn(-sc.alpha_s, q0, a);
@@ -238,9 +240,10 @@ __device__ __forceinline__ float luq_quotient_raw(float x, const LuqScale& sc) {
   const float r1 = __fmaf_rn(-sc.alpha_s, q1, a);
   return __fmaf_rn(r1, sc.recip, q1);
 }
+template <bool PW2 = false>
 __device__ __forceinline__ float luq_quotient(float x, const LuqScale& sc) {
-  // an overflowing or non-finite quotient turns into NaN above; both belong to the top level
-  return fminf(luq_quotient_raw(x, sc), static_cast<float>(1 << LUQ_KMAX));   // fminf(NaN, c) = c
+  // an overflowing or non-finite quotient turns into NaN or Inf above; both belong to the top level
+  return fminf(luq_quotient_raw<PW2>(x, sc), static_cast<float>(1 << LUQ_KMAX));   // fminf(NaN, c) = c
 }
 
 // Per element: lower code and the 32-bit threshold of the up-decision, from the
@@ -263,23 +266,36 @@ __device__ __forceinline__ uint32_t luq_nibble(uint32_t xbits, uint32_t lo_code,
   return c ? (((xbits >> 28) & 8u) | c) : 0u;
 }
 
-// NS: number of samples known at compile time (1, 2) or 0 = read n_samples at run time
-template <bool BF16, int NS>
+// 2^ceil(log2 m) for a positive finite m (power-of-two LUQ: the maximum is rounded up, never down)
+__device__ __forceinline__ float pw2_ceil(float m) {
+  const uint32_t b = __float_as_uint(m);
+  if (m > 0.0f && b < 0x7F800000u && (b & 0x007FFFFFu) != 0u) return __uint_as_float((b & 0x7F800000u) + 0x00800000u);
+  return m;
+}
+
+// NS: number of samples known at compile time (1, 2) or 0 = read n_samples at run time.
+// PW2: the scale is a power of two, the quotient an exact scaling (one multiply).
+// TRACK: the tensor's own max|x| is reduced on the way (in-hindsight estimation: the scale
+// in d_amax is an estimate from earlier steps, the measured maximum feeds the next one).
+template <bool BF16, int NS, bool PW2, bool TRACK>
 __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restrict__ x, size_t n,
                                                              const float* __restrict__ d_amax,
                                                              const __grid_constant__ PhiloxKeySet keys,
                                                              int n_samples_rt,
                                                              uint8_t* __restrict__ codes,
                                                              float* __restrict__ d_alpha,
+                                                             unsigned int* __restrict__ measured_bits,
                                                              unsigned int* __restrict__ status) {
   const int n_samples = NS > 0 ? NS : n_samples_rt;
   constexpr int kElems = Item<BF16>::kElems;
-  const float mx = __ldg(d_amax);
+  const float mx = PW2 ? pw2_ceil(__ldg(d_amax)) : __ldg(d_amax);
   const bool first = blockIdx.x == 0 && threadIdx.x == 0;
   const bool ok = scale_usable(mx, first ? status : nullptr);
   const float alpha = ok ? mx * (1.0f / static_cast<float>(1 << LUQ_KMAX)) : 0.0f;  // exact scaling
   if (first) *d_alpha = alpha;
-  const LuqScale sc = luq_scale(ok ? alpha : 1.0f);
+  LuqScale sc = luq_scale(ok ? alpha : 1.0f);
+  if constexpr (PW2) { sc.pre = 1.0f; sc.alpha_s = ok ? alpha : 1.0f; sc.recip = 1.0f / sc.alpha_s; }  // exact
+  uint32_t seen = 0;   // running max of |x| bit patterns (TRACK)
 
   const size_t plane = n / 2;
   const bool aligned = (plane % (kElems / 2)) == 0;  // planes start on a store boundary
@@ -296,12 +312,16 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
     bool in_range = false;
 #pragma unroll
     for (int j = 0; j < kElems; ++j) in_range |= !(fabsf(v[j]) < alpha);
+    if constexpr (TRACK) {
+#pragma unroll
+      for (int j = 0; j < kElems; ++j) seen = max(seen, __float_as_uint(v[j]) & 0x7FFFFFFFu);
+    }
     // the vote needs every lane of the warp here: only the full-tile loop qualifies
     if (whole_warp && !__any_sync(0xFFFFFFFFu, in_range)) {
       uint32_t thr[kElems], sn[kElems];
 #pragma unroll
       for (int j = 0; j < kElems; ++j) {
-        thr[j] = __float2uint_rz(luq_quotient_raw(v[j], sc) * 4294967296.0f);
+        thr[j] = __float2uint_rz(luq_quotient_raw<PW2>(v[j], sc) * 4294967296.0f);
         sn[j] = ((__float_as_uint(v[j]) >> 28) & 8u) | 1u;
       }
 #pragma unroll
@@ -323,7 +343,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
     }
     uint32_t lo_code[kElems], thr[kElems];
 #pragma unroll
-    for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient(v[j], sc), lo_code[j], thr[j]);
+    for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient<PW2>(v[j], sc), lo_code[j], thr[j]);
 #pragma unroll
     for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
       if (NS == 0 && s >= n_samples) break;
@@ -356,9 +376,18 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
       for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) process(i, __ldg(p + i), false);
   } else {
     const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
-    for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < items; i += stride)
+    for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < items; i += stride) {
       for (int s = 0; s < n_samples; ++s) Item<BF16>::store(codes + plane * s, i, 0u, aligned || s == 0);
+      if constexpr (TRACK) {   // an unusable estimate still needs this tensor's maximum for the next step
+        float v[kElems];
+        Item<BF16>::widen(__ldg(p + i), v);
+#pragma unroll
+        for (int j = 0; j < kElems; ++j) seen = max(seen, __float_as_uint(v[j]) & 0x7FFFFFFFu);
+      }
+    }
   }
+  if (TRACK && first)
+    for (size_t e = items * kElems; e < n; ++e) seen = max(seen, __float_as_uint(Item<BF16>::load1(x, e)) & 0x7FFFFFFFu);
   if (first) {  // tail: fewer elements than one piece, two per byte
     for (int s = 0; s < n_samples; ++s) {
       const PhiloxKeys& ks = keys.s[s];
@@ -369,7 +398,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
           if (ok && idx < n) {
             const float xv = Item<BF16>::load1(x, idx);
             uint32_t lc, th;
-            luq_bin(luq_quotient(xv, sc), lc, th);
+            luq_bin(luq_quotient<PW2>(xv, sc), lc, th);
             const uint4 r = philox_block(idx >> 2, ks);
             const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
             nib[h] = luq_nibble(__float_as_uint(xv), lc, th, rw[idx & 3]);
@@ -379,6 +408,27 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
       }
     }
   }
+  if constexpr (TRACK) {   // block maximum -> one atomicMax; Inf/NaN patterns win and raise the flag
+    seen = __reduce_max_sync(0xFFFFFFFFu, seen);
+    __shared__ uint32_t warp_seen[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_seen[threadIdx.x >> 5] = seen;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      seen = threadIdx.x < kThreads / 32 ? warp_seen[threadIdx.x] : 0u;
+      seen = __reduce_max_sync(0xFFFFFFFFu, seen);
+      if (threadIdx.x == 0 && seen != 0) {
+        atomicMax(measured_bits, seen);
+        if (seen >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
+      }
+    }
+  }
+}
+
+// In-hindsight update after a tracked quantization: m_hat <- (1 - eta) * measured + eta * m_hat,
+// every operation rounded once in binary32.
+__global__ void hindsight_update_kernel(float* __restrict__ m_hat, const float* __restrict__ measured, float eta) {
+  const float keep = __fsub_rn(1.0f, eta);
+  *m_hat = __fadd_rn(__fmul_rn(keep, *measured), __fmul_rn(eta, *m_hat));
 }
 
 // Diagnostic: the quotient t = |x| / alpha exactly as the quantizer forms it
@@ -446,37 +496,68 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
 }
 
 namespace {
-template <bool BF16>
+template <bool BF16, bool PW2, bool TRACK>
 int launch_luq(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys, int n_samples,
-               uint8_t* d_codes, float* d_alpha, cudaStream_t st) {
+               uint8_t* d_codes, float* d_alpha, unsigned int* d_measured, cudaStream_t st) {
   const size_t thread_items = n / Item<BF16>::kElems / kTileItems + 1;
   if (n_samples == 1) {
-    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 1>, thread_items);
-    quant_luq_kernel<BF16, 1><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 1, d_codes, d_alpha, ctx->d_status);
+    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 1, PW2, TRACK>, thread_items);
+    quant_luq_kernel<BF16, 1, PW2, TRACK><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 1, d_codes, d_alpha,
+                                                                     d_measured, ctx->d_status);
   } else if (n_samples == 2) {
-    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 2>, thread_items);
-    quant_luq_kernel<BF16, 2><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 2, d_codes, d_alpha, ctx->d_status);
+    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 2, PW2, TRACK>, thread_items);
+    quant_luq_kernel<BF16, 2, PW2, TRACK><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 2, d_codes, d_alpha,
+                                                                     d_measured, ctx->d_status);
   } else {
-    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 0>, thread_items);
-    quant_luq_kernel<BF16, 0><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, n_samples, d_codes, d_alpha,
-                                                        ctx->d_status);
+    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 0, PW2, TRACK>, thread_items);
+    quant_luq_kernel<BF16, 0, PW2, TRACK><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, n_samples, d_codes,
+                                                                     d_alpha, d_measured, ctx->d_status);
   }
   return static_cast<int>(cudaGetLastError());
 }
-}  // namespace
 
-int luq_launch_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
-                          uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, cudaStream_t st) {
+PhiloxKeySet expand_keys(uint64_t seed, int n_samples) {
   PhiloxKeySet keys{};
   for (int s = 0; s < n_samples; ++s) {   // sample s is keyed by seed + s
     const uint64_t key = seed + static_cast<uint64_t>(s);
     uint32_t a = static_cast<uint32_t>(key), b = static_cast<uint32_t>(key >> 32);
     for (int r = 0; r < 10; ++r) { keys.s[s].k0[r] = a; keys.s[s].k1[r] = b; a += 0x9E3779B9u; b += 0xBB67AE85u; }
   }
-  const int rc = dtype == LUQ_BF16 ? launch_luq<true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, st)
-                                   : launch_luq<false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, st);
+  return keys;
+}
+}  // namespace
+
+// flags: bit 0 = power-of-two scale, bit 1 = track this tensor's maximum into d_measured
+int luq_launch_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
+                          uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, cudaStream_t st) {
+  return luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes, d_alpha, 0, nullptr, st);
+}
+
+int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
+                             int n_samples, uint8_t* d_codes, float* d_alpha, int flags, float* d_measured,
+                             cudaStream_t st) {
+  const PhiloxKeySet keys = expand_keys(seed, n_samples);
+  unsigned int* meas = reinterpret_cast<unsigned int*>(d_measured);
+  const bool bf = dtype == LUQ_BF16;
+  int rc;
+  switch ((flags & 3) | (bf ? 4 : 0)) {
+    case 0: rc = launch_luq<false, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    case 1: rc = launch_luq<false, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    case 2: rc = launch_luq<false, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    case 3: rc = launch_luq<false, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    case 4: rc = launch_luq<true, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    case 5: rc = launch_luq<true, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    case 6: rc = launch_luq<true, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    default: rc = launch_luq<true, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+  }
   ctx->launches += 1;
   return rc;
+}
+
+int luq_launch_hindsight_update(luq_ctx* ctx, float* d_mhat, const float* d_measured, float eta, cudaStream_t st) {
+  hindsight_update_kernel<<<1, 1, 0, st>>>(d_mhat, d_measured, eta);
+  ctx->launches += 1;
+  return static_cast<int>(cudaGetLastError());
 }
 
 int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,

@@ -332,3 +332,70 @@ def test_division_free_quotient_equals_ieee_division(ctx):
         total += int(check.sum())
     assert total > 50_000_000
     assert ctx.status() == 0
+
+
+# ----------------------------------------- power-of-two scale, in-hindsight maximum ----
+
+@pytest.mark.parametrize("n", [10, 4098, (1 << 20) + 2])
+@pytest.mark.parametrize("dtype,ns", [("f32", 1), ("f32", 2), ("bf16", 3)])
+def test_quant_grad_pw2_bit_exact(ctx, n, dtype, ns):
+    x = luq_inputs(n, 5000 + n)
+    if dtype == "bf16":
+        x = inputs.to_bf16_bits(x)
+    mx, _ = oracle.amax(x)
+    want, a_want, fl = oracle.quant_luq_pw2(x, mx, 77 + n, ns)
+    xd = to_dev(x)
+    codes, alpha = ctx.quant_grad_pw2(xd, ctx.amax(xd), 77 + n, ns)
+    assert fl == 0 and alpha.item() == a_want
+    np.testing.assert_array_equal(codes.cpu().numpy().reshape(ns, -1), want)
+    # a maximum that already is a power of two is used as it is; one just above it doubles
+    for m in (np.float32(0.25), np.nextafter(np.float32(0.25), np.float32(1))):
+        want, a_want, _ = oracle.quant_luq_pw2(x, m, 3, 1)
+        codes, alpha = ctx.quant_grad_pw2(xd, scalar(float(m)), 3, 1)
+        assert alpha.item() == a_want
+        np.testing.assert_array_equal(codes.cpu().numpy(), want)
+    assert ctx.status() == 0
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("pw2", [False, True])
+def test_hindsight_sequence_matches_oracle(ctx, dtype, pw2):
+    """Six steps with tensors whose scale jumps around: the estimate lags, some steps clip.
+    Codes, alpha, the measured maximum and the estimate must match the oracle bit for bit."""
+    n, eta, ns = 200_006, 0.1, 2
+    scales = [1.0, 0.4, 5.0, 0.05, 2.0, 1.0]
+    base = inputs.log_uniform_magnitudes(n, -20, 2, 31)
+    first = (base * np.float32(scales[0])).astype(np.float32)
+    m_hat_o = oracle.amax(inputs.to_bf16_bits(first) if dtype == "bf16" else first)[0]
+    m_hat_d = scalar(float(m_hat_o))
+    clipped = 0
+    for step, sc in enumerate(scales):
+        x = (base * np.float32(sc)).astype(np.float32)
+        x[step] = np.float32(0.0)
+        if dtype == "bf16":
+            x = inputs.to_bf16_bits(x)
+        want, a_want, fl, meas_want, next_want = oracle.quant_luq_hindsight(x, m_hat_o, eta, seed=step, n_samples=ns, pw2=pw2)
+        codes, alpha, measured = ctx.quant_grad_hindsight(to_dev(x), m_hat_d, eta, step, ns, pw2)
+        assert fl == 0 and alpha.item() == a_want and measured.item() == meas_want
+        assert m_hat_d.item() == next_want
+        np.testing.assert_array_equal(codes.cpu().numpy().reshape(ns, -1), want)
+        clipped += int(meas_want > m_hat_o)
+        m_hat_o = next_want
+    assert clipped >= 2
+    assert ctx.status() == 0
+
+
+def test_hindsight_unusable_estimate_recovers(ctx):
+    x = luq_inputs(50_000, 4)
+    xd = to_dev(x)
+    m_hat = scalar(0.0)
+    codes, alpha, measured = ctx.quant_grad_hindsight(xd, m_hat, 0.1, 1)
+    assert alpha.item() == 0 and not codes.any().item()
+    assert measured.item() == oracle.amax(x)[0]
+    assert m_hat.item() == oracle.hindsight_next(measured.item(), 0.0, 0.1)
+    assert ctx.status() == 0
+    codes, alpha, _ = ctx.quant_grad_hindsight(xd, m_hat, 0.1, 2)
+    assert alpha.item() > 0 and codes.any().item()
+    with pytest.raises(binding.LuqError):
+        ctx.quant_grad_hindsight(xd, m_hat, 1.5, 1)
+    assert ctx.status() == 0
