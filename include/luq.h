@@ -62,6 +62,7 @@ extern "C" {
                               2 (default): chosen per product - int8 where INT4 codes are expanded inside the
                               kernel, e4m3 where both operands are pre-expanded planes */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
+#define LUQ_OPT_PAIRS 3    /* 1: products whose operands are both 8-bit planes run on CTA pairs (cta_group::2) */
 
 #define LUQ_MAX_SAMPLES 8
 

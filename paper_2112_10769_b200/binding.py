@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libluq_b200.so")
 
 LUQ_F32, LUQ_BF16 = 0, 1
 STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT = 1, 2, 4
-OPT_MMA_KIND, OPT_SPLITS = 1, 2
+OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS = 1, 2, 3
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",

@@ -54,6 +54,7 @@ int luq_create(luq_ctx** out, int device) {
   c->sm_count = prop.multiProcessorCount;
   c->mma_kind = LUQ_DEFAULT_MMA_KIND;
   c->forced_splits = 0;
+  c->use_pairs = 0;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;
   c->d_status = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
@@ -89,6 +90,10 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
     case LUQ_OPT_SPLITS:
       if (value < 0 || value > 1024) return LUQ_ERR_ARG;
       ctx->forced_splits = value;
+      return LUQ_OK;
+    case LUQ_OPT_PAIRS:
+      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      ctx->use_pairs = value;
       return LUQ_OK;
     default:
       return LUQ_ERR_UNSUPPORTED;

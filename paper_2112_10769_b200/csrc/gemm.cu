@@ -474,6 +474,214 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   }
 }
 
+// ---------------------------------------------------------------------------
+// CTA-pair kernel (cluster of two, tcgen05 cta_group::2) for products whose two
+// operands both arrive as planes.  A pair computes a 256 x 256 tile: each CTA
+// loads its own 128 rows of A and its own 128 columns of B, one thread of the
+// leader issues 256 x 256 x 32 MMAs that run on both SMs, each SM accumulates its
+// 128 rows in its own tensor memory.  Per SM and stage that is 32 KB of operands
+// instead of 48 KB - the operand fetch, not the tensor core, bounded the
+// single-CTA kernel.
+//   warp 0      TMA producer (its own A slab and B half; bytes counted on the leader's barrier)
+//   warp 1      MMA issue (leader only); owns the tensor-memory allocation in both CTAs
+//   warps 2-5   epilogue of this CTA's 128 rows
+// Barriers: full[s] lives in the leader (one arrival, 64 KB of transactions from both
+// CTAs); empty[s] and acc_full[b] exist in both CTAs and are signalled by one
+// multicast commit; acc_empty[b] lives in the leader and counts the eight epilogue warps.
+// ---------------------------------------------------------------------------
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * kExpandedSlab;             // A slab + half of B
+constexpr int kPairThreads = 32 * 6;
+struct PairSmem {
+  static constexpr int ring = 0;
+  static constexpr int staging = ring + kPairStages * kPairStageBytes;
+  static constexpr int barriers = staging + 4 * 2 * kStageBox;
+  static constexpr int num_barriers = 2 * kPairStages + 4;
+  static constexpr int tmem_slot = barriers + 8 * num_barriers;
+  static constexpr int abort_flag = tmem_slot + 4;
+  static constexpr int total = abort_flag + 4;
+  static constexpr int smem_bytes = total + 1024;
+  static_assert(smem_bytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+};
+
+template <int KIND, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(kPairThreads, 1)
+luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                     const __grid_constant__ CUtensorMap tm_out, const GemmParams p) {
+  constexpr int ES = kPairStages;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* const gen = smem_raw + (base - raw);
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+
+  const uint32_t bar0 = base + PairSmem::barriers;
+  auto full = [&](uint32_t s) { return bar0 + 8u * s; };
+  auto empty = [&](uint32_t s) { return bar0 + 8u * (ES + s); };
+  auto acc_full = [&](uint32_t b) { return bar0 + 8u * (2 * ES + b); };
+  auto acc_empty = [&](uint32_t b) { return bar0 + 8u * (2 * ES + 2 + b); };
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + PairSmem::tmem_slot);
+  volatile uint32_t* const abort_flag = reinterpret_cast<volatile uint32_t*>(gen + PairSmem::abort_flag);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < ES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 0 && lane == 0) { tma_prefetch_desc(&tm_a); tma_prefetch_desc(&tm_b); tma_prefetch_desc(&tm_out); }
+  if (warp == 1) {  // the same warp of both CTAs allocates tensor memory for the pair
+    tmem_alloc_pair(base + PairSmem::tmem_slot, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();   // barriers of both CTAs are initialised before either signals the other
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_m2 = (p.tiles_m + 1) / 2;               // 256-row tiles
+  const int tiles = tiles_m2 * p.tiles_n;
+  const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+  const int total_iters = p.n_samples * p.num_kb;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- producer
+    if (lane == 0) {
+      uint32_t issued = 0, stage = 0, phase = 0;
+      bool ok = true;
+      for (int t = pair; ok && t < tiles; t += pairs) {
+        const int m0 = (t % tiles_m2) * 256 + static_cast<int>(rank) * 128;    // this CTA's rows of A
+        const int n0 = (t / tiles_m2) * BN + static_cast<int>(rank) * 128;     // this CTA's columns of B
+        int sample = 0, kb = 0;
+        for (int k_it = 0; k_it < total_iters; ++k_it) {
+          if (!mbar_wait(empty(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t full_leader = mapa_shared(full(stage), 0);
+          const uint32_t dst = base + PairSmem::ring + stage * kPairStageBytes;
+          if (leader) mbar_arrive_expect_tx(full(stage), 2 * kPairStageBytes);   // both CTAs' bytes
+          if constexpr (A_MN) tma_pair_load_3d(dst, &tm_a, full_leader, m0, kb * BK, sample);
+          else tma_pair_load_3d(dst, &tm_a, full_leader, kb * BK, m0, sample);
+          if constexpr (B_MN) tma_pair_load_2d(dst + kExpandedSlab, &tm_b, full_leader, n0, kb * BK);
+          else tma_pair_load_2d(dst + kExpandedSlab, &tm_b, full_leader, kb * BK, n0);
+          ++issued;
+          if (++kb == p.num_kb) { kb = 0; ++sample; }
+          if (++stage == static_cast<uint32_t>(ES)) { stage = 0; phase ^= 1u; }
+        }
+      }
+      (void)issued;
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------- MMA issue (leader only)
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = (KIND == 0 ? (1u << 4) : (2u << 4)) | ((KIND == 0 ? 0u : 1u) << 7) |
+                                 ((KIND == 0 ? 0u : 1u) << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+                                 (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
+      const uint32_t a0 = base + PairSmem::ring, b0 = a0 + kExpandedSlab;
+      const uint64_t da0 = A_MN ? umma_desc_sw128(a0, kExpandedSlab, 1024) : umma_desc_sw128(a0, 16, 1024);
+      const uint64_t db0 = B_MN ? umma_desc_sw128(b0, kExpandedSlab, 1024) : umma_desc_sw128(b0, 16, 1024);
+      constexpr uint64_t kStepA = (A_MN ? 32 * 128 : 32) >> 4, kStepB = (B_MN ? 32 * 128 : 32) >> 4;
+      constexpr uint64_t kStageStep = kPairStageBytes >> 4;
+      uint32_t stage = 0, phase = 0, tile_it = 0;
+      bool ok = true;
+      for (int t = pair; ok && t < tiles; t += pairs, ++tile_it) {
+        const uint32_t buf = tile_it & 1u;
+        if (!mbar_wait_cluster(acc_empty(buf), ((tile_it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + buf * BN;
+        uint32_t accumulate = 0;
+        for (int k_it = 0; k_it < total_iters; ++k_it) {
+          if (!mbar_wait_cluster(full(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t da = da0 + stage * kStageStep, db = db0 + stage * kStageStep;
+#pragma unroll
+          for (int kk = 0; kk < BK / 32; ++kk) {
+            tc_mma_pair<KIND>(tmem_d, da + kk * kStepA, db + kk * kStepB, idesc, accumulate);
+            accumulate = 1;
+          }
+          tc_commit_pair(empty(stage));
+          if (++stage == static_cast<uint32_t>(ES)) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit_pair(acc_full(buf));
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;
+    const float scale = (__ldg(p.scale_a) * __ldg(p.scale_b)) * p.post_scale;
+    const uint32_t stage0 = base + PairSmem::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
+    uint8_t* const stage0_gen = gen + PairSmem::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
+    const int sw = lane & 7;
+    uint32_t tile_it = 0, box_it = 0;
+    bool ok = true;
+    for (int t = pair; ok && t < tiles; t += pairs, ++tile_it) {
+      const long long row0 = static_cast<long long>(t % tiles_m2) * 256 + rank * 128 + quarter * 32;
+      const long long col_base = static_cast<long long>(t / tiles_m2) * BN;
+      const uint32_t buf = tile_it & 1u;
+      if (!mbar_wait(acc_full(buf), (tile_it >> 1) & 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+      auto emit = [&](const uint32_t (&r)[32], int c) {
+        const long long col0 = col_base + c * 32;
+        if (row0 < p.Mo && col0 < p.No) {   // warp-uniform
+          const uint32_t b = box_it & 1u;
+          ++box_it;
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
+          uint8_t* const rowp = stage0_gen + b * kStageBox + lane * 128;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            float4 v;
+            if constexpr (KIND == 0) {
+              v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                              __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+            } else {
+              v = make_float4(static_cast<float>(static_cast<int>(r[4 * j])), static_cast<float>(static_cast<int>(r[4 * j + 1])),
+                              static_cast<float>(static_cast<int>(r[4 * j + 2])), static_cast<float>(static_cast<int>(r[4 * j + 3])));
+            }
+            v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
+            *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tm_out, stage0 + b * kStageBox, static_cast<int>(col0), static_cast<int>(row0));
+            bulk_commit();
+          }
+        }
+      };
+      uint32_t r0[32], r1[32];
+      tmem_ld_32x32(taddr, r0);
+      tmem_ld_wait();
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; c += 2) {
+        tmem_ld_32x32(taddr + (c + 1) * 32, r1);
+        emit(r0, c);
+        tmem_ld_wait();
+        if (c + 2 < BN / 32) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
+        emit(r1, c + 1);
+        tmem_ld_wait();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(acc_empty(buf), 0));   // tell the leader this half is drained
+    }
+    if (lane == 0) bulk_wait<0>();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  cluster_sync_all();   // neither CTA leaves (or frees tensor memory) while its peer may still signal it
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, LUQ_STATUS_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 // Sums the partial tiles of a split contraction in a fixed order, applies the
 // scales and writes the output.  One thread per float4 of a tile.
 __global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restrict__ ws, float* __restrict__ out,
@@ -577,6 +785,26 @@ int launch_planes(bool a_plane, bool b_plane, const CUtensorMap& ta, const CUten
   if (a_plane) return launch<KIND, A_MN, B_MN, A_LUQ, true, false>(ta, tb, to, p, grid, st);
   if (b_plane) return launch<KIND, A_MN, B_MN, A_LUQ, false, true>(ta, tb, to, p, grid, st);
   return launch<KIND, A_MN, B_MN, A_LUQ, false, false>(ta, tb, to, p, grid, st);
+}
+
+template <int KIND, bool A_MN, bool B_MN>
+int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const GemmParams& p, int pairs,
+                cudaStream_t st) {
+  auto kernel = luq_gemm_pair_kernel<KIND, A_MN, B_MN>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::smem_bytes);
+  if (e != cudaSuccess) return static_cast<int>(e);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(kPairThreads, 1, 1);
+  cfg.dynamicSmemBytes = PairSmem::smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, to, p);
+  return static_cast<int>(e);
 }
 
 template <int KIND>
@@ -700,6 +928,26 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   else bad |= encode_out_map(ctx->encode_tiled, &to, a.d_out, a.Mo, a.No);
   if (bad) return LUQ_ERR_CUDA;
 
+  // CTA pairs when both operands are planes (no expansion inside the kernel) and the contraction
+  // is not split: option LUQ_OPT_PAIRS (default on)
+  if (ctx->use_pairs && a_plane && b_plane && p.splits == 1 && p.tiles_m >= 2) {
+    const long long pair_tiles = static_cast<long long>((p.tiles_m + 1) / 2) * p.tiles_n;
+    const int max_pairs = ctx->sm_count / 2;
+    const int pairs = static_cast<int>(pair_tiles < max_pairs ? pair_tiles : max_pairs);
+    const int sel2 = (ctx->mma_kind ? 4 : 0) | (a.a_mn ? 2 : 0) | (a.b_mn ? 1 : 0);
+    switch (sel2) {
+      case 0: rc = launch_pair<0, false, false>(ta, tb, to, p, pairs, st); break;
+      case 1: rc = launch_pair<0, false, true>(ta, tb, to, p, pairs, st); break;
+      case 3: rc = launch_pair<0, true, true>(ta, tb, to, p, pairs, st); break;
+      case 4: rc = launch_pair<1, false, false>(ta, tb, to, p, pairs, st); break;
+      case 5: rc = launch_pair<1, false, true>(ta, tb, to, p, pairs, st); break;
+      case 7: rc = launch_pair<1, true, true>(ta, tb, to, p, pairs, st); break;
+      default: return LUQ_ERR_UNSUPPORTED;
+    }
+    if (rc == 0) ctx->launches += 1;
+    return rc;
+  }
+
   const int grid = static_cast<int>(units < ctx->sm_count ? units : ctx->sm_count);
   const int sel = (ctx->mma_kind ? 4 : 0) | (a.a_mn ? 2 : 0) | (a.b_mn ? 1 : 0);
   if (a.b_kind != 0 || (a.a_kind == 1) != (sel & 3 ? true : false)) return LUQ_ERR_UNSUPPORTED;
@@ -821,6 +1069,7 @@ extern "C" int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_al
   local.workspace_bytes = kStaticScratchBytes;
   local.mma_kind = LUQ_DEFAULT_MMA_KIND;
   local.forced_splits = 0;
+  local.use_pairs = 0;
   local.launches = 0;
   local.encode_tiled = s->encode_tiled;
 
