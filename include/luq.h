@@ -58,13 +58,26 @@ extern "C" {
 #define LUQ_STATUS_TIMEOUT 4   /* a bounded wait inside a kernel expired; outputs unspecified */
 
 /* options for luq_set_option */
-#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands; 1: kind::i8 on int8 operands;
-                              2 (default): chosen per product - int8 where INT4 codes are expanded inside the
-                              kernel, e4m3 where both operands are pre-expanded planes */
+#define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands (operand bytes passed to a GEMM are then
+                              ignored); 1: kind::i8 on int8 operands; 2 (default): int8, except e4m3 where an
+                              int32 accumulator could wrap (contractions beyond about 2^18 terms) */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
 #define LUQ_OPT_PAIRS 3    /* 1: products whose operands are both 8-bit planes run on CTA pairs (cta_group::2) */
 
 #define LUQ_MAX_SAMPLES 8
+
+/* Operand bytes ("d_*_operand" arguments, all optional: pass NULL to leave them out).
+ * The 4-bit codes are the format of the paper (Sec. 3, Sec. 4) and what is stored;
+ * the tensor cores of this GPU read 8-bit operands, so a GEMM has to widen every
+ * code once per tile that reads it.  A quantizer can write the widened form next to
+ * the codes in the same pass, and a GEMM given those bytes fetches them instead of
+ * widening the codes again.  They carry the same integers as the codes, so every
+ * result is bit-identical with or without them.  Layout: one int8 per element, in
+ * the element order of the tensor (sample planes one after the other, rows*cols
+ * bytes each).  INT4: 16 * q (the code nibble in the high half of the byte).  LUQ:
+ * +-2^(c-1) for code c >= 1, 0 for c = 0.  16-byte aligned.  A GEMM uses them where
+ * at least two of its tiles re-read the operand and the contraction is long, and
+ * reads the codes otherwise; the codes must always be passed. */
 
 typedef struct luq_ctx luq_ctx;
 
@@ -91,7 +104,7 @@ int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, 
  * d_clip is usually the tensor max from luq_amax; any caller clip is allowed.
  * rows*cols must be even.  d_codes: rows*cols/2 bytes.  d_scale: one float. */
 int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
-                   const float* d_clip, uint8_t* d_codes, float* d_scale, void* stream);
+                   const float* d_clip, uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
 
 /* Q_FP = LUQ (Sec. 4): alpha = max / 2^kmax (Eq. alpha); |x| < alpha becomes
  * sign*alpha with probability |x|/alpha, else 0 (Eq. StochasticPruning);
@@ -104,7 +117,7 @@ int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t
  * smaller value clips to the top level.  d_alpha receives alpha. */
 int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
                    const float* d_amax, uint64_t seed, int n_samples,
-                   uint8_t* d_codes, float* d_alpha, void* stream);
+                   uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream);
 
 /* LUQ with a power-of-two scale (Appendix A.7, LUQ_PW2): as luq_quant_grad, but
  * alpha = 2^ceil(log2 max) / 2^kmax - the maximum is rounded UP to a power of two,
@@ -112,7 +125,7 @@ int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t
  * exponent shift.  d_alpha receives the power-of-two alpha. */
 int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
                        const float* d_amax, uint64_t seed, int n_samples,
-                       uint8_t* d_codes, float* d_alpha, void* stream);
+                       uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream);
 
 /* LUQ with the in-hindsight maximum (Sec. 7 "Reducing the data movement", Appendix
  * A.5.4): the tensor is quantized in ONE pass with the estimate *d_mhat made from
@@ -124,7 +137,8 @@ int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, si
  * *d_mhat before the first step, e.g. with luq_amax.  0 <= eta <= 1. */
 int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
                              float* d_mhat, float eta, int pw2, uint64_t seed, int n_samples,
-                             uint8_t* d_codes, float* d_alpha, float* d_measured_max, void* stream);
+                             uint8_t* d_codes, float* d_alpha, float* d_measured_max, int8_t* d_operand,
+                             void* stream);
 
 /* Diagnostic for the division-free quotient inside luq_quant_grad (reading of
  * Eq. StochasticPruning / Eq. unbiasedFpQ: the probabilities are functions of
@@ -136,8 +150,8 @@ int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_
 /* Forward GEMM (Eq. Forward; scale factoring of Appendix A.1):
  *   Z[m,n] = (sa*sw) * sum_k qA[m,k] * qW[n,k]        fp32 accumulate, fp32 out.
  * a_codes [M x K/2], w_codes [N x K/2].  K must be a multiple of 32. */
-int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa,
-                 const uint8_t* d_w_codes, const float* d_sw,
+int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
+                 const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
                  float* d_z, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Backward GEMM (Eq. Backward), SMP average fused (Sec. 5.1):
@@ -145,7 +159,7 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa,
  * g_codes: n_samples planes [M x N/2]; w_codes [N x K/2].
  * N and K must be multiples of 32. */
 int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
-                 const uint8_t* d_w_codes, const float* d_sw,
+                 const int8_t* d_g_operand, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
                  float* d_da, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Update GEMM (Eq. Update), SMP average fused (Sec. 5.1):
@@ -154,7 +168,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
  * N and K must be multiples of 32.  Uses the context's split workspace when
  * the output has few tiles (contraction over M is split across CTAs). */
 int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
-                   const uint8_t* d_a_codes, const float* d_sa,
+                   const int8_t* d_g_operand, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
                    float* d_dw, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Update GEMM without any allocation.  (The paper has no counterpart; this entry

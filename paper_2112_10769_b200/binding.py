@@ -46,15 +46,15 @@ def load() -> ctypes.CDLL:
         L.luq_set_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
         L.luq_kmax.argtypes = []
         L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
-        L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp]
-        L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp]
-        L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp]
+        L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
+        L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
+        L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, ctypes.c_int, u64,
-                                               ctypes.c_int, vp, vp, vp, vp]
+                                               ctypes.c_int, vp, vp, vp, vp, vp]
         L.luq_debug_quotient.argtypes = [vp, vp, sz, vp, vp, vp]
-        L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
-        L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
-        L.luq_gemm_wgrad.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_gemm_wgrad.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_wgrad_static.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
         L.luq_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int)]
         L.luq_launch_count.argtypes = [vp]
@@ -75,6 +75,15 @@ def _dtype_code(t: torch.Tensor) -> int:
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+def _opt(t, numel: int):
+    """Pointer of an optional int8 operand-byte tensor (None -> NULL), size and type checked."""
+    if t is None:
+        return None
+    if t.dtype != torch.int8 or t.numel() < numel or not t.is_contiguous():
+        raise TypeError(f"operand bytes: contiguous int8 tensor of at least {numel} elements expected")
+    return t.data_ptr()
 
 
 def _check(rc: int, what: str):
@@ -118,40 +127,46 @@ class Context:
                "luq_amax")
         return out
 
+    # `operand` (optional, int8, one byte per element and sample): filled with the tensor-core
+    # operand bytes in the same pass; hand it to the GEMMs together with the codes.
     def quant_int4(self, x: torch.Tensor, clip: torch.Tensor, codes: torch.Tensor | None = None,
-                   scale: torch.Tensor | None = None):
+                   scale: torch.Tensor | None = None, operand: torch.Tensor | None = None):
         rows, cols = (x.shape[0], x.numel() // max(x.shape[0], 1)) if x.dim() > 1 else (1, x.numel())
         codes = torch.empty(x.numel() // 2, dtype=torch.uint8, device=x.device) if codes is None else codes
         scale = torch.empty(1, dtype=torch.float32, device=x.device) if scale is None else scale
         _check(load().luq_quant_int4(self.handle, x.data_ptr(), _dtype_code(x), rows, cols, clip.data_ptr(),
-                                     codes.data_ptr(), scale.data_ptr(), _stream()), "luq_quant_int4")
+                                     codes.data_ptr(), scale.data_ptr(), _opt(operand, x.numel()), _stream()),
+               "luq_quant_int4")
         return codes, scale
 
     def quant_grad(self, g: torch.Tensor, amax: torch.Tensor, seed: int, n_samples: int = 1,
-                   codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None):
+                   codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None,
+                   operand: torch.Tensor | None = None):
         rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
         if codes is None:
             codes = torch.empty((n_samples, g.numel() // 2), dtype=torch.uint8, device=g.device)
         alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
         _check(load().luq_quant_grad(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
                                      seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
-                                     _stream()), "luq_quant_grad")
+                                     _opt(operand, n_samples * g.numel()), _stream()), "luq_quant_grad")
         return codes, alpha
 
     def quant_grad_pw2(self, g: torch.Tensor, amax: torch.Tensor, seed: int, n_samples: int = 1,
-                       codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None):
+                       codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None,
+                       operand: torch.Tensor | None = None):
         rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
         if codes is None:
             codes = torch.empty((n_samples, g.numel() // 2), dtype=torch.uint8, device=g.device)
         alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
         _check(load().luq_quant_grad_pw2(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
                                          seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
-                                         _stream()), "luq_quant_grad_pw2")
+                                         _opt(operand, n_samples * g.numel()), _stream()), "luq_quant_grad_pw2")
         return codes, alpha
 
     def quant_grad_hindsight(self, g: torch.Tensor, m_hat: torch.Tensor, eta: float, seed: int, n_samples: int = 1,
                              pw2: bool = False, codes: torch.Tensor | None = None,
-                             alpha: torch.Tensor | None = None, measured: torch.Tensor | None = None):
+                             alpha: torch.Tensor | None = None, measured: torch.Tensor | None = None,
+                             operand: torch.Tensor | None = None):
         """One pass: quantize with the estimate in `m_hat`, measure this tensor's maximum into
         `measured`, replace `m_hat` by the estimate for the next step."""
         rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
@@ -161,7 +176,8 @@ class Context:
         measured = torch.empty(1, dtype=torch.float32, device=g.device) if measured is None else measured
         _check(load().luq_quant_grad_hindsight(self.handle, g.data_ptr(), _dtype_code(g), rows, cols,
                                                m_hat.data_ptr(), eta, int(pw2), seed & (2 ** 64 - 1), n_samples,
-                                               codes.data_ptr(), alpha.data_ptr(), measured.data_ptr(), _stream()),
+                                               codes.data_ptr(), alpha.data_ptr(), measured.data_ptr(),
+                                               _opt(operand, n_samples * g.numel()), _stream()),
                "luq_quant_grad_hindsight")
         return codes, alpha, measured
 
@@ -171,26 +187,30 @@ class Context:
                                          _stream()), "luq_debug_quotient")
         return out
 
-    def gemm_fwd(self, a_codes, sa, w_codes, sw, M: int, N: int, K: int, out: torch.Tensor | None = None):
+    def gemm_fwd(self, a_codes, sa, w_codes, sw, M: int, N: int, K: int, out: torch.Tensor | None = None,
+                 a_operand: torch.Tensor | None = None, w_operand: torch.Tensor | None = None):
         out = torch.empty((M, N), dtype=torch.float32, device=a_codes.device) if out is None else out
-        _check(load().luq_gemm_fwd(self.handle, a_codes.data_ptr(), sa.data_ptr(), w_codes.data_ptr(),
-                                   sw.data_ptr(), out.data_ptr(), M, N, K, _stream()), "luq_gemm_fwd")
+        _check(load().luq_gemm_fwd(self.handle, a_codes.data_ptr(), sa.data_ptr(), _opt(a_operand, M * K),
+                                   w_codes.data_ptr(), sw.data_ptr(), _opt(w_operand, N * K), out.data_ptr(),
+                                   M, N, K, _stream()), "luq_gemm_fwd")
         return out
 
     def gemm_bwd(self, g_codes, alpha, n_samples: int, w_codes, sw, M: int, N: int, K: int,
-                 out: torch.Tensor | None = None):
+                 out: torch.Tensor | None = None, g_operand: torch.Tensor | None = None,
+                 w_operand: torch.Tensor | None = None):
         out = torch.empty((M, K), dtype=torch.float32, device=g_codes.device) if out is None else out
         _check(load().luq_gemm_bwd(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
-                                   w_codes.data_ptr(), sw.data_ptr(), out.data_ptr(), M, N, K, _stream()),
-               "luq_gemm_bwd")
+                                   _opt(g_operand, n_samples * M * N), w_codes.data_ptr(), sw.data_ptr(),
+                                   _opt(w_operand, N * K), out.data_ptr(), M, N, K, _stream()), "luq_gemm_bwd")
         return out
 
     def gemm_wgrad(self, g_codes, alpha, n_samples: int, a_codes, sa, M: int, N: int, K: int,
-                   out: torch.Tensor | None = None):
+                   out: torch.Tensor | None = None, g_operand: torch.Tensor | None = None,
+                   a_operand: torch.Tensor | None = None):
         out = torch.empty((N, K), dtype=torch.float32, device=g_codes.device) if out is None else out
         _check(load().luq_gemm_wgrad(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
-                                     a_codes.data_ptr(), sa.data_ptr(), out.data_ptr(), M, N, K, _stream()),
-               "luq_gemm_wgrad")
+                                     _opt(g_operand, n_samples * M * N), a_codes.data_ptr(), sa.data_ptr(),
+                                     _opt(a_operand, M * K), out.data_ptr(), M, N, K, _stream()), "luq_gemm_wgrad")
         return out
 
     def status(self) -> int:

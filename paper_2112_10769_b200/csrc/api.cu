@@ -111,70 +111,69 @@ int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, 
 }
 
 int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, const float* d_clip,
-                   uint8_t* d_codes, float* d_scale, void* stream) {
+                   uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream) {
   if (!ctx || !d_clip || !d_scale || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
   const size_t n = rows * cols;
   if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
   if (n & 1u) return LUQ_ERR_ARG;
   if (n && (!d_x || !d_codes)) return LUQ_ERR_ARG;
-  if (!aligned16(d_x) || !aligned16(d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_codes) || !aligned16(d_operand)) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
-  return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, d_clip, d_codes, d_scale, as_stream(stream)));
-}
-
-int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
-                   uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, void* stream) {
-  if (!ctx || !d_amax || !d_alpha || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
-  if (n_samples < 1 || n_samples > LUQ_MAX_SAMPLES) return LUQ_ERR_ARG;
-  const size_t n = rows * cols;
-  if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
-  if (n & 1u) return LUQ_ERR_ARG;
-  if (n && (!d_g || !d_codes)) return LUQ_ERR_ARG;
-  if (!aligned16(d_g) || !aligned16(d_codes)) return LUQ_ERR_ARG;
-  DeviceGuard guard(ctx->device);
-  if (!guard.ok) return LUQ_ERR_CUDA;
-  return cuda_rc(luq_launch_quant_grad(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes, d_alpha,
+  return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, d_clip, d_codes, n ? d_operand : nullptr, d_scale,
                                        as_stream(stream)));
 }
 
 static int quant_grad_args(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
-                           int n_samples, const uint8_t* d_codes, const float* d_alpha, size_t* n_out) {
+                           int n_samples, const uint8_t* d_codes, const float* d_alpha, const int8_t* d_operand,
+                           size_t* n_out) {
   if (!ctx || !d_amax || !d_alpha || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
   if (n_samples < 1 || n_samples > LUQ_MAX_SAMPLES) return LUQ_ERR_ARG;
   const size_t n = rows * cols;
   if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
   if (n & 1u) return LUQ_ERR_ARG;
   if (n && (!d_g || !d_codes)) return LUQ_ERR_ARG;
-  if (!aligned16(d_g) || !aligned16(d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_g) || !aligned16(d_codes) || !aligned16(d_operand)) return LUQ_ERR_ARG;
   *n_out = n;
   return LUQ_OK;
 }
 
-int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
-                       uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, void* stream) {
+int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
+                   uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream) {
   size_t n = 0;
-  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, &n);
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, d_operand, &n);
   if (rc) return rc;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
-  return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes, d_alpha, 1, nullptr,
-                                          as_stream(stream)));
+  return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
+                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, as_stream(stream)));
+}
+
+int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
+                       uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, int8_t* d_operand,
+                       void* stream) {
+  size_t n = 0;
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, d_operand, &n);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
+                                          n ? d_operand : nullptr, d_alpha, 1, nullptr, as_stream(stream)));
 }
 
 int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, float* d_mhat,
                              float eta, int pw2, uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha,
-                             float* d_measured_max, void* stream) {
+                             float* d_measured_max, int8_t* d_operand, void* stream) {
   size_t n = 0;
-  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_mhat, n_samples, d_codes, d_alpha, &n);
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_mhat, n_samples, d_codes, d_alpha, d_operand, &n);
   if (rc) return rc;
   if (!d_measured_max || !(eta >= 0.0f && eta <= 1.0f) || (pw2 != 0 && pw2 != 1)) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   cudaStream_t st = as_stream(stream);
   if (cudaMemsetAsync(d_measured_max, 0, sizeof(float), st) != cudaSuccess) return LUQ_ERR_CUDA;
-  int e = luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_mhat, seed, n_samples, d_codes, d_alpha, 2 | pw2,
-                                   d_measured_max, st);
+  int e = luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_mhat, seed, n_samples, d_codes, n ? d_operand : nullptr,
+                                   d_alpha, 2 | pw2, d_measured_max, st);
   if (e) return cuda_rc(e);
   return cuda_rc(luq_launch_hindsight_update(ctx, d_mhat, d_measured_max, eta, st));
 }
@@ -186,19 +185,21 @@ int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_
   return cuda_rc(luq_launch_debug_quotient(ctx, d_x, n, d_amax, d_t, as_stream(stream)));
 }
 
-static int gemm_common(luq_ctx* ctx, const uint8_t* x, const float* sx, const uint8_t* y, const float* sy,
-                       float* out, int64_t M, int64_t N, int64_t K, int n_samples) {
+static int gemm_common(luq_ctx* ctx, const uint8_t* x, const float* sx, const int8_t* xo, const uint8_t* y,
+                       const float* sy, const int8_t* yo, float* out, int64_t M, int64_t N, int64_t K,
+                       int n_samples) {
   if (!ctx || !sx || !sy) return LUQ_ERR_ARG;
   if (M < 0 || N < 0 || K < 0 || M > (1ll << 31) || N > (1ll << 31) || K > (1ll << 31)) return LUQ_ERR_ARG;
   if (n_samples < 1 || n_samples > LUQ_MAX_SAMPLES) return LUQ_ERR_ARG;
   if (M && N && K && (!x || !y || !out)) return LUQ_ERR_ARG;
-  if (!aligned16(x) || !aligned16(y) || !aligned16(out)) return LUQ_ERR_ARG;
+  if (!aligned16(x) || !aligned16(y) || !aligned16(out) || !aligned16(xo) || !aligned16(yo)) return LUQ_ERR_ARG;
   return LUQ_OK;
 }
 
-int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, const uint8_t* d_w_codes,
-                 const float* d_sw, float* d_z, int64_t M, int64_t N, int64_t K, void* stream) {
-  int rc = gemm_common(ctx, d_a_codes, d_sa, d_w_codes, d_sw, d_z, M, N, K, 1);
+int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
+                 const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand, float* d_z, int64_t M,
+                 int64_t N, int64_t K, void* stream) {
+  int rc = gemm_common(ctx, d_a_codes, d_sa, d_a_operand, d_w_codes, d_sw, d_w_operand, d_z, M, N, K, 1);
   if (rc) return rc;
   if (K % 32 || N % 4) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);
@@ -206,6 +207,7 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, cons
   luq_gemm_args a{};
   a.a_codes = d_a_codes; a.a_kind = 0; a.a_mn = 0; a.n_samples = 1;
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 0;
+  a.a_operand = d_a_operand; a.b_operand = d_w_operand;
   a.d_scale_a = d_sa; a.d_scale_b = d_sw; a.d_out = d_z; a.Mo = M; a.No = N; a.Kc = K;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;
@@ -213,9 +215,9 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, cons
 }
 
 int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
-                 const uint8_t* d_w_codes, const float* d_sw, float* d_da, int64_t M, int64_t N, int64_t K,
-                 void* stream) {
-  int rc = gemm_common(ctx, d_g_codes, d_alpha, d_w_codes, d_sw, d_da, M, N, K, n_samples);
+                 const int8_t* d_g_operand, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
+                 float* d_da, int64_t M, int64_t N, int64_t K, void* stream) {
+  int rc = gemm_common(ctx, d_g_codes, d_alpha, d_g_operand, d_w_codes, d_sw, d_w_operand, d_da, M, N, K, n_samples);
   if (rc) return rc;
   if (N % 32 || K % 32) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);
@@ -223,6 +225,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
   luq_gemm_args a{};
   a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 0; a.n_samples = n_samples;   // G[M x N]: contraction n contiguous
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 1;                            // W[N x K]: rows are the contraction
+  a.a_operand = d_g_operand; a.b_operand = d_w_operand;
   a.d_scale_a = d_alpha; a.d_scale_b = d_sw; a.d_out = d_da; a.Mo = M; a.No = K; a.Kc = N;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;
@@ -230,9 +233,9 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
 }
 
 int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
-                   const uint8_t* d_a_codes, const float* d_sa, float* d_dw, int64_t M, int64_t N, int64_t K,
-                   void* stream) {
-  int rc = gemm_common(ctx, d_g_codes, d_alpha, d_a_codes, d_sa, d_dw, M, N, K, n_samples);
+                   const int8_t* d_g_operand, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
+                   float* d_dw, int64_t M, int64_t N, int64_t K, void* stream) {
+  int rc = gemm_common(ctx, d_g_codes, d_alpha, d_g_operand, d_a_codes, d_sa, d_a_operand, d_dw, M, N, K, n_samples);
   if (rc) return rc;
   if (N % 32 || K % 32) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);
@@ -240,6 +243,7 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
   luq_gemm_args a{};
   a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 1; a.n_samples = n_samples;   // G[M x N]: rows are the contraction
   a.b_codes = d_a_codes; a.b_kind = 0; a.b_mn = 1;                            // A[M x K]: rows are the contraction
+  a.a_operand = d_g_operand; a.b_operand = d_a_operand;
   a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.Mo = N; a.No = K; a.Kc = M;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;

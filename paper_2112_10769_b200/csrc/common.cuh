@@ -7,7 +7,7 @@
 #include "luq.h"
 
 #define LUQ_KMAX 4  // alpha = max / 2^LUQ_KMAX (Eq. alpha with b = 3)
-#define LUQ_DEFAULT_MMA_KIND 2  // chosen per product: int8 where INT4 codes are expanded in the kernel, else e4m3
+#define LUQ_DEFAULT_MMA_KIND 2  // automatic: int8, the type of the operand bytes the quantizers can emit
 
 struct luq_ctx {
   int device;
@@ -24,15 +24,14 @@ struct luq_ctx {
 
 // internal launchers (defined in quant.cu / gemm.cu); return a cudaError_t as int
 int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, cudaStream_t st);
+// d_operand (may be null): int8 operand bytes, one per element (and per sample), written with the codes
 int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
-                          uint8_t* d_codes, float* d_scale, cudaStream_t st);
-int luq_launch_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
-                          uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, cudaStream_t st);
+                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, cudaStream_t st);
 
 // flags: bit 0 = power-of-two scale, bit 1 = also reduce max|x| of this tensor into d_measured (pre-zeroed)
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
-                             int n_samples, uint8_t* d_codes, float* d_alpha, int flags, float* d_measured,
-                             cudaStream_t st);
+                             int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
+                             float* d_measured, cudaStream_t st);
 int luq_launch_hindsight_update(luq_ctx* ctx, float* d_mhat, const float* d_measured, float eta, cudaStream_t st);
 int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,
                               cudaStream_t st);
@@ -43,6 +42,7 @@ int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const fl
 struct luq_gemm_args {
   const uint8_t* a_codes; int a_kind; int a_mn; int n_samples;
   const uint8_t* b_codes; int b_kind; int b_mn;
+  const int8_t* a_operand; const int8_t* b_operand;   // int8 operand bytes from the quantizer, or null
   const float* d_scale_a; const float* d_scale_b;
   float* d_out; int64_t Mo, No, Kc;
   float* d_workspace; size_t workspace_bytes;   // split partial tiles (caller-chosen memory)

@@ -209,6 +209,9 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const int units = p.tiles_m * p.tiles_n * p.splits;
   const int total_iters = p.n_samples * p.num_kb;
 
+  // consecutive tiles walk down the rows of one column panel: the CTAs that run at the same time share the panel of B
+  auto tile_m = [&](int tile) { return tile % p.tiles_m; };
+  auto tile_n = [&](int tile) { return tile / p.tiles_m; };
   auto unit_range = [&](int u, int& tile, int& it_begin, int& it_end) {
     tile = u / p.splits;
     const int sp = u - tile * p.splits;
@@ -226,8 +229,8 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
         int tile, it_begin, it_end;
         unit_range(u, tile, it_begin, it_end);
-        const int m0 = (tile % p.tiles_m) * BM;
-        const int n0 = (tile / p.tiles_m) * BN;
+        const int m0 = tile_m(tile) * BM;
+        const int n0 = tile_n(tile) * BN;
         int sample = it_begin / p.num_kb;
         int kb = it_begin - sample * p.num_kb;
         for (int k_it = it_begin; k_it < it_end; ++k_it) {
@@ -268,8 +271,8 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
         int tile, it_begin, it_end;
         unit_range(u, tile, it_begin, it_end);
-        const int m0 = (tile % p.tiles_m) * BM;
-        const int n0 = (tile / p.tiles_m) * BN;
+        const int m0 = tile_m(tile) * BM;
+        const int n0 = tile_n(tile) * BN;
         int sample = it_begin / p.num_kb;
         int kb = it_begin - sample * p.num_kb;
         for (int k_it = it_begin; k_it < it_end; ++k_it) {
@@ -354,9 +357,9 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       int tile, it_begin, it_end;
       unit_range(u, tile, it_begin, it_end);
       // a split stores its whole partial tile at row u*128 of the workspace
-      const long long row0 = (p.splits == 1 ? static_cast<long long>(tile % p.tiles_m) * BM
+      const long long row0 = (p.splits == 1 ? static_cast<long long>(tile_m(tile)) * BM
                                             : static_cast<long long>(u) * BM) + quarter * 32;
-      const long long col_base = p.splits == 1 ? static_cast<long long>(tile / p.tiles_m) * BN : 0;
+      const long long col_base = p.splits == 1 ? static_cast<long long>(tile_n(tile)) * BN : 0;
       const long long row_limit = p.splits == 1 ? p.Mo : static_cast<long long>(units) * BM;
       const long long col_limit = p.splits == 1 ? p.No : BN;
       const uint32_t buf = tile_it & 1u;
@@ -859,53 +862,66 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   }
   const long long units = tiles * p.splits;
 
-  // Operand planes: an operand that at least two tiles re-read is expanded once, if the
-  // workspace behind the split region has room for it.  A product with a short contraction
-  // is bound by its output stream and hides the in-kernel expansion completely (measured:
-  // the backward product of the ResNet shape, 2 blocks per tile), so it keeps the codes.
+  // Operand type.  "Automatic" is int8: INT4 codes expand to it in three instructions per eight
+  // codes, and it is the type of the operand bytes the quantizers can write themselves.
+  // Where an int32 accumulator could wrap (a very long contraction) it is e4m3 with fp32 accumulators.
+  const long long worst_product = static_cast<long long>(a.a_kind == 0 ? 7 * 16 : 64) * (a.b_kind == 0 ? 7 * 16 : 64);
+  const bool int32_safe = worst_product * a.Kc * a.n_samples < (1ll << 31);
+  if (ctx->mma_kind == 2) ctx->mma_kind = int32_safe ? 1 : 0;
+  if (ctx->mma_kind == 1 && !int32_safe) return LUQ_ERR_ARG;
+  // Operand planes: an operand that at least two tiles re-read is fetched as bytes.  The caller's
+  // bytes (written by the quantizer, int8) are taken as they are; otherwise the codes are expanded
+  // once into the workspace behind the split region, if there is room.  A product with a short
+  // contraction is bound by its output stream and hides the in-kernel expansion completely
+  // (measured: the backward product of the ResNet shape, 2 blocks per tile), so it keeps the codes.
   const size_t a_plane_bytes = static_cast<size_t>(a.Mo) * a.Kc * a.n_samples;
   const size_t b_plane_bytes = static_cast<size_t>(a.No) * a.Kc;
   size_t plane_room = (a.d_workspace && a.workspace_bytes > kSplitRegionBytes) ? a.workspace_bytes - kSplitRegionBytes : 0;
   uint8_t* plane_ptr = a.d_workspace ? reinterpret_cast<uint8_t*>(a.d_workspace) + kSplitRegionBytes : nullptr;
   auto packed_ok = [](size_t bytes) { return bytes % 32 == 0; };   // whole 16-byte pieces of packed codes
-  bool b_plane = false, a_plane = false;
+  const uint8_t* a_given = ctx->mma_kind == 1 ? reinterpret_cast<const uint8_t*>(a.a_operand) : nullptr;
+  const uint8_t* b_given = ctx->mma_kind == 1 ? reinterpret_cast<const uint8_t*>(a.b_operand) : nullptr;
+  bool b_plane = false, a_plane = false, b_expand = false, a_expand = false;
   const bool long_contraction = total_iters >= 8;
-  uint8_t* b_plane_ptr = nullptr; uint8_t* a_plane_ptr = nullptr;
-  if (long_contraction && p.tiles_m >= 2 && packed_ok(b_plane_bytes) && b_plane_bytes <= plane_room) {
-    b_plane = true; b_plane_ptr = plane_ptr;
-    const size_t used = (b_plane_bytes + 1023) & ~static_cast<size_t>(1023);
-    plane_ptr += used; plane_room -= used <= plane_room ? used : plane_room;
+  const uint8_t* b_plane_ptr = nullptr; const uint8_t* a_plane_ptr = nullptr;
+  if (long_contraction && p.tiles_m >= 2) {
+    if (b_given) {
+      b_plane = true; b_plane_ptr = b_given;
+    } else if (packed_ok(b_plane_bytes) && b_plane_bytes <= plane_room) {
+      b_plane = b_expand = true; b_plane_ptr = plane_ptr;
+      const size_t used = (b_plane_bytes + 1023) & ~static_cast<size_t>(1023);
+      plane_ptr += used; plane_room -= used <= plane_room ? used : plane_room;
+    }
   }
-  if (long_contraction && p.tiles_n >= 2 && packed_ok(a_plane_bytes) && a_plane_bytes <= plane_room) {
-    a_plane = true; a_plane_ptr = plane_ptr;
+  if (long_contraction && p.tiles_n >= 2) {
+    if (a_given) {
+      a_plane = true; a_plane_ptr = a_given;
+    } else if (packed_ok(a_plane_bytes) && a_plane_bytes <= plane_room) {
+      a_plane = a_expand = true; a_plane_ptr = plane_ptr;
+    }
   }
-  // Operand type.  "Automatic" takes int8 whenever an INT4 operand is expanded inside the
-  // kernel (three instructions per eight codes instead of a table lookup) and e4m3 when both
-  // operands arrive as planes (fp32 accumulators spare the epilogue the int-to-float conversions).
-  if (ctx->mma_kind == 2) ctx->mma_kind = (a_plane && b_plane) ? 0 : 1;
   p.lut_a = make_lut(ctx->mma_kind, a.a_kind);
   p.lut_b = make_lut(ctx->mma_kind, a.b_kind);
   // int8 operands carry INT4 integers as 16*q: undo with an exact power of two
   float pow2 = 1.0f;
   if (ctx->mma_kind == 1) {
-    const int a_mag = a.a_kind == 0 ? 7 * 16 : 64, b_mag = a.b_kind == 0 ? 7 * 16 : 64;
     if (a.a_kind == 0) pow2 *= 1.0f / 16.0f;
     if (a.b_kind == 0) pow2 *= 1.0f / 16.0f;
-    const long long worst = static_cast<long long>(a_mag) * b_mag;   // largest |operand product|
-    if (worst * a.Kc * a.n_samples >= (1ll << 31)) return LUQ_ERR_ARG;  // the int32 accumulator could wrap
   }
   p.post_scale = (1.0f / static_cast<float>(a.n_samples)) * pow2;
 
   int rc = 0;
-  if (b_plane) {
-    rc = ctx->mma_kind ? launch_expand<1>(a.b_kind == 1, a.b_codes, b_plane_ptr, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st)
-                       : launch_expand<0>(a.b_kind == 1, a.b_codes, b_plane_ptr, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st);
+  if (b_expand) {
+    uint8_t* dst = const_cast<uint8_t*>(b_plane_ptr);   // workspace memory
+    rc = ctx->mma_kind ? launch_expand<1>(a.b_kind == 1, a.b_codes, dst, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st)
+                       : launch_expand<0>(a.b_kind == 1, a.b_codes, dst, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st);
     if (rc != 0) return rc;
     ctx->launches += 1;
   }
-  if (a_plane) {
-    rc = ctx->mma_kind ? launch_expand<1>(a.a_kind == 1, a.a_codes, a_plane_ptr, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st)
-                       : launch_expand<0>(a.a_kind == 1, a.a_codes, a_plane_ptr, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st);
+  if (a_expand) {
+    uint8_t* dst = const_cast<uint8_t*>(a_plane_ptr);   // workspace memory
+    rc = ctx->mma_kind ? launch_expand<1>(a.a_kind == 1, a.a_codes, dst, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st)
+                       : launch_expand<0>(a.a_kind == 1, a.a_codes, dst, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st);
     if (rc != 0) return rc;
     ctx->launches += 1;
   }

@@ -67,6 +67,17 @@ template <bool BF16> struct Item {
       for (int b = 0; b < kElems / 2; ++b) plane_base[item * (kElems / 2) + b] = static_cast<uint8_t>(word >> (8 * b));
     }
   }
+  // store the operand bytes of one piece (4 bytes for fp32 input, 8 for bf16); w[j] holds elements 4j..4j+3
+  static __device__ __forceinline__ void store_bytes(int8_t* bytes_base, size_t item, const uint32_t (&w)[kElems / 4],
+                                                     bool aligned) {
+    if (aligned) {
+      if constexpr (BF16) reinterpret_cast<uint2*>(bytes_base)[item] = make_uint2(w[0], w[1]);
+      else reinterpret_cast<uint32_t*>(bytes_base)[item] = w[0];
+    } else {
+#pragma unroll
+      for (int b = 0; b < kElems; ++b) bytes_base[item * kElems + b] = static_cast<int8_t>(w[b / 4] >> (8 * (b % 4)));
+    }
+  }
 };
 
 // ------------------------------------------------------------------ amax ----
@@ -139,10 +150,13 @@ __device__ __forceinline__ uint32_t int4_code(float x, float inv) {
   return (y == y) ? code : 0u;        // NaN element -> 0
 }
 
-template <bool BF16>
+// PLANE: the tensor-core operand bytes (int8, 16 * q: the code nibble in the high half of the
+// byte) are written next to the packed codes, one byte per element in element order.
+template <bool BF16, bool PLANE>
 __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __restrict__ x, size_t n,
                                                               const float* __restrict__ d_clip,
                                                               uint8_t* __restrict__ codes,
+                                                              int8_t* __restrict__ operand,
                                                               float* __restrict__ d_scale,
                                                               unsigned int* __restrict__ status) {
   constexpr int kElems = Item<BF16>::kElems;
@@ -154,14 +168,19 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
 
   const size_t items = n / kElems;
   const uint4* p = reinterpret_cast<const uint4*>(x);
-  auto encode = [&](const uint4& u) -> uint32_t {
-    if (!ok) return 0u;
+  auto emit = [&](size_t item, const uint4& u) {
     float v[kElems];
     Item<BF16>::widen(u, v);
     uint32_t word = 0;
+    uint32_t bytes[kElems / 4] = {};
 #pragma unroll
-    for (int j = 0; j < kElems; ++j) word |= int4_code(v[j], inv) << (4 * j);
-    return word;
+    for (int j = 0; j < kElems; ++j) {
+      const uint32_t code = ok ? int4_code(v[j], inv) : 0u;
+      word |= code << (4 * j);
+      if constexpr (PLANE) bytes[j / 4] |= code << (8 * (j % 4) + 4);
+    }
+    Item<BF16>::store(codes, item, word, true);
+    if constexpr (PLANE) Item<BF16>::store_bytes(operand, item, bytes, true);
   };
   // The tensor was just read front to back by the max reduction; its tail is what the
   // L2 still holds, so this pass walks the tiles from the back.
@@ -172,16 +191,19 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i0 + j * kThreads);
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) Item<BF16>::store(codes, i0 + j * kThreads, encode(u[j]), true);
+    for (int j = 0; j < kUnroll; ++j) emit(i0 + j * kThreads, u[j]);
   }
   if (blockIdx.x == gridDim.x - 1)
-    for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads)
-      Item<BF16>::store(codes, i, encode(__ldg(p + i)), true);
+    for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) emit(i, __ldg(p + i));
   if (first) {  // tail: fewer elements than one piece, two per byte
     for (size_t e = items * kElems; e < n; e += 2) {
       const uint32_t lo = ok ? int4_code(Item<BF16>::load1(x, e), inv) : 0u;
       const uint32_t hi = (ok && e + 1 < n) ? int4_code(Item<BF16>::load1(x, e + 1), inv) : 0u;
       codes[e >> 1] = static_cast<uint8_t>(lo | (hi << 4));
+      if constexpr (PLANE) {
+        operand[e] = static_cast<int8_t>(lo << 4);
+        if (e + 1 < n) operand[e + 1] = static_cast<int8_t>(hi << 4);
+      }
     }
   }
 }
@@ -265,6 +287,11 @@ __device__ __forceinline__ uint32_t luq_nibble(uint32_t xbits, uint32_t lo_code,
   const uint32_t c = lo_code + (word < thr ? 1u : 0u);
   return c ? (((xbits >> 28) & 8u) | c) : 0u;
 }
+// the tensor-core operand byte of a LUQ nibble: int8 value +-2^(c-1), 0 for code 0
+__device__ __forceinline__ uint32_t luq_operand_byte(uint32_t nibble) {
+  const uint32_t mag = (1u << (nibble & 7u)) >> 1;
+  return ((nibble & 8u) ? 0u - mag : mag) & 0xFFu;
+}
 
 // 2^ceil(log2 m) for a positive finite m (power-of-two LUQ: the maximum is rounded up, never down)
 __device__ __forceinline__ float pw2_ceil(float m) {
@@ -277,12 +304,15 @@ __device__ __forceinline__ float pw2_ceil(float m) {
 // PW2: the scale is a power of two, the quotient an exact scaling (one multiply).
 // TRACK: the tensor's own max|x| is reduced on the way (in-hindsight estimation: the scale
 // in d_amax is an estimate from earlier steps, the measured maximum feeds the next one).
-template <bool BF16, int NS, bool PW2, bool TRACK>
+// PLANE: the tensor-core operand bytes (int8, +-2^(c-1)) of every sample are written next to
+// the packed codes, one byte per element, sample s at offset s * n.
+template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
 __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restrict__ x, size_t n,
                                                              const float* __restrict__ d_amax,
                                                              const __grid_constant__ PhiloxKeySet keys,
                                                              int n_samples_rt,
                                                              uint8_t* __restrict__ codes,
+                                                             int8_t* __restrict__ operand,
                                                              float* __restrict__ d_alpha,
                                                              unsigned int* __restrict__ measured_bits,
                                                              unsigned int* __restrict__ status) {
@@ -299,6 +329,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
 
   const size_t plane = n / 2;
   const bool aligned = (plane % (kElems / 2)) == 0;  // planes start on a store boundary
+  const bool aligned_op = (n % kElems) == 0;
   const size_t items = n / kElems;
   const uint4* p = reinterpret_cast<const uint4*>(x);
 
@@ -318,26 +349,32 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
     }
     // the vote needs every lane of the warp here: only the full-tile loop qualifies
     if (whole_warp && !__any_sync(0xFFFFFFFFu, in_range)) {
-      uint32_t thr[kElems], sn[kElems];
+      uint32_t thr[kElems], sn[kElems], ob[kElems];
 #pragma unroll
       for (int j = 0; j < kElems; ++j) {
         thr[j] = __float2uint_rz(luq_quotient_raw<PW2>(v[j], sc) * 4294967296.0f);
         sn[j] = ((__float_as_uint(v[j]) >> 28) & 8u) | 1u;
+        if constexpr (PLANE) ob[j] = (__float_as_uint(v[j]) >> 31) ? 0xFFu : 0x01u;   // -1 or +1
       }
 #pragma unroll
       for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
         if (NS == 0 && s >= n_samples) break;
         const PhiloxKeys& ks = keys.s[s];
         uint32_t word = 0;
+        uint32_t bytes[kElems / 4] = {};
 #pragma unroll
         for (int b = 0; b < kElems / 4; ++b) {
           const uint4 r = philox_block(item * (kElems / 4) + b, ks);
           const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            word += (rw[j] < thr[4 * b + j] ? sn[4 * b + j] : 0u) << (4 * (4 * b + j));
+          for (int j = 0; j < 4; ++j) {
+            const bool up = rw[j] < thr[4 * b + j];
+            word += (up ? sn[4 * b + j] : 0u) << (4 * (4 * b + j));
+            if constexpr (PLANE) bytes[b] += (up ? ob[4 * b + j] : 0u) << (8 * j);
+          }
         }
         Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
+        if constexpr (PLANE) Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
       }
       return;
     }
@@ -349,16 +386,20 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
       if (NS == 0 && s >= n_samples) break;
       const PhiloxKeys& ks = keys.s[s];
       uint32_t word = 0;
+      uint32_t bytes[kElems / 4] = {};
 #pragma unroll
       for (int b = 0; b < kElems / 4; ++b) {
         const uint4 r = philox_block(item * (kElems / 4) + b, ks);
         const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          word |= luq_nibble(__float_as_uint(v[4 * b + j]), lo_code[4 * b + j], thr[4 * b + j], rw[j])
-                  << (4 * (4 * b + j));
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t nib = luq_nibble(__float_as_uint(v[4 * b + j]), lo_code[4 * b + j], thr[4 * b + j], rw[j]);
+          word |= nib << (4 * (4 * b + j));
+          if constexpr (PLANE) bytes[b] |= luq_operand_byte(nib) << (8 * j);
+        }
       }
       Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
+      if constexpr (PLANE) Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
     }
   };
 
@@ -377,7 +418,13 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
   } else {
     const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
     for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < items; i += stride) {
-      for (int s = 0; s < n_samples; ++s) Item<BF16>::store(codes + plane * s, i, 0u, aligned || s == 0);
+      for (int s = 0; s < n_samples; ++s) {
+        Item<BF16>::store(codes + plane * s, i, 0u, aligned || s == 0);
+        if constexpr (PLANE) {
+          const uint32_t zero[kElems / 4] = {};
+          Item<BF16>::store_bytes(operand + n * s, i, zero, aligned_op || s == 0);
+        }
+      }
       if constexpr (TRACK) {   // an unusable estimate still needs this tensor's maximum for the next step
         float v[kElems];
         Item<BF16>::widen(__ldg(p + i), v);
@@ -405,6 +452,10 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
           }
         }
         codes[plane * s + (e >> 1)] = static_cast<uint8_t>(nib[0] | (nib[1] << 4));
+        if constexpr (PLANE) {
+          operand[n * s + e] = static_cast<int8_t>(luq_operand_byte(nib[0]));
+          if (e + 1 < n) operand[n * s + e + 1] = static_cast<int8_t>(luq_operand_byte(nib[1]));
+        }
       }
     }
   }
@@ -482,38 +533,58 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
   return static_cast<int>(cudaGetLastError());
 }
 
-int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
-                          uint8_t* d_codes, float* d_scale, cudaStream_t st) {
-  if (dtype == LUQ_BF16) {
-    const int grid = grid_for(ctx, quant_int4_kernel<true>, n / 8 / kTileItems + 1);
-    quant_int4_kernel<true><<<grid, kThreads, 0, st>>>(d_x, n, d_clip, d_codes, d_scale, ctx->d_status);
-  } else {
-    const int grid = grid_for(ctx, quant_int4_kernel<false>, n / 4 / kTileItems + 1);
-    quant_int4_kernel<false><<<grid, kThreads, 0, st>>>(d_x, n, d_clip, d_codes, d_scale, ctx->d_status);
-  }
-  ctx->launches += 1;
+namespace {
+template <bool BF16, bool PLANE>
+int launch_int4(luq_ctx* ctx, const void* d_x, size_t n, const float* d_clip, uint8_t* d_codes, int8_t* d_operand,
+                float* d_scale, cudaStream_t st) {
+  const int grid = grid_for(ctx, quant_int4_kernel<BF16, PLANE>, n / Item<BF16>::kElems / kTileItems + 1);
+  quant_int4_kernel<BF16, PLANE><<<grid, kThreads, 0, st>>>(d_x, n, d_clip, d_codes, d_operand, d_scale, ctx->d_status);
   return static_cast<int>(cudaGetLastError());
+}
+}  // namespace
+
+int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
+                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, cudaStream_t st) {
+  const bool bf = dtype == LUQ_BF16;
+  int rc;
+  if (d_operand) rc = bf ? launch_int4<true, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, st)
+                         : launch_int4<false, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, st);
+  else rc = bf ? launch_int4<true, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, st)
+               : launch_int4<false, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, st);
+  ctx->launches += 1;
+  return rc;
 }
 
 namespace {
+template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
+int launch_luq_ns(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys,
+                  int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, unsigned int* d_measured,
+                  cudaStream_t st) {
+  const size_t tiles = n / Item<BF16>::kElems / kTileItems + 1;
+  const int grid = grid_for(ctx, quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, tiles);
+  quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, n_samples, d_codes,
+                                                                           d_operand, d_alpha, d_measured,
+                                                                           ctx->d_status);
+  return static_cast<int>(cudaGetLastError());
+}
+
+template <bool BF16, bool PW2, bool TRACK, bool PLANE>
+int launch_luq_plane(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys,
+                     int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, unsigned int* d_measured,
+                     cudaStream_t st) {
+  if (n_samples == 1)
+    return launch_luq_ns<BF16, 1, PW2, TRACK, PLANE>(ctx, d_g, n, d_amax, keys, 1, d_codes, d_operand, d_alpha, d_measured, st);
+  if (n_samples == 2)
+    return launch_luq_ns<BF16, 2, PW2, TRACK, PLANE>(ctx, d_g, n, d_amax, keys, 2, d_codes, d_operand, d_alpha, d_measured, st);
+  return launch_luq_ns<BF16, 0, PW2, TRACK, PLANE>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, d_measured, st);
+}
+
 template <bool BF16, bool PW2, bool TRACK>
 int launch_luq(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys, int n_samples,
-               uint8_t* d_codes, float* d_alpha, unsigned int* d_measured, cudaStream_t st) {
-  const size_t thread_items = n / Item<BF16>::kElems / kTileItems + 1;
-  if (n_samples == 1) {
-    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 1, PW2, TRACK>, thread_items);
-    quant_luq_kernel<BF16, 1, PW2, TRACK><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 1, d_codes, d_alpha,
-                                                                     d_measured, ctx->d_status);
-  } else if (n_samples == 2) {
-    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 2, PW2, TRACK>, thread_items);
-    quant_luq_kernel<BF16, 2, PW2, TRACK><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, 2, d_codes, d_alpha,
-                                                                     d_measured, ctx->d_status);
-  } else {
-    const int grid = grid_for(ctx, quant_luq_kernel<BF16, 0, PW2, TRACK>, thread_items);
-    quant_luq_kernel<BF16, 0, PW2, TRACK><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, n_samples, d_codes,
-                                                                     d_alpha, d_measured, ctx->d_status);
-  }
-  return static_cast<int>(cudaGetLastError());
+               uint8_t* d_codes, int8_t* d_operand, float* d_alpha, unsigned int* d_measured, cudaStream_t st) {
+  if (d_operand)
+    return launch_luq_plane<BF16, PW2, TRACK, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, d_measured, st);
+  return launch_luq_plane<BF16, PW2, TRACK, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, nullptr, d_alpha, d_measured, st);
 }
 
 PhiloxKeySet expand_keys(uint64_t seed, int n_samples) {
@@ -528,27 +599,22 @@ PhiloxKeySet expand_keys(uint64_t seed, int n_samples) {
 }  // namespace
 
 // flags: bit 0 = power-of-two scale, bit 1 = track this tensor's maximum into d_measured
-int luq_launch_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
-                          uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, cudaStream_t st) {
-  return luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes, d_alpha, 0, nullptr, st);
-}
-
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
-                             int n_samples, uint8_t* d_codes, float* d_alpha, int flags, float* d_measured,
-                             cudaStream_t st) {
+                             int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
+                             float* d_measured, cudaStream_t st) {
   const PhiloxKeySet keys = expand_keys(seed, n_samples);
   unsigned int* meas = reinterpret_cast<unsigned int*>(d_measured);
   const bool bf = dtype == LUQ_BF16;
   int rc;
   switch ((flags & 3) | (bf ? 4 : 0)) {
-    case 0: rc = launch_luq<false, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
-    case 1: rc = launch_luq<false, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
-    case 2: rc = launch_luq<false, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
-    case 3: rc = launch_luq<false, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
-    case 4: rc = launch_luq<true, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
-    case 5: rc = launch_luq<true, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
-    case 6: rc = launch_luq<true, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
-    default: rc = launch_luq<true, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_alpha, meas, st); break;
+    case 0: rc = launch_luq<false, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+    case 1: rc = launch_luq<false, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+    case 2: rc = launch_luq<false, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+    case 3: rc = launch_luq<false, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+    case 4: rc = launch_luq<true, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+    case 5: rc = launch_luq<true, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+    case 6: rc = launch_luq<true, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+    default: rc = launch_luq<true, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
   }
   ctx->launches += 1;
   return rc;

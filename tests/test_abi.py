@@ -41,9 +41,9 @@ def test_constants_and_messages(lib):
 def test_null_arguments_are_rejected_without_a_gpu(lib):
     assert lib.luq_create(None, 0) == binding.ERR_ARG
     assert lib.luq_amax(None, None, 0, 0, None, None) == binding.ERR_ARG
-    assert lib.luq_quant_int4(None, None, 0, 0, 0, None, None, None, None) == binding.ERR_ARG
-    assert lib.luq_quant_grad(None, None, 0, 0, 0, None, 0, 1, None, None, None) == binding.ERR_ARG
-    assert lib.luq_gemm_fwd(None, None, None, None, None, None, 1, 1, 32, None) == binding.ERR_ARG
+    assert lib.luq_quant_int4(None, None, 0, 0, 0, None, None, None, None, None) == binding.ERR_ARG
+    assert lib.luq_quant_grad(None, None, 0, 0, 0, None, 0, 1, None, None, None, None) == binding.ERR_ARG
+    assert lib.luq_gemm_fwd(None, None, None, None, None, None, None, None, 1, 1, 32, None) == binding.ERR_ARG
     assert lib.luq_status(None, None, None) == binding.ERR_ARG
     assert lib.luq_destroy(None) == 0
     assert lib.luq_launch_count(None) == 0

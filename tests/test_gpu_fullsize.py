@@ -46,19 +46,26 @@ def check_entries(got, ref):
     assert (np.abs(got - ref) <= RTOL * np.abs(ref) + floor).all()
 
 
+@pytest.mark.parametrize("operand_bytes", [True, False])
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg5"])
-def test_layer_configs_full_size(ctx, name):
+def test_layer_configs_full_size(ctx, name, operand_bytes):
+    """operand_bytes=True is the configuration bench.py times: the quantizers also write the 8-bit
+    operand form of W and G (and of A for wide layers) and the GEMMs are handed those bytes."""
     cfg = inputs.CONFIGS[name]
     M, K, N, ns, seed = cfg.M, cfg.K, cfg.N, cfg.n_samples, cfg.luq_seed
     A, W, G = inputs.layer_inputs(cfg)
     Ad, Wd, Gd = to_dev(A), to_dev(W), to_dev(G)
     mA, mW, mG = ctx.amax(Ad), ctx.amax(Wd), ctx.amax(Gd)
-    ca, sa = ctx.quant_int4(Ad, mA)
-    cw, sw = ctx.quant_int4(Wd, mW)
-    cg, al = ctx.quant_grad(Gd, mG, seed, ns)
-    Z = ctx.gemm_fwd(ca, sa, cw, sw, M, N, K)
-    dA = ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K)
-    dW = ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K)
+    i8 = lambda n: torch.empty(n, dtype=torch.int8, device="cuda")  # noqa: E731
+    bW = i8(N * K) if operand_bytes else None
+    bG = i8(ns * M * N) if operand_bytes else None
+    bA = i8(M * K) if operand_bytes and N >= 1024 else None
+    ca, sa = ctx.quant_int4(Ad, mA, operand=bA)
+    cw, sw = ctx.quant_int4(Wd, mW, operand=bW)
+    cg, al = ctx.quant_grad(Gd, mG, seed, ns, operand=bG)
+    Z = ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=bA, w_operand=bW)
+    dA = ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bG, w_operand=bW)
+    dW = ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K, g_operand=bG, a_operand=bA)
     assert ctx.status() == 0
 
     # maxima, scales and every code, bit for bit
