@@ -57,10 +57,13 @@ int luq_create(luq_ctx** out, int device) {
   c->use_pairs = 0;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;
-  c->d_status = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
-  bool ok = cudaMalloc(&c->d_status, sizeof(unsigned int)) == cudaSuccess &&
+  c->d_status = nullptr; c->d_scratch = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
+  // status word and the grid-maximum scratch share one small allocation
+  const size_t small_bytes = (64 + LUQ_SCRATCH_WORDS) * sizeof(unsigned int);
+  bool ok = cudaMalloc(&c->d_status, small_bytes) == cudaSuccess &&
             cudaMalloc(&c->d_workspace, kWorkspaceBytes) == cudaSuccess;
-  ok = ok && cudaMemset(c->d_status, 0, sizeof(unsigned int)) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_status, 0, small_bytes) == cudaSuccess;
+  if (ok) c->d_scratch = c->d_status + 64;
   if (ok) {
     cudaDriverEntryPointQueryResult q;
     ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q) == cudaSuccess &&
@@ -146,7 +149,7 @@ int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, as_stream(stream)));
+                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, nullptr, 0.0f, as_stream(stream)));
 }
 
 int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
@@ -158,7 +161,7 @@ int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, si
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 1, nullptr, as_stream(stream)));
+                                          n ? d_operand : nullptr, d_alpha, 1, nullptr, nullptr, 0.0f, as_stream(stream)));
 }
 
 int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, float* d_mhat,
@@ -170,12 +173,10 @@ int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t ro
   if (!d_measured_max || !(eta >= 0.0f && eta <= 1.0f) || (pw2 != 0 && pw2 != 1)) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
-  cudaStream_t st = as_stream(stream);
-  if (cudaMemsetAsync(d_measured_max, 0, sizeof(float), st) != cudaSuccess) return LUQ_ERR_CUDA;
-  int e = luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_mhat, seed, n_samples, d_codes, n ? d_operand : nullptr,
-                                   d_alpha, 2 | pw2, d_measured_max, st);
-  if (e) return cuda_rc(e);
-  return cuda_rc(luq_launch_hindsight_update(ctx, d_mhat, d_measured_max, eta, st));
+  // one kernel: quantize with the estimate, measure, and let the last block replace the estimate
+  return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_mhat, seed, n_samples, d_codes,
+                                          n ? d_operand : nullptr, d_alpha, 2 | pw2, d_measured_max, d_mhat, eta,
+                                          as_stream(stream)));
 }
 
 int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream) {

@@ -144,6 +144,8 @@ __device__ __forceinline__ void expand32(const uint4& w, const uint4& lut, uint4
 template <int KIND, bool LUQ_CODES>
 __global__ void __launch_bounds__(256) expand_plane_kernel(const uint4* __restrict__ codes, uint4* __restrict__ plane,
                                                            size_t pieces, uint4 lut) {
+  pdl_wait();
+  pdl_trigger();
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
   for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < pieces; i += stride) {
     uint4 o0, o1;
@@ -205,6 +207,10 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // set-up done (barriers, tensor memory, descriptor prefetch): from here on global memory is
+  // touched, which has to wait for the preceding kernel of the stream
+  pdl_wait();
+  pdl_trigger();
 
   const int units = p.tiles_m * p.tiles_n * p.splits;
   const int total_iters = p.n_samples * p.num_kb;
@@ -546,6 +552,10 @@ luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   cluster_sync_all();   // barriers of both CTAs are initialised before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // set-up done (barriers, tensor memory, descriptor prefetch): from here on global memory is
+  // touched, which has to wait for the preceding kernel of the stream
+  pdl_wait();
+  pdl_trigger();
 
   const int tiles_m2 = (p.tiles_m + 1) / 2;               // 256-row tiles
   const int tiles = tiles_m2 * p.tiles_n;
@@ -692,6 +702,8 @@ __global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restri
                                                            const float* __restrict__ scale_b, float post_scale,
                                                            int tiles, int tiles_m, int splits, long long Mo,
                                                            long long No) {
+  pdl_wait();
+  pdl_trigger();
   const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<long long>(tiles) * (kTileFloats / 4)) return;
   const int tile = static_cast<int>(idx / (kTileFloats / 4));
@@ -777,8 +789,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, 
   constexpr int smem = Cfg<A_PLANE, B_PLANE>::smem_bytes;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return static_cast<int>(e);
-  kernel<<<grid, Cfg<A_PLANE, B_PLANE>::threads, smem, st>>>(ta, tb, to, p);
-  return static_cast<int>(cudaGetLastError());
+  return static_cast<int>(luq_launch_kernel(kernel, grid, Cfg<A_PLANE, B_PLANE>::threads, smem, st, true, 1, ta, tb, to, p));
 }
 
 template <int KIND, bool A_MN, bool B_MN, bool A_LUQ>
@@ -796,17 +807,7 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap&
   auto kernel = luq_gemm_pair_kernel<KIND, A_MN, B_MN>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::smem_bytes);
   if (e != cudaSuccess) return static_cast<int>(e);
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3(kPairThreads, 1, 1);
-  cfg.dynamicSmemBytes = PairSmem::smem_bytes;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, kernel, ta, tb, to, p);
+  e = luq_launch_kernel(kernel, 2 * pairs, kPairThreads, PairSmem::smem_bytes, st, true, 2, ta, tb, to, p);
   return static_cast<int>(e);
 }
 
@@ -818,13 +819,11 @@ int launch_expand(bool luq_codes, const uint8_t* codes, uint8_t* plane, size_t p
   const size_t cap = static_cast<size_t>(sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  if (luq_codes)
-    expand_plane_kernel<KIND, true><<<static_cast<int>(blocks), 256, 0, st>>>(
-        reinterpret_cast<const uint4*>(codes), reinterpret_cast<uint4*>(plane), pieces, lut);
-  else
-    expand_plane_kernel<KIND, false><<<static_cast<int>(blocks), 256, 0, st>>>(
-        reinterpret_cast<const uint4*>(codes), reinterpret_cast<uint4*>(plane), pieces, lut);
-  return static_cast<int>(cudaGetLastError());
+  const uint4* src = reinterpret_cast<const uint4*>(codes);
+  uint4* dst = reinterpret_cast<uint4*>(plane);
+  const int grid = static_cast<int>(blocks);
+  return static_cast<int>(luq_codes ? luq_launch_kernel(expand_plane_kernel<KIND, true>, grid, 256, 0, st, true, 1, src, dst, pieces, lut)
+                                    : luq_launch_kernel(expand_plane_kernel<KIND, false>, grid, 256, 0, st, true, 1, src, dst, pieces, lut));
 }
 
 constexpr size_t kSplitRegionBytes = 20u << 20;   // the first 20 MiB of a workspace hold split partial tiles
@@ -980,10 +979,9 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   ctx->launches += 1;
   if (p.splits > 1) {
     const long long work = tiles * (kTileFloats / 4);
-    split_reduce_kernel<<<static_cast<int>((work + 255) / 256), 256, 0, st>>>(
-        a.d_workspace, a.d_out, a.d_scale_a, a.d_scale_b, p.post_scale, static_cast<int>(tiles), p.tiles_m, p.splits,
-        a.Mo, a.No);
-    rc = static_cast<int>(cudaGetLastError());
+    rc = static_cast<int>(luq_launch_kernel(split_reduce_kernel, static_cast<int>((work + 255) / 256), 256, 0, st, true, 1,
+                                            a.d_workspace, a.d_out, a.d_scale_a, a.d_scale_b, p.post_scale,
+                                            static_cast<int>(tiles), p.tiles_m, p.splits, a.Mo, a.No));
     if (rc == 0) ctx->launches += 1;
   }
   return rc;

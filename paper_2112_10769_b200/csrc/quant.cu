@@ -80,17 +80,57 @@ template <bool BF16> struct Item {
   }
 };
 
+// Grid-wide maximum without a pre-zeroed output: every block leaves its maximum in the
+// context's scratch array and takes a ticket; the block that draws the last ticket reduces the
+// array, resets the ticket counter and returns true in its thread 0 with the result in `m`.
+// scratch[0] is the ticket counter (zero between kernels), scratch[1 + b] block b's maximum.
+__device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* scratch) {
+  __shared__ uint32_t warp_max[kThreads / 32];
+  __shared__ bool last;
+  m = __reduce_max_sync(0xFFFFFFFFu, m);
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if (threadIdx.x == 0) {
+      __stcg(scratch + 1 + blockIdx.x, m);
+      __threadfence();
+      last = atomicAdd(scratch, 1u) == gridDim.x - 1;
+    }
+  }
+  __syncthreads();
+  if (!last) return false;
+  __threadfence();
+  m = 0;
+  for (unsigned int b = threadIdx.x; b < gridDim.x; b += kThreads) m = max(m, __ldcg(scratch + 1 + b));
+  m = __reduce_max_sync(0xFFFFFFFFu, m);
+  __syncthreads();            // warp_max is reused
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if (threadIdx.x == 0) { *scratch = 0u; return true; }
+  }
+  return false;
+}
+
 // ------------------------------------------------------------------ amax ----
 // |x| as an unsigned bit pattern is monotone in |x| for finite values, and every
 // Inf/NaN pattern is larger than every finite one: one unsigned max does both
 // the reduction and the non-finite detection.  Warp shuffle reduction (redux),
-// then one shared-memory step per block, then one atomicMax per block.
+// then one shared-memory step per block, then the last block to finish reduces the
+// block maxima (no pre-zeroed output, no atomics on it).
 constexpr int kAmaxUnroll = 4;
 constexpr int kAmaxCtasPerSm = 8;
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__ x, size_t n,
                                                         unsigned int* __restrict__ out_bits,
+                                                        unsigned int* __restrict__ scratch,
                                                         unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
   constexpr int kElems = Item<BF16>::kElems;
   constexpr int kUnroll = kAmaxUnroll;
   constexpr int kTileItems = kThreads * kUnroll;
@@ -125,17 +165,9 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
   if (blockIdx.x == 0 && threadIdx.x < n - items * kElems)
     m = max(m, __float_as_uint(Item<BF16>::load1(x, items * kElems + threadIdx.x)) & 0x7FFFFFFFu);
 
-  m = __reduce_max_sync(0xFFFFFFFFu, m);
-  __shared__ uint32_t warp_max[kThreads / 32];
-  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
-    m = __reduce_max_sync(0xFFFFFFFFu, m);
-    if (threadIdx.x == 0 && m != 0) {
-      atomicMax(out_bits, m);
-      if (m >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
-    }
+  if (grid_max_last_block(m, scratch)) {
+    *out_bits = m;
+    if (m >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
   }
 }
 
@@ -159,6 +191,8 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
                                                               int8_t* __restrict__ operand,
                                                               float* __restrict__ d_scale,
                                                               unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
   constexpr int kElems = Item<BF16>::kElems;
   const float clip = __ldg(d_clip);
   const bool first = blockIdx.x == 0 && threadIdx.x == 0;
@@ -303,22 +337,29 @@ __device__ __forceinline__ float pw2_ceil(float m) {
 // NS: number of samples known at compile time (1, 2) or 0 = read n_samples at run time.
 // PW2: the scale is a power of two, the quotient an exact scaling (one multiply).
 // TRACK: the tensor's own max|x| is reduced on the way (in-hindsight estimation: the scale
-// in d_amax is an estimate from earlier steps, the measured maximum feeds the next one).
+// in d_amax is an estimate from earlier steps, the measured maximum feeds the next one); the
+// block that finishes last writes the measured maximum and replaces the estimate by
+// (1 - eta) * measured + eta * estimate, every operation rounded once in binary32.
 // PLANE: the tensor-core operand bytes (int8, +-2^(c-1)) of every sample are written next to
 // the packed codes, one byte per element, sample s at offset s * n.
 template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
 __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restrict__ x, size_t n,
-                                                             const float* __restrict__ d_amax,
+                                                             const float* d_amax,
                                                              const __grid_constant__ PhiloxKeySet keys,
                                                              int n_samples_rt,
                                                              uint8_t* __restrict__ codes,
                                                              int8_t* __restrict__ operand,
                                                              float* __restrict__ d_alpha,
                                                              unsigned int* __restrict__ measured_bits,
+                                                             float* d_estimate, float eta,
+                                                             unsigned int* __restrict__ scratch,
                                                              unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
   const int n_samples = NS > 0 ? NS : n_samples_rt;
   constexpr int kElems = Item<BF16>::kElems;
-  const float mx = PW2 ? pw2_ceil(__ldg(d_amax)) : __ldg(d_amax);
+  const float given = *d_amax;   // with TRACK the last block overwrites it after every block has read it
+  const float mx = PW2 ? pw2_ceil(given) : given;
   const bool first = blockIdx.x == 0 && threadIdx.x == 0;
   const bool ok = scale_usable(mx, first ? status : nullptr);
   const float alpha = ok ? mx * (1.0f / static_cast<float>(1 << LUQ_KMAX)) : 0.0f;  // exact scaling
@@ -459,27 +500,14 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
       }
     }
   }
-  if constexpr (TRACK) {   // block maximum -> one atomicMax; Inf/NaN patterns win and raise the flag
-    seen = __reduce_max_sync(0xFFFFFFFFu, seen);
-    __shared__ uint32_t warp_seen[kThreads / 32];
-    if ((threadIdx.x & 31) == 0) warp_seen[threadIdx.x >> 5] = seen;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-      seen = threadIdx.x < kThreads / 32 ? warp_seen[threadIdx.x] : 0u;
-      seen = __reduce_max_sync(0xFFFFFFFFu, seen);
-      if (threadIdx.x == 0 && seen != 0) {
-        atomicMax(measured_bits, seen);
-        if (seen >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
-      }
+  if constexpr (TRACK) {   // Inf/NaN patterns win the maximum and raise the flag
+    if (grid_max_last_block(seen, scratch)) {
+      *measured_bits = seen;
+      if (seen >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
+      const float keep = __fsub_rn(1.0f, eta);
+      *d_estimate = __fadd_rn(__fmul_rn(keep, __uint_as_float(seen)), __fmul_rn(eta, given));
     }
   }
-}
-
-// In-hindsight update after a tracked quantization: m_hat <- (1 - eta) * measured + eta * m_hat,
-// every operation rounded once in binary32.
-__global__ void hindsight_update_kernel(float* __restrict__ m_hat, const float* __restrict__ measured, float eta) {
-  const float keep = __fsub_rn(1.0f, eta);
-  *m_hat = __fadd_rn(__fmul_rn(keep, *measured), __fmul_rn(eta, *m_hat));
 }
 
 // Diagnostic: the quotient t = |x| / alpha exactly as the quantizer forms it
@@ -487,6 +515,8 @@ __global__ void hindsight_update_kernel(float* __restrict__ m_hat, const float* 
 __global__ void __launch_bounds__(kThreads) luq_quotient_kernel(const float* __restrict__ x, size_t n,
                                                                 const float* __restrict__ d_amax,
                                                                 float* __restrict__ out) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
   const float alpha = __ldg(d_amax) * (1.0f / static_cast<float>(1 << LUQ_KMAX));
   const LuqScale sc = luq_scale(alpha);
   const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
@@ -509,7 +539,8 @@ int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 3
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1)
     per_sm = 1;
   if (per_sm > max_per_sm) per_sm = max_per_sm;
-  const size_t cap = static_cast<size_t>(ctx->sm_count) * per_sm;
+  size_t cap = static_cast<size_t>(ctx->sm_count) * per_sm;
+  if (cap > LUQ_SCRATCH_WORDS - 1) cap = LUQ_SCRATCH_WORDS - 1;   // one scratch word per block of a reducing kernel
   if (tiles < 1) tiles = 1;
   if (tiles <= cap) return static_cast<int>(tiles);
   const size_t rounds = (tiles + cap - 1) / cap;
@@ -519,18 +550,18 @@ int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 3
 }  // namespace
 
 int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, cudaStream_t st) {
-  cudaError_t e = cudaMemsetAsync(d_amax, 0, sizeof(float), st);
-  if (e != cudaSuccess) return static_cast<int>(e);
-  if (n == 0) return 0;
+  if (n == 0) return static_cast<int>(cudaMemsetAsync(d_amax, 0, sizeof(float), st));
+  unsigned int* out = reinterpret_cast<unsigned int*>(d_amax);
+  cudaError_t e;
   if (dtype == LUQ_BF16) {
     const int grid = grid_for(ctx, amax_kernel<true>, n / 8 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
-    amax_kernel<true><<<grid, kThreads, 0, st>>>(d_x, n, reinterpret_cast<unsigned int*>(d_amax), ctx->d_status);
+    e = luq_launch_kernel(amax_kernel<true>, grid, kThreads, 0, st, false, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
   } else {
     const int grid = grid_for(ctx, amax_kernel<false>, n / 4 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
-    amax_kernel<false><<<grid, kThreads, 0, st>>>(d_x, n, reinterpret_cast<unsigned int*>(d_amax), ctx->d_status);
+    e = luq_launch_kernel(amax_kernel<false>, grid, kThreads, 0, st, false, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
   }
   ctx->launches += 1;
-  return static_cast<int>(cudaGetLastError());
+  return static_cast<int>(e);
 }
 
 namespace {
@@ -538,8 +569,8 @@ template <bool BF16, bool PLANE>
 int launch_int4(luq_ctx* ctx, const void* d_x, size_t n, const float* d_clip, uint8_t* d_codes, int8_t* d_operand,
                 float* d_scale, cudaStream_t st) {
   const int grid = grid_for(ctx, quant_int4_kernel<BF16, PLANE>, n / Item<BF16>::kElems / kTileItems + 1);
-  quant_int4_kernel<BF16, PLANE><<<grid, kThreads, 0, st>>>(d_x, n, d_clip, d_codes, d_operand, d_scale, ctx->d_status);
-  return static_cast<int>(cudaGetLastError());
+  return static_cast<int>(luq_launch_kernel(quant_int4_kernel<BF16, PLANE>, grid, kThreads, 0, st, false, 1, d_x, n, d_clip,
+                                            d_codes, d_operand, d_scale, ctx->d_status));
 }
 }  // namespace
 
@@ -556,37 +587,6 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
 }
 
 namespace {
-template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
-int launch_luq_ns(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys,
-                  int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, unsigned int* d_measured,
-                  cudaStream_t st) {
-  const size_t tiles = n / Item<BF16>::kElems / kTileItems + 1;
-  const int grid = grid_for(ctx, quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, tiles);
-  quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE><<<grid, kThreads, 0, st>>>(d_g, n, d_amax, keys, n_samples, d_codes,
-                                                                           d_operand, d_alpha, d_measured,
-                                                                           ctx->d_status);
-  return static_cast<int>(cudaGetLastError());
-}
-
-template <bool BF16, bool PW2, bool TRACK, bool PLANE>
-int launch_luq_plane(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys,
-                     int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, unsigned int* d_measured,
-                     cudaStream_t st) {
-  if (n_samples == 1)
-    return launch_luq_ns<BF16, 1, PW2, TRACK, PLANE>(ctx, d_g, n, d_amax, keys, 1, d_codes, d_operand, d_alpha, d_measured, st);
-  if (n_samples == 2)
-    return launch_luq_ns<BF16, 2, PW2, TRACK, PLANE>(ctx, d_g, n, d_amax, keys, 2, d_codes, d_operand, d_alpha, d_measured, st);
-  return launch_luq_ns<BF16, 0, PW2, TRACK, PLANE>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, d_measured, st);
-}
-
-template <bool BF16, bool PW2, bool TRACK>
-int launch_luq(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys, int n_samples,
-               uint8_t* d_codes, int8_t* d_operand, float* d_alpha, unsigned int* d_measured, cudaStream_t st) {
-  if (d_operand)
-    return launch_luq_plane<BF16, PW2, TRACK, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, d_measured, st);
-  return launch_luq_plane<BF16, PW2, TRACK, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, nullptr, d_alpha, d_measured, st);
-}
-
 PhiloxKeySet expand_keys(uint64_t seed, int n_samples) {
   PhiloxKeySet keys{};
   for (int s = 0; s < n_samples; ++s) {   // sample s is keyed by seed + s
@@ -596,41 +596,59 @@ PhiloxKeySet expand_keys(uint64_t seed, int n_samples) {
   }
   return keys;
 }
+
+struct LuqLaunch {
+  luq_ctx* ctx; const void* g; size_t n; const float* amax; PhiloxKeySet keys; int n_samples;
+  uint8_t* codes; int8_t* operand; float* alpha; unsigned int* measured; float* estimate; float eta; cudaStream_t st;
+};
+
+template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
+int launch_luq_ns(const LuqLaunch& a) {
+  const size_t tiles = a.n / Item<BF16>::kElems / kTileItems + 1;
+  const int grid = grid_for(a.ctx, quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, tiles);
+  return static_cast<int>(luq_launch_kernel(quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, grid, kThreads, 0, a.st, false, 1,
+                                            a.g, a.n, a.amax, a.keys, a.n_samples, a.codes, a.operand, a.alpha,
+                                            a.measured, a.estimate, a.eta, a.ctx->d_scratch, a.ctx->d_status));
+}
+template <bool BF16, bool PW2, bool TRACK, bool PLANE>
+int launch_luq_plane(const LuqLaunch& a) {
+  if (a.n_samples == 1) return launch_luq_ns<BF16, 1, PW2, TRACK, PLANE>(a);
+  if (a.n_samples == 2) return launch_luq_ns<BF16, 2, PW2, TRACK, PLANE>(a);
+  return launch_luq_ns<BF16, 0, PW2, TRACK, PLANE>(a);
+}
+template <bool BF16, bool PW2, bool TRACK>
+int launch_luq(const LuqLaunch& a) {
+  return a.operand ? launch_luq_plane<BF16, PW2, TRACK, true>(a) : launch_luq_plane<BF16, PW2, TRACK, false>(a);
+}
 }  // namespace
 
-// flags: bit 0 = power-of-two scale, bit 1 = track this tensor's maximum into d_measured
+// flags: bit 0 = power-of-two scale; bit 1 = in-hindsight: d_amax is the running estimate, the
+// tensor's own maximum goes to d_measured and the estimate is replaced (eta) by the same kernel
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
-                             float* d_measured, cudaStream_t st) {
-  const PhiloxKeySet keys = expand_keys(seed, n_samples);
-  unsigned int* meas = reinterpret_cast<unsigned int*>(d_measured);
-  const bool bf = dtype == LUQ_BF16;
+                             float* d_measured, float* d_estimate, float eta, cudaStream_t st) {
+  const LuqLaunch a{ctx, d_g, n, d_amax, expand_keys(seed, n_samples), n_samples, d_codes, d_operand, d_alpha,
+                    reinterpret_cast<unsigned int*>(d_measured), d_estimate, eta, st};
   int rc;
-  switch ((flags & 3) | (bf ? 4 : 0)) {
-    case 0: rc = launch_luq<false, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
-    case 1: rc = launch_luq<false, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
-    case 2: rc = launch_luq<false, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
-    case 3: rc = launch_luq<false, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
-    case 4: rc = launch_luq<true, false, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
-    case 5: rc = launch_luq<true, true, false>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
-    case 6: rc = launch_luq<true, false, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
-    default: rc = launch_luq<true, true, true>(ctx, d_g, n, d_amax, keys, n_samples, d_codes, d_operand, d_alpha, meas, st); break;
+  switch ((flags & 3) | (dtype == LUQ_BF16 ? 4 : 0)) {
+    case 0: rc = launch_luq<false, false, false>(a); break;
+    case 1: rc = launch_luq<false, true, false>(a); break;
+    case 2: rc = launch_luq<false, false, true>(a); break;
+    case 3: rc = launch_luq<false, true, true>(a); break;
+    case 4: rc = launch_luq<true, false, false>(a); break;
+    case 5: rc = launch_luq<true, true, false>(a); break;
+    case 6: rc = launch_luq<true, false, true>(a); break;
+    default: rc = launch_luq<true, true, true>(a); break;
   }
   ctx->launches += 1;
   return rc;
-}
-
-int luq_launch_hindsight_update(luq_ctx* ctx, float* d_mhat, const float* d_measured, float eta, cudaStream_t st) {
-  hindsight_update_kernel<<<1, 1, 0, st>>>(d_mhat, d_measured, eta);
-  ctx->launches += 1;
-  return static_cast<int>(cudaGetLastError());
 }
 
 int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,
                               cudaStream_t st) {
   if (n == 0) return 0;
   const int grid = grid_for(ctx, luq_quotient_kernel, n / kThreads + 1);
-  luq_quotient_kernel<<<grid, kThreads, 0, st>>>(d_x, n, d_amax, d_t);
+  const cudaError_t e = luq_launch_kernel(luq_quotient_kernel, grid, kThreads, 0, st, false, 1, d_x, n, d_amax, d_t);
   ctx->launches += 1;
-  return static_cast<int>(cudaGetLastError());
+  return static_cast<int>(e);
 }
