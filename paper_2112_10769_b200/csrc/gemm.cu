@@ -215,9 +215,12 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const int units = p.tiles_m * p.tiles_n * p.splits;
   const int total_iters = p.n_samples * p.num_kb;
 
-  // consecutive tiles walk down the rows of one column panel: the CTAs that run at the same time share the panel of B
-  auto tile_m = [&](int tile) { return tile % p.tiles_m; };
-  auto tile_n = [&](int tile) { return tile / p.tiles_m; };
+  // Tile order.  Unsplit products walk along the rows of the output: the CTAs that run at the same
+  // time then write whole output rows (an output-bound product gains 6 % of write bandwidth,
+  // measured with the bare store pattern) and share the row panel of A.  Split products keep the
+  // order of the reduction kernel, down the columns.
+  auto tile_m = [&](int tile) { return p.splits == 1 ? tile / p.tiles_n : tile % p.tiles_m; };
+  auto tile_n = [&](int tile) { return p.splits == 1 ? tile % p.tiles_n : tile / p.tiles_m; };
   auto unit_range = [&](int u, int& tile, int& it_begin, int& it_end) {
     tile = u / p.splits;
     const int sp = u - tile * p.splits;
