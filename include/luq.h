@@ -106,6 +106,16 @@ int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, 
 int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
                    const float* d_clip, uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
 
+/* luq_amax followed by luq_quant_int4 with that maximum as the clip, as ONE kernel (the paper's
+ * forward quantization measures the tensor and then quantizes it, Sec. 3; two launches of
+ * streaming kernels cost more than the second pass when the tensor is small).  Every block
+ * first reduces its share of max|x|, the blocks meet at a grid barrier, then all quantize.
+ * *d_amax receives the maximum; codes, scale, operand bytes and status bits are exactly those
+ * of the two separate calls.  The launch is cooperative; the barrier's wait is bounded, and if
+ * it expires LUQ_STATUS_TIMEOUT is raised and no codes are written. */
+int luq_amax_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
+                        float* d_amax, uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
+
 /* Q_FP = LUQ (Sec. 4): alpha = max / 2^kmax (Eq. alpha); |x| < alpha becomes
  * sign*alpha with probability |x|/alpha, else 0 (Eq. StochasticPruning);
  * in-range values round stochastically between the two enclosing powers of two
@@ -118,6 +128,13 @@ int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t
 int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
                    const float* d_amax, uint64_t seed, int n_samples,
                    uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream);
+
+/* luq_amax followed by luq_quant_grad with that maximum, as ONE kernel (Sec. 4: the underflow
+ * threshold follows the maximum of the tensor at hand, measured in every backward pass).
+ * Same construction and guarantees as luq_amax_quant_int4; *d_amax receives the maximum. */
+int luq_amax_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
+                        uint64_t seed, int n_samples, float* d_amax,
+                        uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream);
 
 /* LUQ with a power-of-two scale (Appendix A.7, LUQ_PW2): as luq_quant_grad, but
  * alpha = 2^ceil(log2 max) / 2^kmax - the maximum is rounded UP to a power of two,

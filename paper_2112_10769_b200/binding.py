@@ -21,8 +21,9 @@ OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS = 1, 2, 3
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_quant_grad", "luq_quant_grad_pw2", "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad", "luq_gemm_wgrad_static", "luq_status",
-           "luq_launch_count", "luq_strerror")
+           "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_pw2",
+           "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
+           "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
 _lib = None
 
@@ -47,6 +48,8 @@ def load() -> ctypes.CDLL:
         L.luq_kmax.argtypes = []
         L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
         L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
+        L.luq_amax_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
+        L.luq_amax_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, u64, ctypes.c_int, vp, vp, vp, vp, vp]
         L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, ctypes.c_int, u64,
@@ -138,6 +141,33 @@ class Context:
                                      codes.data_ptr(), scale.data_ptr(), _opt(operand, x.numel()), _stream()),
                "luq_quant_int4")
         return codes, scale
+
+    def amax_quant_int4(self, x: torch.Tensor, amax: torch.Tensor | None = None, codes: torch.Tensor | None = None,
+                        scale: torch.Tensor | None = None, operand: torch.Tensor | None = None):
+        """amax + quant_int4 in one kernel; returns (amax, codes, scale)."""
+        rows, cols = (x.shape[0], x.numel() // max(x.shape[0], 1)) if x.dim() > 1 else (1, x.numel())
+        amax = torch.empty(1, dtype=torch.float32, device=x.device) if amax is None else amax
+        codes = torch.empty(x.numel() // 2, dtype=torch.uint8, device=x.device) if codes is None else codes
+        scale = torch.empty(1, dtype=torch.float32, device=x.device) if scale is None else scale
+        _check(load().luq_amax_quant_int4(self.handle, x.data_ptr(), _dtype_code(x), rows, cols, amax.data_ptr(),
+                                          codes.data_ptr(), scale.data_ptr(), _opt(operand, x.numel()), _stream()),
+               "luq_amax_quant_int4")
+        return amax, codes, scale
+
+    def amax_quant_grad(self, g: torch.Tensor, seed: int, n_samples: int = 1, amax: torch.Tensor | None = None,
+                        codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None,
+                        operand: torch.Tensor | None = None):
+        """amax + quant_grad in one kernel; returns (amax, codes, alpha)."""
+        rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
+        amax = torch.empty(1, dtype=torch.float32, device=g.device) if amax is None else amax
+        if codes is None:
+            codes = torch.empty((n_samples, g.numel() // 2), dtype=torch.uint8, device=g.device)
+        alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
+        _check(load().luq_amax_quant_grad(self.handle, g.data_ptr(), _dtype_code(g), rows, cols,
+                                          seed & (2 ** 64 - 1), n_samples, amax.data_ptr(), codes.data_ptr(),
+                                          alpha.data_ptr(), _opt(operand, n_samples * g.numel()), _stream()),
+               "luq_amax_quant_grad")
+        return amax, codes, alpha
 
     def quant_grad(self, g: torch.Tensor, amax: torch.Tensor, seed: int, n_samples: int = 1,
                    codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None,

@@ -124,7 +124,21 @@ int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, d_clip, d_codes, n ? d_operand : nullptr, d_scale,
-                                       as_stream(stream)));
+                                       nullptr, as_stream(stream)));
+}
+
+int luq_amax_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, float* d_amax,
+                        uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream) {
+  if (!ctx || !d_amax || !d_scale || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  const size_t n = rows * cols;
+  if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
+  if (n & 1u) return LUQ_ERR_ARG;
+  if (n && (!d_x || !d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_codes) || !aligned16(d_operand)) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, nullptr, d_codes, n ? d_operand : nullptr, d_scale,
+                                       d_amax, as_stream(stream)));
 }
 
 static int quant_grad_args(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
@@ -149,7 +163,21 @@ int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, nullptr, 0.0f, as_stream(stream)));
+                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, nullptr, 0.0f, nullptr,
+                                          as_stream(stream)));
+}
+
+int luq_amax_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, uint64_t seed,
+                        int n_samples, float* d_amax, uint8_t* d_codes, float* d_alpha, int8_t* d_operand,
+                        void* stream) {
+  size_t n = 0;
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, d_operand, &n);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, nullptr, seed, n_samples, d_codes,
+                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, nullptr, 0.0f, d_amax,
+                                          as_stream(stream)));
 }
 
 int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
@@ -161,7 +189,8 @@ int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, si
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 1, nullptr, nullptr, 0.0f, as_stream(stream)));
+                                          n ? d_operand : nullptr, d_alpha, 1, nullptr, nullptr, 0.0f, nullptr,
+                                          as_stream(stream)));
 }
 
 int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, float* d_mhat,
@@ -176,7 +205,7 @@ int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t ro
   // one kernel: quantize with the estimate, measure, and let the last block replace the estimate
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_mhat, seed, n_samples, d_codes,
                                           n ? d_operand : nullptr, d_alpha, 2 | pw2, d_measured_max, d_mhat, eta,
-                                          as_stream(stream)));
+                                          nullptr, as_stream(stream)));
 }
 
 int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream) {
@@ -260,6 +289,9 @@ int luq_status(luq_ctx* ctx, void* stream, int* host_flags) {
   if (cudaMemcpyAsync(&flags, ctx->d_status, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return LUQ_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LUQ_ERR_CUDA;
   if (flags) {
+    // a grid barrier that gave up leaves its counters behind: clear them with the status word
+    if ((flags & LUQ_STATUS_TIMEOUT) &&
+        cudaMemsetAsync(ctx->d_scratch, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) return LUQ_ERR_CUDA;
     if (cudaMemsetAsync(ctx->d_status, 0, sizeof(unsigned int), st) != cudaSuccess) return LUQ_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return LUQ_ERR_CUDA;
   }

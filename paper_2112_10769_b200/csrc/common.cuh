@@ -26,15 +26,16 @@ struct luq_ctx {
 // internal launchers (defined in quant.cu / gemm.cu); return a cudaError_t as int
 int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, cudaStream_t st);
 // d_operand (may be null): int8 operand bytes, one per element (and per sample), written with the codes
+// d_amax_out (may be null): fused - the kernel reduces the tensor's maximum itself, uses it as clip, writes it there
 int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
-                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, cudaStream_t st);
+                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_amax_out, cudaStream_t st);
 
 // flags: bit 0 = power-of-two scale; bit 1 = in-hindsight (d_amax is the running estimate: the tensor's own
 // max|x| goes to d_measured and d_estimate (= d_amax) is replaced by (1 - eta) * measured + eta * estimate)
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
-                             float* d_measured, float* d_estimate, float eta, cudaStream_t st);
-#define LUQ_SCRATCH_WORDS 4096  // ticket + block maxima; grids of the reducing kernels stay below it
+                             float* d_measured, float* d_estimate, float eta, float* d_amax_out, cudaStream_t st);
+#define LUQ_SCRATCH_WORDS 4096  // two counters + block maxima; grids of the reducing kernels stay below it
 int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,
                               cudaStream_t st);
 
@@ -54,7 +55,8 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st);
 
 #ifdef __CUDACC__
 
-// Launch helper.  `early` = programmatic dependent launch: the kernel may become resident and set
+// Launch helper.  LUQ_LAUNCH_COOPERATIVE: all blocks of the grid are resident at once (the kernel
+// has a grid barrier inside).  LUQ_LAUNCH_EARLY = programmatic dependent launch: the kernel may become resident and set
 // up (barriers, tensor memory, descriptor prefetch) while its predecessor in the stream drains,
 // and waits in pdl_wait() until that predecessor has completed and its writes are visible.
 // Every kernel of the library calls pdl_wait() before its first access to global memory, so any
@@ -64,9 +66,12 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st);
 // are launched normally: launched early they become resident next to a running GEMM CTA, on an
 // SM configured for maximum shared memory, keep that small L1 after the GEMM has gone and lose
 // a third of their bandwidth (measured: the 462 MB max reduction, 68 -> 96 us).
+#define LUQ_LAUNCH_NORMAL 0
+#define LUQ_LAUNCH_EARLY 1
+#define LUQ_LAUNCH_COOPERATIVE 2
 template <typename... KArgs, typename... Args>
 cudaError_t luq_launch_kernel(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
-                              bool early, unsigned cluster_x, Args&&... args) {
+                              int mode, unsigned cluster_x, Args&&... args) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
   cfg.blockDim = dim3(static_cast<unsigned>(block), 1, 1);
@@ -74,9 +79,15 @@ cudaError_t luq_launch_kernel(void (*kernel)(KArgs...), int grid, int block, siz
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   unsigned n = 0;
-  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[n].val.programmaticStreamSerializationAllowed = 1;
-  if (early) ++n;
+  if (mode == LUQ_LAUNCH_EARLY) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  } else if (mode == LUQ_LAUNCH_COOPERATIVE) {
+    attr[n].id = cudaLaunchAttributeCooperative;
+    attr[n].val.cooperative = 1;
+    ++n;
+  }
   if (cluster_x > 1) {
     attr[n].id = cudaLaunchAttributeClusterDimension;
     attr[n].val.clusterDim.x = cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;

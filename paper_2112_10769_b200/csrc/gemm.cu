@@ -792,7 +792,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, 
   constexpr int smem = Cfg<A_PLANE, B_PLANE>::smem_bytes;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return static_cast<int>(e);
-  return static_cast<int>(luq_launch_kernel(kernel, grid, Cfg<A_PLANE, B_PLANE>::threads, smem, st, true, 1, ta, tb, to, p));
+  return static_cast<int>(luq_launch_kernel(kernel, grid, Cfg<A_PLANE, B_PLANE>::threads, smem, st, LUQ_LAUNCH_EARLY, 1, ta, tb, to, p));
 }
 
 template <int KIND, bool A_MN, bool B_MN, bool A_LUQ>
@@ -810,7 +810,7 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap&
   auto kernel = luq_gemm_pair_kernel<KIND, A_MN, B_MN>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem::smem_bytes);
   if (e != cudaSuccess) return static_cast<int>(e);
-  e = luq_launch_kernel(kernel, 2 * pairs, kPairThreads, PairSmem::smem_bytes, st, true, 2, ta, tb, to, p);
+  e = luq_launch_kernel(kernel, 2 * pairs, kPairThreads, PairSmem::smem_bytes, st, LUQ_LAUNCH_EARLY, 2, ta, tb, to, p);
   return static_cast<int>(e);
 }
 
@@ -825,8 +825,8 @@ int launch_expand(bool luq_codes, const uint8_t* codes, uint8_t* plane, size_t p
   const uint4* src = reinterpret_cast<const uint4*>(codes);
   uint4* dst = reinterpret_cast<uint4*>(plane);
   const int grid = static_cast<int>(blocks);
-  return static_cast<int>(luq_codes ? luq_launch_kernel(expand_plane_kernel<KIND, true>, grid, 256, 0, st, true, 1, src, dst, pieces, lut)
-                                    : luq_launch_kernel(expand_plane_kernel<KIND, false>, grid, 256, 0, st, true, 1, src, dst, pieces, lut));
+  return static_cast<int>(luq_codes ? luq_launch_kernel(expand_plane_kernel<KIND, true>, grid, 256, 0, st, LUQ_LAUNCH_EARLY, 1, src, dst, pieces, lut)
+                                    : luq_launch_kernel(expand_plane_kernel<KIND, false>, grid, 256, 0, st, LUQ_LAUNCH_EARLY, 1, src, dst, pieces, lut));
 }
 
 constexpr size_t kSplitRegionBytes = 20u << 20;   // the first 20 MiB of a workspace hold split partial tiles
@@ -982,7 +982,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   ctx->launches += 1;
   if (p.splits > 1) {
     const long long work = tiles * (kTileFloats / 4);
-    rc = static_cast<int>(luq_launch_kernel(split_reduce_kernel, static_cast<int>((work + 255) / 256), 256, 0, st, true, 1,
+    rc = static_cast<int>(luq_launch_kernel(split_reduce_kernel, static_cast<int>((work + 255) / 256), 256, 0, st, LUQ_LAUNCH_EARLY, 1,
                                             a.d_workspace, a.d_out, a.d_scale_a, a.d_scale_b, p.post_scale,
                                             static_cast<int>(tiles), p.tiles_m, p.splits, a.Mo, a.No));
     if (rc == 0) ctx->launches += 1;

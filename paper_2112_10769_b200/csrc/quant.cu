@@ -83,7 +83,8 @@ template <bool BF16> struct Item {
 // Grid-wide maximum without a pre-zeroed output: every block leaves its maximum in the
 // context's scratch array and takes a ticket; the block that draws the last ticket reduces the
 // array, resets the ticket counter and returns true in its thread 0 with the result in `m`.
-// scratch[0] is the ticket counter (zero between kernels), scratch[1 + b] block b's maximum.
+// scratch[0] is the ticket counter (zero between kernels), scratch[1] the departure counter of
+// the fused kernels' grid barrier, scratch[2 + b] block b's maximum.
 __device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* scratch) {
   __shared__ uint32_t warp_max[kThreads / 32];
   __shared__ bool last;
@@ -94,7 +95,7 @@ __device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* s
     m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
     m = __reduce_max_sync(0xFFFFFFFFu, m);
     if (threadIdx.x == 0) {
-      __stcg(scratch + 1 + blockIdx.x, m);
+      __stcg(scratch + 2 + blockIdx.x, m);
       __threadfence();
       last = atomicAdd(scratch, 1u) == gridDim.x - 1;
     }
@@ -103,7 +104,7 @@ __device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* s
   if (!last) return false;
   __threadfence();
   m = 0;
-  for (unsigned int b = threadIdx.x; b < gridDim.x; b += kThreads) m = max(m, __ldcg(scratch + 1 + b));
+  for (unsigned int b = threadIdx.x; b < gridDim.x; b += kThreads) m = max(m, __ldcg(scratch + 2 + b));
   m = __reduce_max_sync(0xFFFFFFFFu, m);
   __syncthreads();            // warp_max is reused
   if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
@@ -171,6 +172,90 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
   }
 }
 
+// ------------------------------------------------- fused max (phase one) ----
+// A quantizer launched "fused" first reduces max|x| itself: every block folds its share of the
+// tensor, leaves its maximum in the scratch array and waits at a grid barrier; then every block
+// reduces the array, so all of them hold the tensor's maximum without a second launch.  The
+// launch is cooperative (one wave, all blocks resident).  The wait is bounded: when it expires
+// the block raises LUQ_STATUS_TIMEOUT and the kernel returns without writing codes.
+constexpr uint32_t kBarrierPolls = 4u << 20;   // x 200 ns of sleep: the better part of a second
+
+template <bool BF16>
+__device__ __forceinline__ bool fused_grid_max(const void* __restrict__ x, size_t n, unsigned int* scratch,
+                                               unsigned int* status, uint32_t& result) {
+  constexpr int kElems = Item<BF16>::kElems;
+  const size_t items = n / kElems;
+  const uint4* p = reinterpret_cast<const uint4*>(x);
+  uint32_t m = 0;
+  auto fold = [&](const uint4& u) {
+    if constexpr (BF16) {
+      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        m = max(m, (w[j] << 16) & 0x7FFFFFFFu);
+        m = max(m, w[j] & 0x7FFF0000u);
+      }
+    } else {
+      m = max(m, u.x & 0x7FFFFFFFu); m = max(m, u.y & 0x7FFFFFFFu);
+      m = max(m, u.z & 0x7FFFFFFFu); m = max(m, u.w & 0x7FFFFFFFu);
+    }
+  };
+  const size_t full_tiles = items / kTileItems;
+  for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {   // front to back; phase two walks back to front
+    const uint4* q = p + t * kTileItems + threadIdx.x;
+    uint4 u[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(q + j * kThreads);
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) fold(u[j]);
+  }
+  if (blockIdx.x == gridDim.x - 1)
+    for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) fold(__ldg(p + i));
+  if (blockIdx.x == 0 && threadIdx.x < n - items * kElems)
+    m = max(m, __float_as_uint(Item<BF16>::load1(x, items * kElems + threadIdx.x)) & 0x7FFFFFFFu);
+
+  __shared__ uint32_t warp_max[kThreads / 32];
+  __shared__ uint32_t arrived;
+  m = __reduce_max_sync(0xFFFFFFFFu, m);
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if (threadIdx.x == 0) {
+      __stcg(scratch + 2 + blockIdx.x, m);
+      __threadfence();
+      atomicAdd(scratch, 1u);
+      uint32_t seen = 0, polls = 0;
+      for (;;) {
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(scratch) : "memory");
+        if (seen >= gridDim.x || ++polls > kBarrierPolls) break;
+        __nanosleep(200);
+      }
+      arrived = seen;
+    }
+  }
+  __syncthreads();
+  if (arrived < gridDim.x) {                    // the barrier gave up: some block never arrived
+    if (threadIdx.x == 0) atomicOr(status, LUQ_STATUS_TIMEOUT);
+    return false;
+  }
+  __threadfence();
+  m = 0;
+  for (unsigned int b = threadIdx.x; b < gridDim.x; b += kThreads) m = max(m, __ldcg(scratch + 2 + b));
+  m = __reduce_max_sync(0xFFFFFFFFu, m);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) m = max(m, warp_max[w]);
+  // the last block to leave the barrier resets both counters for the next kernel
+  if (threadIdx.x == 0 && atomicAdd(scratch + 1, 1u) == gridDim.x - 1) { scratch[0] = 0u; scratch[1] = 0u; }
+  result = m;
+  return true;
+}
+
 // ------------------------------------------------------------------ INT4 ----
 // clamp, then add 1.5 * 2^23: the sum's low mantissa bits hold the integer rounded to
 // nearest-even, already in two's complement (clamping before rounding equals clamping
@@ -186,16 +271,25 @@ __device__ __forceinline__ uint32_t int4_code(float x, float inv) {
 // byte) are written next to the packed codes, one byte per element in element order.
 template <bool BF16, bool PLANE>
 __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __restrict__ x, size_t n,
-                                                              const float* __restrict__ d_clip,
+                                                              const float* d_clip,
                                                               uint8_t* __restrict__ codes,
                                                               int8_t* __restrict__ operand,
                                                               float* __restrict__ d_scale,
+                                                              float* d_amax_out, unsigned int* scratch,
                                                               unsigned int* __restrict__ status) {
   luqdev::pdl_wait();
   luqdev::pdl_trigger();
   constexpr int kElems = Item<BF16>::kElems;
-  const float clip = __ldg(d_clip);
   const bool first = blockIdx.x == 0 && threadIdx.x == 0;
+  float clip;
+  if (d_amax_out != nullptr) {   // fused: the clip is this tensor's maximum, reduced here
+    uint32_t bits;
+    if (!fused_grid_max<BF16>(x, n, scratch, status, bits)) return;
+    clip = __uint_as_float(bits);
+    if (first) *d_amax_out = clip;
+  } else {
+    clip = *d_clip;
+  }
   const bool ok = scale_usable(clip, first ? status : nullptr);
   const float inv = ok ? 7.0f / clip : 0.0f;
   if (first) *d_scale = ok ? clip / 7.0f : 0.0f;
@@ -270,51 +364,55 @@ __device__ __forceinline__ uint4 philox_block(uint64_t block, const PhiloxKeys& 
 }
 
 // The scale of one tensor, prepared once per thread.
-//   alpha = max / 2^kmax (exact).  The quotient t = |x| / alpha must be the IEEE
-//   round-to-nearest quotient.  With y = RN(1/alpha) (correctly rounded) it is
-//   obtained without a division: q0 = a*y is within 1.5 ulp, one residual
-//   correction makes it faithful, a second one (residual now exact) makes it
-//   correctly rounded (Markstein).  For a tiny max both operands are first scaled
-//   by 2^64 (exact) so that no residual that matters falls into the denormal range.
-struct LuqScale { float alpha_s, recip, pre; };
+//   alpha = max / 2^kmax (exact).  Every decision is a function of the IEEE round-to-nearest
+//   quotient t = |x| / alpha, and is taken on Q = t * 2^32 = RN(|x| / beta) with
+//   beta = alpha * 2^-32: scaling by a power of two commutes with the rounding, and the
+//   32-bit threshold of an underflow element is simply trunc(Q).
+//   With y = RN(1/beta) (correctly rounded) Q is obtained without a division: q0 = a*y is
+//   within 1.5 ulp, one residual correction makes it faithful, a second one (residual now
+//   exact) makes it correctly rounded (Markstein).  The residuals are exact as long as they
+//   do not fall below the denormal grid, which holds for alpha >= 2^-71; for a smaller
+//   alpha ("tiny") both operands are first scaled by 2^64 (exact).
+struct LuqScale { float beta, recip, pre; bool tiny; };
 
 __device__ __forceinline__ LuqScale luq_scale(float alpha) {
   LuqScale sc;
-  sc.pre = alpha < 0x1p-44f ? 0x1p64f : 1.0f;
-  sc.alpha_s = alpha * sc.pre;
-  sc.recip = __frcp_rn(sc.alpha_s);
+  sc.tiny = alpha < 0x1p-60f;
+  sc.pre = sc.tiny ? 0x1p64f : 1.0f;
+  sc.beta = alpha * sc.pre * 0x1p-32f;       // exact: alpha lies in [2^-104, 2^96]
+  sc.recip = __frcp_rn(sc.beta);
   return sc;
 }
 
+// Q for a = |x| * pre (the caller applies pre; it is 1 unless the scale is tiny)
 template <bool PW2 = false>
-__device__ __forceinline__ float luq_quotient_raw(float x, const LuqScale& sc) {
-  if constexpr (PW2) return fabsf(x) * sc.recip;   // alpha is a power of two: exact up to the final rounding
-  const float a = fabsf(x) * sc.pre;
+__device__ __forceinline__ float luq_scaled_quotient(float a, const LuqScale& sc) {
+  if constexpr (PW2) return a * sc.recip;   // beta is a power of two: one exact scaling
   const float q0 = a * sc.recip;
-  const float r0 = __fmaf_rn(-sc.alpha_s, q0, a);
+  const float r0 = __fmaf_rn(-sc.beta, q0, a);
   const float q1 = __fmaf_rn(r0, sc.recip, q0);
-  const float r1 = __fmaf_rn(-sc.alpha_s, q1, a);
+  const float r1 = __fmaf_rn(-sc.beta, q1, a);
   return __fmaf_rn(r1, sc.recip, q1);
 }
 template <bool PW2 = false>
-__device__ __forceinline__ float luq_quotient(float x, const LuqScale& sc) {
-  // an overflowing or non-finite quotient turns into NaN or Inf above; both belong to the top level
-  return fminf(luq_quotient_raw<PW2>(x, sc), static_cast<float>(1 << LUQ_KMAX));   // fminf(NaN, c) = c
+__device__ __forceinline__ float luq_quotient_clamped(float x, const LuqScale& sc) {
+  // an overflowing or non-finite quotient turns into NaN or Inf; both belong to the top level
+  return fminf(luq_scaled_quotient<PW2>(fabsf(x) * sc.pre, sc), 0x1p32f * static_cast<float>(1 << LUQ_KMAX));   // fminf(NaN, c) = c
 }
 
 // Per element: lower code and the 32-bit threshold of the up-decision, from the
-// bit fields of t (already clamped to 2^kmax).
+// bit fields of Q = t * 2^32 (already clamped to 2^(kmax+32)).
 //   t >= 1: code 1 + exponent(t), threshold = mantissa << 9 (up-probability
 //           (|x| - lo)/lo); t = 2^kmax gives the top code with threshold 0.
-//   t <  1: code 0, threshold trunc(t * 2^32) (prune-up probability |x|/alpha),
-//           computed as (1.mantissa << 8) >> (126 - exponent field).
-__device__ __forceinline__ void luq_bin(float t, uint32_t& lo_code, uint32_t& thr) {
-  const uint32_t u = __float_as_uint(t);
+//   t <  1: code 0, threshold trunc(Q) (prune-up probability |x|/alpha),
+//           computed as (1.mantissa << 8) >> (158 - exponent field).
+__device__ __forceinline__ void luq_bin(float q, uint32_t& lo_code, uint32_t& thr) {
+  const uint32_t u = __float_as_uint(q);
   const int e = static_cast<int>(u >> 23);
   const uint32_t thr_in = u << 9;
-  const uint32_t thr_under = __funnelshift_rc((u << 8) | 0x80000000u, 0u, static_cast<uint32_t>(126 - e));
-  thr = u >= 0x3F800000u ? thr_in : thr_under;
-  lo_code = static_cast<uint32_t>(max(e - 126, 0));
+  const uint32_t thr_under = __funnelshift_rc((u << 8) | 0x80000000u, 0u, static_cast<uint32_t>(158 - e));
+  thr = u >= 0x4F800000u ? thr_in : thr_under;
+  lo_code = static_cast<uint32_t>(max(e - 158, 0));
 }
 
 __device__ __forceinline__ uint32_t luq_nibble(uint32_t xbits, uint32_t lo_code, uint32_t thr, uint32_t word) {
@@ -352,20 +450,28 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
                                                              float* __restrict__ d_alpha,
                                                              unsigned int* __restrict__ measured_bits,
                                                              float* d_estimate, float eta,
-                                                             unsigned int* __restrict__ scratch,
+                                                             float* d_amax_out, unsigned int* scratch,
                                                              unsigned int* __restrict__ status) {
   luqdev::pdl_wait();
   luqdev::pdl_trigger();
   const int n_samples = NS > 0 ? NS : n_samples_rt;
   constexpr int kElems = Item<BF16>::kElems;
-  const float given = *d_amax;   // with TRACK the last block overwrites it after every block has read it
+  float given;
+  if (!TRACK && d_amax_out != nullptr) {   // fused: the maximum of this tensor, reduced here
+    uint32_t bits;
+    if (!fused_grid_max<BF16>(x, n, scratch, status, bits)) return;
+    given = __uint_as_float(bits);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *d_amax_out = given;
+  } else {
+    given = *d_amax;   // with TRACK the last block overwrites it after every block has read it
+  }
+  const bool back_to_front = !TRACK && d_amax_out != nullptr;   // phase one ended at the tensor's tail
   const float mx = PW2 ? pw2_ceil(given) : given;
   const bool first = blockIdx.x == 0 && threadIdx.x == 0;
   const bool ok = scale_usable(mx, first ? status : nullptr);
   const float alpha = ok ? mx * (1.0f / static_cast<float>(1 << LUQ_KMAX)) : 0.0f;  // exact scaling
   if (first) *d_alpha = alpha;
-  LuqScale sc = luq_scale(ok ? alpha : 1.0f);
-  if constexpr (PW2) { sc.pre = 1.0f; sc.alpha_s = ok ? alpha : 1.0f; sc.recip = 1.0f / sc.alpha_s; }  // exact
+  const LuqScale sc = luq_scale(ok ? alpha : 1.0f);   // with a power-of-two alpha the reciprocal is exact
   uint32_t seen = 0;   // running max of |x| bit patterns (TRACK)
 
   const size_t plane = n / 2;
@@ -389,13 +495,17 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
       for (int j = 0; j < kElems; ++j) seen = max(seen, __float_as_uint(v[j]) & 0x7FFFFFFFu);
     }
     // the vote needs every lane of the warp here: only the full-tile loop qualifies
-    if (whole_warp && !__any_sync(0xFFFFFFFFu, in_range)) {
+    if (whole_warp && !sc.tiny && !__any_sync(0xFFFFFFFFu, in_range)) {
+      // thr: the up-threshold trunc(Q) (Q < 2^32 here).  sn / ob: the element's non-zero nibble
+      // (sign, code 1) and operand byte (-1 or +1), already shifted to their place in the word.
       uint32_t thr[kElems], sn[kElems], ob[kElems];
 #pragma unroll
       for (int j = 0; j < kElems; ++j) {
-        thr[j] = __float2uint_rz(luq_quotient_raw<PW2>(v[j], sc) * 4294967296.0f);
-        sn[j] = ((__float_as_uint(v[j]) >> 28) & 8u) | 1u;
-        if constexpr (PLANE) ob[j] = (__float_as_uint(v[j]) >> 31) ? 0xFFu : 0x01u;   // -1 or +1
+        const uint32_t bits = __float_as_uint(v[j]);
+        thr[j] = __float2uint_rz(luq_scaled_quotient<PW2>(fabsf(v[j]), sc));
+        const int at = 4 * j;   // bit position of the nibble; the sign bit goes to at + 3
+        sn[j] = ((bits >> (28 - at)) & (8u << at)) | (1u << at);
+        if constexpr (PLANE) ob[j] = ((bits >> 31) ? 0xFFu : 0x01u) << (8 * (j % 4));
       }
 #pragma unroll
       for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
@@ -409,9 +519,10 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
           const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const bool up = rw[j] < thr[4 * b + j];
-            word += (up ? sn[4 * b + j] : 0u) << (4 * (4 * b + j));
-            if constexpr (PLANE) bytes[b] += (up ? ob[4 * b + j] : 0u) << (8 * j);
+            if (rw[j] < thr[4 * b + j]) {
+              word |= sn[4 * b + j];
+              if constexpr (PLANE) bytes[b] |= ob[4 * b + j];
+            }
           }
         }
         Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
@@ -421,7 +532,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
     }
     uint32_t lo_code[kElems], thr[kElems];
 #pragma unroll
-    for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient<PW2>(v[j], sc), lo_code[j], thr[j]);
+    for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient_clamped<PW2>(v[j], sc), lo_code[j], thr[j]);
 #pragma unroll
     for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
       if (NS == 0 && s >= n_samples) break;
@@ -447,7 +558,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
   const size_t full_tiles = items / kTileItems;
   if (ok) {
     for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {
-      const size_t i0 = t * kTileItems + threadIdx.x;
+      const size_t i0 = (back_to_front ? full_tiles - 1 - t : t) * kTileItems + threadIdx.x;
       uint4 u[kUnroll];
 #pragma unroll
       for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i0 + j * kThreads);
@@ -486,7 +597,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
           if (ok && idx < n) {
             const float xv = Item<BF16>::load1(x, idx);
             uint32_t lc, th;
-            luq_bin(luq_quotient<PW2>(xv, sc), lc, th);
+            luq_bin(luq_quotient_clamped<PW2>(xv, sc), lc, th);
             const uint4 r = philox_block(idx >> 2, ks);
             const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
             nib[h] = luq_nibble(__float_as_uint(xv), lc, th, rw[idx & 3]);
@@ -520,14 +631,8 @@ __global__ void __launch_bounds__(kThreads) luq_quotient_kernel(const float* __r
   const float alpha = __ldg(d_amax) * (1.0f / static_cast<float>(1 << LUQ_KMAX));
   const LuqScale sc = luq_scale(alpha);
   const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
-  for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < n; i += stride) {
-    const float a = fabsf(x[i]) * sc.pre;
-    const float q0 = a * sc.recip;
-    const float r0 = __fmaf_rn(-sc.alpha_s, q0, a);
-    const float q1 = __fmaf_rn(r0, sc.recip, q0);
-    const float r1 = __fmaf_rn(-sc.alpha_s, q1, a);
-    out[i] = __fmaf_rn(r1, sc.recip, q1);
-  }
+  for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < n; i += stride)
+    out[i] = luq_scaled_quotient<false>(fabsf(x[i]) * sc.pre, sc) * 0x1p-32f;   // t = Q * 2^-32
 }
 
 // Grid for a kernel that walks `tiles` tiles: at most the CTAs the GPU holds at once
@@ -540,7 +645,7 @@ int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 3
     per_sm = 1;
   if (per_sm > max_per_sm) per_sm = max_per_sm;
   size_t cap = static_cast<size_t>(ctx->sm_count) * per_sm;
-  if (cap > LUQ_SCRATCH_WORDS - 1) cap = LUQ_SCRATCH_WORDS - 1;   // one scratch word per block of a reducing kernel
+  if (cap > LUQ_SCRATCH_WORDS - 2) cap = LUQ_SCRATCH_WORDS - 2;   // one scratch word per block of a reducing kernel
   if (tiles < 1) tiles = 1;
   if (tiles <= cap) return static_cast<int>(tiles);
   const size_t rounds = (tiles + cap - 1) / cap;
@@ -555,10 +660,10 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
   cudaError_t e;
   if (dtype == LUQ_BF16) {
     const int grid = grid_for(ctx, amax_kernel<true>, n / 8 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
-    e = luq_launch_kernel(amax_kernel<true>, grid, kThreads, 0, st, false, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
+    e = luq_launch_kernel(amax_kernel<true>, grid, kThreads, 0, st, LUQ_LAUNCH_NORMAL, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
   } else {
     const int grid = grid_for(ctx, amax_kernel<false>, n / 4 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
-    e = luq_launch_kernel(amax_kernel<false>, grid, kThreads, 0, st, false, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
+    e = luq_launch_kernel(amax_kernel<false>, grid, kThreads, 0, st, LUQ_LAUNCH_NORMAL, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
   }
   ctx->launches += 1;
   return static_cast<int>(e);
@@ -567,21 +672,23 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
 namespace {
 template <bool BF16, bool PLANE>
 int launch_int4(luq_ctx* ctx, const void* d_x, size_t n, const float* d_clip, uint8_t* d_codes, int8_t* d_operand,
-                float* d_scale, cudaStream_t st) {
+                float* d_scale, float* d_amax_out, cudaStream_t st) {
   const int grid = grid_for(ctx, quant_int4_kernel<BF16, PLANE>, n / Item<BF16>::kElems / kTileItems + 1);
-  return static_cast<int>(luq_launch_kernel(quant_int4_kernel<BF16, PLANE>, grid, kThreads, 0, st, false, 1, d_x, n, d_clip,
-                                            d_codes, d_operand, d_scale, ctx->d_status));
+  const int mode = d_amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_NORMAL;   // fused: grid barrier inside
+  return static_cast<int>(luq_launch_kernel(quant_int4_kernel<BF16, PLANE>, grid, kThreads, 0, st, mode, 1, d_x, n, d_clip,
+                                            d_codes, d_operand, d_scale, d_amax_out, ctx->d_scratch, ctx->d_status));
 }
 }  // namespace
 
+// d_amax_out non-null: fused - the clip is the tensor's maximum, reduced by the same kernel and written there
 int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
-                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, cudaStream_t st) {
+                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_amax_out, cudaStream_t st) {
   const bool bf = dtype == LUQ_BF16;
   int rc;
-  if (d_operand) rc = bf ? launch_int4<true, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, st)
-                         : launch_int4<false, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, st);
-  else rc = bf ? launch_int4<true, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, st)
-               : launch_int4<false, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, st);
+  if (d_operand) rc = bf ? launch_int4<true, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st)
+                         : launch_int4<false, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st);
+  else rc = bf ? launch_int4<true, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, d_amax_out, st)
+               : launch_int4<false, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, d_amax_out, st);
   ctx->launches += 1;
   return rc;
 }
@@ -599,16 +706,20 @@ PhiloxKeySet expand_keys(uint64_t seed, int n_samples) {
 
 struct LuqLaunch {
   luq_ctx* ctx; const void* g; size_t n; const float* amax; PhiloxKeySet keys; int n_samples;
-  uint8_t* codes; int8_t* operand; float* alpha; unsigned int* measured; float* estimate; float eta; cudaStream_t st;
+  uint8_t* codes; int8_t* operand; float* alpha; unsigned int* measured; float* estimate; float eta;
+  float* amax_out;   // non-null: fused, the maximum is reduced by the same kernel (cooperative launch)
+  cudaStream_t st;
 };
 
 template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
 int launch_luq_ns(const LuqLaunch& a) {
   const size_t tiles = a.n / Item<BF16>::kElems / kTileItems + 1;
   const int grid = grid_for(a.ctx, quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, tiles);
-  return static_cast<int>(luq_launch_kernel(quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, grid, kThreads, 0, a.st, false, 1,
+  const int mode = a.amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_NORMAL;
+  return static_cast<int>(luq_launch_kernel(quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, grid, kThreads, 0, a.st, mode, 1,
                                             a.g, a.n, a.amax, a.keys, a.n_samples, a.codes, a.operand, a.alpha,
-                                            a.measured, a.estimate, a.eta, a.ctx->d_scratch, a.ctx->d_status));
+                                            a.measured, a.estimate, a.eta, a.amax_out, a.ctx->d_scratch,
+                                            a.ctx->d_status));
 }
 template <bool BF16, bool PW2, bool TRACK, bool PLANE>
 int launch_luq_plane(const LuqLaunch& a) {
@@ -626,9 +737,9 @@ int launch_luq(const LuqLaunch& a) {
 // tensor's own maximum goes to d_measured and the estimate is replaced (eta) by the same kernel
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
-                             float* d_measured, float* d_estimate, float eta, cudaStream_t st) {
+                             float* d_measured, float* d_estimate, float eta, float* d_amax_out, cudaStream_t st) {
   const LuqLaunch a{ctx, d_g, n, d_amax, expand_keys(seed, n_samples), n_samples, d_codes, d_operand, d_alpha,
-                    reinterpret_cast<unsigned int*>(d_measured), d_estimate, eta, st};
+                    reinterpret_cast<unsigned int*>(d_measured), d_estimate, eta, d_amax_out, st};
   int rc;
   switch ((flags & 3) | (dtype == LUQ_BF16 ? 4 : 0)) {
     case 0: rc = launch_luq<false, false, false>(a); break;
@@ -648,7 +759,7 @@ int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const fl
                               cudaStream_t st) {
   if (n == 0) return 0;
   const int grid = grid_for(ctx, luq_quotient_kernel, n / kThreads + 1);
-  const cudaError_t e = luq_launch_kernel(luq_quotient_kernel, grid, kThreads, 0, st, false, 1, d_x, n, d_amax, d_t);
+  const cudaError_t e = luq_launch_kernel(luq_quotient_kernel, grid, kThreads, 0, st, LUQ_LAUNCH_NORMAL, 1, d_x, n, d_amax, d_t);
   ctx->launches += 1;
   return static_cast<int>(e);
 }

@@ -168,6 +168,26 @@ def test_quant_grad_bit_exact(ctx, n, dtype, ns):
     assert ctx.status() == 0
 
 
+@pytest.mark.parametrize("exponent", [-103, -99, -80, -62, -59, -45, -20, 60, 95])
+@pytest.mark.parametrize("pw2", [False, True])
+def test_quant_grad_extreme_scales(ctx, exponent, pw2):
+    """Maxima near both ends of the accepted range, and on both sides of the point below which
+    the kernel rescales its operands: codes stay bit-exact (inputs reach into the denormals)."""
+    n = 300_000
+    x = (luq_inputs(n, 400 + exponent).astype(np.float64) * 2.0 ** exponent).astype(np.float32)
+    mx, _ = oracle.amax(x)
+    xd = to_dev(x)
+    if pw2:
+        want, a_want, fl = oracle.quant_luq_pw2(x, mx, 5, 2)
+        codes, alpha = ctx.quant_grad_pw2(xd, ctx.amax(xd), 5, 2)
+    else:
+        want, a_want, fl = oracle.quant_luq(x, mx, 5, 2)
+        codes, alpha = ctx.quant_grad(xd, ctx.amax(xd), 5, 2)
+    assert alpha.item() == a_want
+    np.testing.assert_array_equal(codes.cpu().numpy(), want)
+    assert ctx.status() == fl
+
+
 def test_quant_grad_seed_semantics_and_clipping(ctx):
     x = luq_inputs(50000, 9)
     xd = to_dev(x)
