@@ -63,6 +63,10 @@ extern "C" {
                               int32 accumulator could wrap (contractions beyond about 2^18 terms) */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
 #define LUQ_OPT_PAIRS 3    /* 1: products whose operands are both 8-bit planes run on CTA pairs (cta_group::2) */
+#define LUQ_OPT_LEVELS 4   /* kmax of the gradient quantizers, 1..6 (default luq_kmax() = 4): levels
+                              alpha * 2^0 .. alpha * 2^kmax with alpha = max / 2^kmax, codes 0..kmax+1.  The
+                              other grids of the paper from the same kernels: kmax = 2 is the FP2 grid of
+                              the ablation figure (Sec. 4), kmax = 6 uses the whole 3-bit exponent. */
 
 #define LUQ_MAX_SAMPLES 8
 
@@ -88,9 +92,9 @@ int luq_create(luq_ctx** out, int device);
 int luq_destroy(luq_ctx* ctx);
 int luq_set_option(luq_ctx* ctx, int option, int value);
 
-/* Number of binades between the underflow threshold and the tensor maximum:
+/* Default number of binades between the underflow threshold and the tensor maximum:
  * alpha = max|x| / 2^kmax.  The paper's Eq. (alpha) prints 2^(2^(b-1)) with
- * b = 3, i.e. kmax = 4. */
+ * b = 3, i.e. kmax = 4.  LUQ_OPT_LEVELS changes it per context. */
 int luq_kmax(void);
 
 /* max_i |x_i| of a tensor of n elements (Sec. 4, "Above FP maximum": the top
@@ -135,6 +139,16 @@ int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t
 int luq_amax_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
                         uint64_t seed, int n_samples, float* d_amax,
                         uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream);
+
+/* Biased logarithmic quantization, the "FP4" baseline of the paper's ablation (Sec. 4, Eq. RC):
+ * the grid, scale, code layout and clipping of luq_quant_grad, but deterministic.  In range, the
+ * nearer level in LINEAR distance (round-to-nearest-power: up from 2^n alpha exactly when
+ * |x| >= 3/2 * 2^n alpha, i.e. 2^floor(log2(4/3 * |x|/alpha))); below alpha, the nearer of 0 and alpha
+ * (up when |x| >= alpha/2).  One plane, no seed.  Implemented as the LUQ decision at probability
+ * 1/2: every random word is replaced by 2^31 - 1, no generator runs. */
+int luq_quant_grad_nearest(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
+                           const float* d_amax, uint8_t* d_codes, float* d_alpha, int8_t* d_operand,
+                           void* stream);
 
 /* LUQ with a power-of-two scale (Appendix A.7, LUQ_PW2): as luq_quant_grad, but
  * alpha = 2^ceil(log2 max) / 2^kmax - the maximum is rounded UP to a power of two,

@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
             L.oracle_quant_luq_window.argtypes = [f32p, sz, ctypes.c_uint64, ctypes.c_float, ctypes.c_int,
                                                   ctypes.c_uint64, ctypes.c_int, u8p, intp]
             L.oracle_quant_luq_window.restype = ctypes.c_float
+            L.oracle_quant_fp_nearest.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, u8p, intp]
+            L.oracle_quant_fp_nearest.restype = ctypes.c_float
             L.oracle_pw2_ceil.argtypes = [ctypes.c_float]
             L.oracle_pw2_ceil.restype = ctypes.c_float
             L.oracle_hindsight_next.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float]
@@ -144,6 +146,16 @@ def quant_luq(x: np.ndarray, mx, seed: int, n_samples: int = 1, kmax: int = KMAX
     a = lib().oracle_quant_luq_window(_ptr(xf, ctypes.c_float), xf.size, first_index, np.float32(mx), kmax,
                                       seed & (2**64 - 1), n_samples, _ptr(codes, ctypes.c_uint8),
                                       ctypes.byref(flags))
+    return codes, np.float32(a), flags.value
+
+
+def quant_fp_nearest(x: np.ndarray, mx, kmax: int = KMAX_DEFAULT):
+    """Deterministic round-to-nearest-power on the LUQ grid (Eq. RC); returns (codes[1, n/2], alpha, flags)."""
+    xf = widen(x).reshape(-1)
+    codes = np.zeros((1, (xf.size + 1) // 2), dtype=np.uint8)
+    flags = ctypes.c_int(0)
+    a = lib().oracle_quant_fp_nearest(_ptr(xf, ctypes.c_float), xf.size, np.float32(mx), kmax,
+                                      _ptr(codes, ctypes.c_uint8), ctypes.byref(flags))
     return codes, np.float32(a), flags.value
 
 

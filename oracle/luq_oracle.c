@@ -201,6 +201,42 @@ float oracle_quant_luq_window(const float* x, size_t n, uint64_t first_index, fl
 }
 
 /* ------------------------------------------------------------------------ */
+/* Biased logarithmic quantization: the "FP4" baseline of the ablation         */
+/* (Sec. 4, Eq. RC).  Same grid, scale and code layout as LUQ, no randomness.  */
+/*   in range  : RDNP(2^x) = 2^floor(log2(4/3 * 2^x)): the level nearest in     */
+/*               linear distance; the midpoint of [2^n, 2^(n+1)] is 3/2 * 2^n   */
+/*               and goes up (the floor of an exact integer).                   */
+/*   below alpha (reading: the paper only draws it): the nearer of 0 and alpha, */
+/*               |x| = alpha/2 goes up like the other midpoints.                */
+/*   above max : the top level (cannot happen with mx = the tensor maximum).    */
+/* Written on t = fl32(|x|/alpha), the quantity the LUQ decisions use too.      */
+/* ------------------------------------------------------------------------ */
+float oracle_quant_fp_nearest(const float* x, size_t n, float mx, int kmax, uint8_t* codes, int* flags) {
+  size_t plane = (n + 1) / 2;
+  memset(codes, 0, plane);
+  if (!scale_usable(mx, flags)) return 0.0f;
+  float alpha = oracle_luq_alpha(mx, kmax);
+  for (size_t i = 0; i < n; ++i) {
+    float t = fabsf(x[i]) / alpha;
+    uint32_t sign = bits_of(x[i]) >> 31;
+    uint32_t c;
+    if (!(t < ldexpf(1.0f, kmax))) {      /* at or above the top level, Inf, NaN */
+      c = (uint32_t)kmax + 1u;
+    } else if (t < 1.0f) {
+      c = (t >= 0.5f) ? 1u : 0u;
+    } else {
+      /* floor(log2(4/3 t)): the largest m with 2^m <= 4t/3, i.e. 3 * 2^m <= 4t (exact in double) */
+      int m = 0;
+      while (3.0 * ldexp(1.0, m + 1) <= 4.0 * (double)t) ++m;
+      c = (uint32_t)m + 1u;                /* level alpha * 2^m has code m + 1 */
+    }
+    uint8_t nib = c ? (uint8_t)((sign << 3) | c) : 0;
+    codes[i >> 1] |= (uint8_t)(nib << ((i & 1) * 4));
+  }
+  return alpha;
+}
+
+/* ------------------------------------------------------------------------ */
 /* Power-of-two LUQ (Appendix A.7): alpha_PW2 = 2^ceil(log2 max|x|) / 2^kmax. */
 /* The maximum is rounded UP to a power of two (so nothing is clipped), the   */
 /* quantizer itself is unchanged; every level is then a power of two.         */

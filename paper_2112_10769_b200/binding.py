@@ -17,11 +17,11 @@ LIB_PATH = os.path.join(_HERE, "libluq_b200.so")
 
 LUQ_F32, LUQ_BF16 = 0, 1
 STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT = 1, 2, 4
-OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS = 1, 2, 3
+OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS = 1, 2, 3, 4
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_pw2",
+           "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_pw2",
            "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
@@ -51,6 +51,7 @@ def load() -> ctypes.CDLL:
         L.luq_amax_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_amax_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, u64, ctypes.c_int, vp, vp, vp, vp, vp]
         L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
+        L.luq_quant_grad_nearest.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, ctypes.c_int, u64,
                                                ctypes.c_int, vp, vp, vp, vp, vp]
@@ -179,6 +180,17 @@ class Context:
         _check(load().luq_quant_grad(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
                                      seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
                                      _opt(operand, n_samples * g.numel()), _stream()), "luq_quant_grad")
+        return codes, alpha
+
+    def quant_grad_nearest(self, g: torch.Tensor, amax: torch.Tensor, codes: torch.Tensor | None = None,
+                           alpha: torch.Tensor | None = None, operand: torch.Tensor | None = None):
+        """Deterministic round-to-nearest-power on the LUQ grid (the biased FP4 baseline)."""
+        rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
+        codes = torch.empty((1, g.numel() // 2), dtype=torch.uint8, device=g.device) if codes is None else codes
+        alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
+        _check(load().luq_quant_grad_nearest(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
+                                             codes.data_ptr(), alpha.data_ptr(), _opt(operand, g.numel()),
+                                             _stream()), "luq_quant_grad_nearest")
         return codes, alpha
 
     def quant_grad_pw2(self, g: torch.Tensor, amax: torch.Tensor, seed: int, n_samples: int = 1,

@@ -55,6 +55,7 @@ int luq_create(luq_ctx** out, int device) {
   c->mma_kind = LUQ_DEFAULT_MMA_KIND;
   c->forced_splits = 0;
   c->use_pairs = 0;
+  c->kmax = LUQ_KMAX;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;
   c->d_status = nullptr; c->d_scratch = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
@@ -93,6 +94,10 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
     case LUQ_OPT_SPLITS:
       if (value < 0 || value > 1024) return LUQ_ERR_ARG;
       ctx->forced_splits = value;
+      return LUQ_OK;
+    case LUQ_OPT_LEVELS:
+      if (value < 1 || value > 6) return LUQ_ERR_ARG;
+      ctx->kmax = value;
       return LUQ_OK;
     case LUQ_OPT_PAIRS:
       if (value != 0 && value != 1) return LUQ_ERR_ARG;
@@ -178,6 +183,17 @@ int luq_amax_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, s
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, nullptr, seed, n_samples, d_codes,
                                           n ? d_operand : nullptr, d_alpha, 0, nullptr, nullptr, 0.0f, d_amax,
                                           as_stream(stream)));
+}
+
+int luq_quant_grad_nearest(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
+                           uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream) {
+  size_t n = 0;
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, 1, d_codes, d_alpha, d_operand, &n);
+  if (rc) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, 0, 1, d_codes, n ? d_operand : nullptr,
+                                          d_alpha, 4, nullptr, nullptr, 0.0f, nullptr, as_stream(stream)));
 }
 
 int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,

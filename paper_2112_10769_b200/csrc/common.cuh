@@ -6,7 +6,7 @@
 
 #include "luq.h"
 
-#define LUQ_KMAX 4  // alpha = max / 2^LUQ_KMAX (Eq. alpha with b = 3)
+#define LUQ_KMAX 4  // default level count: alpha = max / 2^LUQ_KMAX (Eq. alpha with b = 3)
 #define LUQ_DEFAULT_MMA_KIND 2  // automatic: int8, the type of the operand bytes the quantizers can emit
 
 struct luq_ctx {
@@ -19,6 +19,7 @@ struct luq_ctx {
   int mma_kind;             // 0 f8f6f4/e4m3, 1 i8, 2 chosen per product
   int forced_splits;        // 0 = automatic
   int use_pairs;            // CTA-pair kernel for products whose operands are both planes
+  int kmax;                 // LUQ levels alpha * 2^0 .. alpha * 2^kmax (1..6, default LUQ_KMAX)
   int64_t launches;
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved at create
 };

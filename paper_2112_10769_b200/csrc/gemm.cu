@@ -1087,6 +1087,7 @@ extern "C" int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_al
   local.mma_kind = LUQ_DEFAULT_MMA_KIND;
   local.forced_splits = 0;
   local.use_pairs = 0;
+  local.kmax = LUQ_KMAX;
   local.launches = 0;
   local.encode_tiled = s->encode_tiled;
 

@@ -342,7 +342,12 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
 // expands it into the ten round keys of every sample and passes them as kernel
 // parameters, so a round is two wide multiplies and two three-input XORs.
 struct PhiloxKeys { uint32_t k0[10]; uint32_t k1[10]; };
-struct PhiloxKeySet { PhiloxKeys s[LUQ_MAX_SAMPLES]; };
+// Per-launch constants of the LUQ kernel: the round keys of every sample, and the grid.
+//   inv_levels = 2^-kmax (alpha = max * inv_levels), q_top = 2^(32 + kmax) (the top level on the
+//   scale of Q).  fixed_word != 0 replaces every random word by that constant: with 0x7FFFFFFF
+//   an element goes up exactly when its up-probability is at least 1/2, which is deterministic
+//   round-to-nearest-power (Eq. RC), ties up.
+struct PhiloxKeySet { PhiloxKeys s[LUQ_MAX_SAMPLES]; uint32_t fixed_word; float inv_levels; float q_top; };
 
 __device__ __forceinline__ void mul_wide(uint32_t a, uint32_t b, uint32_t& lo, uint32_t& hi) {
   asm("{\n\t.reg .b64 t;\n\tmul.wide.u32 t, %2, %3;\n\tmov.b64 {%0, %1}, t;\n\t}" : "=r"(lo), "=r"(hi) : "r"(a), "r"(b));
@@ -395,9 +400,9 @@ __device__ __forceinline__ float luq_scaled_quotient(float a, const LuqScale& sc
   return __fmaf_rn(r1, sc.recip, q1);
 }
 template <bool PW2 = false>
-__device__ __forceinline__ float luq_quotient_clamped(float x, const LuqScale& sc) {
+__device__ __forceinline__ float luq_quotient_clamped(float x, const LuqScale& sc, float q_top) {
   // an overflowing or non-finite quotient turns into NaN or Inf; both belong to the top level
-  return fminf(luq_scaled_quotient<PW2>(fabsf(x) * sc.pre, sc), 0x1p32f * static_cast<float>(1 << LUQ_KMAX));   // fminf(NaN, c) = c
+  return fminf(luq_scaled_quotient<PW2>(fabsf(x) * sc.pre, sc), q_top);   // fminf(NaN, c) = c
 }
 
 // Per element: lower code and the 32-bit threshold of the up-decision, from the
@@ -469,7 +474,11 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
   const float mx = PW2 ? pw2_ceil(given) : given;
   const bool first = blockIdx.x == 0 && threadIdx.x == 0;
   const bool ok = scale_usable(mx, first ? status : nullptr);
-  const float alpha = ok ? mx * (1.0f / static_cast<float>(1 << LUQ_KMAX)) : 0.0f;  // exact scaling
+  const float alpha = ok ? mx * keys.inv_levels : 0.0f;  // exact scaling
+  const uint32_t fixed_word = keys.fixed_word;
+  auto random_words = [&](uint64_t block, const PhiloxKeys& ks) {
+    return fixed_word ? make_uint4(fixed_word, fixed_word, fixed_word, fixed_word) : philox_block(block, ks);
+  };
   if (first) *d_alpha = alpha;
   const LuqScale sc = luq_scale(ok ? alpha : 1.0f);   // with a power-of-two alpha the reciprocal is exact
   uint32_t seen = 0;   // running max of |x| bit patterns (TRACK)
@@ -515,7 +524,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
         uint32_t bytes[kElems / 4] = {};
 #pragma unroll
         for (int b = 0; b < kElems / 4; ++b) {
-          const uint4 r = philox_block(item * (kElems / 4) + b, ks);
+          const uint4 r = random_words(item * (kElems / 4) + b, ks);
           const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -532,7 +541,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
     }
     uint32_t lo_code[kElems], thr[kElems];
 #pragma unroll
-    for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient_clamped<PW2>(v[j], sc), lo_code[j], thr[j]);
+    for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient_clamped<PW2>(v[j], sc, keys.q_top), lo_code[j], thr[j]);
 #pragma unroll
     for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
       if (NS == 0 && s >= n_samples) break;
@@ -541,7 +550,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
       uint32_t bytes[kElems / 4] = {};
 #pragma unroll
       for (int b = 0; b < kElems / 4; ++b) {
-        const uint4 r = philox_block(item * (kElems / 4) + b, ks);
+        const uint4 r = random_words(item * (kElems / 4) + b, ks);
         const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -597,8 +606,8 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
           if (ok && idx < n) {
             const float xv = Item<BF16>::load1(x, idx);
             uint32_t lc, th;
-            luq_bin(luq_quotient_clamped<PW2>(xv, sc), lc, th);
-            const uint4 r = philox_block(idx >> 2, ks);
+            luq_bin(luq_quotient_clamped<PW2>(xv, sc, keys.q_top), lc, th);
+            const uint4 r = random_words(idx >> 2, ks);
             const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
             nib[h] = luq_nibble(__float_as_uint(xv), lc, th, rw[idx & 3]);
           }
@@ -625,10 +634,10 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
 // (before the clamp to the top level), for comparison with an IEEE division.
 __global__ void __launch_bounds__(kThreads) luq_quotient_kernel(const float* __restrict__ x, size_t n,
                                                                 const float* __restrict__ d_amax,
-                                                                float* __restrict__ out) {
+                                                                float inv_levels, float* __restrict__ out) {
   luqdev::pdl_wait();
   luqdev::pdl_trigger();
-  const float alpha = __ldg(d_amax) * (1.0f / static_cast<float>(1 << LUQ_KMAX));
+  const float alpha = __ldg(d_amax) * inv_levels;
   const LuqScale sc = luq_scale(alpha);
   const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
   for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < n; i += stride)
@@ -694,8 +703,11 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
 }
 
 namespace {
-PhiloxKeySet expand_keys(uint64_t seed, int n_samples) {
+PhiloxKeySet expand_keys(uint64_t seed, int n_samples, int kmax, uint32_t fixed_word) {
   PhiloxKeySet keys{};
+  keys.fixed_word = fixed_word;
+  keys.inv_levels = 1.0f / static_cast<float>(1 << kmax);
+  keys.q_top = 4294967296.0f * static_cast<float>(1 << kmax);
   for (int s = 0; s < n_samples; ++s) {   // sample s is keyed by seed + s
     const uint64_t key = seed + static_cast<uint64_t>(s);
     uint32_t a = static_cast<uint32_t>(key), b = static_cast<uint32_t>(key >> 32);
@@ -734,11 +746,13 @@ int launch_luq(const LuqLaunch& a) {
 }  // namespace
 
 // flags: bit 0 = power-of-two scale; bit 1 = in-hindsight: d_amax is the running estimate, the
-// tensor's own maximum goes to d_measured and the estimate is replaced (eta) by the same kernel
+// tensor's own maximum goes to d_measured and the estimate is replaced (eta) by the same kernel;
+// bit 2 = deterministic round-to-nearest-power instead of the random words
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
                              float* d_measured, float* d_estimate, float eta, float* d_amax_out, cudaStream_t st) {
-  const LuqLaunch a{ctx, d_g, n, d_amax, expand_keys(seed, n_samples), n_samples, d_codes, d_operand, d_alpha,
+  const LuqLaunch a{ctx, d_g, n, d_amax, expand_keys(seed, n_samples, ctx->kmax, (flags & 4) ? 0x7FFFFFFFu : 0u),
+                    n_samples, d_codes, d_operand, d_alpha,
                     reinterpret_cast<unsigned int*>(d_measured), d_estimate, eta, d_amax_out, st};
   int rc;
   switch ((flags & 3) | (dtype == LUQ_BF16 ? 4 : 0)) {
@@ -759,7 +773,8 @@ int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const fl
                               cudaStream_t st) {
   if (n == 0) return 0;
   const int grid = grid_for(ctx, luq_quotient_kernel, n / kThreads + 1);
-  const cudaError_t e = luq_launch_kernel(luq_quotient_kernel, grid, kThreads, 0, st, LUQ_LAUNCH_NORMAL, 1, d_x, n, d_amax, d_t);
+  const cudaError_t e = luq_launch_kernel(luq_quotient_kernel, grid, kThreads, 0, st, LUQ_LAUNCH_NORMAL, 1, d_x, n, d_amax,
+                                          1.0f / static_cast<float>(1 << ctx->kmax), d_t);
   ctx->launches += 1;
   return static_cast<int>(e);
 }

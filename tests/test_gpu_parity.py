@@ -419,3 +419,91 @@ def test_hindsight_unusable_estimate_recovers(ctx):
     with pytest.raises(binding.LuqError):
         ctx.quant_grad_hindsight(xd, m_hat, 1.5, 1)
     assert ctx.status() == 0
+
+
+# ------------------------------- other grids from the same kernels: level count, nearest power ----
+
+@pytest.mark.parametrize("kmax", [1, 2, 3, 5, 6])
+@pytest.mark.parametrize("dtype,ns", [("f32", 1), ("bf16", 2)])
+def test_quant_grad_other_level_counts(ctx, kmax, dtype, ns):
+    n = 500_002
+    x = inputs.log_uniform_magnitudes(n, -12, 1, 60 + kmax)       # every level of every grid occurs
+    if dtype == "bf16":
+        x = inputs.to_bf16_bits(x)
+    mx, _ = oracle.amax(x)
+    xd = to_dev(x)
+    ctx.set_option(binding.OPT_LEVELS, kmax)
+    try:
+        want, a_want, _ = oracle.quant_luq(x, mx, 21, ns, kmax=kmax)
+        ob = torch.empty(ns * n, dtype=torch.int8, device="cuda")
+        codes, alpha = ctx.quant_grad(xd, ctx.amax(xd), 21, ns, operand=ob)
+        assert alpha.item() == a_want == oracle.luq_alpha(mx, kmax)
+        np.testing.assert_array_equal(codes.cpu().numpy(), want)
+        assert set(np.unique(oracle.unpack(want[0], n) & 7)) == set(range(kmax + 2))
+        got = ob.cpu().numpy().reshape(ns, n)
+        for s in range(ns):
+            np.testing.assert_array_equal(got[s], oracle.dequant(want[s], n, 1.0, "luq").astype(np.int8))
+        want, a_want, _ = oracle.quant_luq_pw2(x, mx, 22, ns, kmax=kmax)
+        codes, alpha = ctx.quant_grad_pw2(xd, ctx.amax(xd), 22, ns)
+        assert alpha.item() == a_want
+        np.testing.assert_array_equal(codes.cpu().numpy(), want)
+        _, codes, alpha = ctx.amax_quant_grad(xd, 21, ns)
+        np.testing.assert_array_equal(codes.cpu().numpy(), oracle.quant_luq(x, mx, 21, ns, kmax=kmax)[0])
+    finally:
+        ctx.set_option(binding.OPT_LEVELS, 4)
+    with pytest.raises(binding.LuqError):
+        ctx.set_option(binding.OPT_LEVELS, 7)
+    assert ctx.status() == 0
+
+
+def test_gemms_with_the_widest_grid(ctx):
+    """kmax = 6: gradient levels up to 64 alpha; the GEMMs must still be exact."""
+    M, K, N, ns = 384, 256, 288, 2
+    A, W, G = inputs.small_layer(M, K, N, 91)
+    ctx.set_option(binding.OPT_LEVELS, 6)
+    try:
+        Ad, Wd, Gd = to_dev(A), to_dev(W), to_dev(G)
+        ca, sa = ctx.quant_int4(Ad, ctx.amax(Ad))
+        cw, sw = ctx.quant_int4(Wd, ctx.amax(Wd))
+        cg, al = ctx.quant_grad(Gd, ctx.amax(Gd), 3, ns)
+        og, oal, _ = oracle.quant_luq(G, oracle.amax(G)[0], 3, ns, kmax=6)
+        np.testing.assert_array_equal(cg.cpu().numpy(), og)
+        assert (oracle.unpack(og[0], M * N) & 7).max() == 7
+        for kind in (0, 1):
+            ctx.set_option(binding.OPT_MMA_KIND, kind)
+            dA = ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K)
+            dW = ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K)
+            assert_gemm_close(dA.cpu().numpy(), oracle.gemm_bwd(og, oal, ns, cw.cpu().numpy(), sw.item(), M, N, K))
+            assert_gemm_close(dW.cpu().numpy(), oracle.gemm_wgrad(og, oal, ns, ca.cpu().numpy(), sa.item(), M, N, K))
+    finally:
+        ctx.set_option(binding.OPT_MMA_KIND, 2)
+        ctx.set_option(binding.OPT_LEVELS, 4)
+    assert ctx.status() == 0
+
+
+@pytest.mark.parametrize("n", [10, 4098, (1 << 20) + 2])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("kmax", [2, 4])
+def test_quant_grad_nearest_power_bit_exact(ctx, n, dtype, kmax):
+    x = luq_inputs(n, 700 + n)
+    mx0 = np.abs(x).max()
+    # values on and around the midpoints of the bins, where the deterministic decision flips
+    al = np.float32(mx0) / np.float32(2 ** kmax)
+    mids = np.array([al * 0.5, al * 1.5, al * 3, al * 6], dtype=np.float32)
+    k = min(n - 2, 12)
+    x[-k:] = np.concatenate([mids, np.nextafter(mids, np.float32(0)), np.nextafter(mids, np.float32(np.inf))])[:k]
+    if dtype == "bf16":
+        x = inputs.to_bf16_bits(x)
+    mx, _ = oracle.amax(x)
+    xd = to_dev(x)
+    ctx.set_option(binding.OPT_LEVELS, kmax)
+    try:
+        want, a_want, _ = oracle.quant_fp_nearest(x, mx, kmax)
+        ob = torch.empty(n, dtype=torch.int8, device="cuda")
+        codes, alpha = ctx.quant_grad_nearest(xd, ctx.amax(xd), operand=ob)
+        assert alpha.item() == a_want
+        np.testing.assert_array_equal(codes.cpu().numpy(), want)
+        np.testing.assert_array_equal(ob.cpu().numpy(), oracle.dequant(want[0], n, 1.0, "luq").astype(np.int8))
+    finally:
+        ctx.set_option(binding.OPT_LEVELS, 4)
+    assert ctx.status() == 0

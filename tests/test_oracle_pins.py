@@ -635,3 +635,80 @@ def test_hindsight_step_uses_the_estimate_and_clips_above_it():
     # with the power-of-two option the estimate is rounded up first
     codes2, alpha2, _, _, nxt2 = oracle.quant_luq_hindsight(x, m_hat, 0.1, seed=9, pw2=True)
     assert float(alpha2) * 16 == float(oracle.pw2_ceil(m_hat)) and nxt2 == nxt
+
+
+# ------------------------------------- biased FP4 baseline: round-to-nearest-power (Eq. RC) ----
+
+def _levels(kmax):
+    return np.array([0.0] + [2.0 ** k for k in range(kmax + 1)])
+
+
+@pytest.mark.parametrize("kmax", [2, 4, 6])
+def test_nearest_power_is_the_linear_nearest_level(kmax):
+    """RDNP exists because rounding the EXPONENT to nearest is biased; Eq. (RC) shifts it so that the
+    chosen level is the nearest one in linear distance.  Brute force over the levels, away from ties."""
+    rng = np.random.default_rng(70 + kmax)
+    mx = np.float32(3.7)
+    alpha = float(oracle.luq_alpha(mx, kmax))
+    t = np.exp2(rng.uniform(-6, kmax, 20000))
+    lv = _levels(kmax)
+    mids = (lv[:-1] + lv[1:]) / 2
+    t = t[np.min(np.abs(t[:, None] - mids[None, :]), axis=1) > 1e-4]
+    x = (t * alpha * np.where(rng.random(t.size) < 0.5, -1, 1)).astype(np.float32)
+    if x.size % 2:
+        x = x[:-1]
+    codes, a, fl = oracle.quant_fp_nearest(x, mx, kmax)
+    assert fl == 0 and float(a) == alpha
+    got = oracle.dequant(codes[0], x.size, 1.0, "luq")
+    tt = np.abs(x.astype(np.float64)) / alpha
+    want = lv[np.argmin(np.abs(tt[:, None] - lv[None, :]), axis=1)] * np.sign(x)
+    np.testing.assert_array_equal(got, want)
+
+
+def test_nearest_power_matches_the_printed_formulas():
+    """2^floor(log2(4/3 * 2^x)) and the printed 2^RDN(x - 0.085), evaluated in float64 away from ties."""
+    shift = golden()["rdnp_shift"][0]                      # -0.085, printed in Eq. (RC)
+    rng = np.random.default_rng(5)
+    xs = rng.uniform(0.0, 4.0, 20000)                       # exponents inside the range of kmax = 4
+    frac = (xs + math.log2(4 / 3)) % 1.0
+    xs = xs[np.minimum(frac, 1 - frac) > 1e-3]
+    mx = np.float32(16.0)                                   # alpha = 1
+    x = np.exp2(xs).astype(np.float32)
+    if x.size % 2:
+        x, xs = x[:-1], xs[:-1]
+    xs = np.log2(x.astype(np.float64))
+    codes, a, _ = oracle.quant_fp_nearest(x, mx, 4)
+    assert float(a) == 1.0
+    got = oracle.dequant(codes[0], x.size, 1.0, "luq")
+    np.testing.assert_array_equal(got, np.exp2(np.floor(xs + math.log2(4 / 3))))
+    np.testing.assert_array_equal(got, np.exp2(np.rint(xs + shift)))
+
+
+def test_nearest_power_ties_underflow_clipping_and_bias():
+    mx = np.float32(16.0)
+    x = np.array([1.5, 3.0, 6.0, 12.0, 0.5, 0.49999997, 0.0, -0.75, 1.0, 2.0, 16.0, 40.0, -1.4999999, 11.999999],
+                 dtype=np.float32)
+    codes, _, _ = oracle.quant_fp_nearest(x, mx, 4)
+    got = oracle.dequant(codes[0], x.size, 1.0, "luq")
+    # midpoints go up (the floor of an exact power of two), alpha/2 goes up, values above max clip
+    np.testing.assert_array_equal(got, [2, 4, 8, 16, 1, 0, 0, -1, 1, 2, 16, 16, -1, 8])
+    # on-grid values are fixed points
+    grid = np.array([0, 1, 2, 4, 8, 16, -1, -2, -4, -8, -16, 0], dtype=np.float32)
+    c2, _, _ = oracle.quant_fp_nearest(grid, mx, 4)
+    np.testing.assert_array_equal(oracle.dequant(c2[0], grid.size, 1.0, "luq"), grid)
+    # it is biased, unlike LUQ: for a log-uniform density on one bin the mean error is
+    # (2 ln 2 - ln 1.5 - 1) / ln 2 of the bin's lower edge (closed form of the two integrals)
+    n = 1 << 20
+    u = (np.arange(n) + 0.5) / n
+    t = np.exp2(u).astype(np.float32)                       # log-uniform on [1, 2), alpha = 1
+    c3, _, _ = oracle.quant_fp_nearest(t, mx, 4)
+    err = (oracle.dequant(c3[0], n, 1.0, "luq") - t.astype(np.float64)).mean()
+    closed = (2 * math.log(2) - math.log(1.5) - 1) / math.log(2)
+    assert abs(err - closed) < 1e-5 and closed < -0.02
+    # and it is the LUQ decision taken at probability one half: up exactly when the up-threshold >= 2^31
+    xr = inputs.log_uniform_magnitudes(20000, -6, 4.5, 9)
+    m2 = np.float32(np.abs(xr).max())
+    lo, hi, thr = oracle.luq_bins(xr, m2)
+    c4, al, _ = oracle.quant_fp_nearest(xr, m2, 4)
+    got = np.abs(oracle.dequant(c4[0], xr.size, 1.0, "luq"))
+    np.testing.assert_array_equal(got, np.where(thr >= 2 ** 31, hi, lo))
