@@ -202,3 +202,40 @@ def test_gemm_reads_the_bytes_it_is_given(ctx):
         ctx.set_option(binding.OPT_MMA_KIND, 2)
     assert torch.equal(Z_e4m3, ctx.gemm_fwd(ca, sa, cw, sw, M, N, K))
     assert ctx.status() == 0
+
+
+@pytest.mark.parametrize("mma_kind", [0, 2])
+def test_cta_pair_kernel_matches_the_single_cta_kernel(ctx, mma_kind):
+    """LUQ_OPT_PAIRS: products whose operands both arrive as bytes and whose contraction is not split
+    run on CTA pairs (256-row tiles, cta_group::2).  Same integers, same epilogue: bit-identical.
+    The shape has more tiles than half the SMs (no split) and ragged edges in both directions."""
+    M, K, N, ns = 2176, 1024, 2304, 2
+    A, W, G = inputs.small_layer(M, K, N, 123)
+    (ca, sa, ba), (cw, sw, bw), (cg, al, bg) = layer_with_bytes(ctx, A, W, G, seed=5, ns=ns)
+    ctx.set_option(binding.OPT_MMA_KIND, mma_kind)
+    try:
+        single = (ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=ba, w_operand=bw),
+                  ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bg, w_operand=bw),
+                  ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K, g_operand=bg, a_operand=ba))
+        launches = ctx.launches
+        ctx.set_option(binding.OPT_PAIRS, 1)
+        paired = (ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=ba, w_operand=bw),
+                  ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bg, w_operand=bw),
+                  ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K, g_operand=bg, a_operand=ba))
+    finally:
+        ctx.set_option(binding.OPT_PAIRS, 0)
+        ctx.set_option(binding.OPT_MMA_KIND, 2)
+    assert ctx.status() == 0
+    for s, p in zip(single, paired):
+        assert torch.equal(s, p)
+    oa, ow, og = ca.cpu().numpy(), cw.cpu().numpy(), cg.cpu().numpy().reshape(ns, -1)
+    r = np.array([0, 127, 128, 255, 256, 1000, M - 1, M - 1, 0], dtype=np.int64)
+    c = np.array([0, 255, 256, 1, N - 1, 777, N - 1, 0, N - 1], dtype=np.int64)
+    assert_gemm_close(paired[0].cpu().numpy()[r, c],
+                      oracle.gemm_entries("fwd", oa, sa.item(), 1, ow, sw.item(), M, N, K, r, c))
+    ck = np.minimum(c, K - 1)
+    assert_gemm_close(paired[1].cpu().numpy()[r, ck],
+                      oracle.gemm_entries("bwd", og, al.item(), ns, ow, sw.item(), M, N, K, r, ck))
+    rn = np.minimum(r, N - 1)
+    assert_gemm_close(paired[2].cpu().numpy()[rn, ck],
+                      oracle.gemm_entries("wgrad", og, al.item(), ns, oa, sa.item(), M, N, K, rn, ck))
