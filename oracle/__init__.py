@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
             L.oracle_amax.restype = ctypes.c_float
             L.oracle_quant_int4.argtypes = [f32p, sz, ctypes.c_float, u8p, intp]
             L.oracle_quant_int4.restype = ctypes.c_float
+            L.oracle_quant_uint4.argtypes = [f32p, sz, ctypes.c_float, u8p, intp]
+            L.oracle_quant_uint4.restype = ctypes.c_float
             L.oracle_luq_alpha.argtypes = [ctypes.c_float, ctypes.c_int]
             L.oracle_luq_alpha.restype = ctypes.c_float
             L.oracle_quant_luq.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, ctypes.c_uint64,
@@ -128,6 +130,16 @@ def quant_int4(x: np.ndarray, clip):
     flags = ctypes.c_int(0)
     s = lib().oracle_quant_int4(_ptr(xf, ctypes.c_float), xf.size, np.float32(clip),
                                 _ptr(codes, ctypes.c_uint8), ctypes.byref(flags))
+    return codes, np.float32(s), flags.value
+
+
+def quant_uint4(x: np.ndarray, clip):
+    """Unsigned INT4 (range [0, clip], s = clip/15) for non-negative tensors.  Returns (codes, scale, flags)."""
+    xf = widen(x).reshape(-1)
+    codes = np.zeros((xf.size + 1) // 2, dtype=np.uint8)
+    flags = ctypes.c_int(0)
+    s = lib().oracle_quant_uint4(_ptr(xf, ctypes.c_float), xf.size, np.float32(clip),
+                                 _ptr(codes, ctypes.c_uint8), ctypes.byref(flags))
     return codes, np.float32(s), flags.value
 
 
@@ -206,10 +218,10 @@ def unpack(codes: np.ndarray, n: int) -> np.ndarray:
 
 
 def dequant(codes: np.ndarray, n: int, scale, kind: str) -> np.ndarray:
-    """Values of a packed plane in float64.  kind: 'int4' or 'luq'."""
+    """Values of a packed plane in float64.  kind: 'int4', 'luq' or 'uint4'."""
     codes = np.ascontiguousarray(codes).reshape(-1)
     out = np.zeros(n, dtype=np.float64)
-    lib().oracle_dequant(_ptr(codes, ctypes.c_uint8), n, float(scale), 0 if kind == "int4" else 1,
+    lib().oracle_dequant(_ptr(codes, ctypes.c_uint8), n, float(scale), {"int4": 0, "luq": 1, "uint4": 2}[kind],
                          _ptr(out, ctypes.c_double))
     return out
 

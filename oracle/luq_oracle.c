@@ -125,6 +125,30 @@ float oracle_quant_int4(const float* x, size_t n, float clip, uint8_t* codes, in
   return s;
 }
 
+/* ------------------------------------------------------------------------ */
+/* Unsigned INT4 for tensors that cannot be negative (post-ReLU activations).  */
+/* Appendix "Quantization formats": scale = Delta / (2^b - 1), Delta the        */
+/* quantized range: for the range [0, clip] and b = 4, s = clip/15 and the      */
+/* codes are the integers 0..15 (all sixteen levels on one side of zero).       */
+/* Round to nearest, ties to even; negative inputs clamp to 0.                  */
+/* ------------------------------------------------------------------------ */
+float oracle_quant_uint4(const float* x, size_t n, float clip, uint8_t* codes, int* flags) {
+  if (!scale_usable(clip, flags)) { memset(codes, 0, (n + 1) / 2); return 0.0f; }
+  float s = clip / 15.0f;
+  float inv = 15.0f / clip;
+  memset(codes, 0, (n + 1) / 2);
+  for (size_t i = 0; i < n; ++i) {
+    float y = x[i] * inv;
+    float r = rintf(y);
+    if (r > 15.0f) r = 15.0f;
+    if (r < 0.0f) r = 0.0f;
+    if (r != r) r = 0.0f; /* NaN element -> 0 */
+    uint8_t nib = (uint8_t)((int)r & 0xF);
+    codes[i >> 1] |= (uint8_t)(nib << ((i & 1) * 4));
+  }
+  return s;
+}
+
 int oracle_int4_value(uint8_t nibble) { /* two's complement 4 bit */
   int v = nibble & 0xF;
   return v >= 8 ? v - 16 : v;
@@ -287,10 +311,12 @@ double oracle_luq_value(uint8_t nibble) { /* in units of alpha */
 /* ------------------------------------------------------------------------ */
 /* Dequantise and multiply: the plain definition (Appendix A.1: the scale is  */
 /* a single high-precision factor, all MACs act on the low-precision values). */
-/* kind: 0 = INT4 codes (value q*scale), 1 = LUQ codes (value +-scale*2^(c-1)) */
+/* kind: 0 = INT4 codes (value q*scale), 1 = LUQ codes (value +-scale*2^(c-1)),  */
+/*       2 = unsigned INT4 codes (value nibble*scale)                            */
 /* ------------------------------------------------------------------------ */
 static double code_value(const uint8_t* codes, size_t idx, int kind) {
   uint8_t nib = (codes[idx >> 1] >> ((idx & 1) * 4)) & 0xF;
+  if (kind == 2) return (double)nib;
   return kind ? oracle_luq_value(nib) : (double)oracle_int4_value(nib);
 }
 

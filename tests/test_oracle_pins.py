@@ -712,3 +712,42 @@ def test_nearest_power_ties_underflow_clipping_and_bias():
     c4, al, _ = oracle.quant_fp_nearest(xr, m2, 4)
     got = np.abs(oracle.dequant(c4[0], xr.size, 1.0, "luq"))
     np.testing.assert_array_equal(got, np.where(thr >= 2 ** 31, hi, lo))
+
+
+# ------------------------------------------------- unsigned INT4 for non-negative tensors ----
+
+def test_uint4_grid_error_bound_and_edges():
+    rng = np.random.default_rng(11)
+    x = np.maximum(rng.standard_normal(100_000), 0).astype(np.float32)      # post-ReLU: half zeros
+    clip, _ = oracle.amax(x)
+    codes, s, fl = oracle.quant_uint4(x, clip)
+    assert fl == 0 and s == np.float32(clip) / np.float32(15)
+    q = oracle.unpack(codes, x.size)
+    assert q.max() == 15 and q.min() == 0                                   # the maximum takes the top code
+    deq = oracle.dequant(codes, x.size, float(s), "uint4")
+    np.testing.assert_array_equal(deq, q.astype(np.float64) * float(s))
+    assert np.abs(deq - x).max() <= float(s) / 2 * (1 + 1e-6)               # round to nearest
+    assert (q[x == 0] == 0).all()
+    # half the step of the signed grid on the same range: Delta/(2^b - 1) with all levels on one side
+    _, s_signed, _ = oracle.quant_int4(x, clip)
+    assert abs(float(s) / float(s_signed) - 7 / 15) < 1e-6
+    # negative inputs clamp to zero, values above the clip to 15, ties go to even, NaN to 0
+    c = np.float32(15.0)
+    y = np.array([-3.0, 0.5, 1.5, 2.5, 14.5, 15.5, 99.0, np.nan, 7.49, 7.51], dtype=np.float32)
+    cy, sy, _ = oracle.quant_uint4(y, c)
+    assert sy == 1.0
+    np.testing.assert_array_equal(oracle.unpack(cy, y.size), [0, 0, 2, 2, 14, 15, 15, 0, 7, 8])
+    # idempotent on its own grid, and brute force against the nearest of the sixteen levels
+    g = (np.arange(16, dtype=np.float32) * np.float32(0.25))
+    cg, sg, _ = oracle.quant_uint4(g, np.float32(3.75))
+    np.testing.assert_array_equal(oracle.unpack(cg, 16), np.arange(16))
+    z = rng.uniform(0, 3.75, 4000).astype(np.float32)
+    z = z[np.abs((z / 0.25) % 1.0 - 0.5) > 1e-3]
+    z = z[: z.size // 2 * 2]
+    cz, _, _ = oracle.quant_uint4(z, np.float32(3.75))
+    want = np.argmin(np.abs(z.astype(np.float64)[:, None] - g.astype(np.float64)[None, :]), axis=1)
+    np.testing.assert_array_equal(oracle.unpack(cz, z.size), want)
+    # unusable clips behave like the signed quantizer's
+    for bad, flag in ((0.0, 0), (np.inf, oracle.FLAG_NONFINITE), (1e-35, oracle.FLAG_RANGE)):
+        cb, sb, fb = oracle.quant_uint4(x[:10], np.float32(bad))
+        assert sb == 0 and not cb.any() and fb == flag
