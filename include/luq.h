@@ -16,6 +16,7 @@
  *   - Packed codes: two 4-bit codes per byte along the contiguous dimension,
  *     element 2j in the low nibble, element 2j+1 in the high nibble.
  *       INT4 : two's-complement integer q in [-7, 7]; value q * scale.
+ *       UINT4: (optional, non-negative tensors) integer q in [0, 15]; value q * scale.
  *       LUQ  : bit 3 = sign, bits 0..2 = c; c = 0 is zero (always nibble 0x0),
  *              c >= 1 is alpha * 2^(c-1).  With the compiled level count
  *              (luq_kmax() = 4) the codes 0..5 occur.
@@ -63,6 +64,10 @@ extern "C" {
                               int32 accumulator could wrap (contractions beyond about 2^18 terms) */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
 #define LUQ_OPT_PAIRS 3    /* 1: products whose operands are both 8-bit planes run on CTA pairs (cta_group::2) */
+#define LUQ_OPT_UNSIGNED_ACTIVATIONS 5 /* 1: the activation codes given to luq_gemm_fwd and luq_gemm_wgrad are
+                              unsigned INT4 (from luq_quant_uint4).  Such an operand is always fetched as bytes:
+                              pass the operand bytes luq_quant_uint4 wrote, or the GEMM expands a plane into the
+                              context workspace (LUQ_ERR_WORKSPACE if it does not fit: 76 MiB). */
 #define LUQ_OPT_LEVELS 4   /* kmax of the gradient quantizers, 1..6 (default luq_kmax() = 4): levels
                               alpha * 2^0 .. alpha * 2^kmax with alpha = max / 2^kmax, codes 0..kmax+1.  The
                               other grids of the paper from the same kernels: kmax = 2 is the FP2 grid of
@@ -109,6 +114,15 @@ int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, 
  * rows*cols must be even.  d_codes: rows*cols/2 bytes.  d_scale: one float. */
 int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
                    const float* d_clip, uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
+
+/* Unsigned INT4 for tensors that cannot be negative (post-ReLU activations).  Appendix
+ * "Quantization formats": scale = Delta / (2^b - 1) with Delta the quantized range - for the
+ * range [0, clip] all sixteen codes lie on one side of zero:
+ *   scale = clip / 15, q = clamp(rint(x * (15 / clip)), 0, 15), ties to even; code nibble = q.
+ * Half the step of luq_quant_int4 on the same range.  Operand bytes (optional): int8 q.
+ * Use with LUQ_OPT_UNSIGNED_ACTIVATIONS = 1 on the context whose GEMMs read the codes. */
+int luq_quant_uint4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
+                    const float* d_clip, uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
 
 /* luq_amax followed by luq_quant_int4 with that maximum as the clip, as ONE kernel (the paper's
  * forward quantization measures the tensor and then quantizes it, Sec. 3; two launches of

@@ -17,11 +17,11 @@ LIB_PATH = os.path.join(_HERE, "libluq_b200.so")
 
 LUQ_F32, LUQ_BF16 = 0, 1
 STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT = 1, 2, 4
-OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS = 1, 2, 3, 4
+OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS, OPT_UNSIGNED_ACTIVATIONS = 1, 2, 3, 4, 5
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_pw2",
+           "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_pw2",
            "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
@@ -48,6 +48,7 @@ def load() -> ctypes.CDLL:
         L.luq_kmax.argtypes = []
         L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
         L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
+        L.luq_quant_uint4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_amax_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_amax_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, u64, ctypes.c_int, vp, vp, vp, vp, vp]
         L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
@@ -141,6 +142,17 @@ class Context:
         _check(load().luq_quant_int4(self.handle, x.data_ptr(), _dtype_code(x), rows, cols, clip.data_ptr(),
                                      codes.data_ptr(), scale.data_ptr(), _opt(operand, x.numel()), _stream()),
                "luq_quant_int4")
+        return codes, scale
+
+    def quant_uint4(self, x: torch.Tensor, clip: torch.Tensor, codes: torch.Tensor | None = None,
+                    scale: torch.Tensor | None = None, operand: torch.Tensor | None = None):
+        """Unsigned INT4 (0..15, scale = clip / 15) for non-negative tensors."""
+        rows, cols = (x.shape[0], x.numel() // max(x.shape[0], 1)) if x.dim() > 1 else (1, x.numel())
+        codes = torch.empty(x.numel() // 2, dtype=torch.uint8, device=x.device) if codes is None else codes
+        scale = torch.empty(1, dtype=torch.float32, device=x.device) if scale is None else scale
+        _check(load().luq_quant_uint4(self.handle, x.data_ptr(), _dtype_code(x), rows, cols, clip.data_ptr(),
+                                      codes.data_ptr(), scale.data_ptr(), _opt(operand, x.numel()), _stream()),
+               "luq_quant_uint4")
         return codes, scale
 
     def amax_quant_int4(self, x: torch.Tensor, amax: torch.Tensor | None = None, codes: torch.Tensor | None = None,

@@ -56,6 +56,7 @@ int luq_create(luq_ctx** out, int device) {
   c->forced_splits = 0;
   c->use_pairs = 0;
   c->kmax = LUQ_KMAX;
+  c->unsigned_act = 0;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;
   c->d_status = nullptr; c->d_scratch = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
@@ -95,6 +96,10 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
       if (value < 0 || value > 1024) return LUQ_ERR_ARG;
       ctx->forced_splits = value;
       return LUQ_OK;
+    case LUQ_OPT_UNSIGNED_ACTIVATIONS:
+      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      ctx->unsigned_act = value;
+      return LUQ_OK;
     case LUQ_OPT_LEVELS:
       if (value < 1 || value > 6) return LUQ_ERR_ARG;
       ctx->kmax = value;
@@ -129,7 +134,21 @@ int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, d_clip, d_codes, n ? d_operand : nullptr, d_scale,
-                                       nullptr, as_stream(stream)));
+                                       nullptr, false, as_stream(stream)));
+}
+
+int luq_quant_uint4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, const float* d_clip,
+                    uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream) {
+  if (!ctx || !d_clip || !d_scale || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  const size_t n = rows * cols;
+  if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
+  if (n & 1u) return LUQ_ERR_ARG;
+  if (n && (!d_x || !d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_codes) || !aligned16(d_operand)) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, d_clip, d_codes, n ? d_operand : nullptr, d_scale,
+                                       nullptr, true, as_stream(stream)));
 }
 
 int luq_amax_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, float* d_amax,
@@ -143,7 +162,7 @@ int luq_amax_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, s
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_int4(ctx, d_x, dtype, n, nullptr, d_codes, n ? d_operand : nullptr, d_scale,
-                                       d_amax, as_stream(stream)));
+                                       d_amax, false, as_stream(stream)));
 }
 
 static int quant_grad_args(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
@@ -251,7 +270,7 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, cons
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   luq_gemm_args a{};
-  a.a_codes = d_a_codes; a.a_kind = 0; a.a_mn = 0; a.n_samples = 1;
+  a.a_codes = d_a_codes; a.a_kind = ctx->unsigned_act ? 2 : 0; a.a_mn = 0; a.n_samples = 1;
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 0;
   a.a_operand = d_a_operand; a.b_operand = d_w_operand;
   a.d_scale_a = d_sa; a.d_scale_b = d_sw; a.d_out = d_z; a.Mo = M; a.No = N; a.Kc = K;
@@ -288,7 +307,7 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
   if (!guard.ok) return LUQ_ERR_CUDA;
   luq_gemm_args a{};
   a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 1; a.n_samples = n_samples;   // G[M x N]: rows are the contraction
-  a.b_codes = d_a_codes; a.b_kind = 0; a.b_mn = 1;                            // A[M x K]: rows are the contraction
+  a.b_codes = d_a_codes; a.b_kind = ctx->unsigned_act ? 2 : 0; a.b_mn = 1;    // A[M x K]: rows are the contraction
   a.a_operand = d_g_operand; a.b_operand = d_a_operand;
   a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.Mo = N; a.No = K; a.Kc = M;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;

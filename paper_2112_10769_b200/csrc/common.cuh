@@ -19,6 +19,7 @@ struct luq_ctx {
   int mma_kind;             // 0 f8f6f4/e4m3, 1 i8, 2 chosen per product
   int forced_splits;        // 0 = automatic
   int use_pairs;            // CTA-pair kernel for products whose operands are both planes
+  int unsigned_act;         // activation codes handed to the forward / update GEMMs are unsigned INT4
   int kmax;                 // LUQ levels alpha * 2^0 .. alpha * 2^kmax (1..6, default LUQ_KMAX)
   int64_t launches;
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved at create
@@ -28,8 +29,10 @@ struct luq_ctx {
 int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, cudaStream_t st);
 // d_operand (may be null): int8 operand bytes, one per element (and per sample), written with the codes
 // d_amax_out (may be null): fused - the kernel reduces the tensor's maximum itself, uses it as clip, writes it there
+// is_unsigned: the grid 0..15 with scale clip/15 instead of -7..7 with clip/7 (not with d_amax_out)
 int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
-                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_amax_out, cudaStream_t st);
+                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_amax_out, bool is_unsigned,
+                          cudaStream_t st);
 
 // flags: bit 0 = power-of-two scale; bit 1 = in-hindsight (d_amax is the running estimate: the tensor's own
 // max|x| goes to d_measured and d_estimate (= d_amax) is replaced by (1 - eta) * measured + eta * estimate)
@@ -42,7 +45,7 @@ int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const fl
 
 // One GEMM  D[Mo x No] = scale * sum_s sum_k opA_s[mo,k] * opB[no,k].
 //   a_mn / b_mn: operand is stored contraction-major (rows = k) instead of
-//   k-contiguous (rows = mo / no).  a_kind / b_kind: 0 INT4 codes, 1 LUQ codes.
+//   k-contiguous (rows = mo / no).  a_kind / b_kind: 0 INT4 codes, 1 LUQ codes, 2 unsigned INT4 codes.
 struct luq_gemm_args {
   const uint8_t* a_codes; int a_kind; int a_mn; int n_samples;
   const uint8_t* b_codes; int b_kind; int b_mn;

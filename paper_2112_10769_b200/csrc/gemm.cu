@@ -731,7 +731,8 @@ __global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restri
 // mantissa); kind 1: two's-complement int8.  Every INT4 integer and every LUQ
 // level 2^0..2^6 is exact in both.
 uint8_t e4m3_of_int(int v) {
-  static const uint8_t mag[9] = {0x00, 0x38, 0x40, 0x44, 0x48, 0x4A, 0x4C, 0x4E, 0x50};
+  static const uint8_t mag[16] = {0x00, 0x38, 0x40, 0x44, 0x48, 0x4A, 0x4C, 0x4E,
+                                  0x50, 0x51, 0x52, 0x53, 0x54, 0x55, 0x56, 0x57};
   const int a = v < 0 ? -v : v;
   return static_cast<uint8_t>(mag[a] | (v < 0 ? 0x80 : 0));
 }
@@ -741,6 +742,8 @@ uint4 make_lut(int mma_kind, int operand_kind) {
     if (operand_kind == 0) {               // INT4 two's complement
       const int v = n < 8 ? n : n - 16;
       t[n] = mma_kind == 0 ? e4m3_of_int(v) : static_cast<uint8_t>(static_cast<int8_t>(v));
+    } else if (operand_kind == 2) {        // unsigned INT4: the nibble is the value, 0..15
+      t[n] = mma_kind == 0 ? e4m3_of_int(n) : static_cast<uint8_t>(n);
     } else {                               // LUQ: sign | c, value +-2^(c-1)
       const int c = n & 7, neg = n >> 3;
       if (c == 0) t[n] = 0;
@@ -867,7 +870,8 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   // Operand type.  "Automatic" is int8: INT4 codes expand to it in three instructions per eight
   // codes, and it is the type of the operand bytes the quantizers can write themselves.
   // Where an int32 accumulator could wrap (a very long contraction) it is e4m3 with fp32 accumulators.
-  const long long worst_product = static_cast<long long>(a.a_kind == 0 ? 7 * 16 : 64) * (a.b_kind == 0 ? 7 * 16 : 64);
+  auto worst = [](int kind) { return kind == 0 ? 7 * 16 : kind == 2 ? 15 : 64; };   // largest |operand byte|
+  const long long worst_product = static_cast<long long>(worst(a.a_kind)) * worst(a.b_kind);
   const bool int32_safe = worst_product * a.Kc * a.n_samples < (1ll << 31);
   if (ctx->mma_kind == 2) ctx->mma_kind = int32_safe ? 1 : 0;
   if (ctx->mma_kind == 1 && !int32_safe) return LUQ_ERR_ARG;
@@ -886,20 +890,27 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   bool b_plane = false, a_plane = false, b_expand = false, a_expand = false;
   const bool long_contraction = total_iters >= 8;
   const uint8_t* b_plane_ptr = nullptr; const uint8_t* a_plane_ptr = nullptr;
-  if (long_contraction && p.tiles_m >= 2) {
+  // Unsigned INT4 codes (kind 2) have no expansion inside the GEMM kernels: such an operand is
+  // always fetched as bytes, the caller's or a plane expanded here.
+  const bool b_must = a.b_kind == 2, a_must = a.a_kind == 2;
+  if (b_must || (long_contraction && p.tiles_m >= 2)) {
     if (b_given) {
       b_plane = true; b_plane_ptr = b_given;
     } else if (packed_ok(b_plane_bytes) && b_plane_bytes <= plane_room) {
       b_plane = b_expand = true; b_plane_ptr = plane_ptr;
       const size_t used = (b_plane_bytes + 1023) & ~static_cast<size_t>(1023);
       plane_ptr += used; plane_room -= used <= plane_room ? used : plane_room;
+    } else if (b_must) {
+      return LUQ_ERR_WORKSPACE;
     }
   }
-  if (long_contraction && p.tiles_n >= 2) {
+  if (a_must || (long_contraction && p.tiles_n >= 2)) {
     if (a_given) {
       a_plane = true; a_plane_ptr = a_given;
     } else if (packed_ok(a_plane_bytes) && a_plane_bytes <= plane_room) {
       a_plane = a_expand = true; a_plane_ptr = plane_ptr;
+    } else if (a_must) {
+      return LUQ_ERR_WORKSPACE;
     }
   }
   p.lut_a = make_lut(ctx->mma_kind, a.a_kind);
@@ -915,15 +926,15 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   int rc = 0;
   if (b_expand) {
     uint8_t* dst = const_cast<uint8_t*>(b_plane_ptr);   // workspace memory
-    rc = ctx->mma_kind ? launch_expand<1>(a.b_kind == 1, a.b_codes, dst, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st)
-                       : launch_expand<0>(a.b_kind == 1, a.b_codes, dst, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st);
+    rc = ctx->mma_kind ? launch_expand<1>(a.b_kind != 0, a.b_codes, dst, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st)
+                       : launch_expand<0>(a.b_kind != 0, a.b_codes, dst, b_plane_bytes / 2, p.lut_b, ctx->sm_count, st);
     if (rc != 0) return rc;
     ctx->launches += 1;
   }
   if (a_expand) {
     uint8_t* dst = const_cast<uint8_t*>(a_plane_ptr);   // workspace memory
-    rc = ctx->mma_kind ? launch_expand<1>(a.a_kind == 1, a.a_codes, dst, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st)
-                       : launch_expand<0>(a.a_kind == 1, a.a_codes, dst, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st);
+    rc = ctx->mma_kind ? launch_expand<1>(a.a_kind != 0, a.a_codes, dst, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st)
+                       : launch_expand<0>(a.a_kind != 0, a.a_codes, dst, a_plane_bytes / 2, p.lut_a, ctx->sm_count, st);
     if (rc != 0) return rc;
     ctx->launches += 1;
   }
@@ -968,7 +979,11 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
 
   const int grid = static_cast<int>(units < ctx->sm_count ? units : ctx->sm_count);
   const int sel = (ctx->mma_kind ? 4 : 0) | (a.a_mn ? 2 : 0) | (a.b_mn ? 1 : 0);
-  if (a.b_kind != 0 || (a.a_kind == 1) != (sel & 3 ? true : false)) return LUQ_ERR_UNSUPPORTED;
+  // the kernels expand signed INT4 codes in B, and in A signed INT4 (forward) or LUQ codes (backward,
+  // update); any other kind of operand must have arrived as bytes
+  if ((a.b_kind != 0 && !b_plane) || (!a_plane && (a.a_kind == 1) != (sel & 3 ? true : false)) ||
+      (a.a_kind == 2 && !a_plane))
+    return LUQ_ERR_UNSUPPORTED;
   switch (sel) {
     case 0: rc = launch_planes<0, false, false, false>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
     case 1: rc = launch_planes<0, false, true, true>(a_plane, b_plane, ta, tb, to, p, grid, st); break;
@@ -1088,6 +1103,7 @@ extern "C" int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_al
   local.forced_splits = 0;
   local.use_pairs = 0;
   local.kmax = LUQ_KMAX;
+  local.unsigned_act = 0;
   local.launches = 0;
   local.encode_tiled = s->encode_tiled;
 

@@ -267,9 +267,18 @@ __device__ __forceinline__ uint32_t int4_code(float x, float inv) {
   return (y == y) ? code : 0u;        // NaN element -> 0
 }
 
+// the same for the unsigned grid 0..15 (the clamp keeps negative inputs at 0)
+__device__ __forceinline__ uint32_t uint4_code(float x, float inv) {
+  const float y = x * inv;
+  const float c = fminf(fmaxf(y, 0.0f), 15.0f);
+  const uint32_t code = __float_as_uint(c + 12582912.0f) & 0xFu;
+  return (y == y) ? code : 0u;
+}
+
 // PLANE: the tensor-core operand bytes (int8, 16 * q: the code nibble in the high half of the
 // byte) are written next to the packed codes, one byte per element in element order.
-template <bool BF16, bool PLANE>
+// UNSIGNED: the grid 0..15 with scale clip / 15 (non-negative tensors); operand byte = q.
+template <bool BF16, bool PLANE, bool UNSIGNED>
 __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __restrict__ x, size_t n,
                                                               const float* d_clip,
                                                               uint8_t* __restrict__ codes,
@@ -291,8 +300,11 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
     clip = *d_clip;
   }
   const bool ok = scale_usable(clip, first ? status : nullptr);
-  const float inv = ok ? 7.0f / clip : 0.0f;
-  if (first) *d_scale = ok ? clip / 7.0f : 0.0f;
+  constexpr float kTop = UNSIGNED ? 15.0f : 7.0f;
+  constexpr int kByteShift = UNSIGNED ? 0 : 4;
+  const float inv = ok ? kTop / clip : 0.0f;
+  if (first) *d_scale = ok ? clip / kTop : 0.0f;
+  auto code_of = [&](float v) { return UNSIGNED ? uint4_code(v, inv) : int4_code(v, inv); };
 
   const size_t items = n / kElems;
   const uint4* p = reinterpret_cast<const uint4*>(x);
@@ -303,9 +315,9 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
     uint32_t bytes[kElems / 4] = {};
 #pragma unroll
     for (int j = 0; j < kElems; ++j) {
-      const uint32_t code = ok ? int4_code(v[j], inv) : 0u;
+      const uint32_t code = ok ? code_of(v[j]) : 0u;
       word |= code << (4 * j);
-      if constexpr (PLANE) bytes[j / 4] |= code << (8 * (j % 4) + 4);
+      if constexpr (PLANE) bytes[j / 4] |= code << (8 * (j % 4) + kByteShift);
     }
     Item<BF16>::store(codes, item, word, true);
     if constexpr (PLANE) Item<BF16>::store_bytes(operand, item, bytes, true);
@@ -325,12 +337,12 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
     for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) emit(i, __ldg(p + i));
   if (first) {  // tail: fewer elements than one piece, two per byte
     for (size_t e = items * kElems; e < n; e += 2) {
-      const uint32_t lo = ok ? int4_code(Item<BF16>::load1(x, e), inv) : 0u;
-      const uint32_t hi = (ok && e + 1 < n) ? int4_code(Item<BF16>::load1(x, e + 1), inv) : 0u;
+      const uint32_t lo = ok ? code_of(Item<BF16>::load1(x, e)) : 0u;
+      const uint32_t hi = (ok && e + 1 < n) ? code_of(Item<BF16>::load1(x, e + 1)) : 0u;
       codes[e >> 1] = static_cast<uint8_t>(lo | (hi << 4));
       if constexpr (PLANE) {
-        operand[e] = static_cast<int8_t>(lo << 4);
-        if (e + 1 < n) operand[e + 1] = static_cast<int8_t>(hi << 4);
+        operand[e] = static_cast<int8_t>(lo << kByteShift);
+        if (e + 1 < n) operand[e + 1] = static_cast<int8_t>(hi << kByteShift);
       }
     }
   }
@@ -679,25 +691,33 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
 }
 
 namespace {
-template <bool BF16, bool PLANE>
+template <bool BF16, bool PLANE, bool UNSIGNED>
 int launch_int4(luq_ctx* ctx, const void* d_x, size_t n, const float* d_clip, uint8_t* d_codes, int8_t* d_operand,
                 float* d_scale, float* d_amax_out, cudaStream_t st) {
-  const int grid = grid_for(ctx, quant_int4_kernel<BF16, PLANE>, n / Item<BF16>::kElems / kTileItems + 1);
+  const int grid = grid_for(ctx, quant_int4_kernel<BF16, PLANE, UNSIGNED>, n / Item<BF16>::kElems / kTileItems + 1);
   const int mode = d_amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_NORMAL;   // fused: grid barrier inside
-  return static_cast<int>(luq_launch_kernel(quant_int4_kernel<BF16, PLANE>, grid, kThreads, 0, st, mode, 1, d_x, n, d_clip,
-                                            d_codes, d_operand, d_scale, d_amax_out, ctx->d_scratch, ctx->d_status));
+  return static_cast<int>(luq_launch_kernel(quant_int4_kernel<BF16, PLANE, UNSIGNED>, grid, kThreads, 0, st, mode, 1, d_x, n,
+                                            d_clip, d_codes, d_operand, d_scale, d_amax_out, ctx->d_scratch,
+                                            ctx->d_status));
+}
+template <bool BF16, bool PLANE>
+int launch_int4_grid(bool is_unsigned, luq_ctx* ctx, const void* d_x, size_t n, const float* d_clip, uint8_t* d_codes,
+                     int8_t* d_operand, float* d_scale, float* d_amax_out, cudaStream_t st) {
+  return is_unsigned ? launch_int4<BF16, PLANE, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st)
+                     : launch_int4<BF16, PLANE, false>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st);
 }
 }  // namespace
 
 // d_amax_out non-null: fused - the clip is the tensor's maximum, reduced by the same kernel and written there
 int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
-                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_amax_out, cudaStream_t st) {
+                          uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_amax_out, bool is_unsigned,
+                          cudaStream_t st) {
   const bool bf = dtype == LUQ_BF16;
   int rc;
-  if (d_operand) rc = bf ? launch_int4<true, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st)
-                         : launch_int4<false, true>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st);
-  else rc = bf ? launch_int4<true, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, d_amax_out, st)
-               : launch_int4<false, false>(ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, d_amax_out, st);
+  if (d_operand) rc = bf ? launch_int4_grid<true, true>(is_unsigned, ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st)
+                         : launch_int4_grid<false, true>(is_unsigned, ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st);
+  else rc = bf ? launch_int4_grid<true, false>(is_unsigned, ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, d_amax_out, st)
+               : launch_int4_grid<false, false>(is_unsigned, ctx, d_x, n, d_clip, d_codes, nullptr, d_scale, d_amax_out, st);
   ctx->launches += 1;
   return rc;
 }
