@@ -1,0 +1,90 @@
+"""A linear layer trained with the 4-bit path, as a ``torch.autograd.Function``.
+
+Argument marshalling only: every step runs in the library's kernels (Sec. 3, Eqs. Forward /
+Backward / Update; Sec. 4 LUQ; Sec. 5.1 SMP).
+
+    forward    Z  = Q_INT(A) . Q_INT(W)^T
+    backward   dA = mean_s Q_FP,s(G) . Q_INT(W)
+    update     dW = mean_s Q_FP,s(G)^T . Q_INT(A)
+
+``A`` is ``[M, K]`` (leading dimensions are flattened), ``W`` is ``[N, K]`` as in ``torch.nn.Linear``.
+The INT4 codes of the forward pass are kept for the backward pass (the paper's update GEMM re-uses the
+quantized activations), together with the 8-bit operand bytes of W and G that the GEMMs re-read.
+Shapes must satisfy the GEMMs' divisibility rules (K and N multiples of 32).
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding
+
+_contexts: dict[int, binding.Context] = {}
+
+
+def context(device: torch.device) -> binding.Context:
+    """One library context per device, created on first use."""
+    index = device.index if device.index is not None else torch.cuda.current_device()
+    if index not in _contexts:
+        _contexts[index] = binding.Context(index)
+    return _contexts[index]
+
+
+class LuqLinearFunction(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int):
+        lib = context(a.device)
+        a2 = a.reshape(-1, a.shape[-1]).contiguous()
+        w2 = w.contiguous()
+        M, K = a2.shape
+        N = w2.shape[0]
+        w_bytes = torch.empty(N * K, dtype=torch.int8, device=a.device)
+        ca, sa = lib.quant_int4(a2, lib.amax(a2))
+        cw, sw = lib.quant_int4(w2, lib.amax(w2), operand=w_bytes)
+        z = lib.gemm_fwd(ca, sa, cw, sw, M, N, K, w_operand=w_bytes)
+        ctx.save_for_backward(ca, sa, cw, sw, w_bytes)
+        ctx.dims = (M, N, K, a.shape, a.dtype, w.dtype)
+        ctx.seed, ctx.n_samples = int(seed), int(n_samples)
+        return z.reshape(*a.shape[:-1], N).to(a.dtype)
+
+    @staticmethod
+    def backward(ctx, grad_out: torch.Tensor):
+        ca, sa, cw, sw, w_bytes = ctx.saved_tensors
+        M, N, K, a_shape, a_dtype, w_dtype = ctx.dims
+        ns = ctx.n_samples
+        lib = context(grad_out.device)
+        g2 = grad_out.reshape(M, N).contiguous()
+        g_bytes = torch.empty(ns * M * N, dtype=torch.int8, device=g2.device)
+        cg, alpha = lib.quant_grad(g2, lib.amax(g2), ctx.seed, ns, operand=g_bytes)
+        da = dw = None
+        if ctx.needs_input_grad[0]:
+            da = lib.gemm_bwd(cg, alpha, ns, cw, sw, M, N, K, g_operand=g_bytes, w_operand=w_bytes)
+            da = da.reshape(a_shape).to(a_dtype)
+        if ctx.needs_input_grad[1]:
+            dw = lib.gemm_wgrad(cg, alpha, ns, ca, sa, M, N, K, g_operand=g_bytes).to(w_dtype)
+        return da, dw, None, None
+
+
+def luq_linear(a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int = 1) -> torch.Tensor:
+    """``a @ w.T`` with INT4 operands forward and LUQ-FP4 gradients backward.  ``seed`` keys the
+    stochastic rounding of this call's backward pass: give every layer and step its own."""
+    return LuqLinearFunction.apply(a, w, seed, n_samples)
+
+
+class LuqLinear(torch.nn.Module):
+    """``torch.nn.Linear`` without bias whose three GEMMs run on the 4-bit path.  The seed of the
+    gradient quantizer advances with every forward call."""
+
+    def __init__(self, in_features: int, out_features: int, n_samples: int = 1, seed: int = 0,
+                 device=None, dtype=torch.float32):
+        super().__init__()
+        w = torch.empty(out_features, in_features, device=device, dtype=dtype)
+        torch.nn.init.kaiming_uniform_(w, a=5 ** 0.5)
+        self.weight = torch.nn.Parameter(w)
+        self.n_samples = n_samples
+        self.base_seed = seed
+        self.calls = 0
+
+    def forward(self, a: torch.Tensor) -> torch.Tensor:
+        seed = self.base_seed + self.calls * self.n_samples     # sample s of a call uses seed + s
+        self.calls += 1
+        return luq_linear(a, self.weight, seed, self.n_samples)

@@ -1,0 +1,58 @@
+"""The autograd wrapper is argument marshalling: its outputs and gradients must be exactly what the
+C-ABI calls give, and those are checked against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2112_10769_b200 import autograd, inputs
+
+from test_gpu_parity import assert_gemm_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_function_matches_the_oracle(dtype):
+    M, K, N, ns, seed = 384, 256, 288, 2, 17
+    A, W, G = inputs.small_layer(M, K, N, 4)
+    a = torch.from_numpy(A).cuda().to(dtype).requires_grad_(True)
+    w = torch.from_numpy(W).cuda().to(dtype).requires_grad_(True)
+    g = torch.from_numpy(G).cuda().to(dtype)
+    z = autograd.luq_linear(a, w, seed, ns)
+    z.backward(g)
+    # the oracle on the same (possibly bf16-rounded) inputs
+    to_np = (lambda t: t.detach().float().cpu().numpy()) if dtype == torch.float32 else \
+        (lambda t: t.detach().view(torch.int16).cpu().numpy().view(np.uint16))
+    An, Wn, Gn = to_np(a), to_np(w), to_np(g)
+    oa, sa, _ = oracle.quant_int4(An, oracle.amax(An)[0])
+    ow, sw, _ = oracle.quant_int4(Wn, oracle.amax(Wn)[0])
+    og, al, _ = oracle.quant_luq(Gn, oracle.amax(Gn)[0], seed, ns)
+    refs = (oracle.gemm_fwd(oa, sa, ow, sw, M, N, K), oracle.gemm_bwd(og, al, ns, ow, sw, M, N, K),
+            oracle.gemm_wgrad(og, al, ns, oa, sa, M, N, K))
+    for got, ref in zip((z, a.grad, w.grad), refs):
+        assert got.dtype == dtype
+        got = got.detach().float().cpu().numpy().astype(np.float64)
+        if dtype == torch.float32:
+            assert_gemm_close(got, ref)
+        else:   # the result is rounded once more, to bf16
+            assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-12 * np.abs(ref).max()).all()
+
+
+def test_module_trains_a_small_regression():
+    torch.manual_seed(0)
+    K, N, M = 128, 64, 512
+    target = torch.randn(N, K, device="cuda") / K ** 0.5
+    layer = autograd.LuqLinear(K, N, n_samples=2, seed=100, device="cuda")
+    opt = torch.optim.SGD(layer.parameters(), lr=0.2)
+    losses = []
+    for _ in range(60):
+        x = torch.randn(M, K, device="cuda")
+        loss = (layer(x) - x @ target.T).pow(2).sum(1).mean()     # gradient 2 (W - target) for white inputs
+        opt.zero_grad()
+        loss.backward()
+        opt.step()
+        losses.append(loss.item())
+    assert layer.calls == 60
+    assert losses[-1] < 0.2 * losses[0]          # the 4-bit forward noise sets the floor; no divergence
+    assert autograd.context(torch.device("cuda", 0)).status() == 0
