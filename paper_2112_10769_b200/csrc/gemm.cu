@@ -10,8 +10,9 @@
 //   warp 0       TMA producer for packed slabs (128 rows x 64 bytes) -> packed ring
 //   warp 6       TMA producer for operand planes (128 rows x 128 bytes, already
 //                8-bit, 128-byte swizzle) -> straight into the operand ring
-//   warps 7-22   converters: packed nibbles -> 8-bit operands, written in the
-//                128-byte swizzled layout the tensor core reads
+//   warps 7-..   converters (8 or 16 warps, by how many operands arrive packed): packed
+//                nibbles -> 8-bit operands, written in the 128-byte swizzled layout the
+//                tensor core reads
 //   warp 1       one thread issues tcgen05.mma (128 x 256 x 32 per instruction),
 //                accumulators live in tensor memory, two buffers of 256 columns
 //   warps 2-5    epilogue: tcgen05.ld -> scale -> swizzled staging -> TMA store
@@ -21,9 +22,14 @@
 // Shared-memory bandwidth bounds the in-kernel expansion (TMA write + converter
 // read + converter write + tensor-core read of every operand byte).  An operand
 // that many tiles re-read (the weights; the gradient in the backward and update
-// products) is therefore expanded once by a small kernel into an 8-bit "plane"
-// in the context workspace and fetched by TMA in its final layout; only operands
+// products) is therefore fetched as bytes, by TMA in its final layout: the bytes
+// the quantizer wrote beside the codes if the caller passes them, else an 8-bit
+// "plane" that a small kernel expands into the context workspace.  Only operands
 // used by a single row or column of tiles are expanded inside the GEMM.
+//
+// A second kernel (luq_gemm_pair_kernel, option LUQ_OPT_PAIRS) runs products
+// whose operands both arrive as bytes on CTA pairs: tcgen05 cta_group::2, one
+// 256-row tile per pair, each CTA fetching half of B.
 //
 // Operand bytes.  kind::f8f6f4: e4m3 through a 16-entry byte table (PRMT).
 // kind::i8: LUQ levels +-2^(c-1) through the table; INT4 integers without a
@@ -958,7 +964,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   if (bad) return LUQ_ERR_CUDA;
 
   // CTA pairs when both operands are planes (no expansion inside the kernel) and the contraction
-  // is not split: option LUQ_OPT_PAIRS (default on)
+  // is not split: option LUQ_OPT_PAIRS (off unless set)
   if (ctx->use_pairs && a_plane && b_plane && p.splits == 1 && p.tiles_m >= 2) {
     const long long pair_tiles = static_cast<long long>((p.tiles_m + 1) / 2) * p.tiles_n;
     const int max_pairs = ctx->sm_count / 2;

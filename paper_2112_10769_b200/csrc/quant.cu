@@ -1,12 +1,17 @@
 // Memory-bound kernels of the path: tensor max, INT4 round-to-nearest
-// quantize-and-pack, LUQ stochastic quantize-and-pack (Philox, n samples).
+// quantize-and-pack (signed, and unsigned for non-negative tensors), LUQ stochastic
+// quantize-and-pack (Philox, n samples) with its variants: power-of-two scale,
+// in-hindsight maximum, other level counts, deterministic nearest power.
 //
-// All three stream the input once.  The unit of work is one 16-byte load
+// All stream the input once.  The unit of work is one 16-byte load
 // (4 fp32 or 8 bf16 elements); consecutive lanes take consecutive 16-byte
 // pieces, so every load instruction of a warp covers 512 contiguous bytes and
 // the packed codes leave as contiguous 64- or 128-byte warp stores.  Grids are
 // sized to the number of CTAs the GPU holds at once (SM count x occupancy) and
 // walk the tensor in contiguous 16 KB tiles, several loads in flight per thread.
+// Every quantizer can also write the codes' 8-bit tensor-core form ("operand
+// bytes") in the same pass, and can be launched "fused": it then reduces the
+// tensor's maximum itself (first phase, grid barrier) instead of reading it.
 //
 // Compile this file without FMA contraction and with IEEE division: code
 // decisions must be bit-identical to a scalar IEEE implementation.
