@@ -68,6 +68,10 @@ extern "C" {
                               unsigned INT4 (from luq_quant_uint4).  Such an operand is always fetched as bytes:
                               pass the operand bytes luq_quant_uint4 wrote, or the GEMM expands a plane into the
                               context workspace (LUQ_ERR_WORKSPACE if it does not fit: 76 MiB). */
+#define LUQ_OPT_OUTPUT_BF16 6 /* 1: luq_gemm_fwd / bwd / wgrad write bf16 outputs (the fp32 result rounded to
+                              nearest even) instead of fp32: half the output traffic, which is what bounds the
+                              backward product of a wide layer.  The output's row length must then be a
+                              multiple of 8 elements.  Not available in luq_gemm_wgrad_static. */
 #define LUQ_OPT_LEVELS 4   /* kmax of the gradient quantizers, 1..6 (default luq_kmax() = 4): levels
                               alpha * 2^0 .. alpha * 2^kmax with alpha = max / 2^kmax, codes 0..kmax+1.  The
                               other grids of the paper from the same kernels: kmax = 2 is the FP2 grid of
@@ -192,12 +196,15 @@ int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t ro
  * equal the IEEE binary32 quotient wherever that quotient is a normal number. */
 int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream);
 
-/* Forward GEMM (Eq. Forward; scale factoring of Appendix A.1):
+/* The three GEMMs write fp32 outputs (void* d_z / d_da / d_dw point to floats) unless
+ * LUQ_OPT_OUTPUT_BF16 is set on the context, in which case they point to bf16 values.
+ *
+ * Forward GEMM (Eq. Forward; scale factoring of Appendix A.1):
  *   Z[m,n] = (sa*sw) * sum_k qA[m,k] * qW[n,k]        fp32 accumulate, fp32 out.
  * a_codes [M x K/2], w_codes [N x K/2].  K must be a multiple of 32. */
 int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
                  const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
-                 float* d_z, int64_t M, int64_t N, int64_t K, void* stream);
+                 void* d_z, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Backward GEMM (Eq. Backward), SMP average fused (Sec. 5.1):
  *   dA[m,k] = (alpha*sw/n_samples) * sum_s sum_n qG_s[m,n] * qW[n,k].
@@ -205,7 +212,7 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, cons
  * N and K must be multiples of 32. */
 int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
                  const int8_t* d_g_operand, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
-                 float* d_da, int64_t M, int64_t N, int64_t K, void* stream);
+                 void* d_da, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Update GEMM (Eq. Update), SMP average fused (Sec. 5.1):
  *   dW[n,k] = (alpha*sa/n_samples) * sum_s sum_m qG_s[m,n] * qA[m,k].
@@ -214,7 +221,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
  * the output has few tiles (contraction over M is split across CTAs). */
 int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
                    const int8_t* d_g_operand, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
-                   float* d_dw, int64_t M, int64_t N, int64_t K, void* stream);
+                   void* d_dw, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Update GEMM without any allocation.  (The paper has no counterpart; this entry
  * point exists for the sake of callers.)

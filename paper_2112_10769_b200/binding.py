@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libluq_b200.so")
 
 LUQ_F32, LUQ_BF16 = 0, 1
 STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT = 1, 2, 4
-OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS, OPT_UNSIGNED_ACTIVATIONS = 1, 2, 3, 4, 5
+OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS, OPT_UNSIGNED_ACTIVATIONS, OPT_OUTPUT_BF16 = 1, 2, 3, 4, 5, 6
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
@@ -120,6 +120,17 @@ class Context:
 
     def set_option(self, option: int, value: int):
         _check(load().luq_set_option(self.handle, option, value), "luq_set_option")
+        if option == OPT_OUTPUT_BF16:
+            self.out_dtype = torch.bfloat16 if value else torch.float32
+
+    def _out(self, out, rows: int, cols: int, device):
+        """Output tensor of a GEMM: the caller's (type checked) or a new one of the context's output type."""
+        dtype = getattr(self, "out_dtype", torch.float32)
+        if out is None:
+            return torch.empty((rows, cols), dtype=dtype, device=device)
+        if out.dtype != dtype or out.numel() < rows * cols or not out.is_contiguous():
+            raise TypeError(f"GEMM output: contiguous {dtype} tensor of {rows} x {cols} expected")
+        return out
 
     @property
     def launches(self) -> int:
@@ -243,7 +254,7 @@ class Context:
 
     def gemm_fwd(self, a_codes, sa, w_codes, sw, M: int, N: int, K: int, out: torch.Tensor | None = None,
                  a_operand: torch.Tensor | None = None, w_operand: torch.Tensor | None = None):
-        out = torch.empty((M, N), dtype=torch.float32, device=a_codes.device) if out is None else out
+        out = self._out(out, M, N, a_codes.device)
         _check(load().luq_gemm_fwd(self.handle, a_codes.data_ptr(), sa.data_ptr(), _opt(a_operand, M * K),
                                    w_codes.data_ptr(), sw.data_ptr(), _opt(w_operand, N * K), out.data_ptr(),
                                    M, N, K, _stream()), "luq_gemm_fwd")
@@ -252,7 +263,7 @@ class Context:
     def gemm_bwd(self, g_codes, alpha, n_samples: int, w_codes, sw, M: int, N: int, K: int,
                  out: torch.Tensor | None = None, g_operand: torch.Tensor | None = None,
                  w_operand: torch.Tensor | None = None):
-        out = torch.empty((M, K), dtype=torch.float32, device=g_codes.device) if out is None else out
+        out = self._out(out, M, K, g_codes.device)
         _check(load().luq_gemm_bwd(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
                                    _opt(g_operand, n_samples * M * N), w_codes.data_ptr(), sw.data_ptr(),
                                    _opt(w_operand, N * K), out.data_ptr(), M, N, K, _stream()), "luq_gemm_bwd")
@@ -261,7 +272,7 @@ class Context:
     def gemm_wgrad(self, g_codes, alpha, n_samples: int, a_codes, sa, M: int, N: int, K: int,
                    out: torch.Tensor | None = None, g_operand: torch.Tensor | None = None,
                    a_operand: torch.Tensor | None = None):
-        out = torch.empty((N, K), dtype=torch.float32, device=g_codes.device) if out is None else out
+        out = self._out(out, N, K, g_codes.device)
         _check(load().luq_gemm_wgrad(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
                                      _opt(g_operand, n_samples * M * N), a_codes.data_ptr(), sa.data_ptr(),
                                      _opt(a_operand, M * K), out.data_ptr(), M, N, K, _stream()), "luq_gemm_wgrad")

@@ -57,6 +57,7 @@ int luq_create(luq_ctx** out, int device) {
   c->use_pairs = 0;
   c->kmax = LUQ_KMAX;
   c->unsigned_act = 0;
+  c->out_bf16 = 0;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;
   c->d_status = nullptr; c->d_scratch = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
@@ -95,6 +96,10 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
     case LUQ_OPT_SPLITS:
       if (value < 0 || value > 1024) return LUQ_ERR_ARG;
       ctx->forced_splits = value;
+      return LUQ_OK;
+    case LUQ_OPT_OUTPUT_BF16:
+      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      ctx->out_bf16 = value;
       return LUQ_OK;
     case LUQ_OPT_UNSIGNED_ACTIVATIONS:
       if (value != 0 && value != 1) return LUQ_ERR_ARG;
@@ -251,7 +256,7 @@ int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_
 }
 
 static int gemm_common(luq_ctx* ctx, const uint8_t* x, const float* sx, const int8_t* xo, const uint8_t* y,
-                       const float* sy, const int8_t* yo, float* out, int64_t M, int64_t N, int64_t K,
+                       const float* sy, const int8_t* yo, const void* out, int64_t M, int64_t N, int64_t K,
                        int n_samples) {
   if (!ctx || !sx || !sy) return LUQ_ERR_ARG;
   if (M < 0 || N < 0 || K < 0 || M > (1ll << 31) || N > (1ll << 31) || K > (1ll << 31)) return LUQ_ERR_ARG;
@@ -262,7 +267,7 @@ static int gemm_common(luq_ctx* ctx, const uint8_t* x, const float* sx, const in
 }
 
 int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
-                 const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand, float* d_z, int64_t M,
+                 const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand, void* d_z, int64_t M,
                  int64_t N, int64_t K, void* stream) {
   int rc = gemm_common(ctx, d_a_codes, d_sa, d_a_operand, d_w_codes, d_sw, d_w_operand, d_z, M, N, K, 1);
   if (rc) return rc;
@@ -273,7 +278,7 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, cons
   a.a_codes = d_a_codes; a.a_kind = ctx->unsigned_act ? 2 : 0; a.a_mn = 0; a.n_samples = 1;
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 0;
   a.a_operand = d_a_operand; a.b_operand = d_w_operand;
-  a.d_scale_a = d_sa; a.d_scale_b = d_sw; a.d_out = d_z; a.Mo = M; a.No = N; a.Kc = K;
+  a.d_scale_a = d_sa; a.d_scale_b = d_sw; a.d_out = d_z; a.out_bf16 = ctx->out_bf16; a.Mo = M; a.No = N; a.Kc = K;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;
   return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
@@ -281,7 +286,7 @@ int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, cons
 
 int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
                  const int8_t* d_g_operand, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
-                 float* d_da, int64_t M, int64_t N, int64_t K, void* stream) {
+                 void* d_da, int64_t M, int64_t N, int64_t K, void* stream) {
   int rc = gemm_common(ctx, d_g_codes, d_alpha, d_g_operand, d_w_codes, d_sw, d_w_operand, d_da, M, N, K, n_samples);
   if (rc) return rc;
   if (N % 32 || K % 32) return LUQ_ERR_ARG;
@@ -291,7 +296,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
   a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 0; a.n_samples = n_samples;   // G[M x N]: contraction n contiguous
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 1;                            // W[N x K]: rows are the contraction
   a.a_operand = d_g_operand; a.b_operand = d_w_operand;
-  a.d_scale_a = d_alpha; a.d_scale_b = d_sw; a.d_out = d_da; a.Mo = M; a.No = K; a.Kc = N;
+  a.d_scale_a = d_alpha; a.d_scale_b = d_sw; a.d_out = d_da; a.out_bf16 = ctx->out_bf16; a.Mo = M; a.No = K; a.Kc = N;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;
   return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));
@@ -299,7 +304,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
 
 int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
                    const int8_t* d_g_operand, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
-                   float* d_dw, int64_t M, int64_t N, int64_t K, void* stream) {
+                   void* d_dw, int64_t M, int64_t N, int64_t K, void* stream) {
   int rc = gemm_common(ctx, d_g_codes, d_alpha, d_g_operand, d_a_codes, d_sa, d_a_operand, d_dw, M, N, K, n_samples);
   if (rc) return rc;
   if (N % 32 || K % 32) return LUQ_ERR_ARG;
@@ -309,7 +314,7 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
   a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 1; a.n_samples = n_samples;   // G[M x N]: rows are the contraction
   a.b_codes = d_a_codes; a.b_kind = ctx->unsigned_act ? 2 : 0; a.b_mn = 1;    // A[M x K]: rows are the contraction
   a.a_operand = d_g_operand; a.b_operand = d_a_operand;
-  a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.Mo = N; a.No = K; a.Kc = M;
+  a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.out_bf16 = ctx->out_bf16; a.Mo = N; a.No = K; a.Kc = M;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;
   return cuda_rc(luq_launch_gemm(ctx, a, as_stream(stream)));

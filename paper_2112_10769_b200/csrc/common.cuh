@@ -19,6 +19,7 @@ struct luq_ctx {
   int mma_kind;             // 0 f8f6f4/e4m3, 1 i8, 2 chosen per product
   int forced_splits;        // 0 = automatic
   int use_pairs;            // CTA-pair kernel for products whose operands are both planes
+  int out_bf16;             // the GEMMs write bf16 outputs
   int unsigned_act;         // activation codes handed to the forward / update GEMMs are unsigned INT4
   int kmax;                 // LUQ levels alpha * 2^0 .. alpha * 2^kmax (1..6, default LUQ_KMAX)
   int64_t launches;
@@ -51,7 +52,8 @@ struct luq_gemm_args {
   const uint8_t* b_codes; int b_kind; int b_mn;
   const int8_t* a_operand; const int8_t* b_operand;   // int8 operand bytes from the quantizer, or null
   const float* d_scale_a; const float* d_scale_b;
-  float* d_out; int64_t Mo, No, Kc;
+  void* d_out; int out_bf16;   // fp32 [Mo x No], or bf16 when out_bf16
+  int64_t Mo, No, Kc;
   float* d_workspace; size_t workspace_bytes;   // split partial tiles (caller-chosen memory)
   int allow_split;
 };

@@ -104,6 +104,7 @@ struct GemmParams {
   long long Mo, No, Kc;
   int n_samples;
   int tiles_m, tiles_n;
+  int out_bf16;          // the output tensor is bf16 (round to nearest even of the fp32 result), not fp32
   int num_kb;          // contraction blocks per sample plane
   int splits;          // contraction splits per tile
   int iters_per_split;
@@ -129,6 +130,12 @@ __device__ __forceinline__ void expand8_int4_x16(uint32_t w, uint32_t& lo, uint3
   const uint32_t odd = w & 0xF0F0F0F0u;
   if constexpr (PERMUTED) { lo = even; hi = odd; }
   else { lo = __byte_perm(even, odd, 0x5140); hi = __byte_perm(even, odd, 0x7362); }
+}
+// two fp32 values -> two bf16 (round to nearest even), the first in the low half
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
 // 32 packed codes (16 bytes) -> 32 operand bytes in element order
 template <int KIND, bool LUQ_CODES, bool PERMUTED>
@@ -366,6 +373,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const uint32_t stage0 = base + C::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
     uint8_t* const stage0_gen = gen + C::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
     const int sw = lane & 7;
+    const bool out_bf16 = p.out_bf16 && p.splits == 1;   // partial tiles of a split stay fp32
     uint32_t tile_it = 0, box_it = 0;
     bool ok = true;
     for (int u = blockIdx.x; ok && u < units; u += gridDim.x, ++tile_it) {
@@ -389,19 +397,29 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           ++box_it;
           if (lane == 0) bulk_wait_read<1>();          // the store that last read this box is done
           __syncwarp();
-          uint8_t* const rowp = stage0_gen + b * kStageBox + lane * 128;
+          auto value = [&](int i) {
+            const float acc = KIND == 0 ? __uint_as_float(r[i]) : static_cast<float>(static_cast<int>(r[i]));
+            return acc * scale;
+          };
+          if (out_bf16) {
+            // 32 columns of bf16 = 64 bytes per row: four 16-byte pieces, 64-byte swizzle (piece ^ row/2)
+            uint8_t* const rowp = stage0_gen + b * kStageBox + lane * 64;
+            const int sw64 = (lane >> 1) & 3;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            float4 v;
-            if constexpr (KIND == 0) {
-              v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                              __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-            } else {
-              v = make_float4(static_cast<float>(static_cast<int>(r[4 * j])), static_cast<float>(static_cast<int>(r[4 * j + 1])),
-                              static_cast<float>(static_cast<int>(r[4 * j + 2])), static_cast<float>(static_cast<int>(r[4 * j + 3])));
+            for (int j = 0; j < 4; ++j) {
+              uint4 v;
+              v.x = pack_bf16x2(value(8 * j), value(8 * j + 1));
+              v.y = pack_bf16x2(value(8 * j + 2), value(8 * j + 3));
+              v.z = pack_bf16x2(value(8 * j + 4), value(8 * j + 5));
+              v.w = pack_bf16x2(value(8 * j + 6), value(8 * j + 7));
+              *reinterpret_cast<uint4*>(rowp + ((j ^ sw64) << 4)) = v;
             }
-            v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
-            *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
+          } else {
+            uint8_t* const rowp = stage0_gen + b * kStageBox + lane * 128;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) =
+                  make_float4(value(4 * j), value(4 * j + 1), value(4 * j + 2), value(4 * j + 3));
           }
           fence_proxy_async();
           __syncwarp();
@@ -706,11 +724,11 @@ luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 
 // Sums the partial tiles of a split contraction in a fixed order, applies the
 // scales and writes the output.  One thread per float4 of a tile.
-__global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restrict__ ws, float* __restrict__ out,
+__global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restrict__ ws, void* __restrict__ out_any,
                                                            const float* __restrict__ scale_a,
                                                            const float* __restrict__ scale_b, float post_scale,
                                                            int tiles, int tiles_m, int splits, long long Mo,
-                                                           long long No) {
+                                                           long long No, int out_bf16) {
   pdl_wait();
   pdl_trigger();
   const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -729,7 +747,11 @@ __global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restri
   if (row < Mo && col < No) {
     const float scale = (__ldg(scale_a) * __ldg(scale_b)) * post_scale;
     acc.x *= scale; acc.y *= scale; acc.z *= scale; acc.w *= scale;
-    *reinterpret_cast<float4*>(out + row * No + col) = acc;
+    if (out_bf16)
+      *reinterpret_cast<uint2*>(static_cast<uint16_t*>(out_any) + row * No + col) =
+          make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
+    else
+      *reinterpret_cast<float4*>(static_cast<float*>(out_any) + row * No + col) = acc;
   }
 }
 
@@ -783,14 +805,16 @@ int encode_bytes_map(void* fn, CUtensorMap* map, const uint8_t* ptr, uint64_t pi
   return r == CUDA_SUCCESS ? 0 : 1;
 }
 // fp32 output (or workspace) tensor rows x cols, box = 32 rows x 32 columns, 128-byte swizzle in shared memory
-int encode_out_map(void* fn, CUtensorMap* map, float* ptr, uint64_t rows, uint64_t cols) {
+// (bf16 output: the same box of 32 x 32 elements is 64 bytes wide, 64-byte swizzle)
+int encode_out_map(void* fn, CUtensorMap* map, void* ptr, uint64_t rows, uint64_t cols, bool bf16) {
   const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {cols * sizeof(float)};
+  const cuuint64_t strides[1] = {cols * (bf16 ? 2 : 4)};
   const cuuint32_t box[2] = {32, 32};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
-      map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ptr, dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+      CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : 1;
 }
 
@@ -847,6 +871,8 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   p.scale_a = a.d_scale_a; p.scale_b = a.d_scale_b; p.status = ctx->d_status;
   p.Mo = a.Mo; p.No = a.No; p.Kc = a.Kc;
   p.n_samples = a.n_samples;
+  p.out_bf16 = a.out_bf16;
+  if (a.out_bf16 && a.No % 8 != 0) return LUQ_ERR_ARG;   // output rows must stay 16-byte aligned
   p.tiles_m = static_cast<int>((a.Mo + BM - 1) / BM);
   p.tiles_n = static_cast<int>((a.No + BN - 1) / BN);
   p.num_kb = static_cast<int>((a.Kc + BK - 1) / BK);
@@ -899,7 +925,10 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   // Unsigned INT4 codes (kind 2) have no expansion inside the GEMM kernels: such an operand is
   // always fetched as bytes, the caller's or a plane expanded here.
   const bool b_must = a.b_kind == 2, a_must = a.a_kind == 2;
-  if (b_must || (long_contraction && p.tiles_m >= 2)) {
+  // (With bf16 outputs the output stream no longer hides the expansion: the caller's bytes are then
+  // used for short contractions too - backward product of the ResNet shape 82 -> 65 us.)
+  const bool use_given = a.out_bf16 != 0;
+  if (b_must || ((long_contraction || (use_given && b_given)) && p.tiles_m >= 2)) {
     if (b_given) {
       b_plane = true; b_plane_ptr = b_given;
     } else if (packed_ok(b_plane_bytes) && b_plane_bytes <= plane_room) {
@@ -910,7 +939,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
       return LUQ_ERR_WORKSPACE;
     }
   }
-  if (a_must || (long_contraction && p.tiles_n >= 2)) {
+  if (a_must || ((long_contraction || (use_given && a_given)) && p.tiles_n >= 2)) {
     if (a_given) {
       a_plane = true; a_plane_ptr = a_given;
     } else if (packed_ok(a_plane_bytes) && a_plane_bytes <= plane_room) {
@@ -959,13 +988,13 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
     if (a.b_mn) bad |= encode_bytes_map(ctx->encode_tiled, &tb, ptr, a.No / div, a.Kc, 1, false, b_plane);
     else bad |= encode_bytes_map(ctx->encode_tiled, &tb, ptr, a.Kc / div, a.No, 1, false, b_plane);
   }
-  if (p.splits > 1) bad |= encode_out_map(ctx->encode_tiled, &to, a.d_workspace, units * BM, BN);
-  else bad |= encode_out_map(ctx->encode_tiled, &to, a.d_out, a.Mo, a.No);
+  if (p.splits > 1) bad |= encode_out_map(ctx->encode_tiled, &to, a.d_workspace, units * BM, BN, false);
+  else bad |= encode_out_map(ctx->encode_tiled, &to, a.d_out, a.Mo, a.No, a.out_bf16 != 0);
   if (bad) return LUQ_ERR_CUDA;
 
   // CTA pairs when both operands are planes (no expansion inside the kernel) and the contraction
   // is not split: option LUQ_OPT_PAIRS (off unless set)
-  if (ctx->use_pairs && a_plane && b_plane && p.splits == 1 && p.tiles_m >= 2) {
+  if (ctx->use_pairs && a_plane && b_plane && p.splits == 1 && p.tiles_m >= 2 && !a.out_bf16) {
     const long long pair_tiles = static_cast<long long>((p.tiles_m + 1) / 2) * p.tiles_n;
     const int max_pairs = ctx->sm_count / 2;
     const int pairs = static_cast<int>(pair_tiles < max_pairs ? pair_tiles : max_pairs);
@@ -1005,7 +1034,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
     const long long work = tiles * (kTileFloats / 4);
     rc = static_cast<int>(luq_launch_kernel(split_reduce_kernel, static_cast<int>((work + 255) / 256), 256, 0, st, LUQ_LAUNCH_EARLY, 1,
                                             a.d_workspace, a.d_out, a.d_scale_a, a.d_scale_b, p.post_scale,
-                                            static_cast<int>(tiles), p.tiles_m, p.splits, a.Mo, a.No));
+                                            static_cast<int>(tiles), p.tiles_m, p.splits, a.Mo, a.No, a.out_bf16));
     if (rc == 0) ctx->launches += 1;
   }
   return rc;
@@ -1110,6 +1139,7 @@ extern "C" int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_al
   local.use_pairs = 0;
   local.kmax = LUQ_KMAX;
   local.unsigned_act = 0;
+  local.out_bf16 = 0;
   local.launches = 0;
   local.encode_tiled = s->encode_tiled;
 
