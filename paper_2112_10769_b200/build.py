@@ -7,6 +7,7 @@ with fast-math, flush-to-zero or approximate division.
 """
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 import sys
@@ -21,26 +22,49 @@ COMMON = ["-std=c++17", "-O3", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path
 UNITS = {"quant.cu": ["-fmad=false"], "gemm.cu": [], "api.cu": []}
 
 
-def _stale(target: str, deps) -> bool:
-    if not os.path.exists(target):
+def _digest(paths, extra=()) -> str:
+    """Content hash of the inputs of one build step (a copied tree keeps contents, not timestamps)."""
+    h = hashlib.sha256()
+    for item in extra:
+        h.update(str(item).encode())
+    for path in paths:
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def _stale(target: str, digest: str) -> bool:
+    stamp = target + ".sha"
+    if not os.path.exists(target) or not os.path.exists(stamp):
         return True
-    t = os.path.getmtime(target)
-    return any(os.path.getmtime(d) > t for d in deps)
+    with open(stamp) as f:
+        return f.read().strip() != digest
+
+
+def _stamp(target: str, digest: str) -> None:
+    with open(target + ".sha", "w") as f:
+        f.write(digest)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "nvcc")
-    headers = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "luq.h"), os.path.abspath(__file__)]
-    objs = []
+    headers = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "luq.h")]
+    objs, digests = [], []
     for name, extra in UNITS.items():
         src = os.path.join(CSRC, name)
         obj = os.path.join(CSRC, name.replace(".cu", ".o"))
         objs.append(obj)
-        if force or _stale(obj, [src] + headers):
+        flags = ARCH + COMMON[:5] + extra        # the flags that change the code (not the include paths)
+        digest = _digest([src] + headers, flags)
+        digests.append(digest)
+        if force or _stale(obj, digest):
             cmd = [nvcc] + ARCH + COMMON + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
             subprocess.run(cmd, check=True)
-    if force or _stale(LIB, objs):
+            _stamp(obj, digest)
+    link_digest = _digest([], digests)
+    if force or _stale(LIB, link_digest):
         subprocess.run([nvcc] + ARCH + ["-shared", "-o", LIB] + objs, check=True)
+        _stamp(LIB, link_digest)
     return LIB
 
 
