@@ -352,6 +352,11 @@ def run_ours(args):
     # this step run for tens of microseconds at the full SM clock, far from the power cap under which
     # the sustained figure (1.3 GHz) was taken.
     fp8_peak = 2.0 * peaks["bf16_tflops"]
+    props = torch.cuda.get_device_properties(local)
+    clocks_summary = sampler.summary()
+
+    def sampler_max_mhz():
+        return float(clocks_summary.get("sm_max_mhz") or 1965.0)
     kernels = {}
     for k, ms in per_kernel_ms.items():
         b, f = alg[k]
@@ -362,6 +367,15 @@ def run_ours(args):
             ach, peak, unit = b / (ms * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s"
         else:
             ach, peak, unit = f / (ms * 1e-3) / 1e12, fp8_peak, "TFLOP/s"
+        if k == "quant_grad_G":
+            # The LUQ quantizer is bound by instruction issue, not by HBM: per 32 elements about 21 issue
+            # cycles of decision and packing plus, per sample, 20 for the five wide multiplies of
+            # Philox4x32-10 (4 issue cycles each, measured) and 3 for the operand bytes.  Peak = what
+            # 4 sub-partitions per SM issue at the SM clock.
+            cycles = 21 + ns * (20 + 3)
+            alu_peak = props.multi_processor_count * 4 * sampler_max_mhz() * 1e6 * 32 / cycles / 1e9   # Gelt/s
+            if alu_peak * 1e9 < (peaks["hbm_gbs"] * 1e9) / (b / (M * N)):
+                bound, ach, peak, unit = "alu", M * N / (ms * 1e-3) / 1e9, round(alu_peak, 1), "Gelt/s"
         kernels[k] = {"ms": round(ms, 5), "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit,
                       "frac": round(ach / peak, 4), "tflops": round(f / (ms * 1e-3) / 1e12, 2) if f else None,
                       "gbs": round(b / (ms * 1e-3) / 1e9, 1)}
@@ -371,7 +385,9 @@ def run_ours(args):
                 "frac": d["frac"],
                 "traffic": NCU_TRAFFIC_BYTES.get(dominant) if (args.workload == "cfg2" and not args.rows) else None,
                 "algorithmic_bytes": alg[dominant][0], "algorithmic_flops": alg[dominant][1],
-                "peak_source": f"{peaks['source']}" + (" hbm copy" if d["bound"] == "hbm" else " bf16 burst x2 (8-bit operands)")}
+                "peak_source": {"hbm": f"{peaks['source']} hbm copy",
+                                "tensor": f"{peaks['source']} bf16 burst x2 (8-bit operands)",
+                                "alu": "derived: issue cycles per element x SM sub-partitions x SM clock"}[d["bound"]]}
 
     # ---- end to end: host buffers in, host buffers out, through the same calls
     e2e = None
@@ -458,7 +474,7 @@ def run_ours(args):
                                        ((per_kernel_ms["amax_G"] + per_kernel_ms["quant_grad_G"]) * 1e-3) / 1e9, 1),
             "ms_per_step_with_per_kernel_events": round(instrumented_ms, 5),
             "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline,
-            "gpu_launches": int(launches), "clocks": sampler.summary(),
+            "gpu_launches": int(launches), "clocks": clocks_summary,
         }
         print(json.dumps(line))
     ctx.close()
