@@ -75,6 +75,7 @@ class ClockSampler(threading.Thread):
         self.index = index
         self.samples = []
         self.stop_flag = threading.Event()
+        self.ready = threading.Event()       # set after the first sample (NVML start-up can take a second)
         self.error = None
 
     def run(self):
@@ -91,9 +92,11 @@ class ClockSampler(threading.Thread):
                 except Exception:
                     rs = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
                 self.samples.append((sm, pw, rs))
+                self.ready.set()
                 self.stop_flag.wait(0.01)
         except Exception as e:  # pragma: no cover
             self.error = repr(e)
+            self.ready.set()
 
     def summary(self):
         if not self.samples:
@@ -316,7 +319,7 @@ def run_ours(args):
 
     sampler = ClockSampler(gpu_physical_index(local))
     sampler.start()
-    time.sleep(0.3)
+    sampler.ready.wait(10.0)
     # The timed region: K steps, two events around the whole of it.
     launches0 = ctx.launches
     barrier()

@@ -62,16 +62,15 @@ int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st);
 #ifdef __CUDACC__
 
 // Launch helper.  LUQ_LAUNCH_COOPERATIVE: all blocks of the grid are resident at once (the kernel
-// has a grid barrier inside).  LUQ_LAUNCH_EARLY = programmatic dependent launch: the kernel may become resident and set
-// up (barriers, tensor memory, descriptor prefetch) while its predecessor in the stream drains,
-// and waits in pdl_wait() until that predecessor has completed and its writes are visible.
-// Every kernel of the library calls pdl_wait() before its first access to global memory, so any
-// of them may be launched this way; it is used for the GEMM-side kernels only.  Their CTAs need
-// most of an SM's shared memory and cannot share an SM with the predecessor's, so all they
-// overlap is launch latency and set-up.  The small-footprint streaming kernels (max, quantizers)
-// are launched normally: launched early they become resident next to a running GEMM CTA, on an
-// SM configured for maximum shared memory, keep that small L1 after the GEMM has gone and lose
-// a third of their bandwidth (measured: the 462 MB max reduction, 68 -> 96 us).
+// has a grid barrier inside).  LUQ_LAUNCH_EARLY = programmatic dependent launch: the kernel may
+// become resident and set up (barriers, tensor memory, descriptor prefetch) while its predecessor
+// in the stream drains, and waits in pdl_wait() until that predecessor has completed and its writes
+// are visible.  Every kernel of the library calls pdl_wait() before its first access to global
+// memory, and all but the cooperative ones are launched this way.  One trap, measured: a small
+// streaming block that becomes resident beside a running GEMM block sits on an SM carved for
+// maximum shared memory and keeps that small L1 after the GEMM has gone (the 462 MB max reduction:
+// 68 -> 96 us).  The streaming kernels therefore state a preference for the largest L1 carve-out,
+// which keeps their blocks off such an SM until it is free.
 #define LUQ_LAUNCH_NORMAL 0
 #define LUQ_LAUNCH_EARLY 1
 #define LUQ_LAUNCH_COOPERATIVE 2

@@ -667,6 +667,10 @@ __global__ void __launch_bounds__(kThreads) luq_quotient_kernel(const float* __r
 template <typename K>
 int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 30) {
   int per_sm = 0;
+  // These kernels are launched early (see luq_launch_kernel).  With a preference for the largest L1
+  // their blocks do not become resident on an SM that is still carved for a GEMM block's shared
+  // memory, where they would keep a small L1 for their whole life.
+  cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxL1);
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1)
     per_sm = 1;
   if (per_sm > max_per_sm) per_sm = max_per_sm;
@@ -686,10 +690,10 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
   cudaError_t e;
   if (dtype == LUQ_BF16) {
     const int grid = grid_for(ctx, amax_kernel<true>, n / 8 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
-    e = luq_launch_kernel(amax_kernel<true>, grid, kThreads, 0, st, LUQ_LAUNCH_NORMAL, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
+    e = luq_launch_kernel(amax_kernel<true>, grid, kThreads, 0, st, LUQ_LAUNCH_EARLY, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
   } else {
     const int grid = grid_for(ctx, amax_kernel<false>, n / 4 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
-    e = luq_launch_kernel(amax_kernel<false>, grid, kThreads, 0, st, LUQ_LAUNCH_NORMAL, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
+    e = luq_launch_kernel(amax_kernel<false>, grid, kThreads, 0, st, LUQ_LAUNCH_EARLY, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
   }
   ctx->launches += 1;
   return static_cast<int>(e);
@@ -700,7 +704,7 @@ template <bool BF16, bool PLANE, bool UNSIGNED>
 int launch_int4(luq_ctx* ctx, const void* d_x, size_t n, const float* d_clip, uint8_t* d_codes, int8_t* d_operand,
                 float* d_scale, float* d_amax_out, cudaStream_t st) {
   const int grid = grid_for(ctx, quant_int4_kernel<BF16, PLANE, UNSIGNED>, n / Item<BF16>::kElems / kTileItems + 1);
-  const int mode = d_amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_NORMAL;   // fused: grid barrier inside
+  const int mode = d_amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_EARLY;   // fused: grid barrier inside
   return static_cast<int>(luq_launch_kernel(quant_int4_kernel<BF16, PLANE, UNSIGNED>, grid, kThreads, 0, st, mode, 1, d_x, n,
                                             d_clip, d_codes, d_operand, d_scale, d_amax_out, ctx->d_scratch,
                                             ctx->d_status));
@@ -752,7 +756,7 @@ template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
 int launch_luq_ns(const LuqLaunch& a) {
   const size_t tiles = a.n / Item<BF16>::kElems / kTileItems + 1;
   const int grid = grid_for(a.ctx, quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, tiles);
-  const int mode = a.amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_NORMAL;
+  const int mode = a.amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_EARLY;
   return static_cast<int>(luq_launch_kernel(quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, grid, kThreads, 0, a.st, mode, 1,
                                             a.g, a.n, a.amax, a.keys, a.n_samples, a.codes, a.operand, a.alpha,
                                             a.measured, a.estimate, a.eta, a.amax_out, a.ctx->d_scratch,
