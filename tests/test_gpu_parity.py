@@ -507,3 +507,40 @@ def test_quant_grad_nearest_power_bit_exact(ctx, n, dtype, kmax):
     finally:
         ctx.set_option(binding.OPT_LEVELS, 4)
     assert ctx.status() == 0
+
+
+def test_back_to_back_steps_equal_a_synchronised_step(ctx):
+    """Every kernel may become resident while its predecessor drains; nothing may be read or written
+    before the predecessor has finished.  Thirty steps queued without a host synchronisation, buffers
+    re-used, must leave exactly what one synchronised step leaves."""
+    M, K, N, ns = 1152, 1056, 800, 2
+    A, W, G = inputs.small_layer(M, K, N, 5)
+    Ad, Wd, Gd = to_dev(A), to_dev(W), to_dev(G)
+    dev = Ad.device
+    f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)   # noqa: E731
+    u8 = lambda *s: torch.empty(s, dtype=torch.uint8, device=dev)      # noqa: E731
+    i8 = lambda n: torch.empty(n, dtype=torch.int8, device=dev)        # noqa: E731
+    mA, mW, mG, sA, sW, aG = (f32(1) for _ in range(6))
+    cA, cW, cG = u8(M * K // 2), u8(N * K // 2), u8(ns, M * N // 2)
+    bW, bG = i8(N * K), i8(ns * M * N)
+    Z, dA, dW = f32(M, N), f32(M, K), f32(N, K)
+
+    def step(seed):
+        ctx.amax(Ad, mA); ctx.amax(Wd, mW)
+        ctx.quant_int4(Ad, mA, cA, sA); ctx.quant_int4(Wd, mW, cW, sW, bW)
+        ctx.gemm_fwd(cA, sA, cW, sW, M, N, K, Z, None, bW)
+        ctx.amax(Gd, mG); ctx.quant_grad(Gd, mG, seed, ns, cG, aG, bG)
+        ctx.gemm_bwd(cG, aG, ns, cW, sW, M, N, K, dA, bG, bW)
+        ctx.gemm_wgrad(cG, aG, ns, cA, sA, M, N, K, dW, bG, None)
+
+    step(29)
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (cA, cW, cG, Z, dA, dW, mA, mW, mG, sA, sW, aG)]
+    for t in (cA, cW, cG, Z, dA, dW):
+        t.zero_()
+    for seed in range(30):          # different seeds: every step really rewrites the gradient codes
+        step(seed)
+    torch.cuda.synchronize()
+    for got, ref in zip((cA, cW, cG, Z, dA, dW, mA, mW, mG, sA, sW, aG), want):
+        assert torch.equal(got, ref)
+    assert ctx.status() == 0
