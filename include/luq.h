@@ -196,6 +196,12 @@ int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t ro
  * equal the IEEE binary32 quotient wherever that quotient is a normal number. */
 int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream);
 
+/* Diagnostic for the bounded waits (the paper has no counterpart): launches one thread that waits on a
+ * barrier nothing ever arrives on, with a short limit.  The wait expires, the kernel raises
+ * LUQ_STATUS_TIMEOUT the way the GEMM roles and the fused quantizers do, and returns normally; the
+ * context stays usable and luq_status() reports and clears the bit. */
+int luq_debug_expire_wait(luq_ctx* ctx, void* stream);
+
 /* The three GEMMs write fp32 outputs (void* d_z / d_da / d_dw point to floats) unless
  * LUQ_OPT_OUTPUT_BF16 is set on the context, in which case they point to bf16 values.
  *

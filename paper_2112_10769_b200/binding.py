@@ -22,7 +22,7 @@ ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
            "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_pw2",
-           "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
+           "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_debug_expire_wait", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
 _lib = None
@@ -56,6 +56,7 @@ def load() -> ctypes.CDLL:
         L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, ctypes.c_int, u64,
                                                ctypes.c_int, vp, vp, vp, vp, vp]
+        L.luq_debug_expire_wait.argtypes = [vp, vp]
         L.luq_debug_quotient.argtypes = [vp, vp, sz, vp, vp, vp]
         L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, i64, i64, i64, vp]
@@ -245,6 +246,10 @@ class Context:
                                                _opt(operand, n_samples * g.numel()), _stream()),
                "luq_quant_grad_hindsight")
         return codes, alpha, measured
+
+    def debug_expire_wait(self):
+        """Launches a kernel whose bounded wait runs out; status() then reports STATUS_TIMEOUT."""
+        _check(load().luq_debug_expire_wait(self.handle, _stream()), "luq_debug_expire_wait")
 
     def debug_quotient(self, x: torch.Tensor, amax: torch.Tensor) -> torch.Tensor:
         out = torch.empty_like(x, dtype=torch.float32)

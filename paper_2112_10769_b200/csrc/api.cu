@@ -248,6 +248,13 @@ int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t ro
                                           nullptr, as_stream(stream)));
 }
 
+int luq_debug_expire_wait(luq_ctx* ctx, void* stream) {
+  if (!ctx) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_expire_wait(ctx, as_stream(stream)));
+}
+
 int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream) {
   if (!ctx || !d_amax || (n && (!d_x || !d_t))) return LUQ_ERR_ARG;
   DeviceGuard guard(ctx->device);

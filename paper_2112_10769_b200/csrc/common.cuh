@@ -58,6 +58,7 @@ struct luq_gemm_args {
   int allow_split;
 };
 int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st);
+int luq_launch_expire_wait(luq_ctx* ctx, cudaStream_t st);
 
 #ifdef __CUDACC__
 

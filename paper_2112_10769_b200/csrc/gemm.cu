@@ -862,6 +862,22 @@ int launch_expand(bool luq_codes, const uint8_t* codes, uint8_t* plane, size_t p
                                     : luq_launch_kernel(expand_plane_kernel<KIND, false>, grid, 256, 0, st, LUQ_LAUNCH_EARLY, 1, src, dst, pieces, lut));
 }
 
+// Diagnostic: a bounded wait that is left to run out.  One thread initialises an mbarrier that
+// nothing ever arrives on, polls it a fixed number of times, then reports the expiry the way the
+// GEMM roles do (status bit, normal return).  The context stays usable.
+__global__ void expire_wait_kernel(unsigned int* status, uint32_t polls) {
+  __shared__ __align__(8) uint64_t bar;
+  pdl_wait();
+  pdl_trigger();
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    fence_barrier_init();
+    bool arrived = false;
+    for (uint32_t i = 0; i < polls && !arrived; ++i) arrived = mbar_test(smem_u32(&bar), 0);
+    if (!arrived) atomicOr(status, LUQ_STATUS_TIMEOUT);
+  }
+}
+
 constexpr size_t kSplitRegionBytes = 20u << 20;   // the first 20 MiB of a workspace hold split partial tiles
 
 }  // namespace
@@ -1038,6 +1054,12 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
     if (rc == 0) ctx->launches += 1;
   }
   return rc;
+}
+
+int luq_launch_expire_wait(luq_ctx* ctx, cudaStream_t st) {
+  const cudaError_t e = luq_launch_kernel(expire_wait_kernel, 1, 32, 0, st, LUQ_LAUNCH_EARLY, 1, ctx->d_status, 1u << 16);
+  ctx->launches += 1;
+  return static_cast<int>(e);
 }
 
 int luq_launch_gemm(luq_ctx* ctx_in, const luq_gemm_args& a, cudaStream_t st) {

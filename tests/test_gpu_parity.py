@@ -544,3 +544,18 @@ def test_back_to_back_steps_equal_a_synchronised_step(ctx):
     for got, ref in zip((cA, cW, cG, Z, dA, dW, mA, mW, mG, sA, sW, aG), want):
         assert torch.equal(got, ref)
     assert ctx.status() == 0
+
+
+def test_an_expired_wait_is_reported_and_the_context_stays_usable(ctx):
+    """The library's waits are bounded: when one runs out the kernel raises a status bit and returns.
+    The diagnostic kernel waits on a barrier nothing arrives on (no fault, no hang)."""
+    x = to_dev(luq_inputs(100_000, 8))
+    before, _ = ctx.quant_grad(x, ctx.amax(x), 3, 1)
+    assert ctx.status() == 0
+    ctx.debug_expire_wait()
+    assert ctx.status() == binding.STATUS_TIMEOUT
+    assert ctx.status() == 0                       # reading the status clears it
+    after, _ = ctx.quant_grad(x, ctx.amax(x), 3, 1)
+    _, fused, _ = ctx.amax_quant_grad(x, 3, 1)     # also the kernels that share the scratch counters
+    assert torch.equal(before, after) and torch.equal(before, fused)
+    assert ctx.status() == 0
