@@ -119,6 +119,17 @@ int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, 
 int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
                    const float* d_clip, uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
 
+/* luq_amax and luq_quant_int4 for several tensors of one element type in ONE launch each (the
+ * forward pass of a layer quantizes its activations and its weights; a small tensor's launch and
+ * reduction latency then hides behind the large one's stream).  count <= 4.  The arrays are HOST
+ * arrays of `count` entries holding device pointers / element counts; results are exactly those
+ * of the separate calls.  n[i] even for luq_quant_int4_multi; d_operand[i] may be NULL. */
+int luq_amax_multi(luq_ctx* ctx, int count, const void* const* d_x, int dtype, const size_t* n,
+                   float* const* d_amax, void* stream);
+int luq_quant_int4_multi(luq_ctx* ctx, int count, const void* const* d_x, int dtype, const size_t* n,
+                         const float* const* d_clip, uint8_t* const* d_codes, float* const* d_scale,
+                         int8_t* const* d_operand, void* stream);
+
 /* Unsigned INT4 for tensors that cannot be negative (post-ReLU activations).  Appendix
  * "Quantization formats": scale = Delta / (2^b - 1) with Delta the quantized range - for the
  * range [0, clip] all sixteen codes lie on one side of zero:

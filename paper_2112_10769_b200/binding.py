@@ -21,7 +21,7 @@ OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS, OPT_UNSIGNED_ACTIVATIONS, OPT_O
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_pw2",
+           "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_pw2",
            "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_debug_expire_wait", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
@@ -48,6 +48,8 @@ def load() -> ctypes.CDLL:
         L.luq_kmax.argtypes = []
         L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
         L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
+        L.luq_amax_multi.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int, vp, vp, vp]
+        L.luq_quant_int4_multi.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
         L.luq_quant_uint4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_amax_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_amax_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, u64, ctypes.c_int, vp, vp, vp, vp, vp]
@@ -155,6 +157,32 @@ class Context:
                                      codes.data_ptr(), scale.data_ptr(), _opt(operand, x.numel()), _stream()),
                "luq_quant_int4")
         return codes, scale
+
+    # ---- several tensors in one launch (host arrays of device pointers) -----------------------
+    @staticmethod
+    def _ptr_array(tensors):
+        return (ctypes.c_void_p * len(tensors))(*[None if t is None else t.data_ptr() for t in tensors])
+
+    def amax_multi(self, xs, outs=None):
+        """max|x| of up to four tensors of one element type in one launch."""
+        outs = [torch.empty(1, dtype=torch.float32, device=x.device) for x in xs] if outs is None else outs
+        n = (ctypes.c_size_t * len(xs))(*[x.numel() for x in xs])
+        _check(load().luq_amax_multi(self.handle, len(xs), self._ptr_array(xs), _dtype_code(xs[0]), n,
+                                     self._ptr_array(outs), _stream()), "luq_amax_multi")
+        return outs
+
+    def quant_int4_multi(self, xs, clips, codes=None, scales=None, operands=None):
+        """quant_int4 of up to four tensors of one element type in one launch; operands[i] may be None."""
+        codes = [torch.empty(x.numel() // 2, dtype=torch.uint8, device=x.device) for x in xs] if codes is None else codes
+        scales = [torch.empty(1, dtype=torch.float32, device=x.device) for x in xs] if scales is None else scales
+        operands = [None] * len(xs) if operands is None else operands
+        for x, o in zip(xs, operands):
+            _opt(o, x.numel())
+        n = (ctypes.c_size_t * len(xs))(*[x.numel() for x in xs])
+        _check(load().luq_quant_int4_multi(self.handle, len(xs), self._ptr_array(xs), _dtype_code(xs[0]), n,
+                                           self._ptr_array(clips), self._ptr_array(codes), self._ptr_array(scales),
+                                           self._ptr_array(operands), _stream()), "luq_quant_int4_multi")
+        return codes, scales
 
     def quant_uint4(self, x: torch.Tensor, clip: torch.Tensor, codes: torch.Tensor | None = None,
                     scale: torch.Tensor | None = None, operand: torch.Tensor | None = None):

@@ -62,7 +62,7 @@ int luq_create(luq_ctx** out, int device) {
   c->workspace_bytes = kWorkspaceBytes;
   c->d_status = nullptr; c->d_scratch = nullptr; c->d_workspace = nullptr; c->encode_tiled = nullptr;
   // status word and the grid-maximum scratch share one small allocation
-  const size_t small_bytes = (64 + LUQ_SCRATCH_WORDS) * sizeof(unsigned int);
+  const size_t small_bytes = (64 + static_cast<size_t>(LUQ_SCRATCH_WORDS)) * sizeof(unsigned int);
   bool ok = cudaMalloc(&c->d_status, small_bytes) == cudaSuccess &&
             cudaMalloc(&c->d_workspace, kWorkspaceBytes) == cudaSuccess;
   ok = ok && cudaMemset(c->d_status, 0, small_bytes) == cudaSuccess;
@@ -126,6 +126,35 @@ int luq_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_amax, 
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_amax(ctx, d_x, dtype, n, d_amax, as_stream(stream)));
+}
+
+int luq_amax_multi(luq_ctx* ctx, int count, const void* const* d_x, int dtype, const size_t* n,
+                   float* const* d_amax, void* stream) {
+  if (!ctx || count < 1 || count > LUQ_SCRATCH_MULTI || !d_x || !n || !d_amax) return LUQ_ERR_ARG;
+  if (dtype != LUQ_F32 && dtype != LUQ_BF16) return LUQ_ERR_ARG;
+  for (int t = 0; t < count; ++t) {
+    if (!d_amax[t] || (n[t] && !d_x[t]) || !aligned16(d_x[t]) || (reinterpret_cast<uintptr_t>(d_amax[t]) & 3u))
+      return LUQ_ERR_ARG;
+  }
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_amax_multi(ctx, count, d_x, n, d_amax, dtype, as_stream(stream)));
+}
+
+int luq_quant_int4_multi(luq_ctx* ctx, int count, const void* const* d_x, int dtype, const size_t* n,
+                         const float* const* d_clip, uint8_t* const* d_codes, float* const* d_scale,
+                         int8_t* const* d_operand, void* stream) {
+  if (!ctx || count < 1 || count > LUQ_SCRATCH_MULTI || !d_x || !n || !d_clip || !d_codes || !d_scale || !d_operand)
+    return LUQ_ERR_ARG;
+  if (dtype != LUQ_F32 && dtype != LUQ_BF16) return LUQ_ERR_ARG;
+  for (int t = 0; t < count; ++t) {
+    if (!d_clip[t] || !d_scale[t] || (n[t] & 1u) || (n[t] && (!d_x[t] || !d_codes[t]))) return LUQ_ERR_ARG;
+    if (!aligned16(d_x[t]) || !aligned16(d_codes[t]) || !aligned16(d_operand[t])) return LUQ_ERR_ARG;
+  }
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_int4_multi(ctx, count, d_x, n, d_clip, d_codes, d_scale, d_operand, dtype,
+                                             as_stream(stream)));
 }
 
 int luq_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, const float* d_clip,

@@ -40,7 +40,19 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
                              float* d_measured, float* d_estimate, float eta, float* d_amax_out, cudaStream_t st);
-#define LUQ_SCRATCH_WORDS 4096  // two counters + block maxima; grids of the reducing kernels stay below it
+// Scratch words for grid-wide maxima.  Words 0 .. LUQ_SCRATCH_SINGLE-1: the one-tensor kernels (two
+// counters + one word per block).  Then LUQ_SCRATCH_MULTI regions of LUQ_SCRATCH_REGION words, one per
+// tensor of a several-tensor launch.  Grids of the reducing kernels stay below the region sizes.
+#define LUQ_SCRATCH_SINGLE 4096
+#define LUQ_SCRATCH_REGION 2048
+#define LUQ_SCRATCH_MULTI 4
+#define LUQ_SCRATCH_WORDS (LUQ_SCRATCH_SINGLE + LUQ_SCRATCH_MULTI * LUQ_SCRATCH_REGION)
+// several tensors of one element type in one launch (count <= LUQ_SCRATCH_MULTI); host arrays
+int luq_launch_amax_multi(luq_ctx* ctx, int count, const void* const* d_x, const size_t* n, float* const* d_amax,
+                          int dtype, cudaStream_t st);
+int luq_launch_quant_int4_multi(luq_ctx* ctx, int count, const void* const* d_x, const size_t* n,
+                                const float* const* d_clip, uint8_t* const* d_codes, float* const* d_scale,
+                                int8_t* const* d_operand, int dtype, cudaStream_t st);
 int luq_launch_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t,
                               cudaStream_t st);
 

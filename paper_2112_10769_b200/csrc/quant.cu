@@ -88,9 +88,12 @@ template <bool BF16> struct Item {
 // Grid-wide maximum without a pre-zeroed output: every block leaves its maximum in the
 // context's scratch array and takes a ticket; the block that draws the last ticket reduces the
 // array, resets the ticket counter and returns true in its thread 0 with the result in `m`.
+// `rank` of `count` is the block's place among the blocks that work on this tensor (the whole grid,
+// or a share of it in the kernels that take several tensors in one launch).
 // scratch[0] is the ticket counter (zero between kernels), scratch[1] the departure counter of
 // the fused kernels' grid barrier, scratch[2 + b] block b's maximum.
-__device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* scratch) {
+__device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* scratch, unsigned int rank,
+                                                    unsigned int count) {
   __shared__ uint32_t warp_max[kThreads / 32];
   __shared__ bool last;
   m = __reduce_max_sync(0xFFFFFFFFu, m);
@@ -100,16 +103,16 @@ __device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* s
     m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
     m = __reduce_max_sync(0xFFFFFFFFu, m);
     if (threadIdx.x == 0) {
-      __stcg(scratch + 2 + blockIdx.x, m);
+      __stcg(scratch + 2 + rank, m);
       __threadfence();
-      last = atomicAdd(scratch, 1u) == gridDim.x - 1;
+      last = atomicAdd(scratch, 1u) == count - 1;
     }
   }
   __syncthreads();
   if (!last) return false;
   __threadfence();
   m = 0;
-  for (unsigned int b = threadIdx.x; b < gridDim.x; b += kThreads) m = max(m, __ldcg(scratch + 2 + b));
+  for (unsigned int b = threadIdx.x; b < count; b += kThreads) m = max(m, __ldcg(scratch + 2 + b));
   m = __reduce_max_sync(0xFFFFFFFFu, m);
   __syncthreads();            // warp_max is reused
   if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
@@ -131,12 +134,9 @@ __device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* s
 constexpr int kAmaxUnroll = 4;
 constexpr int kAmaxCtasPerSm = 8;
 template <bool BF16>
-__global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__ x, size_t n,
-                                                        unsigned int* __restrict__ out_bits,
-                                                        unsigned int* __restrict__ scratch,
-                                                        unsigned int* __restrict__ status) {
-  luqdev::pdl_wait();
-  luqdev::pdl_trigger();
+__device__ __forceinline__ void amax_body(const void* __restrict__ x, size_t n, unsigned int* __restrict__ out_bits,
+                                          unsigned int* __restrict__ scratch, unsigned int* __restrict__ status,
+                                          unsigned int rank, unsigned int count) {
   constexpr int kElems = Item<BF16>::kElems;
   constexpr int kUnroll = kAmaxUnroll;
   constexpr int kTileItems = kThreads * kUnroll;
@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
     }
   };
   const size_t full_tiles = items / kTileItems;
-  for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {
+  for (size_t t = rank; t < full_tiles; t += count) {
     const uint4* q = p + t * kTileItems + threadIdx.x;
     uint4 u[kUnroll];
 #pragma unroll
@@ -165,16 +165,46 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) fold(u[j]);
   }
-  if (blockIdx.x == gridDim.x - 1)   // pieces after the last full tile
+  if (rank == count - 1)   // pieces after the last full tile
     for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) fold(__ldg(p + i));
   // ragged tail: fewer elements than one piece
-  if (blockIdx.x == 0 && threadIdx.x < n - items * kElems)
+  if (rank == 0 && threadIdx.x < n - items * kElems)
     m = max(m, __float_as_uint(Item<BF16>::load1(x, items * kElems + threadIdx.x)) & 0x7FFFFFFFu);
 
-  if (grid_max_last_block(m, scratch)) {
+  if (grid_max_last_block(m, scratch, rank, count)) {
     *out_bits = m;
     if (m >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
   }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__ x, size_t n,
+                                                        unsigned int* __restrict__ out_bits,
+                                                        unsigned int* __restrict__ scratch,
+                                                        unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
+  amax_body<BF16>(x, n, out_bits, scratch, status, blockIdx.x, gridDim.x);
+}
+
+// Several tensors in one launch (a layer's activations and weights, say): the blocks are dealt out
+// to the tensors in proportion to their sizes, each tensor has its own 1024-word region of the
+// scratch array.  A small tensor's launch and reduction latency hides behind the large one's stream.
+constexpr int kMultiMax = LUQ_SCRATCH_MULTI;
+struct MultiAmax {
+  const void* x[kMultiMax]; size_t n[kMultiMax]; unsigned int* out[kMultiMax];
+  unsigned int first_block[kMultiMax + 1]; int count;
+};
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) amax_multi_kernel(const __grid_constant__ MultiAmax a,
+                                                              unsigned int* __restrict__ scratch,
+                                                              unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
+  int t = 0;
+  while (t + 1 < a.count && blockIdx.x >= a.first_block[t + 1]) ++t;
+  amax_body<BF16>(a.x[t], a.n[t], a.out[t], scratch + LUQ_SCRATCH_SINGLE + t * LUQ_SCRATCH_REGION, status,
+                  blockIdx.x - a.first_block[t], a.first_block[t + 1] - a.first_block[t]);
 }
 
 // ------------------------------------------------- fused max (phase one) ----
@@ -284,26 +314,12 @@ __device__ __forceinline__ uint32_t uint4_code(float x, float inv) {
 // byte) are written next to the packed codes, one byte per element in element order.
 // UNSIGNED: the grid 0..15 with scale clip / 15 (non-negative tensors); operand byte = q.
 template <bool BF16, bool PLANE, bool UNSIGNED>
-__global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __restrict__ x, size_t n,
-                                                              const float* d_clip,
-                                                              uint8_t* __restrict__ codes,
-                                                              int8_t* __restrict__ operand,
-                                                              float* __restrict__ d_scale,
-                                                              float* d_amax_out, unsigned int* scratch,
-                                                              unsigned int* __restrict__ status) {
-  luqdev::pdl_wait();
-  luqdev::pdl_trigger();
+__device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size_t n, float clip,
+                                                uint8_t* __restrict__ codes, int8_t* __restrict__ operand,
+                                                float* __restrict__ d_scale, unsigned int* __restrict__ status,
+                                                unsigned int rank, unsigned int count) {
   constexpr int kElems = Item<BF16>::kElems;
-  const bool first = blockIdx.x == 0 && threadIdx.x == 0;
-  float clip;
-  if (d_amax_out != nullptr) {   // fused: the clip is this tensor's maximum, reduced here
-    uint32_t bits;
-    if (!fused_grid_max<BF16>(x, n, scratch, status, bits)) return;
-    clip = __uint_as_float(bits);
-    if (first) *d_amax_out = clip;
-  } else {
-    clip = *d_clip;
-  }
+  const bool first = rank == 0 && threadIdx.x == 0;
   const bool ok = scale_usable(clip, first ? status : nullptr);
   constexpr float kTop = UNSIGNED ? 15.0f : 7.0f;
   constexpr int kByteShift = UNSIGNED ? 0 : 4;
@@ -330,7 +346,7 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
   // The tensor was just read front to back by the max reduction; its tail is what the
   // L2 still holds, so this pass walks the tiles from the back.
   const size_t full_tiles = items / kTileItems;
-  for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {
+  for (size_t t = rank; t < full_tiles; t += count) {
     const size_t i0 = (full_tiles - 1 - t) * kTileItems + threadIdx.x;
     uint4 u[kUnroll];
 #pragma unroll
@@ -338,7 +354,7 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) emit(i0 + j * kThreads, u[j]);
   }
-  if (blockIdx.x == gridDim.x - 1)
+  if (rank == count - 1)
     for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) emit(i, __ldg(p + i));
   if (first) {  // tail: fewer elements than one piece, two per byte
     for (size_t e = items * kElems; e < n; e += 2) {
@@ -351,6 +367,49 @@ __global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __rest
       }
     }
   }
+}
+
+template <bool BF16, bool PLANE, bool UNSIGNED>
+__global__ void __launch_bounds__(kThreads) quant_int4_kernel(const void* __restrict__ x, size_t n,
+                                                              const float* d_clip,
+                                                              uint8_t* __restrict__ codes,
+                                                              int8_t* __restrict__ operand,
+                                                              float* __restrict__ d_scale,
+                                                              float* d_amax_out, unsigned int* scratch,
+                                                              unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
+  float clip;
+  if (d_amax_out != nullptr) {   // fused: the clip is this tensor's maximum, reduced here
+    uint32_t bits;
+    if (!fused_grid_max<BF16>(x, n, scratch, status, bits)) return;
+    clip = __uint_as_float(bits);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *d_amax_out = clip;
+  } else {
+    clip = *d_clip;
+  }
+  quant_int4_body<BF16, PLANE, UNSIGNED>(x, n, clip, codes, operand, d_scale, status, blockIdx.x, gridDim.x);
+}
+
+// several tensors in one launch, see amax_multi_kernel; a tensor without operand bytes passes null
+struct MultiInt4 {
+  const void* x[kMultiMax]; size_t n[kMultiMax]; const float* clip[kMultiMax]; uint8_t* codes[kMultiMax];
+  int8_t* operand[kMultiMax]; float* scale[kMultiMax];
+  unsigned int first_block[kMultiMax + 1]; int count;
+};
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) quant_int4_multi_kernel(const __grid_constant__ MultiInt4 a,
+                                                                    unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
+  int t = 0;
+  while (t + 1 < a.count && blockIdx.x >= a.first_block[t + 1]) ++t;
+  const unsigned int rank = blockIdx.x - a.first_block[t], count = a.first_block[t + 1] - a.first_block[t];
+  const float clip = *a.clip[t];
+  if (a.operand[t] != nullptr)
+    quant_int4_body<BF16, true, false>(a.x[t], a.n[t], clip, a.codes[t], a.operand[t], a.scale[t], status, rank, count);
+  else
+    quant_int4_body<BF16, false, false>(a.x[t], a.n[t], clip, a.codes[t], nullptr, a.scale[t], status, rank, count);
 }
 
 // ------------------------------------------------------------------- LUQ ----
@@ -638,7 +697,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
     }
   }
   if constexpr (TRACK) {   // Inf/NaN patterns win the maximum and raise the flag
-    if (grid_max_last_block(seen, scratch)) {
+    if (grid_max_last_block(seen, scratch, blockIdx.x, gridDim.x)) {
       *measured_bits = seen;
       if (seen >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
       const float keep = __fsub_rn(1.0f, eta);
@@ -675,7 +734,7 @@ int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 3
     per_sm = 1;
   if (per_sm > max_per_sm) per_sm = max_per_sm;
   size_t cap = static_cast<size_t>(ctx->sm_count) * per_sm;
-  if (cap > LUQ_SCRATCH_WORDS - 2) cap = LUQ_SCRATCH_WORDS - 2;   // one scratch word per block of a reducing kernel
+  if (cap > LUQ_SCRATCH_REGION - 2) cap = LUQ_SCRATCH_REGION - 2;   // one scratch word per block of a reducing kernel
   if (tiles < 1) tiles = 1;
   if (tiles <= cap) return static_cast<int>(tiles);
   const size_t rounds = (tiles + cap - 1) / cap;
@@ -694,6 +753,78 @@ int luq_launch_amax(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d
   } else {
     const int grid = grid_for(ctx, amax_kernel<false>, n / 4 / (kThreads * kAmaxUnroll) + 1, kAmaxCtasPerSm);
     e = luq_launch_kernel(amax_kernel<false>, grid, kThreads, 0, st, LUQ_LAUNCH_EARLY, 1, d_x, n, out, ctx->d_scratch, ctx->d_status);
+  }
+  ctx->launches += 1;
+  return static_cast<int>(e);
+}
+
+namespace {
+// Blocks of a several-tensor launch: one wave of the GPU, dealt out in proportion to the tensors'
+// tile counts, at least one block each.
+template <typename K>
+void deal_blocks(const luq_ctx* ctx, K kernel, int count, const size_t* tiles, unsigned int* first_block) {
+  int per_sm = 0;
+  cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxL1);
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1)
+    per_sm = 1;
+  const size_t cap = static_cast<size_t>(ctx->sm_count) * per_sm;
+  size_t total = 0;
+  for (int t = 0; t < count; ++t) total += tiles[t];
+  first_block[0] = 0;
+  for (int t = 0; t < count; ++t) {
+    size_t blocks = total <= cap ? tiles[t] : tiles[t] * cap / total;
+    if (blocks < 1) blocks = 1;
+    if (blocks > LUQ_SCRATCH_REGION - 2) blocks = LUQ_SCRATCH_REGION - 2;
+    first_block[t + 1] = first_block[t] + static_cast<unsigned int>(blocks);
+  }
+}
+}  // namespace
+
+int luq_launch_amax_multi(luq_ctx* ctx, int count, const void* const* d_x, const size_t* n, float* const* d_amax,
+                          int dtype, cudaStream_t st) {
+  MultiAmax a{};
+  size_t tiles[kMultiMax];
+  const bool bf = dtype == LUQ_BF16;
+  for (int t = 0; t < count; ++t) {
+    a.x[t] = d_x[t]; a.n[t] = n[t]; a.out[t] = reinterpret_cast<unsigned int*>(d_amax[t]);
+    tiles[t] = n[t] / (bf ? 8 : 4) / (kThreads * kAmaxUnroll) + 1;
+  }
+  a.count = count;
+  cudaError_t e;
+  if (bf) {
+    deal_blocks(ctx, amax_multi_kernel<true>, count, tiles, a.first_block);
+    e = luq_launch_kernel(amax_multi_kernel<true>, static_cast<int>(a.first_block[count]), kThreads, 0, st,
+                          LUQ_LAUNCH_EARLY, 1, a, ctx->d_scratch, ctx->d_status);
+  } else {
+    deal_blocks(ctx, amax_multi_kernel<false>, count, tiles, a.first_block);
+    e = luq_launch_kernel(amax_multi_kernel<false>, static_cast<int>(a.first_block[count]), kThreads, 0, st,
+                          LUQ_LAUNCH_EARLY, 1, a, ctx->d_scratch, ctx->d_status);
+  }
+  ctx->launches += 1;
+  return static_cast<int>(e);
+}
+
+int luq_launch_quant_int4_multi(luq_ctx* ctx, int count, const void* const* d_x, const size_t* n,
+                                const float* const* d_clip, uint8_t* const* d_codes, float* const* d_scale,
+                                int8_t* const* d_operand, int dtype, cudaStream_t st) {
+  MultiInt4 a{};
+  size_t tiles[kMultiMax];
+  const bool bf = dtype == LUQ_BF16;
+  for (int t = 0; t < count; ++t) {
+    a.x[t] = d_x[t]; a.n[t] = n[t]; a.clip[t] = d_clip[t]; a.codes[t] = d_codes[t]; a.scale[t] = d_scale[t];
+    a.operand[t] = n[t] ? d_operand[t] : nullptr;
+    tiles[t] = n[t] / (bf ? 8 : 4) / kTileItems + 1;
+  }
+  a.count = count;
+  cudaError_t e;
+  if (bf) {
+    deal_blocks(ctx, quant_int4_multi_kernel<true>, count, tiles, a.first_block);
+    e = luq_launch_kernel(quant_int4_multi_kernel<true>, static_cast<int>(a.first_block[count]), kThreads, 0, st,
+                          LUQ_LAUNCH_EARLY, 1, a, ctx->d_status);
+  } else {
+    deal_blocks(ctx, quant_int4_multi_kernel<false>, count, tiles, a.first_block);
+    e = luq_launch_kernel(quant_int4_multi_kernel<false>, static_cast<int>(a.first_block[count]), kThreads, 0, st,
+                          LUQ_LAUNCH_EARLY, 1, a, ctx->d_status);
   }
   ctx->launches += 1;
   return static_cast<int>(e);
