@@ -320,17 +320,38 @@ def run_ours(args):
     sampler = ClockSampler(gpu_physical_index(local))
     sampler.start()
     sampler.ready.wait(10.0)
-    # The timed region: K steps, two events around the whole of it.
+    # No call of the path allocates or synchronises with the host, so one step is captured in a CUDA
+    # graph and replayed: the small configurations are bound by launch rate otherwise.
     launches0 = ctx.launches
+    step()
+    launches_per_step = ctx.launches - launches0
+    run_step, launch_mode = step, "direct calls"
+    if not args.no_graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    step()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            run_step, launch_mode = graph.replay, "CUDA graph of the step's calls, replayed"
+        except Exception as e:  # pragma: no cover
+            launch_mode = f"direct calls (graph capture failed: {e!r})"
+    # The timed region: K steps, two events around the whole of it.
     barrier()
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(args.steps):
-        step()
+        run_step()
     t1.record()
     barrier()
     total_ms = t0.elapsed_time(t1)
-    launches = ctx.launches - launches0
+    launches = launches_per_step * args.steps
     total_ms = replicas.max_over_ranks(total_ms, dev)
     assert ctx.status() == 0
     ms_per_step = total_ms / args.steps
@@ -471,6 +492,7 @@ def run_ours(args):
             "config": {"workload": f"{args.workload}: M={M} K={K} N={N}, {cfg.dtype} inputs, "
                                    f"LUQ seed {seed}, {ns} sample(s)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "launch": launch_mode,
                        "l2": "inputs (%d MB of activations per step) against a 126 MB L2; no explicit flush" % (A.numel() * A.element_size() >> 20)},
             "luq_quantizer_gbs": kernels["quant_grad_G"]["gbs"],
             "amax_plus_luq_gbs": round((alg["amax_G"][0] + alg["quant_grad_G"][0]) /
@@ -494,6 +516,7 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD, choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"],
                     help="layer shape (the headline number is cfg2), or cfg4 = the quantizer bandwidth sweep")
     ap.add_argument("--rows", type=int, default=None, help="truncate the batch dimension M (small profiling runs)")
+    ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of a replayed CUDA graph")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs")
     ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1, 2],
                     help="tensor-core operand type: 0 e4m3 (kind::f8f6f4), 1 int8 (kind::i8), 2 per product; default: the library's")

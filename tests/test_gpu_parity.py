@@ -559,3 +559,45 @@ def test_an_expired_wait_is_reported_and_the_context_stays_usable(ctx):
     _, fused, _ = ctx.amax_quant_grad(x, 3, 1)     # also the kernels that share the scratch counters
     assert torch.equal(before, after) and torch.equal(before, fused)
     assert ctx.status() == 0
+
+
+def test_a_step_can_be_captured_in_a_cuda_graph(ctx):
+    """No call of the path allocates or synchronises with the host, so a whole step can be captured
+    once and replayed; the replay must leave what the direct calls leave."""
+    cfg = inputs.CONFIGS["cfg1"]
+    A, W, G = inputs.layer_inputs(cfg)
+    M, K, N, ns = cfg.M, cfg.K, cfg.N, 2
+    Ad, Wd, Gd = to_dev(A), to_dev(W), to_dev(G)
+    f32 = lambda *s: torch.empty(s, dtype=torch.float32, device="cuda")   # noqa: E731
+    u8 = lambda *s: torch.empty(s, dtype=torch.uint8, device="cuda")      # noqa: E731
+    mA, mW, mG, sA, sW, aG = (f32(1) for _ in range(6))
+    cA, cW, cG = u8(M * K // 2), u8(N * K // 2), u8(ns, M * N // 2)
+    bW, bG = torch.empty(N * K, dtype=torch.int8, device="cuda"), torch.empty(ns * M * N, dtype=torch.int8, device="cuda")
+    Z, dA, dW = f32(M, N), f32(M, K), f32(N, K)
+
+    def step():
+        ctx.amax_multi([Ad, Wd], [mA, mW])
+        ctx.quant_int4_multi([Ad, Wd], [mA, mW], [cA, cW], [sA, sW], [None, bW])
+        ctx.gemm_fwd(cA, sA, cW, sW, M, N, K, Z, None, bW)
+        ctx.amax_quant_grad(Gd, 5, ns, mG, cG, aG, bG)
+        ctx.gemm_bwd(cG, aG, ns, cW, sW, M, N, K, dA, bG, bW)
+        ctx.gemm_wgrad(cG, aG, ns, cA, sA, M, N, K, dW, bG, None)
+
+    step()
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (cA, cW, cG, Z, dA, dW)]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()                                   # warm up on the capture stream
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+        for t in (cA, cW, cG, Z, dA, dW):
+            t.zero_()
+        for _ in range(3):
+            graph.replay()
+    torch.cuda.synchronize()
+    for got, ref in zip((cA, cW, cG, Z, dA, dW), want):
+        assert torch.equal(got, ref)
+    assert ctx.status() == 0
