@@ -320,21 +320,45 @@ def run_ours(args):
     sampler = ClockSampler(gpu_physical_index(local))
     sampler.start()
     sampler.ready.wait(10.0)
+    # The gradient's max and LUQ pass depend on nothing the forward half of the step produces.  With
+    # --streams 2 (the default) they run on a second stream, through a second context (a context's
+    # scratch and workspace serve one stream at a time), beside the activation/weight quantizers and the
+    # forward GEMM; the backward and update GEMMs wait for both.
+    ctx_g = binding.Context(local) if args.streams == 2 else ctx
+    if args.mma_kind is not None and ctx_g is not ctx:
+        ctx_g.set_option(binding.OPT_MMA_KIND, args.mma_kind)
+    stream_g = torch.cuda.Stream() if args.streams == 2 else None
+
+    def timed_step():
+        if stream_g is None:
+            return step()
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event(); fork.record(main)
+        stream_g.wait_event(fork)
+        with torch.cuda.stream(stream_g):
+            ctx_g.amax(G, mG); ctx_g.quant_grad(G, mG, seed, ns, cG, aG, oG)
+            join = torch.cuda.Event(); join.record(stream_g)
+        for name in ("amax_A", "amax_W", "quant_int4_A", "quant_int4_W", "gemm_fwd"):
+            calls[name]()
+        main.wait_event(join)
+        calls["gemm_bwd"](); calls["gemm_wgrad"]()
+
     # No call of the path allocates or synchronises with the host, so one step is captured in a CUDA
     # graph and replayed: the small configurations are bound by launch rate otherwise.
-    launches0 = ctx.launches
-    step()
-    launches_per_step = ctx.launches - launches0
-    run_step, launch_mode = step, "direct calls"
+    launches0 = ctx.launches + (ctx_g.launches if ctx_g is not ctx else 0)
+    timed_step()
+    launches_per_step = ctx.launches + (ctx_g.launches if ctx_g is not ctx else 0) - launches0
+    run_step, launch_mode = timed_step, "direct calls"
     if not args.no_graph:
         try:
             side = torch.cuda.Stream()
             side.wait_stream(torch.cuda.current_stream())
             with torch.cuda.stream(side):
-                step()
+                timed_step()
+                torch.cuda.synchronize()
                 graph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(graph, stream=side):
-                    step()
+                    timed_step()
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
             graph.replay()
@@ -353,12 +377,18 @@ def run_ours(args):
     total_ms = t0.elapsed_time(t1)
     launches = launches_per_step * args.steps
     total_ms = replicas.max_over_ranks(total_ms, dev)
-    assert ctx.status() == 0
+    assert ctx.status() == 0 and ctx_g.status() == 0
     ms_per_step = total_ms / args.steps
     # The same K steps once more with an event pair around every call, for the per-kernel
     # durations (the 18 extra event records per step lengthen a step, so this pass is not
     # the one the throughput comes from).
     events = {k: [] for k in KERNELS}
+    # 27 host calls per step here: on the short configurations the host would fall behind the GPU and
+    # the idle time would be booked on the kernels.  Hold the GPU back while the host queues the pass.
+    try:
+        torch.cuda._sleep(int(args.steps * 0.35e-3 * 2.0e9))
+    except Exception:  # pragma: no cover
+        pass
     t0.record()
     for _ in range(args.steps):
         step(events)
@@ -493,6 +523,8 @@ def run_ours(args):
                                    f"LUQ seed {seed}, {ns} sample(s)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                        "launch": launch_mode,
+                       "streams": "2: gradient max + LUQ beside the activation/weight quantizers and the forward GEMM"
+                                  if args.streams == 2 else "1",
                        "l2": "inputs (%d MB of activations per step) against a 126 MB L2; no explicit flush" % (A.numel() * A.element_size() >> 20)},
             "luq_quantizer_gbs": kernels["quant_grad_G"]["gbs"],
             "amax_plus_luq_gbs": round((alg["amax_G"][0] + alg["quant_grad_G"][0]) /
@@ -502,6 +534,8 @@ def run_ours(args):
             "gpu_launches": int(launches), "clocks": clocks_summary,
         }
         print(json.dumps(line))
+    if ctx_g is not ctx:
+        ctx_g.close()
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
@@ -516,6 +550,8 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD, choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"],
                     help="layer shape (the headline number is cfg2), or cfg4 = the quantizer bandwidth sweep")
     ap.add_argument("--rows", type=int, default=None, help="truncate the batch dimension M (small profiling runs)")
+    ap.add_argument("--streams", type=int, choices=(1, 2), default=2,
+                    help="2: the gradient's max and LUQ pass run on a second stream beside the forward half")
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of a replayed CUDA graph")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs")
     ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1, 2],
