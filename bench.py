@@ -508,7 +508,7 @@ def run_ours(args):
         torch.cuda.empty_cache()
 
     if rank == 0 and world == 1 and not args.kernel_only:
-        rows = min(2048, M)
+        rows = min(32768, M)   # about 15 s of host time on config 2
         dt, fl, threads = oracle_sample(cfg, rows, ns)
         cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": f"first {rows} of {M} batch rows, all nine stages, {dt:.2f} s"}
