@@ -94,9 +94,12 @@ extern "C" {
 
 typedef struct luq_ctx luq_ctx;
 
-/* Creates a context on `device`: a device status word and the split workspace
- * (96 MiB: partial tiles of split contractions and 8-bit operand planes of the GEMMs).
- * Allocates device memory; call outside stream capture. */
+/* Creates a context on `device`: a device status word, 48 KB of scratch words for grid-wide
+ * maxima, and the workspace (96 MiB: partial tiles of split contractions and 8-bit operand
+ * planes that a GEMM expands itself when the caller passes none).  Allocates device memory;
+ * call outside stream capture.  Every other call of the library allocates nothing and does
+ * not synchronise with the host (luq_status excepted), so a sequence of calls can be captured
+ * in a CUDA graph.  Two streams that run calls concurrently need two contexts. */
 int luq_create(luq_ctx** out, int device);
 int luq_destroy(luq_ctx* ctx);
 int luq_set_option(luq_ctx* ctx, int option, int value);
