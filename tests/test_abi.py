@@ -31,6 +31,28 @@ def test_every_declared_symbol_is_exported(lib):
         assert getattr(lib, n) is not None
 
 
+def declared_arities():
+    """Parameter count of every prototype in the header."""
+    text = open(os.path.join(ROOT, "include", "luq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    out = {}
+    for name, params in re.findall(r"\b(luq_[a-z0-9_]+)\s*\(([^;{]*?)\)\s*;", text, flags=re.S):
+        params = params.strip()
+        out[name] = 0 if params in ("", "void") else params.count(",") + 1
+    return out
+
+
+def test_binding_marshals_as_many_arguments_as_the_header_declares(lib):
+    """The Python binding sets ctypes argtypes for every entry point; a prototype that gains or loses
+    a parameter without the binding following would corrupt the call silently."""
+    arities = declared_arities()
+    assert set(arities) == set(binding.SYMBOLS)
+    for name, count in arities.items():
+        argtypes = getattr(lib, name).argtypes
+        assert argtypes is not None, name
+        assert len(argtypes) == count, (name, len(argtypes), count)
+
+
 def test_constants_and_messages(lib):
     assert lib.luq_kmax() == 4
     assert lib.luq_strerror(0) == b"ok"
