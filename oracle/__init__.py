@@ -66,6 +66,11 @@ def lib() -> ctypes.CDLL:
             L.oracle_quant_luq_window.restype = ctypes.c_float
             L.oracle_quant_fp_nearest.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, u8p, intp]
             L.oracle_quant_fp_nearest.restype = ctypes.c_float
+            L.oracle_quant_fp_ablation.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_int, ctypes.c_uint64,
+                                                   ctypes.c_int, ctypes.c_int, ctypes.c_int, u8p, intp]
+            L.oracle_quant_fp_ablation.restype = ctypes.c_float
+            L.oracle_quant_int4_sr.argtypes = [f32p, sz, ctypes.c_float, ctypes.c_uint64, ctypes.c_int, u8p, intp]
+            L.oracle_quant_int4_sr.restype = ctypes.c_float
             L.oracle_pw2_ceil.argtypes = [ctypes.c_float]
             L.oracle_pw2_ceil.restype = ctypes.c_float
             L.oracle_hindsight_next.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float]
@@ -169,6 +174,30 @@ def quant_fp_nearest(x: np.ndarray, mx, kmax: int = KMAX_DEFAULT):
     a = lib().oracle_quant_fp_nearest(_ptr(xf, ctypes.c_float), xf.size, np.float32(mx), kmax,
                                       _ptr(codes, ctypes.c_uint8), ctypes.byref(flags))
     return codes, np.float32(a), flags.value
+
+
+def quant_fp_ablation(x: np.ndarray, mx, seed: int, sr: bool, su: bool, n_samples: int = 1,
+                      kmax: int = KMAX_DEFAULT):
+    """The ablation's partially unbiased arms on the LUQ grid: `sr` = stochastic rounding inside the
+    range, `su` = stochastic underflow below it, the other region deterministic (nearest).
+    Returns (codes[n_samples, n/2], alpha, flags)."""
+    xf = widen(x).reshape(-1)
+    codes = np.zeros((n_samples, (xf.size + 1) // 2), dtype=np.uint8)
+    flags = ctypes.c_int(0)
+    a = lib().oracle_quant_fp_ablation(_ptr(xf, ctypes.c_float), xf.size, np.float32(mx), kmax, seed, n_samples,
+                                       int(bool(sr)), int(bool(su)), _ptr(codes, ctypes.c_uint8), ctypes.byref(flags))
+    return codes, np.float32(a), flags.value
+
+
+def quant_int4_sr(x: np.ndarray, mx, seed: int, n_samples: int = 1):
+    """The ablation's "INT4 unbiased" arm: grid -7..7 with step max/7 and stochastic rounding (Eq. SR).
+    Returns (codes[n_samples, n/2] as INT4 nibbles, scale, flags)."""
+    xf = widen(x).reshape(-1)
+    codes = np.zeros((n_samples, (xf.size + 1) // 2), dtype=np.uint8)
+    flags = ctypes.c_int(0)
+    s = lib().oracle_quant_int4_sr(_ptr(xf, ctypes.c_float), xf.size, np.float32(mx), seed, n_samples,
+                                   _ptr(codes, ctypes.c_uint8), ctypes.byref(flags))
+    return codes, np.float32(s), flags.value
 
 
 def pw2_ceil(mx) -> np.float32:

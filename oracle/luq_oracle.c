@@ -261,6 +261,91 @@ float oracle_quant_fp_nearest(const float* x, size_t n, float mx, int kmax, uint
 }
 
 /* ------------------------------------------------------------------------ */
+/* Partially unbiased arms of the ablation (Sec. 4, ablation figure and its    */
+/* caption): "SR" makes the quantizer unbiased inside the range, "SU" below     */
+/* it.  The grid, the scale alpha = max/2^kmax and the code layout are LUQ's;   */
+/* each region follows either the stochastic rule or the deterministic one:    */
+/*   |x| <  alpha : su ? sign*alpha w.p. |x|/alpha (Eq. StochasticPruning)      */
+/*                     : the nearer of 0 and alpha, alpha/2 up                   */
+/*   in range     : sr ? up w.p. (|x| - lo)/lo (Eq. unbiasedFpQ)                 */
+/*                     : nearest power, midpoint 3/2 * 2^n up (Eq. RC)           */
+/* sr and su both set is LUQ, both clear is the biased "FP4" baseline.          */
+/* Reading: the paper names the arms and draws them, it does not print them.    */
+/* ------------------------------------------------------------------------ */
+float oracle_quant_fp_ablation(const float* x, size_t n, float mx, int kmax, uint64_t seed, int n_samples,
+                               int sr, int su, uint8_t* codes, int* flags) {
+  size_t plane = (n + 1) / 2;
+  memset(codes, 0, plane * (size_t)n_samples);
+  if (!scale_usable(mx, flags)) return 0.0f;
+  float alpha = oracle_luq_alpha(mx, kmax);
+  float top = ldexpf(1.0f, kmax);
+  for (int s = 0; s < n_samples; ++s) {
+    uint8_t* out = codes + plane * (size_t)s;
+    for (size_t i = 0; i < n; ++i) {
+      float t = fabsf(x[i]) / alpha; /* IEEE binary32 quotient, as in LUQ */
+      uint32_t sign = bits_of(x[i]) >> 31;
+      uint32_t r = oracle_random_word(seed, (uint32_t)s, (uint64_t)i);
+      uint32_t c;
+      if (!(t < top)) {                /* top level, Inf, NaN: nothing to decide */
+        c = (uint32_t)kmax + 1u;
+      } else if (t < 1.0f) {           /* below the range */
+        if (su) c = (r < (uint32_t)(t * 4294967296.0f)) ? 1u : 0u;
+        else c = (t >= 0.5f) ? 1u : 0u;
+      } else {                         /* 2^e <= t < 2^(e+1), level codes e+1 and e+2 */
+        int e = 0;
+        while (ldexpf(1.0f, e + 1) <= t) ++e;
+        float lo = ldexpf(1.0f, e);
+        int up;
+        if (sr) {
+          /* (t - lo)/lo is exact in binary32: t - lo is exact and lo a power of two */
+          float p = (t - lo) / lo;
+          up = r < (uint32_t)(p * 4294967296.0f);
+        } else {
+          up = t >= 1.5f * lo;
+        }
+        c = (uint32_t)(e + 1 + up);
+      }
+      uint8_t nib = c ? (uint8_t)((sign << 3) | c) : 0;
+      out[i >> 1] |= (uint8_t)(nib << ((i & 1) * 4));
+    }
+  }
+  return alpha;
+}
+
+/* ------------------------------------------------------------------------ */
+/* "INT4 unbiased" arm of the ablation: the uniform signed grid -7..7 with     */
+/* stochastic rounding (Sec. 3.1, Eq. SR: up w.p. (x - l)/(u - l)).  The top    */
+/* level is the tensor maximum, so nothing clips: s = max/7.  Taken on the     */
+/* magnitude (the rule is symmetric): y = fl32(|x| * fl32(7/max)), clamped to   */
+/* 7; l = floor(y); up w.p. y - l, decided as r < trunc((y - l) * 2^32);        */
+/* the sign is applied afterwards, the code is the two's-complement nibble.    */
+/* The random word of element i, sample s is the one LUQ would use.            */
+/* ------------------------------------------------------------------------ */
+float oracle_quant_int4_sr(const float* x, size_t n, float mx, uint64_t seed, int n_samples,
+                           uint8_t* codes, int* flags) {
+  size_t plane = (n + 1) / 2;
+  memset(codes, 0, plane * (size_t)n_samples);
+  if (!scale_usable(mx, flags)) return 0.0f;
+  float s7 = mx / 7.0f;
+  float inv = 7.0f / mx;
+  for (int s = 0; s < n_samples; ++s) {
+    uint8_t* out = codes + plane * (size_t)s;
+    for (size_t i = 0; i < n; ++i) {
+      float y = fabsf(x[i]) * inv;
+      if (y != y) y = 0.0f;          /* NaN element -> 0 */
+      if (y > 7.0f) y = 7.0f;
+      float l = floorf(y);
+      float frac = y - l;            /* exact: same binade or below, l <= y */
+      uint32_t r = oracle_random_word(seed, (uint32_t)s, (uint64_t)i);
+      int m = (int)l + (r < (uint32_t)(frac * 4294967296.0f) ? 1 : 0);
+      int q = (bits_of(x[i]) >> 31) ? -m : m;
+      out[i >> 1] |= (uint8_t)((q & 0xF) << ((i & 1) * 4));
+    }
+  }
+  return s7;
+}
+
+/* ------------------------------------------------------------------------ */
 /* Power-of-two LUQ (Appendix A.7): alpha_PW2 = 2^ceil(log2 max|x|) / 2^kmax. */
 /* The maximum is rounded UP to a power of two (so nothing is clipped), the   */
 /* quantizer itself is unchanged; every level is then a power of two.         */

@@ -751,3 +751,161 @@ def test_uint4_grid_error_bound_and_edges():
     for bad, flag in ((0.0, 0), (np.inf, oracle.FLAG_NONFINITE), (1e-35, oracle.FLAG_RANGE)):
         cb, sb, fb = oracle.quant_uint4(x[:10], np.float32(bad))
         assert sb == 0 and not cb.any() and fb == flag
+
+
+# ------------------------------------------ ablation arms (Sec. 4, ablation figure) ----
+
+
+def test_ablation_arms_reduce_to_luq_and_to_the_biased_baseline_region_by_region():
+    """SR+SU is LUQ, neither is the deterministic baseline; a mixed arm has LUQ's codes in its
+    stochastic region and the baseline's in the other."""
+    for kmax in (2, 4):
+        x = luq_test_tensor(seed=91, n=6000)
+        mx, _ = oracle.amax(x)
+        alpha = oracle.luq_alpha(mx, kmax)
+        luq, a0, _ = oracle.quant_luq(x, mx, seed=5, n_samples=2, kmax=kmax)
+        near, _, _ = oracle.quant_fp_nearest(x, mx, kmax=kmax)
+        both, a1, _ = oracle.quant_fp_ablation(x, mx, 5, True, True, n_samples=2, kmax=kmax)
+        none, _, _ = oracle.quant_fp_ablation(x, mx, 5, False, False, n_samples=2, kmax=kmax)
+        assert a0 == a1 == alpha
+        np.testing.assert_array_equal(both, luq)
+        np.testing.assert_array_equal(none[0], near[0])
+        np.testing.assert_array_equal(none[1], near[0])           # no randomness: every sample equal
+        below = np.abs(x) < alpha
+        assert below.sum() > 100 and (~below).sum() > 100
+        for sr, su in ((True, False), (False, True)):
+            got, _, _ = oracle.quant_fp_ablation(x, mx, 5, sr, su, n_samples=2, kmax=kmax)
+            for s in range(2):
+                g = oracle.unpack(got[s], x.size)
+                l = oracle.unpack(luq[s], x.size)
+                d = oracle.unpack(near[0], x.size)
+                np.testing.assert_array_equal(g[below], (l if su else d)[below])
+                np.testing.assert_array_equal(g[~below], (l if sr else d)[~below])
+
+
+def test_ablation_arms_are_unbiased_exactly_where_the_caption_says():
+    """"FP4+SR" is unbiased inside the range and biased below it; stochastic underflow alone the
+    other way round.  The deterministic region's error is the nearest-level error, the same for
+    every seed."""
+    kmax = 4
+    x = inputs.log_uniform_magnitudes(384, -9, 0, 71)
+    mx, _ = oracle.amax(x)
+    alpha = float(oracle.luq_alpha(mx, kmax))
+    below = np.abs(x) < alpha
+    assert below.sum() > 60 and (~below).sum() > 60
+    S = 1500
+    lo, hi, _ = oracle.luq_bins(x, mx, kmax)
+    ax = np.abs(x).astype(np.float64)
+    var_closed = np.maximum((ax - lo * alpha) * (hi * alpha - ax), 0)     # Table 1: Var[SR]
+    for sr, su in ((True, False), (False, True)):
+        acc = np.zeros(x.size)
+        first = None
+        for seed in range(S):
+            codes, a, _ = oracle.quant_fp_ablation(x, mx, seed, sr, su, kmax=kmax)
+            v, _ = decode_luq(codes[0], x.size, a)
+            acc += v
+            if first is None:
+                first = v
+            det = ~below if su else below
+            assert (v[det] == first[det]).all()                            # the deterministic region never moves
+        mean = acc / S
+        sto = below if su else ~below
+        z = np.abs(mean - x)[sto] / np.sqrt(var_closed[sto] / S + 1e-300)
+        assert (z[var_closed[sto] > 0] < 5.5).all()
+        # deterministic region: nearest level, so the error is min(x - l, u - x) (Table 1: Bias[RDN])
+        det = ~sto
+        bias = np.abs(mean - x)[det]
+        want = np.minimum(ax - lo * alpha, hi * alpha - ax)[det]
+        assert np.allclose(bias, want, rtol=1e-5, atol=1e-12)
+        assert bias.max() > 0.1 * alpha
+
+
+def decode_int4(codes, n, s):
+    q = oracle.unpack(codes, n).astype(np.int64)
+    q = np.where(q >= 8, q - 16, q)
+    return q * float(s), q
+
+
+def test_int4_sr_brackets_fixed_points_and_symmetry():
+    rng = np.random.default_rng(17)
+    x = rng.standard_normal(20000).astype(np.float32)
+    mx, _ = oracle.amax(x)
+    codes, s, fl = oracle.quant_int4_sr(x, mx, seed=3, n_samples=2)
+    assert fl == 0 and s == np.float32(mx) / np.float32(7)
+    for p in range(2):
+        v, q = decode_int4(codes[p], x.size, s)
+        assert np.abs(q).max() == 7 and (np.abs(v - x) < float(s) * (1 + 1e-6)).all()   # floor or ceiling of x/s
+        assert (np.sign(v) * np.sign(x) >= 0).all()                                    # never crosses zero
+    assert (codes[0] != codes[1]).any()
+    # the maximum itself takes +-7 with every seed, on-grid values are fixed points, zero stays zero
+    g = (np.arange(-7, 8, dtype=np.float32) * np.float32(0.5))
+    g = np.concatenate([g, np.float32([0.0])])
+    for seed in range(30):
+        cg, sg, _ = oracle.quant_int4_sr(g, np.float32(3.5), seed)
+        vg, _ = decode_int4(cg[0], g.size, sg)
+        np.testing.assert_array_equal(vg, g.astype(np.float64))
+    # Q(-x) = -Q(x) with the same random words
+    cn, _, _ = oracle.quant_int4_sr(-x, mx, seed=3)
+    vn, _ = decode_int4(cn[0], x.size, s)
+    vp, _ = decode_int4(codes[0], x.size, s)
+    np.testing.assert_array_equal(vn, -vp)
+    # values beyond a smaller caller-supplied maximum clamp to the top level; NaN goes to zero
+    y = np.array([9.0, -9.0, np.nan, 7.0, -7.0, 0.25], dtype=np.float32)
+    cy, sy, _ = oracle.quant_int4_sr(y, np.float32(7.0), seed=1)
+    _, qy = decode_int4(cy[0], y.size, sy)
+    assert sy == 1.0 and list(qy[:5]) == [7, -7, 0, 7, -7] and qy[5] in (0, 1)
+    for bad, flag in ((0.0, 0), (np.inf, oracle.FLAG_NONFINITE), (1e-35, oracle.FLAG_RANGE)):
+        cb, sb, fb = oracle.quant_int4_sr(x[:10], np.float32(bad), seed=1)
+        assert sb == 0 and not cb.any() and fb == flag
+
+
+def test_int4_sr_follows_the_random_word_and_is_exactly_half_at_midpoints():
+    x = np.array([0.5, 1.5, -2.5, 0.25, 6.75, -0.125, 3.0], dtype=np.float32)
+    mx = np.float32(7.0)                                                    # s = 1: fractions are exact
+    frac = np.abs(x) - np.floor(np.abs(x))
+    for seed in (0, 9, 123456789):
+        codes, s, _ = oracle.quant_int4_sr(x, mx, seed, n_samples=2)
+        for p in range(2):
+            words = np.array([oracle.random_word(seed, p, i) for i in range(x.size)], dtype=np.float64)
+            up = words < frac * 2.0 ** 32
+            _, q = decode_int4(codes[p], x.size, s)
+            np.testing.assert_array_equal(np.abs(q), np.floor(np.abs(x)) + up)
+    # over many seeds a midpoint goes up half of the time, a quarter point a quarter of the time
+    ups = np.zeros(x.size)
+    S = 4000
+    for seed in range(S):
+        codes, s, _ = oracle.quant_int4_sr(x, mx, seed)
+        _, q = decode_int4(codes[0], x.size, s)
+        ups += np.abs(q) > np.floor(np.abs(x))
+    p_hat = ups / S
+    assert (np.abs(p_hat - frac) < 5 * np.sqrt(frac * (1 - frac) / S) + 1e-12).all()
+
+
+def test_int4_sr_unbiased_with_table1_variance_and_twice_the_rdn_error():
+    """Eq. SR: E[SR(x)] = x and Var = (x - l)(u - x); Table 1: MSE[SR] >= MSE[RDN] - on fractions
+    spread evenly over the bins E[f(1-f)] = 1/6 against E[min(f,1-f)^2] = 1/12, a factor of two."""
+    rng = np.random.default_rng(23)
+    x = rng.uniform(-1, 1, 600).astype(np.float32)
+    x[0] = 1.0
+    mx, _ = oracle.amax(x)
+    S = 1500
+    acc = np.zeros(x.size)
+    acc2 = np.zeros(x.size)
+    s = None
+    for seed in range(S):
+        codes, s, _ = oracle.quant_int4_sr(x, mx, seed)
+        v, _ = decode_int4(codes[0], x.size, s)
+        acc += v
+        acc2 += (v - x) ** 2
+    mean = acc / S
+    y = np.abs(x).astype(np.float64) / float(s)
+    f = y - np.floor(y)
+    var_closed = f * (1 - f) * float(s) ** 2
+    z = np.abs(mean - x) / np.sqrt(var_closed / S + 1e-300)
+    assert (z[var_closed > 1e-12] < 5.5).all()
+    assert abs((acc2 / S).sum() / var_closed.sum() - 1) < 0.05
+    crn, srn, _ = oracle.quant_int4(x, mx)
+    vr, _ = decode_int4(crn, x.size, srn)
+    mse_rdn = ((vr - x) ** 2).mean()
+    mse_sr = (acc2 / S).mean()
+    assert abs(mse_sr / mse_rdn - 2.0) < 0.2
