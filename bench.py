@@ -218,7 +218,13 @@ def run_sweep(args, binding, inputs, torch, local):
                     ("hindsight_pw2", lambda: ctx.quant_grad_hindsight(x, mh, 0.1, 0, ns, True, codes, al, mx), (4 + 0.5 * ns) * n),
                     ("amax_plus_pw2", lambda: (ctx.amax(x, mx), ctx.quant_grad_pw2(x, mx, 0, ns, codes, al)), (8 + 0.5 * ns) * n),
                     # deterministic round-to-nearest-power (the biased FP4 baseline): no generator, one plane
-                    ("amax_plus_nearest", lambda: (ctx.amax(x, mx), ctx.quant_grad_nearest(x, mx, codes, al)), 8.5 * n)):
+                    ("amax_plus_nearest", lambda: (ctx.amax(x, mx), ctx.quant_grad_nearest(x, mx, codes, al)), 8.5 * n),
+                    # the ablation's other arms (quantizer alone, max given): one region of the LUQ grid
+                    # deterministic, and the uniform grid with stochastic rounding
+                    ("ablation_fp4_sr", lambda: ctx.quant_grad_ablation(x, mx, 0, binding.SCHEME_FP4_SR, ns, codes, al),
+                     (4 + 0.5 * ns) * n),
+                    ("ablation_int4_sr", lambda: ctx.quant_grad_ablation(x, mx, 0, binding.SCHEME_INT4_SR, ns, codes, al),
+                     (4 + 0.5 * ns) * n)):
                 ts = []
                 for it in range(reps + 3):
                     flush.fill_(it & 0xFF)

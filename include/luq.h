@@ -72,6 +72,11 @@ extern "C" {
                               nearest even) instead of fp32: half the output traffic, which is what bounds the
                               backward product of a wide layer.  The output's row length must then be a
                               multiple of 8 elements.  Not available in luq_gemm_wgrad_static. */
+#define LUQ_OPT_GRADIENT_INT4 7 /* 1: the gradient codes handed to luq_gemm_bwd / luq_gemm_wgrad are signed INT4
+                              (from luq_quant_grad_ablation with LUQ_SCHEME_INT4_SR; d_alpha is then its
+                              scale max/7).  Such an operand is fetched as bytes: the caller's operand bytes,
+                              or a plane expanded into the context workspace (LUQ_ERR_WORKSPACE beyond 76 MiB).
+                              Not available in luq_gemm_wgrad_static. */
 #define LUQ_OPT_LEVELS 4   /* kmax of the gradient quantizers, 1..6 (default luq_kmax() = 4): levels
                               alpha * 2^0 .. alpha * 2^kmax with alpha = max / 2^kmax, codes 0..kmax+1.  The
                               other grids of the paper from the same kernels: kmax = 2 is the FP2 grid of
@@ -181,6 +186,34 @@ int luq_amax_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, s
 int luq_quant_grad_nearest(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
                            const float* d_amax, uint8_t* d_codes, float* d_alpha, int8_t* d_operand,
                            void* stream);
+
+/* The other gradient quantizers of the paper's ablation (Sec. 4, ablation figure and caption; the
+ * paper names and draws these arms, it does not print them - the readings are stated here).
+ * `scheme` says which region of the LUQ grid is stochastic:
+ *   LUQ_SCHEME_FP4      neither: the biased baseline, the same codes as luq_quant_grad_nearest
+ *   LUQ_SCHEME_FP4_SR   stochastic rounding inside the range (Eq. unbiasedFpQ); below alpha the
+ *                       nearer of 0 and alpha ("FP4 + SR": unbiased inside the range only)
+ *   LUQ_SCHEME_FP4_SU   stochastic underflow below alpha (Eq. StochasticPruning); inside the range
+ *                       round-to-nearest-power (Eq. RC)
+ *   LUQ_SCHEME_LUQ      both: the codes of luq_quant_grad (with the scale of Eq. alpha this is
+ *                       LUQ itself; the figure's "FP4 + SR + SU" arm must differ from it by a
+ *                       range the paper does not give)
+ *   LUQ_SCHEME_INT4_SR  "INT4 unbiased": the uniform grid -7..7 with step max/7 and stochastic
+ *                       rounding (Sec. 3.1, Eq. SR) of the magnitude: y = |x| * fl(7/max), up from
+ *                       floor(y) when word < trunc((y - floor(y)) * 2^32), sign applied afterwards.
+ *                       Codes are INT4 nibbles (two's complement), operand bytes 16 * q, *d_scale
+ *                       receives max/7; elements beyond a smaller caller-supplied maximum take +-7.
+ * For the first four, grid, level count (LUQ_OPT_LEVELS), scale (*d_scale receives alpha), code
+ * layout, sample planes and random words are those of luq_quant_grad.  To multiply with
+ * LUQ_SCHEME_INT4_SR codes set LUQ_OPT_GRADIENT_INT4.  One plain streaming kernel per call. */
+#define LUQ_SCHEME_FP4 0
+#define LUQ_SCHEME_FP4_SR 1
+#define LUQ_SCHEME_FP4_SU 2
+#define LUQ_SCHEME_LUQ 3
+#define LUQ_SCHEME_INT4_SR 4
+int luq_quant_grad_ablation(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols,
+                            const float* d_amax, uint64_t seed, int n_samples, int scheme,
+                            uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
 
 /* LUQ with a power-of-two scale (Appendix A.7, LUQ_PW2): as luq_quant_grad, but
  * alpha = 2^ceil(log2 max) / 2^kmax - the maximum is rounded UP to a power of two,

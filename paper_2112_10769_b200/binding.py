@@ -18,10 +18,12 @@ LIB_PATH = os.path.join(_HERE, "libluq_b200.so")
 LUQ_F32, LUQ_BF16 = 0, 1
 STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT = 1, 2, 4
 OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS, OPT_UNSIGNED_ACTIVATIONS, OPT_OUTPUT_BF16 = 1, 2, 3, 4, 5, 6
+OPT_GRADIENT_INT4 = 7
+SCHEME_FP4, SCHEME_FP4_SR, SCHEME_FP4_SU, SCHEME_LUQ, SCHEME_INT4_SR = 0, 1, 2, 3, 4
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_pw2",
+           "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_ablation", "luq_quant_grad_pw2",
            "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_debug_expire_wait", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
@@ -55,6 +57,7 @@ def load() -> ctypes.CDLL:
         L.luq_amax_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, u64, ctypes.c_int, vp, vp, vp, vp, vp]
         L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_nearest.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
+        L.luq_quant_grad_ablation.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, ctypes.c_int, u64,
                                                ctypes.c_int, vp, vp, vp, vp, vp]
@@ -244,6 +247,21 @@ class Context:
                                              codes.data_ptr(), alpha.data_ptr(), _opt(operand, g.numel()),
                                              _stream()), "luq_quant_grad_nearest")
         return codes, alpha
+
+    def quant_grad_ablation(self, g: torch.Tensor, amax: torch.Tensor, seed: int, scheme: int, n_samples: int = 1,
+                            codes: torch.Tensor | None = None, scale: torch.Tensor | None = None,
+                            operand: torch.Tensor | None = None):
+        """The ablation's other gradient quantizers (SCHEME_*): one region of the LUQ grid deterministic,
+        or the uniform INT4 grid with stochastic rounding.  Returns (codes[n_samples, n/2], scale)."""
+        rows, cols = (g.shape[0], g.numel() // max(g.shape[0], 1)) if g.dim() > 1 else (1, g.numel())
+        if codes is None:
+            codes = torch.empty((n_samples, g.numel() // 2), dtype=torch.uint8, device=g.device)
+        scale = torch.empty(1, dtype=torch.float32, device=g.device) if scale is None else scale
+        _check(load().luq_quant_grad_ablation(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
+                                              seed, n_samples, scheme, codes.data_ptr(), scale.data_ptr(),
+                                              _opt(operand, n_samples * g.numel()), _stream()),
+               "luq_quant_grad_ablation")
+        return codes, scale
 
     def quant_grad_pw2(self, g: torch.Tensor, amax: torch.Tensor, seed: int, n_samples: int = 1,
                        codes: torch.Tensor | None = None, alpha: torch.Tensor | None = None,

@@ -57,6 +57,7 @@ int luq_create(luq_ctx** out, int device) {
   c->use_pairs = 0;
   c->kmax = LUQ_KMAX;
   c->unsigned_act = 0;
+  c->grad_int4 = 0;
   c->out_bf16 = 0;
   c->launches = 0;
   c->workspace_bytes = kWorkspaceBytes;
@@ -104,6 +105,10 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
     case LUQ_OPT_UNSIGNED_ACTIVATIONS:
       if (value != 0 && value != 1) return LUQ_ERR_ARG;
       ctx->unsigned_act = value;
+      return LUQ_OK;
+    case LUQ_OPT_GRADIENT_INT4:
+      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      ctx->grad_int4 = value;
       return LUQ_OK;
     case LUQ_OPT_LEVELS:
       if (value < 1 || value > 6) return LUQ_ERR_ARG;
@@ -249,6 +254,19 @@ int luq_quant_grad_nearest(luq_ctx* ctx, const void* d_g, int dtype, size_t rows
                                           d_alpha, 4, nullptr, nullptr, 0.0f, nullptr, as_stream(stream)));
 }
 
+int luq_quant_grad_ablation(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
+                            uint64_t seed, int n_samples, int scheme, uint8_t* d_codes, float* d_scale,
+                            int8_t* d_operand, void* stream) {
+  size_t n = 0;
+  const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_scale, d_operand, &n);
+  if (rc) return rc;
+  if (scheme < 0 || scheme > LUQ_SCHEME_INT4_SR) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_grad_ablation(ctx, d_g, dtype, n, d_amax, seed, n_samples, scheme, d_codes,
+                                                n ? d_operand : nullptr, d_scale, as_stream(stream)));
+}
+
 int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
                        uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, int8_t* d_operand,
                        void* stream) {
@@ -329,7 +347,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   luq_gemm_args a{};
-  a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 0; a.n_samples = n_samples;   // G[M x N]: contraction n contiguous
+  a.a_codes = d_g_codes; a.a_kind = ctx->grad_int4 ? 0 : 1; a.a_mn = 0; a.n_samples = n_samples;   // G[M x N]: contraction n contiguous
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 1;                            // W[N x K]: rows are the contraction
   a.a_operand = d_g_operand; a.b_operand = d_w_operand;
   a.d_scale_a = d_alpha; a.d_scale_b = d_sw; a.d_out = d_da; a.out_bf16 = ctx->out_bf16; a.Mo = M; a.No = K; a.Kc = N;
@@ -347,7 +365,7 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   luq_gemm_args a{};
-  a.a_codes = d_g_codes; a.a_kind = 1; a.a_mn = 1; a.n_samples = n_samples;   // G[M x N]: rows are the contraction
+  a.a_codes = d_g_codes; a.a_kind = ctx->grad_int4 ? 0 : 1; a.a_mn = 1; a.n_samples = n_samples;   // G[M x N]: rows are the contraction
   a.b_codes = d_a_codes; a.b_kind = ctx->unsigned_act ? 2 : 0; a.b_mn = 1;    // A[M x K]: rows are the contraction
   a.a_operand = d_g_operand; a.b_operand = d_a_operand;
   a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.out_bf16 = ctx->out_bf16; a.Mo = N; a.No = K; a.Kc = M;

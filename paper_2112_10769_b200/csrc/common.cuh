@@ -21,6 +21,7 @@ struct luq_ctx {
   int use_pairs;            // CTA-pair kernel for products whose operands are both planes
   int out_bf16;             // the GEMMs write bf16 outputs
   int unsigned_act;         // activation codes handed to the forward / update GEMMs are unsigned INT4
+  int grad_int4;            // gradient codes handed to the backward / update GEMMs are INT4 (the ablation's uniform arm)
   int kmax;                 // LUQ levels alpha * 2^0 .. alpha * 2^kmax (1..6, default LUQ_KMAX)
   int64_t launches;
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved at create
@@ -40,6 +41,12 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
                              float* d_measured, float* d_estimate, float eta, float* d_amax_out, cudaStream_t st);
+// scheme: bit 0 = stochastic rounding inside the range, bit 1 = stochastic underflow, on the LUQ grid
+// (the other region rounds to the nearest level; d_scale gets alpha); 4 = the uniform grid -7..7 with
+// stochastic rounding (INT4 codes, d_scale gets max/7)
+int luq_launch_quant_grad_ablation(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
+                                   uint64_t seed, int n_samples, int scheme, uint8_t* d_codes, int8_t* d_operand,
+                                   float* d_scale, cudaStream_t st);
 // Scratch words for grid-wide maxima.  Words 0 .. LUQ_SCRATCH_SINGLE-1: the one-tensor kernels (two
 // counters + one word per block).  Then LUQ_SCRATCH_MULTI regions of LUQ_SCRATCH_REGION words, one per
 // tensor of a several-tensor launch.  Grids of the reducing kernels stay below the region sizes.

@@ -940,7 +940,9 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   const uint8_t* b_plane_ptr = nullptr; const uint8_t* a_plane_ptr = nullptr;
   // Unsigned INT4 codes (kind 2) have no expansion inside the GEMM kernels: such an operand is
   // always fetched as bytes, the caller's or a plane expanded here.
-  const bool b_must = a.b_kind == 2, a_must = a.a_kind == 2;
+  // The same holds for signed INT4 codes as the first operand of the backward / update products
+  // (the uniform arm of the gradient ablation): those kernels expand LUQ codes there.
+  const bool b_must = a.b_kind == 2, a_must = a.a_kind == 2 || (a.a_kind == 0 && (a.a_mn || a.b_mn));
   // (With bf16 outputs the output stream no longer hides the expansion: the caller's bytes are then
   // used for short contractions too - backward product of the ResNet shape 82 -> 65 us.)
   const bool use_given = a.out_bf16 != 0;

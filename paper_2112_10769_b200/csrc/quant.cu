@@ -706,6 +706,173 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
   }
 }
 
+// The other gradient quantizers of the ablation (Sec. 4, ablation figure), one plain streaming
+// kernel (no fused maximum, sample count read at run time): same pieces, stores, random words,
+// sample planes and short route as the LUQ kernel.
+//   UNIFORM = false: the LUQ grid with one region deterministic.  word_under / word_range replace
+//     the random word of an element below alpha / inside the range when non-zero; 0x7FFFFFFF makes
+//     that region round to the nearest level ("FP4 + SR": word_under set; stochastic underflow
+//     alone: word_range set).
+//   UNIFORM = true: "INT4 unbiased" - the grid -7..7 with step max/7 and stochastic rounding of
+//     the magnitude: y = |x| * fl(7/max) clamped to 7, l = floor(y), up when word < trunc((y-l)*2^32);
+//     two's-complement nibble, operand byte 16 * q (the INT4 operand form).
+template <bool BF16, bool PLANE, bool UNIFORM>
+__global__ void __launch_bounds__(kThreads) quant_ablation_kernel(const void* __restrict__ x, size_t n,
+                                                                  const float* __restrict__ d_amax,
+                                                                  const __grid_constant__ PhiloxKeySet keys,
+                                                                  int n_samples, uint32_t word_under,
+                                                                  uint32_t word_range,
+                                                                  uint8_t* __restrict__ codes,
+                                                                  int8_t* __restrict__ operand,
+                                                                  float* __restrict__ d_scale,
+                                                                  unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
+  constexpr int kElems = Item<BF16>::kElems;
+  const float given = *d_amax;
+  const bool first = blockIdx.x == 0 && threadIdx.x == 0;
+  const bool ok = scale_usable(given, first ? status : nullptr);
+  const float scale = !ok ? 0.0f : UNIFORM ? given / 7.0f : given * keys.inv_levels;
+  if (first) *d_scale = scale;
+  const float inv = ok ? 7.0f / given : 0.0f;                         // uniform grid only
+  const LuqScale sc = luq_scale(ok && !UNIFORM ? scale : 1.0f);
+
+  // per element: the lower level, the 32-bit threshold of the up-decision, the constant that
+  // replaces the random word (0: none)
+  auto prepare = [&](float v, uint32_t& lo, uint32_t& thr, uint32_t& fixed) {
+    if constexpr (UNIFORM) {
+      const float y = fabsf(v) * inv;
+      const float a = (y == y) ? fminf(y, 7.0f) : 0.0f;               // NaN element -> 0
+      const float l = floorf(a);
+      lo = __float2uint_rz(l);
+      thr = __float2uint_rz((a - l) * 4294967296.0f);                 // a - l is exact
+      fixed = 0u;
+    } else {
+      const float q = luq_quotient_clamped<false>(v, sc, keys.q_top);
+      luq_bin(q, lo, thr);
+      fixed = q < 4294967296.0f ? word_under : word_range;            // Q < 2^32 <=> |x| < alpha
+    }
+  };
+  auto nibble_of = [&](uint32_t xbits, uint32_t lo, uint32_t thr, uint32_t fixed, uint32_t word) -> uint32_t {
+    const uint32_t w = fixed ? fixed : word;
+    if constexpr (UNIFORM) {
+      const uint32_t m = lo + (w < thr ? 1u : 0u);
+      return ((xbits >> 31) ? 0u - m : m) & 0xFu;
+    } else {
+      return luq_nibble(xbits, lo, thr, w);
+    }
+  };
+  auto byte_of = [&](uint32_t nib) -> uint32_t { return UNIFORM ? (nib << 4) : luq_operand_byte(nib); };
+
+  const size_t plane = n / 2;
+  const bool aligned = (plane % (kElems / 2)) == 0;
+  const bool aligned_op = (n % kElems) == 0;
+  const size_t items = n / kElems;
+  const uint4* p = reinterpret_cast<const uint4*>(x);
+
+  auto process = [&](size_t item, const uint4& u, bool whole_warp) {
+    float v[kElems];
+    Item<BF16>::widen(u, v);
+    if constexpr (!UNIFORM) {
+      // the LUQ kernel's short route: a warp whose elements all lie below alpha only decides
+      // between 0 and +-alpha; with a deterministic underflow region no generator runs at all
+      bool in_range = false;
+#pragma unroll
+      for (int j = 0; j < kElems; ++j) in_range |= !(fabsf(v[j]) < scale);
+      if (whole_warp && ok && !sc.tiny && !__any_sync(0xFFFFFFFFu, in_range)) {
+        uint32_t thr[kElems], sn[kElems], ob[kElems];
+#pragma unroll
+        for (int j = 0; j < kElems; ++j) {
+          const uint32_t bits = __float_as_uint(v[j]);
+          thr[j] = __float2uint_rz(luq_scaled_quotient<false>(fabsf(v[j]), sc));
+          const int at = 4 * j;
+          sn[j] = ((bits >> (28 - at)) & (8u << at)) | (1u << at);
+          if constexpr (PLANE) ob[j] = ((bits >> 31) ? 0xFFu : 0x01u) << (8 * (j % 4));
+        }
+        for (int s = 0; s < n_samples; ++s) {
+          const PhiloxKeys& ks = keys.s[s];
+          uint32_t word = 0;
+          uint32_t bytes[kElems / 4] = {};
+#pragma unroll
+          for (int b = 0; b < kElems / 4; ++b) {
+            uint4 r = make_uint4(word_under, word_under, word_under, word_under);
+            if (word_under == 0u) r = philox_block(item * (kElems / 4) + b, ks);
+            const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (rw[j] < thr[4 * b + j]) {
+                word |= sn[4 * b + j];
+                if constexpr (PLANE) bytes[b] |= ob[4 * b + j];
+              }
+            }
+          }
+          Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
+          if constexpr (PLANE) Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
+        }
+        return;
+      }
+    }
+    uint32_t lo[kElems], thr[kElems], fixed[kElems];
+#pragma unroll
+    for (int j = 0; j < kElems; ++j) prepare(v[j], lo[j], thr[j], fixed[j]);
+    for (int s = 0; s < n_samples; ++s) {
+      const PhiloxKeys& ks = keys.s[s];
+      uint32_t word = 0;
+      uint32_t bytes[kElems / 4] = {};
+#pragma unroll
+      for (int b = 0; b < kElems / 4; ++b) {
+        const uint4 r = philox_block(item * (kElems / 4) + b, ks);
+        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int e = 4 * b + j;
+          const uint32_t nib = ok ? nibble_of(__float_as_uint(v[e]), lo[e], thr[e], fixed[e], rw[j]) : 0u;
+          word |= nib << (4 * e);
+          if constexpr (PLANE) bytes[b] |= byte_of(nib) << (8 * j);
+        }
+      }
+      Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
+      if constexpr (PLANE) Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
+    }
+  };
+
+  const size_t full_tiles = items / kTileItems;
+  for (size_t t = blockIdx.x; t < full_tiles; t += gridDim.x) {
+    const size_t i0 = t * kTileItems + threadIdx.x;
+    uint4 u[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i0 + j * kThreads);
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) process(i0 + j * kThreads, u[j], true);
+  }
+  if (blockIdx.x == gridDim.x - 1)
+    for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) process(i, __ldg(p + i), false);
+  if (first) {  // tail: fewer elements than one piece, two per byte
+    for (int s = 0; s < n_samples; ++s) {
+      const PhiloxKeys& ks = keys.s[s];
+      for (size_t e = items * kElems; e < n; e += 2) {
+        uint32_t nib[2] = {0u, 0u};
+        for (int h = 0; h < 2; ++h) {
+          const size_t idx = e + h;
+          if (ok && idx < n) {
+            const float xv = Item<BF16>::load1(x, idx);
+            uint32_t lo, thr, fixed;
+            prepare(xv, lo, thr, fixed);
+            const uint4 r = philox_block(idx >> 2, ks);
+            const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+            nib[h] = nibble_of(__float_as_uint(xv), lo, thr, fixed, rw[idx & 3]);
+          }
+        }
+        codes[plane * s + (e >> 1)] = static_cast<uint8_t>(nib[0] | (nib[1] << 4));
+        if constexpr (PLANE) {
+          operand[n * s + e] = static_cast<int8_t>(byte_of(nib[0]));
+          if (e + 1 < n) operand[n * s + e + 1] = static_cast<int8_t>(byte_of(nib[1]));
+        }
+      }
+    }
+  }
+}
+
 // Diagnostic: the quotient t = |x| / alpha exactly as the quantizer forms it
 // (before the clamp to the top level), for comparison with an IEEE division.
 __global__ void __launch_bounds__(kThreads) luq_quotient_kernel(const float* __restrict__ x, size_t n,
@@ -925,6 +1092,45 @@ int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n,
     case 6: rc = launch_luq<true, false, true>(a); break;
     default: rc = launch_luq<true, true, true>(a); break;
   }
+  ctx->launches += 1;
+  return rc;
+}
+
+namespace {
+template <bool BF16, bool PLANE, bool UNIFORM>
+int launch_ablation(luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax, const PhiloxKeySet& keys, int n_samples,
+                    uint32_t word_under, uint32_t word_range, uint8_t* d_codes, int8_t* d_operand, float* d_scale,
+                    cudaStream_t st) {
+  const int grid = grid_for(ctx, quant_ablation_kernel<BF16, PLANE, UNIFORM>, n / Item<BF16>::kElems / kTileItems + 1);
+  return static_cast<int>(luq_launch_kernel(quant_ablation_kernel<BF16, PLANE, UNIFORM>, grid, kThreads, 0, st,
+                                            LUQ_LAUNCH_EARLY, 1, d_g, n, d_amax, keys, n_samples, word_under, word_range,
+                                            d_codes, d_operand, d_scale, ctx->d_status));
+}
+template <bool BF16, bool PLANE>
+int launch_ablation_grid(bool uniform, luq_ctx* ctx, const void* d_g, size_t n, const float* d_amax,
+                         const PhiloxKeySet& keys, int n_samples, uint32_t word_under, uint32_t word_range,
+                         uint8_t* d_codes, int8_t* d_operand, float* d_scale, cudaStream_t st) {
+  return uniform ? launch_ablation<BF16, PLANE, true>(ctx, d_g, n, d_amax, keys, n_samples, 0u, 0u, d_codes, d_operand, d_scale, st)
+                 : launch_ablation<BF16, PLANE, false>(ctx, d_g, n, d_amax, keys, n_samples, word_under, word_range, d_codes,
+                                                       d_operand, d_scale, st);
+}
+}  // namespace
+
+// scheme: bit 0 = stochastic rounding inside the range, bit 1 = stochastic underflow (the LUQ grid,
+// the other region rounds to the nearest level); 4 = the uniform grid with stochastic rounding
+int luq_launch_quant_grad_ablation(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax,
+                                   uint64_t seed, int n_samples, int scheme, uint8_t* d_codes, int8_t* d_operand,
+                                   float* d_scale, cudaStream_t st) {
+  const PhiloxKeySet keys = expand_keys(seed, n_samples, ctx->kmax, 0u);
+  const bool uniform = scheme == 4;
+  const uint32_t word_range = (scheme & 1) ? 0u : 0x7FFFFFFFu;
+  const uint32_t word_under = (scheme & 2) ? 0u : 0x7FFFFFFFu;
+  const bool bf = dtype == LUQ_BF16;
+  int rc;
+  if (d_operand) rc = bf ? launch_ablation_grid<true, true>(uniform, ctx, d_g, n, d_amax, keys, n_samples, word_under, word_range, d_codes, d_operand, d_scale, st)
+                         : launch_ablation_grid<false, true>(uniform, ctx, d_g, n, d_amax, keys, n_samples, word_under, word_range, d_codes, d_operand, d_scale, st);
+  else rc = bf ? launch_ablation_grid<true, false>(uniform, ctx, d_g, n, d_amax, keys, n_samples, word_under, word_range, d_codes, nullptr, d_scale, st)
+               : launch_ablation_grid<false, false>(uniform, ctx, d_g, n, d_amax, keys, n_samples, word_under, word_range, d_codes, nullptr, d_scale, st);
   ctx->launches += 1;
   return rc;
 }
