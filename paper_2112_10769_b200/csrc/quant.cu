@@ -1,7 +1,9 @@
 // Memory-bound kernels of the path: tensor max, INT4 round-to-nearest
 // quantize-and-pack (signed, and unsigned for non-negative tensors), LUQ stochastic
 // quantize-and-pack (Philox, n samples) with its variants: power-of-two scale,
-// in-hindsight maximum, other level counts, deterministic nearest power.
+// in-hindsight maximum, other level counts, deterministic nearest power, and the
+// ablation's other gradient quantizers (one region deterministic; uniform grid with
+// stochastic rounding).
 //
 // All stream the input once.  The unit of work is one 16-byte load
 // (4 fp32 or 8 bf16 elements); consecutive lanes take consecutive 16-byte
