@@ -39,7 +39,7 @@ KERNELS = ("amax_A", "amax_W", "quant_int4_A", "quant_int4_W", "gemm_fwd",
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the cfg2 kernels, from the ncu
 # capture summarised in profiles/kernels_cfg2_full_size.md (other workloads: None).
 NCU_TRAFFIC_BYTES = {"amax_A": 469.0e6, "quant_int4_A": 511.6e6, "gemm_fwd": 64.1e6, "amax_G": 51.4e6,
-                     "quant_grad_G": 52.3e6, "gemm_bwd": 409.0e6, "gemm_wgrad": 74.3e6, "amax_W": 2.4e6,
+                     "quant_grad_G": 52.3e6, "gemm_bwd": 416.4e6, "gemm_wgrad": 74.3e6, "amax_W": 2.4e6,
                      "quant_int4_W": 2.4e6}
 
 

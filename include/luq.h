@@ -94,8 +94,11 @@ extern "C" {
  * the element order of the tensor (sample planes one after the other, rows*cols
  * bytes each).  INT4: 16 * q (the code nibble in the high half of the byte).  LUQ:
  * +-2^(c-1) for code c >= 1, 0 for c = 0.  16-byte aligned.  A GEMM uses them where
- * at least two of its tiles re-read the operand and the contraction is long, and
- * reads the codes otherwise; the codes must always be passed. */
+ * at least two of its tiles re-read the operand and the contraction is long, or
+ * where the contraction is short (at most four 128-deep stages), the output fp32
+ * and the bytes of BOTH operands are given (such a product is bound by its output
+ * and then stores whole output rows); it reads the codes otherwise.  The codes
+ * must always be passed. */
 
 typedef struct luq_ctx luq_ctx;
 

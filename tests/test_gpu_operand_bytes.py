@@ -186,6 +186,47 @@ def test_gemms_identical_with_and_without_operand_bytes(ctx, M, K, N, ns):
                       oracle.gemm_entries("wgrad", og, al.item(), ns, oa, sa.item(), M, N, K, r, c))
 
 
+@pytest.mark.parametrize("mma_kind", [0, 2])
+@pytest.mark.parametrize("M,K,N,ns", [(1000, 160, 416, 1),    # forward: 2 stages, 13 column chunks (one tile and a part)
+                                      (777, 640, 96, 1),      # backward: 1 stage, ragged rows, 2.5 column tiles
+                                      (1300, 2304, 256, 2),   # backward: 4 stages (two samples), 9 column tiles
+                                      (256, 352, 224, 1)])    # all three: 3, 2 and 2 stages; the update product unsplit (4 tiles)
+def test_whole_row_epilogue_of_short_contractions(ctx, M, K, N, ns, mma_kind):
+    """A product with at most four contraction stages, fp32 output and both operands' bytes stores whole
+    output rows (one 3-D copy per 32-row strip).  Same integers, same scales: bit-identical with the
+    box epilogue of the codes path, ragged rows and partial column tiles included."""
+    A, W, G = inputs.small_layer(M, K, N, 1200 + M)
+    (ca, sa, ba), (cw, sw, bw), (cg, al, bg) = layer_with_bytes(ctx, A, W, G, seed=M, ns=ns)
+    ctx.set_option(binding.OPT_MMA_KIND, mma_kind)
+    try:
+        pairs = []
+        if K <= 512:
+            pairs.append((ctx.gemm_fwd(ca, sa, cw, sw, M, N, K), ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=ba, w_operand=bw)))
+        dA_rows = None
+        if ns * N <= 512:
+            dA_rows = ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bg, w_operand=bw)
+            pairs.append((ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K), dA_rows))
+        if ns * M <= 512:
+            pairs.append((ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K),
+                          ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K, g_operand=bg, a_operand=ba)))
+        assert pairs
+        for plain, rows in pairs:
+            assert torch.equal(plain, rows)
+        if dA_rows is not None and mma_kind == 2:
+            # the bytes are what is multiplied: all-zero gradient bytes give an all-zero product
+            out = torch.full((M, K), 7.0, device="cuda")
+            ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, out, g_operand=torch.zeros_like(bg), w_operand=bw)
+            assert not out.any().item()
+            # and nothing is written outside the output: a guard row after it keeps its pattern
+            buf = torch.full((M + 40, K), 3.0, device="cuda")
+            ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, buf[:M], g_operand=bg, w_operand=bw)
+            assert torch.equal(buf[:M], dA_rows)
+            assert (buf[M:] == 3.0).all().item()
+    finally:
+        ctx.set_option(binding.OPT_MMA_KIND, 2)
+    assert ctx.status() == 0
+
+
 def test_gemm_reads_the_bytes_it_is_given(ctx):
     """Where a product fetches operand bytes, it must fetch the caller's: all-zero bytes give an
     all-zero product.  (With e4m3 operands forced, the int8 bytes are ignored.)"""
