@@ -49,7 +49,7 @@ def _stamp(target: str, digest: str) -> None:
 def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "nvcc")
     headers = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "luq.h")]
-    objs, digests = [], []
+    objs, digests, running = [], [], []
     for name, extra in UNITS.items():
         src = os.path.join(CSRC, name)
         obj = os.path.join(CSRC, name.replace(".cu", ".o"))
@@ -59,8 +59,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         digests.append(digest)
         if force or _stale(obj, digest):
             cmd = [nvcc] + ARCH + COMMON + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
-            subprocess.run(cmd, check=True)
-            _stamp(obj, digest)
+            running.append((subprocess.Popen(cmd), cmd, obj, digest))     # the units compile side by side
+    for proc, cmd, obj, digest in running:
+        if proc.wait() != 0:
+            raise subprocess.CalledProcessError(proc.returncode, cmd)
+        _stamp(obj, digest)
     link_digest = _digest([], digests)
     if force or _stale(LIB, link_digest):
         subprocess.run([nvcc] + ARCH + ["-shared", "-o", LIB] + objs, check=True)
