@@ -225,6 +225,15 @@ def quant_luq_hindsight(x: np.ndarray, m_hat, eta, seed: int, n_samples: int = 1
     return codes, alpha, flags | mflags, measured, hindsight_next(measured, m_hat, eta)
 
 
+def quant_int4_hindsight(x: np.ndarray, c_hat, eta):
+    """One hindsight step for an INT4 tensor (Sec. 7 applied to the forward tensors): quantize x with
+    the clip estimate c_hat made from earlier steps (values beyond it saturate at +-7) and return
+    (codes, scale, flags, measured max of x, c_hat for the next step)."""
+    codes, scale, flags = quant_int4(x, np.float32(c_hat))
+    measured, mflags = amax(x)
+    return codes, scale, flags | mflags, measured, hindsight_next(measured, c_hat, eta)
+
+
 def luq_bins(x: np.ndarray, mx, kmax: int = KMAX_DEFAULT):
     """Per element (lo, hi, thr): candidate levels in units of alpha and the
     32-bit threshold; P(hi) = thr / 2^32."""

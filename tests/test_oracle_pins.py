@@ -909,3 +909,38 @@ def test_int4_sr_unbiased_with_table1_variance_and_twice_the_rdn_error():
     mse_rdn = ((vr - x) ** 2).mean()
     mse_sr = (acc2 / S).mean()
     assert abs(mse_sr / mse_rdn - 2.0) < 0.2
+
+
+# ------------------------------------------ in-hindsight range for the INT4 tensors (Sec. 7) ----
+
+
+def test_int4_hindsight_step_saturates_beyond_the_estimate_and_follows_the_recursion():
+    rng = np.random.default_rng(31)
+    x = rng.standard_normal(6000).astype(np.float32)
+    true_max, _ = oracle.amax(x)
+    c_hat = np.float32(float(true_max) / 3)                  # stale, too small estimate
+    codes, s, fl, measured, nxt = oracle.quant_int4_hindsight(x, c_hat, 0.1)
+    assert fl == 0 and measured == true_max and s == c_hat / np.float32(7)
+    assert nxt == oracle.hindsight_next(true_max, c_hat, 0.1)
+    val, q = decode_int4(codes, x.size, s)
+    beyond = np.abs(x) >= c_hat
+    assert beyond.sum() > 50 and (np.abs(q[beyond]) == 7).all()          # saturation, sign kept
+    assert (np.sign(val[beyond]) == np.sign(x[beyond])).all()
+    inside = ~beyond
+    assert (np.abs(val[inside] - x[inside]) <= float(s) / 2 * (1 + 1e-6)).all()   # nearest inside the range
+    # with an estimate equal to the maximum the step is the plain quantizer
+    plain, s_plain, _ = oracle.quant_int4(x, true_max)
+    same, s_same, _, _, _ = oracle.quant_int4_hindsight(x, true_max, 0.1)
+    np.testing.assert_array_equal(same, plain)
+    assert s_same == s_plain
+    # a constant maximum is approached geometrically: error eta^t after t steps
+    est = np.float32(1.0)
+    for t in range(1, 8):
+        _, _, _, m, est = oracle.quant_int4_hindsight(x, est, 0.25)
+        assert abs(float(est) - float(true_max)) <= abs(1.0 - float(true_max)) * 0.25 ** t * (1 + 1e-5) + 1e-6
+    # a non-finite element is reported, the codes stay defined
+    y = x.copy(); y[5] = np.inf
+    cy, _, fy, my, ny = oracle.quant_int4_hindsight(y, c_hat, 0.1)
+    assert fy & oracle.FLAG_NONFINITE
+    _, qy = decode_int4(cy, y.size, s)
+    assert qy[5] == 7
