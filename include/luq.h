@@ -160,6 +160,19 @@ int luq_quant_uint4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_
 int luq_amax_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
                         float* d_amax, uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream);
 
+/* INT4 with the in-hindsight range (Sec. 7 "Reducing the data movement", Appendix A.5.4, applied to
+ * the forward tensors): the tensor is quantized in ONE pass with the clip estimate *d_chat made from
+ * earlier steps (values beyond it saturate at +-7, as with any caller-supplied clip), its own max|x|
+ * is measured on the way into *d_measured_max, and the estimate for the next step replaces *d_chat:
+ *   c_hat <- (1 - eta) * measured + eta * c_hat     (binary32, one rounding per operation).
+ * This removes the max pass over the tensor, i.e. one of the two reads of the activations.
+ * *d_scale receives c_hat / 7 (the estimate used).  Initialise *d_chat before the first step, e.g.
+ * with luq_amax.  0 <= eta <= 1.  Codes, operand bytes and status bits are those of
+ * luq_quant_int4 called with d_clip = the estimate. */
+int luq_quant_int4_hindsight(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols,
+                             float* d_chat, float eta, uint8_t* d_codes, float* d_scale,
+                             float* d_measured_max, int8_t* d_operand, void* stream);
+
 /* Q_FP = LUQ (Sec. 4): alpha = max / 2^kmax (Eq. alpha); |x| < alpha becomes
  * sign*alpha with probability |x|/alpha, else 0 (Eq. StochasticPruning);
  * in-range values round stochastically between the two enclosing powers of two

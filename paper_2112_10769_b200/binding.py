@@ -23,7 +23,7 @@ SCHEME_FP4, SCHEME_FP4_SR, SCHEME_FP4_SU, SCHEME_LUQ, SCHEME_INT4_SR = 0, 1, 2, 
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
-           "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_ablation", "luq_quant_grad_pw2",
+           "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_int4_hindsight", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_ablation", "luq_quant_grad_pw2",
            "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_debug_expire_wait", "luq_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
@@ -56,6 +56,7 @@ def load() -> ctypes.CDLL:
         L.luq_amax_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_amax_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, u64, ctypes.c_int, vp, vp, vp, vp, vp]
         L.luq_quant_grad.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
+        L.luq_quant_int4_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, vp, vp, vp, vp, vp]
         L.luq_quant_grad_nearest.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_quant_grad_ablation.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp]
         L.luq_quant_grad_pw2.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, u64, ctypes.c_int, vp, vp, vp, vp]
@@ -197,6 +198,20 @@ class Context:
                                       codes.data_ptr(), scale.data_ptr(), _opt(operand, x.numel()), _stream()),
                "luq_quant_uint4")
         return codes, scale
+
+    def quant_int4_hindsight(self, x: torch.Tensor, c_hat: torch.Tensor, eta: float, codes: torch.Tensor | None = None,
+                             scale: torch.Tensor | None = None, measured: torch.Tensor | None = None,
+                             operand: torch.Tensor | None = None):
+        """One pass: INT4 codes with the clip estimate in `c_hat`, this tensor's maximum into `measured`,
+        `c_hat` replaced by the estimate for the next step.  Returns (codes, scale, measured)."""
+        rows, cols = (x.shape[0], x.numel() // max(x.shape[0], 1)) if x.dim() > 1 else (1, x.numel())
+        codes = torch.empty(x.numel() // 2, dtype=torch.uint8, device=x.device) if codes is None else codes
+        scale = torch.empty(1, dtype=torch.float32, device=x.device) if scale is None else scale
+        measured = torch.empty(1, dtype=torch.float32, device=x.device) if measured is None else measured
+        _check(load().luq_quant_int4_hindsight(self.handle, x.data_ptr(), _dtype_code(x), rows, cols, c_hat.data_ptr(),
+                                               eta, codes.data_ptr(), scale.data_ptr(), measured.data_ptr(),
+                                               _opt(operand, x.numel()), _stream()), "luq_quant_int4_hindsight")
+        return codes, scale, measured
 
     def amax_quant_int4(self, x: torch.Tensor, amax: torch.Tensor | None = None, codes: torch.Tensor | None = None,
                         scale: torch.Tensor | None = None, operand: torch.Tensor | None = None):

@@ -190,6 +190,22 @@ int luq_quant_uint4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_
                                        nullptr, true, as_stream(stream)));
 }
 
+int luq_quant_int4_hindsight(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, float* d_chat,
+                             float eta, uint8_t* d_codes, float* d_scale, float* d_measured_max, int8_t* d_operand,
+                             void* stream) {
+  if (!ctx || !d_chat || !d_scale || !d_measured_max || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  if (!(eta >= 0.0f && eta <= 1.0f)) return LUQ_ERR_ARG;
+  const size_t n = rows * cols;
+  if (rows != 0 && n / rows != cols) return LUQ_ERR_ARG;
+  if (n & 1u) return LUQ_ERR_ARG;
+  if (n && (!d_x || !d_codes)) return LUQ_ERR_ARG;
+  if (!aligned16(d_x) || !aligned16(d_codes) || !aligned16(d_operand)) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_quant_int4_hindsight(ctx, d_x, dtype, n, d_chat, eta, d_codes, n ? d_operand : nullptr,
+                                                 d_scale, d_measured_max, as_stream(stream)));
+}
+
 int luq_amax_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t rows, size_t cols, float* d_amax,
                         uint8_t* d_codes, float* d_scale, int8_t* d_operand, void* stream) {
   if (!ctx || !d_amax || !d_scale || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;

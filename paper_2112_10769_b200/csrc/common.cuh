@@ -36,6 +36,11 @@ int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, co
                           uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_amax_out, bool is_unsigned,
                           cudaStream_t st);
 
+// in-hindsight INT4: d_estimate is the clip (values beyond it saturate); the tensor's own max|x| goes to
+// d_measured and d_estimate is replaced by (1 - eta) * measured + eta * estimate, all in one kernel
+int luq_launch_quant_int4_hindsight(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_estimate, float eta,
+                                    uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_measured,
+                                    cudaStream_t st);
 // flags: bit 0 = power-of-two scale; bit 1 = in-hindsight (d_amax is the running estimate: the tensor's own
 // max|x| goes to d_measured and d_estimate (= d_amax) is replaced by (1 - eta) * measured + eta * estimate)
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,

@@ -315,11 +315,17 @@ __device__ __forceinline__ uint32_t uint4_code(float x, float inv) {
 // PLANE: the tensor-core operand bytes (int8, 16 * q: the code nibble in the high half of the
 // byte) are written next to the packed codes, one byte per element in element order.
 // UNSIGNED: the grid 0..15 with scale clip / 15 (non-negative tensors); operand byte = q.
-template <bool BF16, bool PLANE, bool UNSIGNED>
+// TRACK: in-hindsight range - `clip` is an estimate from earlier steps (values beyond it saturate),
+// the tensor's own max|x| is reduced on the way; the block that finishes last writes it to
+// *measured_bits and replaces *d_estimate by (1 - eta) * measured + eta * estimate.
+template <bool BF16, bool PLANE, bool UNSIGNED, bool TRACK = false>
 __device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size_t n, float clip,
                                                 uint8_t* __restrict__ codes, int8_t* __restrict__ operand,
                                                 float* __restrict__ d_scale, unsigned int* __restrict__ status,
-                                                unsigned int rank, unsigned int count) {
+                                                unsigned int rank, unsigned int count,
+                                                unsigned int* __restrict__ measured_bits = nullptr,
+                                                float* d_estimate = nullptr, float eta = 0.0f,
+                                                unsigned int* scratch = nullptr) {
   constexpr int kElems = Item<BF16>::kElems;
   const bool first = rank == 0 && threadIdx.x == 0;
   const bool ok = scale_usable(clip, first ? status : nullptr);
@@ -328,6 +334,7 @@ __device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size
   const float inv = ok ? kTop / clip : 0.0f;
   if (first) *d_scale = ok ? clip / kTop : 0.0f;
   auto code_of = [&](float v) { return UNSIGNED ? uint4_code(v, inv) : int4_code(v, inv); };
+  uint32_t seen = 0;   // running max of |x| bit patterns (TRACK)
 
   const size_t items = n / kElems;
   const uint4* p = reinterpret_cast<const uint4*>(x);
@@ -338,6 +345,7 @@ __device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size
     uint32_t bytes[kElems / 4] = {};
 #pragma unroll
     for (int j = 0; j < kElems; ++j) {
+      if constexpr (TRACK) seen = max(seen, __float_as_uint(v[j]) & 0x7FFFFFFFu);
       const uint32_t code = ok ? code_of(v[j]) : 0u;
       word |= code << (4 * j);
       if constexpr (PLANE) bytes[j / 4] |= code << (8 * (j % 4) + kByteShift);
@@ -360,6 +368,10 @@ __device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size
     for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) emit(i, __ldg(p + i));
   if (first) {  // tail: fewer elements than one piece, two per byte
     for (size_t e = items * kElems; e < n; e += 2) {
+      if constexpr (TRACK) {
+        seen = max(seen, __float_as_uint(Item<BF16>::load1(x, e)) & 0x7FFFFFFFu);
+        if (e + 1 < n) seen = max(seen, __float_as_uint(Item<BF16>::load1(x, e + 1)) & 0x7FFFFFFFu);
+      }
       const uint32_t lo = ok ? code_of(Item<BF16>::load1(x, e)) : 0u;
       const uint32_t hi = (ok && e + 1 < n) ? code_of(Item<BF16>::load1(x, e + 1)) : 0u;
       codes[e >> 1] = static_cast<uint8_t>(lo | (hi << 4));
@@ -369,6 +381,31 @@ __device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size
       }
     }
   }
+  if constexpr (TRACK) {   // Inf/NaN patterns win the maximum and raise the flag
+    if (grid_max_last_block(seen, scratch, rank, count)) {
+      *measured_bits = seen;
+      if (seen >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
+      const float keep = __fsub_rn(1.0f, eta);
+      *d_estimate = __fadd_rn(__fmul_rn(keep, __uint_as_float(seen)), __fmul_rn(eta, clip));
+    }
+  }
+}
+
+// in-hindsight INT4: d_estimate is read as the clip by every block and replaced by the last one
+template <bool BF16, bool PLANE>
+__global__ void __launch_bounds__(kThreads) quant_int4_track_kernel(const void* __restrict__ x, size_t n,
+                                                                    float* d_estimate, float eta,
+                                                                    uint8_t* __restrict__ codes,
+                                                                    int8_t* __restrict__ operand,
+                                                                    float* __restrict__ d_scale,
+                                                                    unsigned int* __restrict__ measured_bits,
+                                                                    unsigned int* scratch,
+                                                                    unsigned int* __restrict__ status) {
+  luqdev::pdl_wait();
+  luqdev::pdl_trigger();
+  const float clip = *d_estimate;
+  quant_int4_body<BF16, PLANE, false, true>(x, n, clip, codes, operand, d_scale, status, blockIdx.x, gridDim.x,
+                                            measured_bits, d_estimate, eta, scratch);
 }
 
 template <bool BF16, bool PLANE, bool UNSIGNED>
@@ -1016,6 +1053,23 @@ int launch_int4_grid(bool is_unsigned, luq_ctx* ctx, const void* d_x, size_t n, 
                      : launch_int4<BF16, PLANE, false>(ctx, d_x, n, d_clip, d_codes, d_operand, d_scale, d_amax_out, st);
 }
 }  // namespace
+
+int luq_launch_quant_int4_hindsight(luq_ctx* ctx, const void* d_x, int dtype, size_t n, float* d_estimate, float eta,
+                                    uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_measured,
+                                    cudaStream_t st) {
+  unsigned int* measured = reinterpret_cast<unsigned int*>(d_measured);
+  const bool bf = dtype == LUQ_BF16;
+  auto go = [&](auto kernel, int elems) {
+    const int grid = grid_for(ctx, kernel, n / elems / kTileItems + 1);
+    return static_cast<int>(luq_launch_kernel(kernel, grid, kThreads, 0, st, LUQ_LAUNCH_EARLY, 1, d_x, n, d_estimate, eta,
+                                              d_codes, d_operand, d_scale, measured, ctx->d_scratch, ctx->d_status));
+  };
+  int rc;
+  if (d_operand) rc = bf ? go(quant_int4_track_kernel<true, true>, 8) : go(quant_int4_track_kernel<false, true>, 4);
+  else rc = bf ? go(quant_int4_track_kernel<true, false>, 8) : go(quant_int4_track_kernel<false, false>, 4);
+  ctx->launches += 1;
+  return rc;
+}
 
 // d_amax_out non-null: fused - the clip is the tensor's maximum, reduced by the same kernel and written there
 int luq_launch_quant_int4(luq_ctx* ctx, const void* d_x, int dtype, size_t n, const float* d_clip,
