@@ -66,6 +66,7 @@ def test_null_arguments_are_rejected_without_a_gpu(lib):
     assert lib.luq_quant_int4(None, None, 0, 0, 0, None, None, None, None, None) == binding.ERR_ARG
     assert lib.luq_quant_grad(None, None, 0, 0, 0, None, 0, 1, None, None, None, None) == binding.ERR_ARG
     assert lib.luq_gemm_fwd(None, None, None, None, None, None, None, None, 1, 1, 32, None) == binding.ERR_ARG
+    assert lib.luq_quant_int4_hindsight(None, None, 0, 0, 0, None, 0.1, None, None, None, None, None) == binding.ERR_ARG
     assert lib.luq_quant_grad_ablation(None, None, 0, 0, 0, None, 0, 1, 0, None, None, None, None) == binding.ERR_ARG
     assert lib.luq_status(None, None, None) == binding.ERR_ARG
     assert lib.luq_destroy(None) == 0
