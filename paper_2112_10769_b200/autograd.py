@@ -11,6 +11,10 @@ Backward / Update; Sec. 4 LUQ; Sec. 5.1 SMP).
 The INT4 codes of the forward pass are kept for the backward pass (the paper's update GEMM re-uses the
 quantized activations), together with the 8-bit operand bytes of W and G that the GEMMs re-read.
 Shapes must satisfy the GEMMs' divisibility rules (K and N multiples of 32).
+
+With ``estimates`` (a float32 tensor of three running maxima: A, W, G) the quantizers take the
+in-hindsight route of Sec. 7: each tensor is quantized in one pass with the estimate made from earlier
+steps while its own maximum is measured and folded into the estimate - no max pass over any tensor.
 """
 from __future__ import annotations
 
@@ -31,19 +35,25 @@ def context(device: torch.device) -> binding.Context:
 
 class LuqLinearFunction(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int):
+    def forward(ctx, a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int,
+                estimates: torch.Tensor | None = None, eta: float = 0.1):
         lib = context(a.device)
         a2 = a.reshape(-1, a.shape[-1]).contiguous()
         w2 = w.contiguous()
         M, K = a2.shape
         N = w2.shape[0]
         w_bytes = torch.empty(N * K, dtype=torch.int8, device=a.device)
-        ca, sa = lib.quant_int4(a2, lib.amax(a2))
-        cw, sw = lib.quant_int4(w2, lib.amax(w2), operand=w_bytes)
+        if estimates is None:
+            ca, sa = lib.quant_int4(a2, lib.amax(a2))
+            cw, sw = lib.quant_int4(w2, lib.amax(w2), operand=w_bytes)
+        else:
+            ca, sa, _ = lib.quant_int4_hindsight(a2, estimates[0:1], eta)
+            cw, sw, _ = lib.quant_int4_hindsight(w2, estimates[1:2], eta, operand=w_bytes)
         z = lib.gemm_fwd(ca, sa, cw, sw, M, N, K, w_operand=w_bytes)
         ctx.save_for_backward(ca, sa, cw, sw, w_bytes)
         ctx.dims = (M, N, K, a.shape, a.dtype, w.dtype)
         ctx.seed, ctx.n_samples = int(seed), int(n_samples)
+        ctx.estimates, ctx.eta = estimates, float(eta)
         return z.reshape(*a.shape[:-1], N).to(a.dtype)
 
     @staticmethod
@@ -54,20 +64,25 @@ class LuqLinearFunction(torch.autograd.Function):
         lib = context(grad_out.device)
         g2 = grad_out.reshape(M, N).contiguous()
         g_bytes = torch.empty(ns * M * N, dtype=torch.int8, device=g2.device)
-        cg, alpha = lib.quant_grad(g2, lib.amax(g2), ctx.seed, ns, operand=g_bytes)
+        if ctx.estimates is None:
+            cg, alpha = lib.quant_grad(g2, lib.amax(g2), ctx.seed, ns, operand=g_bytes)
+        else:
+            cg, alpha, _ = lib.quant_grad_hindsight(g2, ctx.estimates[2:3], ctx.eta, ctx.seed, ns, operand=g_bytes)
         da = dw = None
         if ctx.needs_input_grad[0]:
             da = lib.gemm_bwd(cg, alpha, ns, cw, sw, M, N, K, g_operand=g_bytes, w_operand=w_bytes)
             da = da.reshape(a_shape).to(a_dtype)
         if ctx.needs_input_grad[1]:
             dw = lib.gemm_wgrad(cg, alpha, ns, ca, sa, M, N, K, g_operand=g_bytes).to(w_dtype)
-        return da, dw, None, None
+        return da, dw, None, None, None, None
 
 
-def luq_linear(a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int = 1) -> torch.Tensor:
+def luq_linear(a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int = 1,
+               estimates: torch.Tensor | None = None, eta: float = 0.1) -> torch.Tensor:
     """``a @ w.T`` with INT4 operands forward and LUQ-FP4 gradients backward.  ``seed`` keys the
-    stochastic rounding of this call's backward pass: give every layer and step its own."""
-    return LuqLinearFunction.apply(a, w, seed, n_samples)
+    stochastic rounding of this call's backward pass: give every layer and step its own.
+    ``estimates``: three running maxima (A, W, G) for the in-hindsight route; updated in place."""
+    return LuqLinearFunction.apply(a, w, seed, n_samples, estimates, eta)
 
 
 class LuqLinear(torch.nn.Module):
@@ -75,8 +90,12 @@ class LuqLinear(torch.nn.Module):
     gradient quantizer advances with every forward call."""
 
     def __init__(self, in_features: int, out_features: int, n_samples: int = 1, seed: int = 0,
-                 device=None, dtype=torch.float32):
+                 device=None, dtype=torch.float32, hindsight: bool = False, eta: float = 0.1):
         super().__init__()
+        # in-hindsight maxima of A, W and G (Sec. 7): measured once on the first step, then estimated
+        self.hindsight, self.eta = hindsight, eta
+        self.register_buffer("estimates", torch.zeros(3, device=device, dtype=torch.float32))
+        self._primed = False
         w = torch.empty(out_features, in_features, device=device, dtype=dtype)
         torch.nn.init.kaiming_uniform_(w, a=5 ** 0.5)
         self.weight = torch.nn.Parameter(w)
@@ -87,4 +106,13 @@ class LuqLinear(torch.nn.Module):
     def forward(self, a: torch.Tensor) -> torch.Tensor:
         seed = self.base_seed + self.calls * self.n_samples     # sample s of a call uses seed + s
         self.calls += 1
-        return luq_linear(a, self.weight, seed, self.n_samples)
+        if not self.hindsight:
+            return luq_linear(a, self.weight, seed, self.n_samples)
+        if not self._primed:
+            # the first step has no history: A's and W's maxima are measured; the gradient's estimate
+            # starts at zero, so the first backward pass quantizes G to zero and only measures it
+            lib = context(a.device)
+            lib.amax(a.reshape(-1, a.shape[-1]).contiguous(), self.estimates[0:1])
+            lib.amax(self.weight.detach().contiguous(), self.estimates[1:2])
+            self._primed = True
+        return luq_linear(a, self.weight, seed, self.n_samples, self.estimates, self.eta)

@@ -56,3 +56,41 @@ def test_module_trains_a_small_regression():
     assert layer.calls == 60
     assert losses[-1] < 0.2 * losses[0]          # the 4-bit forward noise sets the floor; no divergence
     assert autograd.context(torch.device("cuda", 0)).status() == 0
+
+
+def test_function_with_in_hindsight_estimates_matches_the_oracle():
+    M, K, N, ns, seed, eta = 384, 256, 288, 2, 23, 0.1
+    A, W, G = inputs.small_layer(M, K, N, 6)
+    a = torch.from_numpy(A).cuda().requires_grad_(True)
+    w = torch.from_numpy(W).cuda().requires_grad_(True)
+    g = torch.from_numpy(G).cuda()
+    start = np.array([oracle.amax(A)[0] * 0.7, oracle.amax(W)[0] * 1.2, oracle.amax(G)[0] * 0.5], dtype=np.float32)
+    est = torch.from_numpy(start.copy()).cuda()
+    z = autograd.luq_linear(a, w, seed, ns, est, eta)
+    z.backward(g)
+    oa, sa, _, ma, na = oracle.quant_int4_hindsight(A, start[0], eta)
+    ow, sw, _, mw, nw = oracle.quant_int4_hindsight(W, start[1], eta)
+    og, al, _, mg, ng = oracle.quant_luq_hindsight(G, start[2], eta, seed, ns)
+    np.testing.assert_array_equal(est.cpu().numpy(), np.array([na, nw, ng], dtype=np.float32))
+    assert_gemm_close(z.detach().cpu().numpy(), oracle.gemm_fwd(oa, float(sa), ow, float(sw), M, N, K))
+    assert_gemm_close(a.grad.cpu().numpy(), oracle.gemm_bwd(og, float(al), ns, ow, float(sw), M, N, K))
+    assert_gemm_close(w.grad.cpu().numpy(), oracle.gemm_wgrad(og, float(al), ns, oa, float(sa), M, N, K))
+
+
+def test_module_trains_with_in_hindsight_maxima():
+    torch.manual_seed(0)
+    K, N, M = 128, 64, 512
+    target = torch.randn(N, K, device="cuda") / K ** 0.5
+    layer = autograd.LuqLinear(K, N, n_samples=2, seed=100, device="cuda", hindsight=True)
+    opt = torch.optim.SGD(layer.parameters(), lr=0.2)
+    losses = []
+    for _ in range(60):
+        x = torch.randn(M, K, device="cuda")
+        loss = (layer(x) - x @ target.T).pow(2).sum(1).mean()
+        opt.zero_grad()
+        loss.backward()
+        opt.step()
+        losses.append(loss.item())
+    assert (layer.estimates > 0).all().item()
+    assert losses[-1] < 0.2 * losses[0]
+    assert autograd.context(torch.device("cuda", 0)).status() == 0
