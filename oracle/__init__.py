@@ -215,13 +215,22 @@ def hindsight_next(measured_max, m_hat, eta) -> np.float32:
     return np.float32(lib().oracle_hindsight_next(np.float32(measured_max), np.float32(m_hat), np.float32(eta)))
 
 
+def _measured_max(x: np.ndarray):
+    """max|x| as a hindsight step measures it: a tensor with an Inf or NaN element has no finite
+    maximum, which the recursion must see (it then keeps its estimate)."""
+    measured, mflags = amax(x)
+    if mflags & FLAG_NONFINITE:
+        measured = np.float32(np.inf)
+    return measured, mflags
+
+
 def quant_luq_hindsight(x: np.ndarray, m_hat, eta, seed: int, n_samples: int = 1, pw2: bool = False,
                         kmax: int = KMAX_DEFAULT):
     """One hindsight step: quantize x with the estimate m_hat (not with its own maximum) and return
     (codes, alpha, flags, measured max of x, m_hat for the next step)."""
     mx_used = pw2_ceil(m_hat) if pw2 else np.float32(m_hat)
     codes, alpha, flags = quant_luq(x, mx_used, seed, n_samples, kmax)
-    measured, mflags = amax(x)
+    measured, mflags = _measured_max(x)
     return codes, alpha, flags | mflags, measured, hindsight_next(measured, m_hat, eta)
 
 
@@ -230,7 +239,7 @@ def quant_int4_hindsight(x: np.ndarray, c_hat, eta):
     the clip estimate c_hat made from earlier steps (values beyond it saturate at +-7) and return
     (codes, scale, flags, measured max of x, c_hat for the next step)."""
     codes, scale, flags = quant_int4(x, np.float32(c_hat))
-    measured, mflags = amax(x)
+    measured, mflags = _measured_max(x)
     return codes, scale, flags | mflags, measured, hindsight_next(measured, c_hat, eta)
 
 
@@ -275,7 +284,7 @@ def gemm_fwd(a_codes, sa, w_codes, sw, M, N, K) -> np.ndarray:
 
 
 def gemm_bwd(g_codes, alpha, n_samples, w_codes, sw, M, N, K) -> np.ndarray:
-    """dA = mean_s(G_d,s) . W_d in float64 (Eq. Backward, SMP average of Sec. 5.1)."""
+    """dA = (sum_s G_d,s . W_d) / n_s in float64 (Eq. Backward; Sec. 5.1 averages the samples' results)."""
     g_codes = np.ascontiguousarray(g_codes).reshape(-1)
     w_codes = np.ascontiguousarray(w_codes).reshape(-1)
     dA = np.zeros((M, K), dtype=np.float64)
@@ -285,7 +294,7 @@ def gemm_bwd(g_codes, alpha, n_samples, w_codes, sw, M, N, K) -> np.ndarray:
 
 
 def gemm_wgrad(g_codes, alpha, n_samples, a_codes, sa, M, N, K) -> np.ndarray:
-    """dW = mean_s(G_d,s)^T . A_d in float64 (Eq. Update, SMP average of Sec. 5.1)."""
+    """dW = (sum_s G_d,s^T . A_d) / n_s in float64 (Eq. Update; Sec. 5.1 averages the samples' weight gradients)."""
     g_codes = np.ascontiguousarray(g_codes).reshape(-1)
     a_codes = np.ascontiguousarray(a_codes).reshape(-1)
     dW = np.zeros((N, K), dtype=np.float64)

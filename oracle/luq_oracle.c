@@ -363,8 +363,17 @@ float oracle_pw2_ceil(float mx) {
 /* paper's runs.  Tensor t is quantized with m_hat^t (values above it clip to  */
 /* the top level) while its own maximum is measured for step t+1.  Evaluated   */
 /* in binary32, each operation rounded once.                                   */
+/* Reading where the paper is silent (it assumes finite tensors and a running  */
+/* estimate that already exists): a measurement that is not finite (an Inf or  */
+/* NaN element) carries no information about the range and leaves the estimate */
+/* as it was, otherwise one overflowed element would make every later estimate */
+/* Inf; an estimate that is itself not a positive finite number (0 before the  */
+/* first step, or Inf/NaN handed in) has no history to blend with and is       */
+/* replaced by the measurement.                                                */
 /* ------------------------------------------------------------------------ */
 float oracle_hindsight_next(float measured_max, float m_hat, float eta) {
+  if (!(measured_max <= 3.402823466e38f)) return m_hat;              /* NaN or Inf measured */
+  if (!(m_hat > 0.0f) || !(m_hat <= 3.402823466e38f)) return measured_max; /* no usable history */
   float keep = 1.0f - eta;
   float a = keep * measured_max;
   float b = eta * m_hat;
@@ -426,49 +435,56 @@ void oracle_gemm_fwd(const uint8_t* a_codes, double sa, const uint8_t* w_codes, 
   free(Ad); free(Wd);
 }
 
-/* mean over samples of dequant(G codes, plane s) -> Gd[M x N] */
-static double* mean_gradient(const uint8_t* g_codes, double alpha, int n_samples,
-                             int64_t M, int64_t N) {
+/* Sample planes of the gradient, each dequantised on its own: Gs[s][M x N] */
+static double* gradient_samples(const uint8_t* g_codes, double alpha, int n_samples,
+                                int64_t M, int64_t N) {
   size_t n = (size_t)(M * N), plane = (n + 1) / 2;
-  double* Gd = (double*)calloc(n, sizeof(double));
+  double* Gs = (double*)malloc(sizeof(double) * n * (size_t)n_samples);
   for (int s = 0; s < n_samples; ++s)
-    for (size_t i = 0; i < n; ++i) Gd[i] += alpha * code_value(g_codes + plane * (size_t)s, i, 1);
-  for (size_t i = 0; i < n; ++i) Gd[i] /= (double)n_samples;
-  return Gd;
+    oracle_dequant(g_codes + plane * (size_t)s, n, alpha, 1, Gs + n * (size_t)s);
+  return Gs;
 }
 
-/* dA[M x K] = mean_s(G_d,s) . W_d   (SMP, Sec. 5.1: average of the samples) */
+/* dA[M x K] = (1/n_s) sum_s G_d,s . W_d.  SMP (Sec. 5.1) averages the RESULTS of the
+ * n_s samples: every sample's product is formed, the products are added, and the
+ * sum is divided by n_s once at the end. */
 void oracle_gemm_bwd(const uint8_t* g_codes, double alpha, int n_samples,
                      const uint8_t* w_codes, double sw,
                      int64_t M, int64_t N, int64_t K, double* dA) {
-  double* Gd = mean_gradient(g_codes, alpha, n_samples, M, N);
+  double* Gs = gradient_samples(g_codes, alpha, n_samples, M, N);
   double* Wd = (double*)malloc(sizeof(double) * (size_t)(N * K));
   oracle_dequant(w_codes, (size_t)(N * K), sw, 0, Wd);
 #pragma omp parallel for schedule(static)
   for (int64_t m = 0; m < M; ++m)
     for (int64_t k = 0; k < K; ++k) {
       double acc = 0.0;
-      for (int64_t n = 0; n < N; ++n) acc += Gd[m * N + n] * Wd[n * K + k];
-      dA[m * K + k] = acc;
+      for (int s = 0; s < n_samples; ++s) {
+        const double* Gd = Gs + (size_t)s * (size_t)(M * N);
+        for (int64_t n = 0; n < N; ++n) acc += Gd[m * N + n] * Wd[n * K + k];
+      }
+      dA[m * K + k] = acc / (double)n_samples;
     }
-  free(Gd); free(Wd);
+  free(Gs); free(Wd);
 }
 
-/* dW[N x K] = mean_s(G_d,s)^T . A_d */
+/* dW[N x K] = (1/n_s) sum_s G_d,s^T . A_d  (Sec. 5.1: the average of the samples' weight gradients) */
 void oracle_gemm_wgrad(const uint8_t* g_codes, double alpha, int n_samples,
                        const uint8_t* a_codes, double sa,
                        int64_t M, int64_t N, int64_t K, double* dW) {
-  double* Gd = mean_gradient(g_codes, alpha, n_samples, M, N);
+  double* Gs = gradient_samples(g_codes, alpha, n_samples, M, N);
   double* Ad = (double*)malloc(sizeof(double) * (size_t)(M * K));
   oracle_dequant(a_codes, (size_t)(M * K), sa, 0, Ad);
 #pragma omp parallel for schedule(static)
   for (int64_t n = 0; n < N; ++n)
     for (int64_t k = 0; k < K; ++k) {
       double acc = 0.0;
-      for (int64_t m = 0; m < M; ++m) acc += Gd[m * N + n] * Ad[m * K + k];
-      dW[n * K + k] = acc;
+      for (int s = 0; s < n_samples; ++s) {
+        const double* Gd = Gs + (size_t)s * (size_t)(M * N);
+        for (int64_t m = 0; m < M; ++m) acc += Gd[m * N + n] * Ad[m * K + k];
+      }
+      dW[n * K + k] = acc / (double)n_samples;
     }
-  free(Gd); free(Ad);
+  free(Gs); free(Ad);
 }
 
 /* Second, independent form (Appendix A.1 scale factoring): integer codes are
@@ -514,7 +530,7 @@ void oracle_gemm_int64(int which, const uint8_t* x_codes, int n_samples, const u
 
 /* Selected output entries of the three products at any size, computed one by
  * one from the codes (same definition as above: dequantise, multiply, add in
- * double).  which: 0 fwd (r=m, c=n), 1 bwd (r=m, c=k), 2 wgrad (r=n, c=k). */
+ * double, the samples' products added and divided by n_s at the end).  which: 0 fwd (r=m, c=n), 1 bwd (r=m, c=k), 2 wgrad (r=n, c=k). */
 void oracle_gemm_entries(int which, const uint8_t* x_codes, double sx, int n_samples,
                          const uint8_t* y_codes, double sy,
                          int64_t M, int64_t N, int64_t K,
@@ -529,19 +545,17 @@ void oracle_gemm_entries(int which, const uint8_t* x_codes, double sx, int n_sam
         acc += (sx * code_value(x_codes, (size_t)(r * K + k), 0)) *
                (sy * code_value(y_codes, (size_t)(c * K + k), 0));
     } else if (which == 1) {
-      for (int64_t n = 0; n < N; ++n) {
-        double g = 0.0;
-        for (int s = 0; s < n_samples; ++s)
-          g += sx * code_value(x_codes + plane * (size_t)s, (size_t)(r * N + n), 1);
-        acc += (g / (double)n_samples) * (sy * code_value(y_codes, (size_t)(n * K + c), 0));
-      }
+      for (int s = 0; s < n_samples; ++s)
+        for (int64_t n = 0; n < N; ++n)
+          acc += (sx * code_value(x_codes + plane * (size_t)s, (size_t)(r * N + n), 1)) *
+                 (sy * code_value(y_codes, (size_t)(n * K + c), 0));
+      acc /= (double)n_samples;
     } else {
-      for (int64_t m = 0; m < M; ++m) {
-        double g = 0.0;
-        for (int s = 0; s < n_samples; ++s)
-          g += sx * code_value(x_codes + plane * (size_t)s, (size_t)(m * N + r), 1);
-        acc += (g / (double)n_samples) * (sy * code_value(y_codes, (size_t)(m * K + c), 0));
-      }
+      for (int s = 0; s < n_samples; ++s)
+        for (int64_t m = 0; m < M; ++m)
+          acc += (sx * code_value(x_codes + plane * (size_t)s, (size_t)(m * N + r), 1)) *
+                 (sy * code_value(y_codes, (size_t)(m * K + c), 0));
+      acc /= (double)n_samples;
     }
     out[e] = acc;
   }

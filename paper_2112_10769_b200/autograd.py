@@ -36,7 +36,7 @@ def context(device: torch.device) -> binding.Context:
 class LuqLinearFunction(torch.autograd.Function):
     @staticmethod
     def forward(ctx, a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int,
-                estimates: torch.Tensor | None = None, eta: float = 0.1):
+                estimates: torch.Tensor | None = None, eta: float = 0.1, primed: list | None = None):
         lib = context(a.device)
         a2 = a.reshape(-1, a.shape[-1]).contiguous()
         w2 = w.contiguous()
@@ -47,13 +47,19 @@ class LuqLinearFunction(torch.autograd.Function):
             ca, sa = lib.quant_int4(a2, lib.amax(a2))
             cw, sw = lib.quant_int4(w2, lib.amax(w2), operand=w_bytes)
         else:
+            if primed is not None:
+                # a tensor seen for the first time has no history: its estimate starts as its own maximum
+                if not primed[0]:
+                    lib.amax(a2, estimates[0:1]); primed[0] = True
+                if not primed[1]:
+                    lib.amax(w2, estimates[1:2]); primed[1] = True
             ca, sa, _ = lib.quant_int4_hindsight(a2, estimates[0:1], eta)
             cw, sw, _ = lib.quant_int4_hindsight(w2, estimates[1:2], eta, operand=w_bytes)
         z = lib.gemm_fwd(ca, sa, cw, sw, M, N, K, w_operand=w_bytes)
         ctx.save_for_backward(ca, sa, cw, sw, w_bytes)
         ctx.dims = (M, N, K, a.shape, a.dtype, w.dtype)
         ctx.seed, ctx.n_samples = int(seed), int(n_samples)
-        ctx.estimates, ctx.eta = estimates, float(eta)
+        ctx.estimates, ctx.eta, ctx.primed = estimates, float(eta), primed
         return z.reshape(*a.shape[:-1], N).to(a.dtype)
 
     @staticmethod
@@ -67,6 +73,10 @@ class LuqLinearFunction(torch.autograd.Function):
         if ctx.estimates is None:
             cg, alpha = lib.quant_grad(g2, lib.amax(g2), ctx.seed, ns, operand=g_bytes)
         else:
+            if ctx.primed is not None and not ctx.primed[2]:
+                # first backward pass: without this the gradient would be quantized with an estimate of
+                # zero, i.e. to all zeros, and every layer below would receive (and measure) nothing
+                lib.amax(g2, ctx.estimates[2:3]); ctx.primed[2] = True
             cg, alpha, _ = lib.quant_grad_hindsight(g2, ctx.estimates[2:3], ctx.eta, ctx.seed, ns, operand=g_bytes)
         da = dw = None
         if ctx.needs_input_grad[0]:
@@ -74,15 +84,18 @@ class LuqLinearFunction(torch.autograd.Function):
             da = da.reshape(a_shape).to(a_dtype)
         if ctx.needs_input_grad[1]:
             dw = lib.gemm_wgrad(cg, alpha, ns, ca, sa, M, N, K, g_operand=g_bytes).to(w_dtype)
-        return da, dw, None, None, None, None
+        return da, dw, None, None, None, None, None
 
 
 def luq_linear(a: torch.Tensor, w: torch.Tensor, seed: int, n_samples: int = 1,
-               estimates: torch.Tensor | None = None, eta: float = 0.1) -> torch.Tensor:
+               estimates: torch.Tensor | None = None, eta: float = 0.1, primed: list | None = None) -> torch.Tensor:
     """``a @ w.T`` with INT4 operands forward and LUQ-FP4 gradients backward.  ``seed`` keys the
     stochastic rounding of this call's backward pass: give every layer and step its own.
-    ``estimates``: three running maxima (A, W, G) for the in-hindsight route; updated in place."""
-    return LuqLinearFunction.apply(a, w, seed, n_samples, estimates, eta)
+    ``estimates``: three running maxima (A, W, G) for the in-hindsight route; updated in place.
+    ``primed``: a list of three booleans, updated in place - an estimate whose flag is False is first
+    set to its tensor's own maximum (one extra max pass, the first time only).  Without it the caller
+    initialises the estimates."""
+    return LuqLinearFunction.apply(a, w, seed, n_samples, estimates, eta, primed)
 
 
 class LuqLinear(torch.nn.Module):
@@ -92,10 +105,13 @@ class LuqLinear(torch.nn.Module):
     def __init__(self, in_features: int, out_features: int, n_samples: int = 1, seed: int = 0,
                  device=None, dtype=torch.float32, hindsight: bool = False, eta: float = 0.1):
         super().__init__()
-        # in-hindsight maxima of A, W and G (Sec. 7): measured once on the first step, then estimated
+        # in-hindsight maxima of A, W and G (Sec. 7): each is measured once, the first time its tensor is
+        # seen (A and W in the first forward pass, G in the first backward pass), then estimated.  An
+        # estimate is "primed" when it is positive; the flags mirror that on the host and are rebuilt
+        # from the buffer when a state dict is loaded, so restored estimates are kept.
         self.hindsight, self.eta = hindsight, eta
         self.register_buffer("estimates", torch.zeros(3, device=device, dtype=torch.float32))
-        self._primed = False
+        self._primed = [False, False, False]
         w = torch.empty(out_features, in_features, device=device, dtype=dtype)
         torch.nn.init.kaiming_uniform_(w, a=5 ** 0.5)
         self.weight = torch.nn.Parameter(w)
@@ -108,11 +124,9 @@ class LuqLinear(torch.nn.Module):
         self.calls += 1
         if not self.hindsight:
             return luq_linear(a, self.weight, seed, self.n_samples)
-        if not self._primed:
-            # the first step has no history: A's and W's maxima are measured; the gradient's estimate
-            # starts at zero, so the first backward pass quantizes G to zero and only measures it
-            lib = context(a.device)
-            lib.amax(a.reshape(-1, a.shape[-1]).contiguous(), self.estimates[0:1])
-            lib.amax(self.weight.detach().contiguous(), self.estimates[1:2])
-            self._primed = True
-        return luq_linear(a, self.weight, seed, self.n_samples, self.estimates, self.eta)
+        return luq_linear(a, self.weight, seed, self.n_samples, self.estimates, self.eta, self._primed)
+
+    def _load_from_state_dict(self, state_dict, prefix, *args, **kwargs):
+        super()._load_from_state_dict(state_dict, prefix, *args, **kwargs)
+        if prefix + "estimates" in state_dict:
+            self._primed[:] = [bool(v > 0) for v in self.estimates.tolist()]

@@ -1167,7 +1167,11 @@ int luq_launch_expire_wait(luq_ctx* ctx, cudaStream_t st) {
 }
 
 int luq_launch_gemm(luq_ctx* ctx_in, const luq_gemm_args& a, cudaStream_t st) {
-  if (a.Mo <= 0 || a.No <= 0 || a.Kc <= 0) return 0;
+  if (a.Mo <= 0 || a.No <= 0) return 0;
+  if (a.Kc <= 0) {  // an empty contraction (an empty batch in the update product): the sum is zero everywhere
+    if (a.d_out == nullptr) return LUQ_ERR_ARG;
+    return static_cast<int>(cudaMemsetAsync(a.d_out, 0, static_cast<size_t>(a.Mo) * a.No * (a.out_bf16 ? 2 : 4), st));
+  }
   luq_ctx ctx_copy = *ctx_in;            // the operand type may be chosen per product below
   luq_ctx* ctx = &ctx_copy;
   const int rc_all = luq_launch_gemm_impl(ctx, a, st);

@@ -127,6 +127,18 @@ __device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* s
   return false;
 }
 
+// In-hindsight update of a running maximum (Sec. 7, App. A.5.4): (1 - eta) * measured + eta * estimate,
+// one rounding per operation.  A measurement that is not finite (an Inf/NaN element) leaves the
+// estimate as it was - one overflowed element must not turn every later estimate into Inf; an
+// estimate that is not a positive finite number (0 before the first step) is replaced by the measurement.
+__device__ __forceinline__ float hindsight_next(uint32_t measured_bits, float estimate, float eta) {
+  if (measured_bits >= 0x7F800000u) return estimate;
+  const uint32_t eb = __float_as_uint(estimate);
+  if (eb == 0u || eb >= 0x7F800000u) return __uint_as_float(measured_bits);   // 0, negative, Inf, NaN
+  const float keep = __fsub_rn(1.0f, eta);
+  return __fadd_rn(__fmul_rn(keep, __uint_as_float(measured_bits)), __fmul_rn(eta, estimate));
+}
+
 // ------------------------------------------------------------------ amax ----
 // |x| as an unsigned bit pattern is monotone in |x| for finite values, and every
 // Inf/NaN pattern is larger than every finite one: one unsigned max does both
@@ -385,8 +397,7 @@ __device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size
     if (grid_max_last_block(seen, scratch, rank, count)) {
       *measured_bits = seen;
       if (seen >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
-      const float keep = __fsub_rn(1.0f, eta);
-      *d_estimate = __fadd_rn(__fmul_rn(keep, __uint_as_float(seen)), __fmul_rn(eta, clip));
+      *d_estimate = hindsight_next(seen, clip, eta);
     }
   }
 }
@@ -739,8 +750,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
     if (grid_max_last_block(seen, scratch, blockIdx.x, gridDim.x)) {
       *measured_bits = seen;
       if (seen >= 0x7F800000u) atomicOr(status, LUQ_STATUS_NONFINITE);
-      const float keep = __fsub_rn(1.0f, eta);
-      *d_estimate = __fadd_rn(__fmul_rn(keep, __uint_as_float(seen)), __fmul_rn(eta, given));
+      *d_estimate = hindsight_next(seen, given, eta);
     }
   }
 }

@@ -36,7 +36,7 @@ def test_function_matches_the_oracle(dtype):
         if dtype == torch.float32:
             assert_gemm_close(got, ref)
         else:   # the result is rounded once more, to bf16
-            assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-12 * np.abs(ref).max()).all()
+            assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref)).all()
 
 
 def test_module_trains_a_small_regression():
@@ -93,4 +93,37 @@ def test_module_trains_with_in_hindsight_maxima():
         losses.append(loss.item())
     assert (layer.estimates > 0).all().item()
     assert losses[-1] < 0.2 * losses[0]
+    assert autograd.context(torch.device("cuda", 0)).status() == 0
+
+
+def test_stacked_layers_get_gradients_on_the_first_step_and_restored_estimates_are_kept():
+    """Every estimate is primed with its tensor's own maximum the first time the tensor is seen - the
+    gradient's in the first backward pass - so the first layer of a stack receives a gradient on step 1;
+    a module restored from a state dict keeps the estimates it was saved with."""
+    torch.manual_seed(1)
+    K = 128
+    layers = torch.nn.Sequential(*[autograd.LuqLinear(K, K, seed=10 * i, device="cuda", hindsight=True)
+                                   for i in range(3)])
+    x = torch.randn(256, K, device="cuda")
+    layers(x).pow(2).mean().backward()
+    for layer in layers:
+        assert layer.weight.grad.abs().max().item() > 0
+        assert (layer.estimates > 0).all().item() and layer._primed == [True, True, True]
+    saved = {k: v.clone() for k, v in layers.state_dict().items()}
+    fresh = torch.nn.Sequential(*[autograd.LuqLinear(K, K, seed=10 * i, device="cuda", hindsight=True)
+                                  for i in range(3)])
+    fresh.load_state_dict(saved)
+    for layer, old in zip(fresh, layers):
+        assert layer._primed == [True, True, True]
+        assert torch.equal(layer.estimates, old.estimates)
+    before = [layer.estimates.clone() for layer in fresh]
+    fresh(x * 0.5).pow(2).mean().backward()
+    eta = 0.1
+    for layer, b in zip(fresh, before):
+        # A's estimate followed the recursion from the restored value: it was not measured afresh
+        assert layer.estimates[0].item() != b[0].item()
+        assert layer.estimates[0].item() > 0.5 * b[0].item() * (1 - eta)
+    first = fresh[0]
+    want = oracle.hindsight_next(oracle.amax((x * 0.5).cpu().numpy())[0], before[0][0].item(), eta)
+    assert first.estimates[0].item() == want
     assert autograd.context(torch.device("cuda", 0)).status() == 0

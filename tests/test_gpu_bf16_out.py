@@ -1,9 +1,11 @@
 """LUQ_OPT_OUTPUT_BF16: the GEMMs round their fp32 result to bf16 (nearest even) in the epilogue.
-The fp32 path is checked against the oracle elsewhere; here the bf16 outputs must be exactly the
-fp32 outputs rounded once."""
+The bf16 outputs must be exactly the fp32 outputs rounded once, and within one bf16 rounding
+(2^-8 relative) of the CPU oracle's float64 product, exact zeros exact."""
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2112_10769_b200 import binding, inputs
 
 from test_gpu_parity import to_dev
@@ -53,6 +55,15 @@ def test_bf16_outputs_are_the_rounded_fp32_outputs(ctx, M, K, N, ns, mma_kind):
     for f, h in zip(full, half):
         assert f.dtype == torch.float32 and h.dtype == torch.bfloat16 and h.shape == f.shape
         assert torch.equal(h, f.to(torch.bfloat16))
+    if M * K * N <= 1152 * 1056 * 800:     # the oracle's triple loops finish in seconds up to here
+        oa, ow, og = ca.cpu().numpy(), cw.cpu().numpy(), cg.cpu().numpy()
+        refs = (oracle.gemm_fwd(oa, sa.item(), ow, sw.item(), M, N, K),
+                oracle.gemm_bwd(og, al.item(), ns, ow, sw.item(), M, N, K),
+                oracle.gemm_wgrad(og, al.item(), ns, oa, sa.item(), M, N, K))
+        for h, ref in zip(half, refs):
+            got = h.float().cpu().numpy().astype(np.float64)
+            assert (got[ref == 0] == 0).all()
+            assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref)).all()
 
 
 def test_bf16_output_rows_must_stay_aligned(ctx):

@@ -79,6 +79,47 @@ def test_unusable_estimate_recovers_and_argument_errors(ctx):
     assert np.isinf(measured.item()) and ctx.status() == binding.STATUS_NONFINITE
 
 
+@pytest.mark.parametrize("kind", ["int4", "luq"])
+def test_a_non_finite_step_does_not_poison_the_estimate(ctx, kind):
+    """Steps [finite, Inf element, finite, finite]: the step with the Inf is flagged and leaves the
+    estimate as it was, so the steps after it quantize normally again; estimates, measured maxima and
+    codes follow the oracle through the whole sequence."""
+    n, eta = 70_002, 0.1
+    base = np.random.default_rng(5).standard_normal(n).astype(np.float32)
+    est_o = np.float32(np.abs(base).max())
+    est_d = scalar(float(est_o))
+    for step in range(4):
+        x = (base * np.float32(1.0 + 0.1 * step)).astype(np.float32)
+        if step == 1:
+            x[n // 2] = np.inf
+        if kind == "int4":
+            want, s_want, fl, meas, nxt = oracle.quant_int4_hindsight(x, est_o, eta)
+            codes, scale, measured = ctx.quant_int4_hindsight(to_dev(x), est_d, eta)
+        else:
+            want, s_want, fl, meas, nxt = oracle.quant_luq_hindsight(x, est_o, eta, seed=step)
+            codes, scale, measured = ctx.quant_grad_hindsight(to_dev(x), est_d, eta, step)
+        np.testing.assert_array_equal(codes.cpu().numpy().reshape(want.shape), want)
+        assert scale.item() == s_want
+        assert measured.item() == meas or (np.isinf(meas) and np.isinf(measured.item()))
+        assert est_d.item() == nxt and np.isfinite(nxt)
+        assert ctx.status() == (binding.STATUS_NONFINITE if step == 1 else 0) == fl
+        if step == 1:
+            assert nxt == est_o                      # unchanged by the non-finite measurement
+        if step >= 2:
+            assert codes.any().item()                # quantizing normally again
+        est_o = nxt
+    # an estimate that is itself unusable is replaced by the first finite measurement
+    for bad in (0.0, float("inf"), float("nan")):
+        est_d = scalar(bad)
+        x = base
+        if kind == "int4":
+            ctx.quant_int4_hindsight(to_dev(x), est_d, eta)
+        else:
+            ctx.quant_grad_hindsight(to_dev(x), est_d, eta, 0)
+        ctx.status()
+        assert est_d.item() == np.abs(base).max() == oracle.hindsight_next(np.abs(base).max(), bad, eta)
+
+
 def test_forward_product_on_hindsight_codes(ctx):
     M, K, N = 1024, 512, 320
     A, W, _ = inputs.small_layer(M, K, N, 77)

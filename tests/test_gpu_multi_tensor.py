@@ -1,5 +1,5 @@
-"""Several tensors in one launch: results must be exactly those of the one-tensor calls (which are
-checked against the oracle elsewhere), whatever the mix of sizes."""
+"""Several tensors in one launch: maxima, codes, scales and operand bytes against the CPU oracle,
+and equal to the one-tensor calls, whatever the mix of sizes."""
 import numpy as np
 import pytest
 import torch
@@ -45,6 +45,9 @@ def test_multi_tensor_calls_equal_the_single_ones(ctx, sizes, dtype):
         np.testing.assert_array_equal(c.cpu().numpy(), want)
         assert s.item() == s_want
         if o is not None:
+            q = oracle.unpack(want, x.numel()).astype(np.int64)       # the oracle's codes, as integers
+            q = np.where(q >= 8, q - 16, q)
+            np.testing.assert_array_equal(o.cpu().numpy(), (16 * q).astype(np.int8))
             ob = torch.empty_like(o)
             ctx.quant_int4(x, m, operand=ob)
             assert torch.equal(o, ob)

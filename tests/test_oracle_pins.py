@@ -614,6 +614,27 @@ def test_hindsight_recursion_closed_form_and_limits():
     assert oracle.hindsight_next(0.7, 0.3, 0.1) == np.float32(np.float32(a) + np.float32(b))
 
 
+def test_hindsight_recursion_ignores_non_finite_measurements_and_replaces_unusable_estimates():
+    """Reading where the paper is silent: an Inf/NaN measurement leaves the estimate unchanged (so the
+    sequence [m, Inf, m, m] never leaves the finite numbers), and an estimate without usable history
+    (0, negative, Inf, NaN) is replaced by the measurement instead of being blended with it."""
+    inf, nan = np.float32(np.inf), np.float32(np.nan)
+    assert oracle.hindsight_next(inf, 3.0, 0.1) == np.float32(3.0)
+    assert oracle.hindsight_next(nan, 3.0, 0.1) == np.float32(3.0)
+    for bad in (0.0, -0.0, -2.0, inf, nan):
+        assert oracle.hindsight_next(2.5, bad, 0.1) == np.float32(2.5)
+    assert np.isnan(oracle.hindsight_next(nan, nan, 0.1)) and oracle.hindsight_next(inf, 0.0, 0.1) == 0
+    m = np.float32(4.0)
+    for measured in (np.float32(2.0), inf, np.float32(2.0), np.float32(2.0)):
+        m = oracle.hindsight_next(measured, m, 0.1)
+        assert np.isfinite(m)
+    # three finite steps from 4 towards 2: 2 + 2 * 0.1^3 up to the binary32 roundings
+    assert abs(float(m) - (2.0 + 2.0 * 0.1 ** 3)) < 1e-6
+    # the ordinary case is untouched: one rounding per operation
+    keep = np.float32(1.0) - np.float32(0.1)
+    assert oracle.hindsight_next(0.7, 0.3, 0.1) == np.float32(keep * np.float32(0.7)) + np.float32(np.float32(0.1) * np.float32(0.3))
+
+
 def test_hindsight_step_uses_the_estimate_and_clips_above_it():
     x = luq_test_tensor(seed=81, n=4000)
     true_max, _ = oracle.amax(x)
