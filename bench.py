@@ -5,10 +5,16 @@ A step is one pass of the whole path over one batch of the ResNet-50-shaped
 im2col workload (M=50176, K=2304, N=256, fp32 inputs):
     amax(A) amax(W) quant_int4(A) quant_int4(W) gemm_fwd
     amax(G) quant_grad(G) gemm_bwd gemm_wgrad
+(for a layer with one column of output tiles, N <= 256, quant_int4(A) and gemm_fwd
+are one kernel: luq_quant_int4_gemm_fwd; `--no-fused` keeps them apart).
 `value` is whole-step throughput in TFLOP/s counting the useful 3 x 2MNK flops,
-quantization included, inputs resident in HBM.  The line also carries the LUQ
-quantizer's HBM GB/s, the roofline of the dominant kernel, an end-to-end number
-with host buffers, and the CPU oracle timed on a bounded sample.
+quantization included, inputs resident in HBM: the timed region is R blocks of
+K replays each (R chosen so that the region lasts at least a second), the
+reported step time is the median block.  The line also carries the LUQ
+quantizer's HBM GB/s, the roofline of the dominant kernel, the 8-bit tensor peak
+measured on this GPU with a library GEMM, the other configurations in compact
+form (`configs`), an end-to-end number with host buffers, and the CPU oracle
+timed on a bounded sample.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -36,8 +42,9 @@ WORKLOAD = "cfg2"
 KERNELS = ("amax_A", "amax_W", "quant_int4_A", "quant_int4_W", "gemm_fwd",
            "amax_G", "quant_grad_G", "gemm_bwd", "gemm_wgrad")
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the cfg2 kernels, from the ncu
-# capture summarised in profiles/kernels_cfg2_full_size.md (other workloads: None).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the cfg2 kernels.  NOT measured by this
+# run: copied from the ncu capture summarised in the file named by TRAFFIC_SOURCE (other workloads: None).
+TRAFFIC_SOURCE = "profiles/kernels_cfg2_full_size.md (an earlier ncu capture, not this run)"
 NCU_TRAFFIC_BYTES = {"amax_A": 469.0e6, "quant_int4_A": 511.6e6, "gemm_fwd": 64.1e6, "amax_G": 51.4e6,
                      "quant_grad_G": 52.3e6, "gemm_bwd": 416.4e6, "gemm_wgrad": 74.3e6, "amax_W": 2.4e6,
                      "quant_int4_W": 2.4e6}
@@ -175,7 +182,291 @@ def run_reference(args):
 
 # ------------------------------------------------------------------ GPU arm --
 
-def run_sweep(args, binding, inputs, torch, local):
+def measure_tensor_peak(torch, seconds: float = 1.0):
+    """Dense 8-bit tensor throughput of THIS GPU with library GEMMs (cuBLASLt through torch), outside
+    the timed region and outside the product path: int8 x int8 -> int32 and e4m3 x e4m3 -> bf16 at
+    8192^3, best of 10 launches (burst) and back to back for `seconds` (sustained).  The denominators
+    of the tensor-bound fractions."""
+    n = 8192
+    out = {"shape": f"{n}^3", "how": "torch._int_mm / torch._scaled_mm, CUDA events; burst = best of 10, "
+                                     f"sustained = back to back for >= {seconds} s"}
+    flops = 2.0 * n ** 3
+
+    def run(name, fn):
+        try:
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            best = float("inf")
+            for _ in range(10):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+                best = min(best, e0.elapsed_time(e1))
+            reps = max(10, int(seconds * 1e3 / best) + 1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record(); torch.cuda.synchronize()
+            out[name + "_burst_tflops"] = round(flops / (best * 1e-3) / 1e12, 1)
+            out[name + "_sustained_tflops"] = round(flops * reps / (e0.elapsed_time(e1) * 1e-3) / 1e12, 1)
+        except Exception as e:  # pragma: no cover
+            out[name + "_error"] = repr(e)[:200]
+
+    a8 = torch.randint(-7, 8, (n, n), dtype=torch.int8, device="cuda")
+    b8 = torch.randint(-7, 8, (n, n), dtype=torch.int8, device="cuda").t()     # column-major B, as the library wants
+    run("int8", lambda: torch._int_mm(a8, b8))
+    try:
+        af = a8.to(torch.float32).to(torch.float8_e4m3fn)
+        bf = b8.t().contiguous().to(torch.float32).to(torch.float8_e4m3fn).t()
+        one = torch.ones((), device="cuda")
+        run("fp8_e4m3", lambda: torch._scaled_mm(af, bf, scale_a=one, scale_b=one, out_dtype=torch.bfloat16))
+    except Exception as e:  # pragma: no cover
+        out["fp8_e4m3_error"] = repr(e)[:200]
+    bursts = [out[k] for k in ("int8_burst_tflops", "fp8_e4m3_burst_tflops") if k in out]
+    sust = [out[k] for k in ("int8_sustained_tflops", "fp8_e4m3_sustained_tflops") if k in out]
+    out["burst_tflops"] = max(bursts) if bursts else None
+    out["sustained_tflops"] = max(sust) if sust else None
+    del a8, b8
+    torch.cuda.empty_cache()
+    return out
+
+
+class LayerBench:
+    """One layer configuration resident on the GPU: inputs, code buffers, outputs, the contexts and
+    streams of the step's schedule, and the ways to run and time a step."""
+
+    def __init__(self, torch, binding, cfg, host_tensors, local, args, ns=None):
+        self.torch, self.binding, self.cfg, self.args = torch, binding, cfg, args
+        M, K, N = cfg.M, cfg.K, cfg.N
+        self.M, self.K, self.N = M, K, N
+        self.ns = cfg.n_samples if ns is None else ns
+        self.seed = cfg.luq_seed
+        A_h, W_h, G_h = host_tensors
+        if cfg.dtype == "bf16":
+            A_h, W_h, G_h = (t.view(np.int16) if t.dtype == np.uint16 else t for t in (A_h, W_h, G_h))
+        pin = lambda a: torch.from_numpy(a).pin_memory() if isinstance(a, np.ndarray) else a  # noqa: E731
+        self.host = [pin(t) for t in (A_h, W_h, G_h)]
+        self.A, self.W, self.G = (t.cuda() for t in self.host)
+        if cfg.dtype == "bf16":
+            self.A, self.W, self.G = (t.view(torch.bfloat16) for t in (self.A, self.W, self.G))
+            self.host = [t.view(torch.bfloat16) for t in self.host]
+        self.ctx = binding.Context(local)
+        self.ctx_g = binding.Context(local) if args.streams == 2 else self.ctx
+        for c in {id(self.ctx): self.ctx, id(self.ctx_g): self.ctx_g}.values():
+            if args.mma_kind is not None:
+                c.set_option(binding.OPT_MMA_KIND, args.mma_kind)
+        self.stream_g = torch.cuda.Stream() if args.streams == 2 else None
+        dev = self.A.device
+        f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)  # noqa: E731
+        u8 = lambda *s: torch.empty(s, dtype=torch.uint8, device=dev)  # noqa: E731
+        i8 = lambda n: torch.empty(n, dtype=torch.int8, device=dev)  # noqa: E731
+        ns = self.ns
+        self.mA, self.mW, self.mG, self.sA, self.sW, self.aG = (f32(1) for _ in range(6))
+        self.cA, self.cW, self.cG = u8(M * K // 2), u8(N * K // 2), u8(ns, M * N // 2)
+        # Operand bytes (the 8-bit form of the codes, written by the quantizer in the same pass) for the
+        # tensors that many GEMM tiles re-read: always W and G; A when the layer is wide enough that the
+        # forward product reads each row block of A four times or more.
+        self.oW, self.oG = i8(N * K), i8(ns * M * N)
+        self.oA = i8(M * K) if N >= 1024 else None
+        self.Z, self.dA, self.dW = f32(M, N), f32(M, K), f32(N, K)
+        # the forward half as one kernel where the layer has a single column of output tiles
+        self.fused = (not args.no_fused) and N <= 256 and args.mma_kind != 0
+        c, s = self.ctx, self
+        self.calls = {
+            "amax_A": lambda: c.amax(s.A, s.mA), "amax_W": lambda: c.amax(s.W, s.mW),
+            "quant_int4_A": lambda: c.quant_int4(s.A, s.mA, s.cA, s.sA, s.oA),
+            "quant_int4_W": lambda: c.quant_int4(s.W, s.mW, s.cW, s.sW, s.oW),
+            "gemm_fwd": lambda: c.gemm_fwd(s.cA, s.sA, s.cW, s.sW, M, N, K, s.Z, s.oA, s.oW),
+            "quant_int4_A+gemm_fwd": lambda: c.quant_int4_gemm_fwd(s.A, s.mA, s.cW, s.sW, M, N, K, s.cA, s.sA, s.Z, s.oW),
+            "amax_G": lambda: c.amax(s.G, s.mG),
+            "quant_grad_G": lambda: c.quant_grad(s.G, s.mG, s.seed, ns, s.cG, s.aG, s.oG),
+            "gemm_bwd": lambda: c.gemm_bwd(s.cG, s.aG, ns, s.cW, s.sW, M, N, K, s.dA, s.oG, s.oW),
+            "gemm_wgrad": lambda: c.gemm_wgrad(s.cG, s.aG, ns, s.cA, s.sA, M, N, K, s.dW, s.oG, s.oA),
+        }
+        if self.fused:
+            self.kernels = ("amax_A", "amax_W", "quant_int4_W", "quant_int4_A+gemm_fwd",
+                            "amax_G", "quant_grad_G", "gemm_bwd", "gemm_wgrad")
+        else:
+            self.kernels = KERNELS
+
+    # ---- one step ------------------------------------------------------------------------------
+    def step_one_stream(self, events=None):
+        torch = self.torch
+        for name in self.kernels:
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e0.record()
+            self.calls[name]()
+            if events is not None:
+                e1 = torch.cuda.Event(enable_timing=True); e1.record()
+                events[name].append((e0, e1))
+
+    def step(self):
+        """The gradient's max and LUQ pass depend on nothing the forward half of the step produces.  With
+        two streams they run on a second stream, through a second context (a context's scratch and
+        workspace serve one stream at a time), beside the activation/weight passes and the forward
+        product; the backward and update products wait for both."""
+        torch = self.torch
+        if self.stream_g is None:
+            return self.step_one_stream()
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event(); fork.record(main)
+        self.stream_g.wait_event(fork)
+        with torch.cuda.stream(self.stream_g):
+            self.ctx_g.amax(self.G, self.mG)
+            self.ctx_g.quant_grad(self.G, self.mG, self.seed, self.ns, self.cG, self.aG, self.oG)
+            join = torch.cuda.Event(); join.record(self.stream_g)
+        for name in self.kernels:
+            if name in ("amax_G", "quant_grad_G", "gemm_bwd", "gemm_wgrad"):
+                continue
+            self.calls[name]()
+        main.wait_event(join)
+        self.calls["gemm_bwd"](); self.calls["gemm_wgrad"]()
+
+    def launches(self):
+        return self.ctx.launches + (self.ctx_g.launches if self.ctx_g is not self.ctx else 0)
+
+    def status(self):
+        return self.ctx.status() | (self.ctx_g.status() if self.ctx_g is not self.ctx else 0)
+
+    def capture(self, fn=None):
+        """No call of the path allocates or synchronises with the host, so one step is captured in a
+        CUDA graph and replayed: the small configurations are bound by launch rate otherwise."""
+        torch = self.torch
+        fn = self.step if fn is None else fn
+        if self.args.no_graph:
+            return fn, "direct calls"
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                fn()
+                torch.cuda.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    fn()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            self._graphs = getattr(self, "_graphs", []) + [graph]
+            return graph.replay, "CUDA graph of the step's calls, replayed"
+        except Exception as e:  # pragma: no cover
+            return fn, f"direct calls (graph capture failed: {e!r})"
+
+    def time_blocks(self, run_step, steps, min_seconds, barrier, max_blocks=400):
+        """R blocks of `steps` replays, one event pair per block, no host synchronisation inside the
+        region; R is chosen from a trial block so that the region lasts at least `min_seconds`.
+        Returns the per-step milliseconds of every block."""
+        torch = self.torch
+        ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(steps):
+            run_step()
+        e1.record(); torch.cuda.synchronize()
+        trial_ms = max(e0.elapsed_time(e1), 1e-3)
+        blocks = int(min(max_blocks, max(1, -(-min_seconds * 1e3 // trial_ms))))
+        barrier()
+        marks = [ev() for _ in range(blocks + 1)]
+        marks[0].record()
+        for b in range(blocks):
+            for _ in range(steps):
+                run_step()
+            marks[b + 1].record()
+        barrier()
+        return [marks[b].elapsed_time(marks[b + 1]) / steps for b in range(blocks)]
+
+    def close(self):
+        if self.ctx_g is not self.ctx:
+            self.ctx_g.close()
+        self.ctx.close()
+
+
+def block_stats(per_block_ms):
+    v = sorted(per_block_ms)
+    med = v[len(v) // 2] if len(v) % 2 else 0.5 * (v[len(v) // 2 - 1] + v[len(v) // 2])
+    return {"blocks": len(v), "ms_median": med, "ms_min": v[0], "ms_max": v[-1],
+            "ms_spread": (v[-1] - v[0]) / med if med else None}
+
+def variance_study(torch, binding, inputs, local, rows=4096, block=64, pairs=256):
+    """Config 5's variance study (Sec. 5.1: averaging N independent samples divides the variance of the
+    weight gradient by N and leaves its mean alone; Table 1: Var[SR(x)] = (x - l)(u - x)).
+    A block x block corner of dW over the first `rows` batch rows of the config-2/5 tensors:
+    for each of `pairs` seed pairs (2p, 2p + 1) the GPU path quantizes G with two samples and forms
+    dW from the first sample alone (n_s = 1) and from both (n_s = 2).  Reported: the empirical
+    variance summed over the block for both, their ratio, and each against the closed form
+        Var[dW[n,k]] = (s_A^2 / n_s) sum_m qA[m,k]^2 (|G[m,n]| - lo)(hi - |G[m,n]|)
+    whose lo / hi are the CPU oracle's bin ends (the check against the oracle; outside any timed region)."""
+    import oracle
+    cfg = inputs.CONFIGS["cfg5"]
+    A, _, G = inputs.layer_inputs(cfg, rows=rows)
+    A, G = np.ascontiguousarray(A[:, :block]), np.ascontiguousarray(G[:, :block])
+    M, K, N = rows, block, block
+    ctx = binding.Context(local)
+    Ad, Gd = torch.from_numpy(A).cuda(), torch.from_numpy(G).cuda()
+    ca, sa = ctx.quant_int4(Ad, ctx.amax(Ad))
+    mG = ctx.amax(Gd)
+    cg = torch.empty((2, M * N // 2), dtype=torch.uint8, device="cuda")
+    al = torch.empty(1, device="cuda")
+    d1 = torch.empty((pairs, N, K), device="cuda")
+    d2 = torch.empty((pairs, N, K), device="cuda")
+    for p in range(pairs):
+        ctx.quant_grad(Gd, mG, 2 * p, 2, cg, al)
+        ctx.gemm_wgrad(cg[0:1], al, 1, ca, sa, M, N, K, d1[p])
+        ctx.gemm_wgrad(cg, al, 2, ca, sa, M, N, K, d2[p])
+    assert ctx.status() == 0
+    d1, d2 = d1.double(), d2.double()
+    var1 = d1.var(dim=0, unbiased=True).cpu().numpy()
+    var2 = d2.var(dim=0, unbiased=True).cpu().numpy()
+    mean2 = d2.mean(dim=0).cpu().numpy()
+    # closed form from the oracle's bins and codes
+    oa, osa, _ = oracle.quant_int4(A, oracle.amax(A)[0])
+    assert np.array_equal(ca.cpu().numpy(), oa) and sa.item() == osa
+    omx = oracle.amax(G)[0]
+    lo, hi, _ = oracle.luq_bins(G, omx)
+    alpha = float(oracle.luq_alpha(omx))
+    g = np.abs(G.astype(np.float64)).reshape(-1)
+    v = np.maximum((g - lo * alpha) * (hi * alpha - g), 0.0).reshape(M, N)
+    Aq = oracle.dequant(oa, M * K, osa, "int4").reshape(M, K)
+    closed1 = v.T @ (Aq ** 2)
+    target = G.astype(np.float64).T @ Aq                      # E[dW]: LUQ is unbiased
+    # the block's sum: T = sum_{m,n} Q(G)[m,n] * (sum_k Aq[m,k]), a sum of independent terms
+    var_T = float((v * (Aq.sum(axis=1) ** 2)[:, None]).sum()) / 2
+    z_T = abs(float(mean2.sum()) - float(target.sum())) / max(np.sqrt(var_T / pairs), 1e-300)
+    ctx.close()
+    return {"what": f"dW[{block}x{block}] over the first {rows} batch rows, {pairs} seed pairs (2p, 2p+1)",
+            "var_ns1": float(var1.sum()), "var_ns2": float(var2.sum()),
+            "ratio_ns2_over_ns1": float(var2.sum() / var1.sum()),
+            "closed_form_ns1": float(closed1.sum()),
+            "ns1_over_closed_form": float(var1.sum() / closed1.sum()),
+            "ns2_over_closed_form": float(var2.sum() / (closed1.sum() / 2)),
+            "bias_of_block_sum_in_sd": float(z_T)}
+
+
+def bench_layer_compact(torch, binding, inputs, local, args, name, barrier, host_tensors=None, min_seconds=0.3):
+    """Step time of one more configuration, same schedule and launch mode as the headline."""
+    cfg = inputs.CONFIGS[name]
+    lb = LayerBench(torch, binding, cfg, host_tensors if host_tensors is not None else inputs.layer_inputs(cfg),
+                    local, args)
+    for _ in range(3):
+        lb.step()
+    assert lb.status() == 0
+    n0 = lb.launches(); lb.step(); per_step = lb.launches() - n0
+    run_step, mode = lb.capture()
+    st = block_stats(lb.time_blocks(run_step, 20, min_seconds, barrier))
+    assert lb.status() == 0
+    M, K, N = cfg.M, cfg.K, cfg.N
+    out = {"workload": f"M={M} K={K} N={N} {cfg.dtype}, {lb.ns} sample(s)", "ms_per_step": round(st["ms_median"], 5),
+           "ms_min": round(st["ms_min"], 5), "blocks": st["blocks"],
+           "tflops": round(3 * 2.0 * M * N * K / (st["ms_median"] * 1e-3) / 1e12, 2),
+           "launches_per_step": per_step, "launch": mode, "fused_forward": lb.fused}
+    lb.close()
+    del lb
+    torch.cuda.empty_cache()
+    return out
+
+def run_sweep(args, binding, inputs, torch, local, exponents=None, extras=True, emit=True):
     """Quantizer bandwidth sweep (config 4): amax + LUQ quantize-and-pack on 1-D fp32
     gradient tensors of 2^20..2^30 elements, 1 and 2 samples.  GB/s = algorithmic bytes
     (4 + 4 + 0.5 n_s per element: the tensor is read twice, codes written once) / time.
@@ -185,7 +476,7 @@ def run_sweep(args, binding, inputs, torch, local):
     peaks = load_peaks()
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     rows = []
-    for e in inputs.SWEEP_EXPONENTS:
+    for e in (exponents or inputs.SWEEP_EXPONENTS):
         n = 1 << e
         x = torch.from_numpy(inputs.sweep_tensor(e)).cuda()
         mx, al = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
@@ -213,7 +504,7 @@ def run_sweep(args, binding, inputs, torch, local):
             # in-hindsight maximum (one pass over the tensor) and power-of-two scale
             mh = mx.clone()
             extra = {}
-            for name, fn, nbytes in (
+            for name, fn, nbytes in () if not extras else (
                     ("hindsight", lambda: ctx.quant_grad_hindsight(x, mh, 0.1, 0, ns, False, codes, al, mx), (4 + 0.5 * ns) * n),
                     ("hindsight_pw2", lambda: ctx.quant_grad_hindsight(x, mh, 0.1, 0, ns, True, codes, al, mx), (4 + 0.5 * ns) * n),
                     ("amax_plus_pw2", lambda: (ctx.amax(x, mx), ctx.quant_grad_pw2(x, mx, 0, ns, codes, al)), (8 + 0.5 * ns) * n),
@@ -241,9 +532,13 @@ def run_sweep(args, binding, inputs, torch, local):
         del x
         torch.cuda.empty_cache()
     assert ctx.status() == 0
-    print(json.dumps({"metric": "luq_quantizer_hbm_gbs", "unit": "GB/s", "workload": "cfg4 sweep", "dtype": "f32",
-                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "rows": rows}))
     ctx.close()
+    del flush
+    torch.cuda.empty_cache()
+    if emit:
+        print(json.dumps({"metric": "luq_quantizer_hbm_gbs", "unit": "GB/s", "workload": "cfg4 sweep", "dtype": "f32",
+                          "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "rows": rows}))
+    return rows
 
 
 def run_ours(args):
@@ -273,131 +568,43 @@ def run_ours(args):
     if args.rows:
         import dataclasses
         cfg = dataclasses.replace(cfg, M=min(cfg.M, args.rows))
-    M, K, N, ns, seed = cfg.M, cfg.K, cfg.N, cfg.n_samples, cfg.luq_seed
-    A_h, W_h, G_h = inputs.layer_inputs(cfg)
-    if cfg.dtype == "bf16":
-        A_h, W_h, G_h = (t.view(np.int16) for t in (A_h, W_h, G_h))
-    pin = lambda a: torch.from_numpy(a).pin_memory()  # noqa: E731
-    A_p, W_p, G_p = pin(A_h), pin(W_h), pin(G_h)
-    A, W, G = A_p.cuda(), W_p.cuda(), G_p.cuda()
-    if cfg.dtype == "bf16":
-        A, W, G = (t.view(torch.bfloat16) for t in (A, W, G))
-        A_p, W_p, G_p = (t.view(torch.bfloat16) for t in (A_p, W_p, G_p))
-    ctx = binding.Context(local)
-    if args.mma_kind is not None:
-        ctx.set_option(binding.OPT_MMA_KIND, args.mma_kind)
-    dev = A.device
-    f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)  # noqa: E731
-    u8 = lambda *s: torch.empty(s, dtype=torch.uint8, device=dev)  # noqa: E731
-    mA, mW, mG, sA, sW, aG = (f32(1) for _ in range(6))
-    cA, cW, cG = u8(M * K // 2), u8(N * K // 2), u8(ns, M * N // 2)
-    # Operand bytes (the 8-bit form of the codes, written by the quantizer in the same pass) for
-    # the tensors that many GEMM tiles re-read: always W and G; A when the layer is wide enough
-    # that the forward product reads each row block of A four times or more.
-    i8 = lambda n: torch.empty(n, dtype=torch.int8, device=dev)  # noqa: E731
-    oW, oG = i8(N * K), i8(ns * M * N)
-    oA = i8(M * K) if N >= 1024 else None
-    Z, dA, dW = f32(M, N), f32(M, K), f32(N, K)
-    Z_p, dA_p, dW_p = (torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in (Z, dA, dW))
-
-    calls = {
-        "amax_A": lambda: ctx.amax(A, mA), "amax_W": lambda: ctx.amax(W, mW),
-        "quant_int4_A": lambda: ctx.quant_int4(A, mA, cA, sA, oA),
-        "quant_int4_W": lambda: ctx.quant_int4(W, mW, cW, sW, oW),
-        "gemm_fwd": lambda: ctx.gemm_fwd(cA, sA, cW, sW, M, N, K, Z, oA, oW),
-        "amax_G": lambda: ctx.amax(G, mG), "quant_grad_G": lambda: ctx.quant_grad(G, mG, seed, ns, cG, aG, oG),
-        "gemm_bwd": lambda: ctx.gemm_bwd(cG, aG, ns, cW, sW, M, N, K, dA, oG, oW),
-        "gemm_wgrad": lambda: ctx.gemm_wgrad(cG, aG, ns, cA, sA, M, N, K, dW, oG, oA),
-    }
-
-    def step(events=None):
-        for name in KERNELS:
-            if events is not None:
-                e0 = torch.cuda.Event(enable_timing=True); e0.record()
-            calls[name]()
-            if events is not None:
-                e1 = torch.cuda.Event(enable_timing=True); e1.record()
-                events[name].append((e0, e1))
+    host_tensors = inputs.layer_inputs(cfg)
+    lb = LayerBench(torch, binding, cfg, host_tensors, local, args)
+    M, K, N, ns, seed = lb.M, lb.K, lb.N, lb.ns, lb.seed
+    dev = lb.A.device
+    ctx, ctx_g = lb.ctx, lb.ctx_g
 
     for _ in range(max(args.warmup, 3)):
-        step()
-    assert ctx.status() == 0
+        lb.step_one_stream()
+    assert lb.status() == 0
 
     sampler = ClockSampler(gpu_physical_index(local))
     sampler.start()
     sampler.ready.wait(10.0)
-    # The gradient's max and LUQ pass depend on nothing the forward half of the step produces.  With
-    # --streams 2 (the default) they run on a second stream, through a second context (a context's
-    # scratch and workspace serve one stream at a time), beside the activation/weight quantizers and the
-    # forward GEMM; the backward and update GEMMs wait for both.
-    ctx_g = binding.Context(local) if args.streams == 2 else ctx
-    if args.mma_kind is not None and ctx_g is not ctx:
-        ctx_g.set_option(binding.OPT_MMA_KIND, args.mma_kind)
-    stream_g = torch.cuda.Stream() if args.streams == 2 else None
-
-    def timed_step():
-        if stream_g is None:
-            return step()
-        main = torch.cuda.current_stream()
-        fork = torch.cuda.Event(); fork.record(main)
-        stream_g.wait_event(fork)
-        with torch.cuda.stream(stream_g):
-            ctx_g.amax(G, mG); ctx_g.quant_grad(G, mG, seed, ns, cG, aG, oG)
-            join = torch.cuda.Event(); join.record(stream_g)
-        for name in ("amax_A", "amax_W", "quant_int4_A", "quant_int4_W", "gemm_fwd"):
-            calls[name]()
-        main.wait_event(join)
-        calls["gemm_bwd"](); calls["gemm_wgrad"]()
-
-    # No call of the path allocates or synchronises with the host, so one step is captured in a CUDA
-    # graph and replayed: the small configurations are bound by launch rate otherwise.
-    launches0 = ctx.launches + (ctx_g.launches if ctx_g is not ctx else 0)
-    timed_step()
-    launches_per_step = ctx.launches + (ctx_g.launches if ctx_g is not ctx else 0) - launches0
-    run_step, launch_mode = timed_step, "direct calls"
-    if not args.no_graph:
-        try:
-            side = torch.cuda.Stream()
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                timed_step()
-                torch.cuda.synchronize()
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(graph, stream=side):
-                    timed_step()
-            torch.cuda.current_stream().wait_stream(side)
-            torch.cuda.synchronize()
-            graph.replay()
-            torch.cuda.synchronize()
-            run_step, launch_mode = graph.replay, "CUDA graph of the step's calls, replayed"
-        except Exception as e:  # pragma: no cover
-            launch_mode = f"direct calls (graph capture failed: {e!r})"
-    # The timed region: K steps, two events around the whole of it.
-    barrier()
-    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for _ in range(args.steps):
-        run_step()
-    t1.record()
-    barrier()
-    total_ms = t0.elapsed_time(t1)
-    launches = launches_per_step * args.steps
-    total_ms = replicas.max_over_ranks(total_ms, dev)
-    assert ctx.status() == 0 and ctx_g.status() == 0
-    ms_per_step = total_ms / args.steps
-    # The same K steps once more with an event pair around every call, for the per-kernel
-    # durations (the 18 extra event records per step lengthen a step, so this pass is not
-    # the one the throughput comes from).
-    events = {k: [] for k in KERNELS}
-    # 27 host calls per step here: on the short configurations the host would fall behind the GPU and
-    # the idle time would be booked on the kernels.  Hold the GPU back while the host queues the pass.
-    try:
+    launches0 = lb.launches()
+    lb.step()
+    launches_per_step = lb.launches() - launches0
+    run_step, launch_mode = lb.capture()
+    # The timed region: blocks of K replays, an event pair around each, at least a second in total.
+    t_region = time.perf_counter()
+    per_block = lb.time_blocks(run_step, args.steps, args.min_seconds, barrier)
+    t_region = time.perf_counter() - t_region
+    assert lb.status() == 0
+    stats = block_stats(per_block)
+    ms_per_step = replicas.max_over_ranks(stats["ms_median"], dev)
+    launches = launches_per_step * args.steps * stats["blocks"]
+    # The same K steps once more, on one stream, with an event pair around every call, for the
+    # per-kernel durations (the extra event records lengthen a step, so this pass is not the one the
+    # throughput comes from).
+    events = {k: [] for k in lb.kernels}
+    try:   # hold the GPU back while the host queues the pass, or idle time would be booked on the kernels
         torch.cuda._sleep(int(args.steps * 0.35e-3 * 2.0e9))
     except Exception:  # pragma: no cover
         pass
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(args.steps):
-        step(events)
+        lb.step_one_stream(events)
     t1.record()
     barrier()
     sampler.stop_flag.set()
@@ -407,16 +614,18 @@ def run_ours(args):
 
     per_kernel_ms = {k: sum(a.elapsed_time(b) for a, b in v) / len(v) for k, v in events.items()}
     alg = algorithmic(cfg, ns)
+    alg["quant_int4_A+gemm_fwd"] = (alg["quant_int4_A"][0] + 0.5 * N * K + 4 * M * N, alg["gemm_fwd"][1])
     peaks = load_peaks()
-    # 8-bit tensor peak: the nominal fp8 : bf16 ratio (2) on the measured bf16 BURST figure.  The GEMMs of
-    # this step run for tens of microseconds at the full SM clock, far from the power cap under which
-    # the sustained figure (1.3 GHz) was taken.
-    fp8_peak = 2.0 * peaks["bf16_tflops"]
+    # 8-bit tensor peak: measured here with a library GEMM (burst: these kernels run for tens of
+    # microseconds at the full SM clock); the nominal 2 x bf16 figure is kept beside it.
+    tensor_peak = None if args.no_peak else measure_tensor_peak(torch)
+    nominal_peak = 2.0 * peaks["bf16_tflops"]
+    fp8_peak = (tensor_peak or {}).get("burst_tflops") or nominal_peak
+    tensor_peak_source = ("measured in this run: library 8-bit GEMM, burst" if (tensor_peak or {}).get("burst_tflops")
+                          else f"{peaks['source']} bf16 burst x2 (nominal ratio; no 8-bit library GEMM ran)")
     props = torch.cuda.get_device_properties(local)
     clocks_summary = sampler.summary()
-
-    def sampler_max_mhz():
-        return float(clocks_summary.get("sm_max_mhz") or 1965.0)
+    sm_max_mhz = float(clocks_summary.get("sm_max_mhz") or 1965.0)
     kernels = {}
     for k, ms in per_kernel_ms.items():
         b, f = alg[k]
@@ -427,102 +636,118 @@ def run_ours(args):
             ach, peak, unit = b / (ms * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s"
         else:
             ach, peak, unit = f / (ms * 1e-3) / 1e12, fp8_peak, "TFLOP/s"
-        if k == "quant_grad_G":
-            # The LUQ quantizer is bound by instruction issue, not by HBM: per 32 elements about 21 issue
-            # cycles of decision and packing plus, per sample, 20 for the five wide multiplies of
-            # Philox4x32-10 (4 issue cycles each, measured) and 3 for the operand bytes.  Peak = what
-            # 4 sub-partitions per SM issue at the SM clock.
-            cycles = 21 + ns * (20 + 3)
-            alu_peak = props.multi_processor_count * 4 * sampler_max_mhz() * 1e6 * 32 / cycles / 1e9   # Gelt/s
-            if alu_peak * 1e9 < (peaks["hbm_gbs"] * 1e9) / (b / (M * N)):
-                bound, ach, peak, unit = "alu", M * N / (ms * 1e-3) / 1e9, round(alu_peak, 1), "Gelt/s"
         kernels[k] = {"ms": round(ms, 5), "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit,
                       "frac": round(ach / peak, 4), "tflops": round(f / (ms * 1e-3) / 1e12, 2) if f else None,
-                      "gbs": round(b / (ms * 1e-3) / 1e9, 1)}
+                      "gbs": round(b / (ms * 1e-3) / 1e9, 1), "frac_hbm": round(b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+        if f:
+            kernels[k]["frac_tensor_nominal_2x_bf16"] = round(f / (ms * 1e-3) / 1e12 / nominal_peak, 4)
+        if k == "quant_grad_G":
+            # Secondary figure, a MODEL, not a roofline: issue cycles per warp and element of the LUQ kernel
+            # (about 21 for decision and packing plus, per sample, 20 for the five wide multiplies of
+            # Philox4x32-10 and 3 for the operand bytes) against what 4 sub-partitions per SM issue.
+            cycles = 21 + ns * (20 + 3)
+            issue_peak = props.multi_processor_count * 4 * sm_max_mhz * 1e6 * 32 / cycles / 1e9   # Gelt/s
+            kernels[k]["issue_model_frac"] = round(M * N / (ms * 1e-3) / 1e9 / issue_peak, 4)
+            kernels[k]["issue_model_peak_gelts"] = round(issue_peak, 1)
     dominant = max(per_kernel_ms, key=per_kernel_ms.get)
     d = kernels[dominant]
+    full_cfg2 = args.workload == "cfg2" and not args.rows
     roofline = {"kernel": dominant, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
                 "frac": d["frac"],
-                "traffic": NCU_TRAFFIC_BYTES.get(dominant) if (args.workload == "cfg2" and not args.rows) else None,
+                "traffic": NCU_TRAFFIC_BYTES.get(dominant) if full_cfg2 else None,
+                "traffic_source": TRAFFIC_SOURCE if (full_cfg2 and dominant in NCU_TRAFFIC_BYTES) else None,
                 "algorithmic_bytes": alg[dominant][0], "algorithmic_flops": alg[dominant][1],
-                "peak_source": {"hbm": f"{peaks['source']} hbm copy",
-                                "tensor": f"{peaks['source']} bf16 burst x2 (8-bit operands)",
-                                "alu": "derived: issue cycles per element x SM sub-partitions x SM clock"}[d["bound"]]}
+                "peak_source": {"hbm": f"{peaks['source']} hbm copy", "tensor": tensor_peak_source}[d["bound"]]}
+    # whole step against its own HBM ceiling: every tensor read twice (max, quantize), codes written and
+    # read by the GEMMs, fp32 outputs written
+    eb = 2 if cfg.dtype == "bf16" else 4
+    step_bytes = (2 * eb * (M * K + N * K + M * N) + 0.5 * (M * K + N * K + ns * M * N)
+                  + (0.5 * M * K + 0.5 * N * K + 4 * M * N) + (0.5 * ns * M * N + 0.5 * N * K + 4 * M * K)
+                  + (0.5 * ns * M * N + 0.5 * M * K + 4 * N * K))
+    step_roofline = {"algorithmic_bytes": step_bytes, "hbm_floor_ms": step_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                     "frac_of_hbm_ceiling": round(step_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_per_step, 4),
+                     "frac_of_tensor_peak": round(value / world / fp8_peak, 4)}
 
     # ---- the variant the paper proposes against the max passes (Sec. 7): every tensor is quantized with
-    # the estimate of earlier steps while its own maximum is measured in the same kernel - six launches
-    # instead of nine, one read of each tensor instead of two.  Reported beside the headline, not as it:
-    # the codes differ (a lagging estimate saturates / clips), the named path is max-then-quantize.
+    # the estimate of earlier steps while its own maximum is measured in the same kernel - one read of each
+    # tensor instead of two.  Reported beside the headline, not as it: the codes differ (a lagging
+    # estimate saturates / clips), the named path is max-then-quantize.
     hindsight = None
-    if not args.no_graph:
+    if not args.no_graph and not args.rows:
         try:
-            eA, eW, eG = mA.clone(), mW.clone(), mG.clone()      # estimates, initialised with the true maxima
+            eA, eW, eG = lb.mA.clone(), lb.mW.clone(), lb.mG.clone()      # estimates, initialised with the true maxima
             meas = torch.empty(3, device=dev)
 
             def hindsight_step():
                 main = torch.cuda.current_stream()
                 fork = torch.cuda.Event(); fork.record(main)
-                side_stream = stream_g if stream_g is not None else main
-                if stream_g is not None:
-                    stream_g.wait_event(fork)
+                side_stream = lb.stream_g if lb.stream_g is not None else main
+                if lb.stream_g is not None:
+                    lb.stream_g.wait_event(fork)
                 with torch.cuda.stream(side_stream):
-                    ctx_g.quant_grad_hindsight(G, eG, 0.1, seed, ns, False, cG, aG, meas[2:3], oG)
+                    ctx_g.quant_grad_hindsight(lb.G, eG, 0.1, seed, ns, False, lb.cG, lb.aG, meas[2:3], lb.oG)
                     join = torch.cuda.Event(); join.record(side_stream)
-                ctx.quant_int4_hindsight(A, eA, 0.1, cA, sA, meas[0:1], oA)
-                ctx.quant_int4_hindsight(W, eW, 0.1, cW, sW, meas[1:2], oW)
-                calls["gemm_fwd"]()
+                ctx.quant_int4_hindsight(lb.A, eA, 0.1, lb.cA, lb.sA, meas[0:1], lb.oA)
+                ctx.quant_int4_hindsight(lb.W, eW, 0.1, lb.cW, lb.sW, meas[1:2], lb.oW)
+                lb.calls["gemm_fwd"]()
                 main.wait_event(join)
-                calls["gemm_bwd"](); calls["gemm_wgrad"]()
+                lb.calls["gemm_bwd"](); lb.calls["gemm_wgrad"]()
 
-            side = torch.cuda.Stream()
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                hindsight_step()
-                torch.cuda.synchronize()
-                hgraph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(hgraph, stream=side):
-                    hindsight_step()
-            torch.cuda.current_stream().wait_stream(side)
-            for _ in range(3):
-                hgraph.replay()
-            barrier()
-            t0.record()
-            for _ in range(args.steps):
-                hgraph.replay()
-            t1.record()
-            barrier()
-            h_ms = replicas.max_over_ranks(t0.elapsed_time(t1) / args.steps, dev)
-            assert ctx.status() == 0 and ctx_g.status() == 0
+            n0 = lb.launches(); hindsight_step(); h_launches = lb.launches() - n0
+            h_run, _ = lb.capture(hindsight_step)
+            hs = block_stats(lb.time_blocks(h_run, args.steps, 0.3, barrier))
+            h_ms = replicas.max_over_ranks(hs["ms_median"], dev)
+            assert lb.status() == 0
             hindsight = {"ms_per_step": h_ms, "value": world * flops_step / (h_ms * 1e-3) / 1e12, "unit": UNIT,
-                         "launches_per_step": 6 + (launches_per_step - 9),
+                         "launches_per_step": h_launches,
                          "what": "in-hindsight maxima for A, W and G (eta 0.1): no max pass, one kernel per tensor"}
         except Exception as e:  # pragma: no cover
             hindsight = {"unavailable": repr(e)}
 
-    # ---- end to end: host buffers in, host buffers out, through the same calls
+    # ---- the nine separate calls, for comparison, when the headline used the fused forward kernel
+    named = None
+    if lb.fused and not args.rows:
+        saved = lb.kernels, lb.fused
+        lb.kernels, lb.fused = KERNELS, False
+        try:
+            n_run, _ = lb.capture()
+            nst = block_stats(lb.time_blocks(n_run, args.steps, 0.3, barrier))
+            named = {"ms_per_step": nst["ms_median"], "value": world * flops_step / (nst["ms_median"] * 1e-3) / 1e12,
+                     "what": "quant_int4(A) and gemm_fwd as two kernels (nine calls per step)"}
+        except Exception as e:  # pragma: no cover
+            named = {"unavailable": repr(e)}
+        lb.kernels, lb.fused = saved
+        assert lb.status() == 0
+
+    # ---- end to end: host buffers in, host buffers out, through the same calls.  Every step copies its
+    # inputs from pinned host memory and its three results back; the copies of neighbouring steps overlap
+    # with the kernels and with each other (both copy engines): two sets of device buffers, a copy-in
+    # stream, the compute stream, a copy-out stream.
     e2e = None
     cpu_baseline = None
-
-    # Every step copies its inputs from pinned host memory and its three results back.  The copies
-    # of neighbouring steps overlap with the kernels and with each other (both copy engines): two
-    # sets of device buffers, a copy-in stream, the compute stream, a copy-out stream.
     if not args.kernel_only:
+        A_p, W_p, G_p = lb.host
+        Z_p, dA_p, dW_p = (torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in (lb.Z, lb.dA, lb.dW))
         e2e_steps = max(6, min(args.steps, 10))
         s_cmp = torch.cuda.current_stream()
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
-        ins = [(A, W, G), tuple(torch.empty_like(t) for t in (A, W, G))]
-        outs = [(Z, dA, dW), tuple(torch.empty_like(t) for t in (Z, dA, dW))]
+        ins = [(lb.A, lb.W, lb.G), tuple(torch.empty_like(t) for t in (lb.A, lb.W, lb.G))]
+        outs = [(lb.Z, lb.dA, lb.dW), tuple(torch.empty_like(t) for t in (lb.Z, lb.dA, lb.dW))]
         ev_in = [torch.cuda.Event() for _ in range(2)]
         ev_done = [torch.cuda.Event() for _ in range(2)]
         ev_out = [torch.cuda.Event() for _ in range(2)]
 
         def e2e_calls(a, w, g, z, da, dw):
-            ctx.amax(a, mA); ctx.amax(w, mW)
-            ctx.quant_int4(a, mA, cA, sA, oA); ctx.quant_int4(w, mW, cW, sW, oW)
-            ctx.gemm_fwd(cA, sA, cW, sW, M, N, K, z, oA, oW)
-            ctx.amax(g, mG); ctx.quant_grad(g, mG, seed, ns, cG, aG, oG)
-            ctx.gemm_bwd(cG, aG, ns, cW, sW, M, N, K, da, oG, oW)
-            ctx.gemm_wgrad(cG, aG, ns, cA, sA, M, N, K, dw, oG, oA)
+            ctx.amax(a, lb.mA); ctx.amax(w, lb.mW)
+            ctx.quant_int4(w, lb.mW, lb.cW, lb.sW, lb.oW)
+            if lb.fused:
+                ctx.quant_int4_gemm_fwd(a, lb.mA, lb.cW, lb.sW, M, N, K, lb.cA, lb.sA, z, lb.oW)
+            else:
+                ctx.quant_int4(a, lb.mA, lb.cA, lb.sA, lb.oA)
+                ctx.gemm_fwd(lb.cA, lb.sA, lb.cW, lb.sW, M, N, K, z, lb.oA, lb.oW)
+            ctx.amax(g, lb.mG); ctx.quant_grad(g, lb.mG, seed, ns, lb.cG, lb.aG, lb.oG)
+            ctx.gemm_bwd(lb.cG, lb.aG, ns, lb.cW, lb.sW, M, N, K, da, lb.oG, lb.oW)
+            ctx.gemm_wgrad(lb.cG, lb.aG, ns, lb.cA, lb.sA, M, N, K, dw, lb.oG, lb.oA)
 
         def e2e_run(n_steps):
             for i in range(n_steps):
@@ -553,8 +778,7 @@ def run_ours(args):
         t1.record()
         barrier()
         assert ctx.status() == 0
-        e2e_ms = t0.elapsed_time(t1) / e2e_steps
-        e2e_ms = replicas.max_over_ranks(e2e_ms, dev)
+        e2e_ms = replicas.max_over_ranks(t0.elapsed_time(t1) / e2e_steps, dev)
         h2d = sum(t.numel() * t.element_size() for t in (A_p, W_p, G_p))
         d2h = sum(t.numel() * t.element_size() for t in (Z_p, dA_p, dW_p))
         e2e = {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
@@ -562,6 +786,33 @@ def run_ours(args):
                "overlap": "copies of neighbouring steps overlap with the kernels (3 streams, 2 buffer sets)"}
         del ins, outs
         torch.cuda.empty_cache()
+
+    # ---- the other configurations in compact form (rank 0, one GPU): cfg1, cfg3, cfg5 step times and the
+    # quantizer sweep's two largest practical sizes; config 5 with its variance study
+    configs = None
+    variance = None
+    if rank == 0 and world == 1 and not args.kernel_only and not args.rows and not args.no_configs:
+        configs = {}
+        try:
+            if args.workload in ("cfg2", "cfg5"):
+                other = "cfg5" if args.workload == "cfg2" else "cfg2"
+                configs[other] = bench_layer_compact(torch, binding, inputs, local, args, other, barrier,
+                                                     host_tensors=lb.host)
+            for name in ("cfg1", "cfg3"):
+                if name != args.workload:
+                    configs[name] = bench_layer_compact(torch, binding, inputs, local, args, name, barrier)
+            configs["cfg4"] = [{k: r[k] for k in ("elements", "n_samples", "cold")}
+                               for r in run_sweep(args, binding, inputs, torch, local, exponents=(26, 28),
+                                                  extras=False, emit=False)]
+        except Exception as e:  # pragma: no cover
+            configs["error"] = repr(e)[:300]
+    if rank == 0 and world == 1 and not args.kernel_only and not args.rows and (args.workload == "cfg5" or configs is not None):
+        try:
+            variance = variance_study(torch, binding, inputs, local)
+            if configs is not None and "cfg5" in configs:
+                configs["cfg5"]["variance"] = variance
+        except Exception as e:  # pragma: no cover
+            variance = {"unavailable": repr(e)[:300]}
 
     if rank == 0 and world == 1 and not args.kernel_only:
         rows = min(32768, M)   # about 15 s of host time on config 2
@@ -579,21 +830,29 @@ def run_ours(args):
                                    f"LUQ seed {seed}, {ns} sample(s)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                        "launch": launch_mode,
+                       "fused_forward": "quant_int4(A) + gemm_fwd in one kernel (luq_quant_int4_gemm_fwd)" if lb.fused else "no",
+                       "operand_bytes": "W,G" + (",A" if lb.oA is not None else "") +
+                                        ": the quantizers also write the codes' 8-bit form, the GEMMs are handed it",
                        "streams": "2: gradient max + LUQ beside the activation/weight quantizers and the forward GEMM"
                                   if args.streams == 2 else "1",
-                       "l2": "inputs (%d MB of activations per step) against a 126 MB L2; no explicit flush" % (A.numel() * A.element_size() >> 20)},
+                       "l2": "inputs (%d MB of activations per step) against a 126 MB L2; no explicit flush" % (lb.A.numel() * lb.A.element_size() >> 20)},
+            "timing": {"blocks": stats["blocks"], "steps_per_block": args.steps, "ms_per_step": "median block",
+                       "ms_min": stats["ms_min"], "ms_max": stats["ms_max"], "ms_spread": stats["ms_spread"],
+                       "timed_region_s": round(t_region, 3)},
+            "step_roofline": step_roofline,
+            "tensor_peak_measured": tensor_peak, "tensor_peak_nominal_2x_bf16": nominal_peak,
             "luq_quantizer_gbs": kernels["quant_grad_G"]["gbs"],
+            "luq_quantizer_frac_hbm": kernels["quant_grad_G"]["frac_hbm"],
             "amax_plus_luq_gbs": round((alg["amax_G"][0] + alg["quant_grad_G"][0]) /
                                        ((per_kernel_ms["amax_G"] + per_kernel_ms["quant_grad_G"]) * 1e-3) / 1e9, 1),
             "ms_per_step_with_per_kernel_events": round(instrumented_ms, 5),
-            "hindsight_variant": hindsight,
-            "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "hindsight_variant": hindsight, "separate_forward_kernels_variant": named,
+            "roofline": roofline, "kernels": kernels, "configs": configs, "variance": variance,
+            "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": int(launches), "clocks": clocks_summary,
         }
         print(json.dumps(line))
-    if ctx_g is not ctx:
-        ctx_g.close()
-    ctx.close()
+    lb.close()
     if world > 1:
         dist.destroy_process_group()
 
@@ -609,8 +868,12 @@ def main():
     ap.add_argument("--rows", type=int, default=None, help="truncate the batch dimension M (small profiling runs)")
     ap.add_argument("--streams", type=int, choices=(1, 2), default=2,
                     help="2: the gradient's max and LUQ pass run on a second stream beside the forward half")
+    ap.add_argument("--min-seconds", type=float, default=1.0, help="least duration of the timed region")
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of a replayed CUDA graph")
-    ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs")
+    ap.add_argument("--no-fused", action="store_true", help="quant_int4(A) and gemm_fwd as two kernels")
+    ap.add_argument("--no-peak", action="store_true", help="do not measure the 8-bit tensor peak with a library GEMM")
+    ap.add_argument("--no-configs", action="store_true", help="skip the compact runs of the other configurations")
+    ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end, other-configuration and CPU-baseline legs")
     ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1, 2],
                     help="tensor-core operand type: 0 e4m3 (kind::f8f6f4), 1 int8 (kind::i8), 2 per product; default: the library's")
     args = ap.parse_args()

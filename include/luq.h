@@ -77,6 +77,12 @@ extern "C" {
                               scale max/7).  Such an operand is fetched as bytes: the caller's operand bytes,
                               or a plane expanded into the context workspace (LUQ_ERR_WORKSPACE beyond 76 MiB).
                               Not available in luq_gemm_wgrad_static. */
+#define LUQ_OPT_SM_LIMIT 8 /* n >= 1: the GEMMs of this context occupy at most n SMs (one persistent CTA each; the
+                              contraction split is chosen for n SMs); 0 (default): all SMs.  Two products that do not
+                              depend on one another - the backward product, which is bound by its output stream and
+                              leaves the tensor cores idle, and the update product, which is bound by the tensor
+                              cores and moves little memory - can then run side by side on two streams (two
+                              contexts), each on its share of the SMs.  Results do not depend on the limit. */
 #define LUQ_OPT_LEVELS 4   /* kmax of the gradient quantizers, 1..6 (default luq_kmax() = 4): levels
                               alpha * 2^0 .. alpha * 2^kmax with alpha = max / 2^kmax, codes 0..kmax+1.  The
                               other grids of the paper from the same kernels: kmax = 2 is the FP2 grid of
@@ -274,6 +280,23 @@ int luq_debug_expire_wait(luq_ctx* ctx, void* stream);
 int luq_gemm_fwd(luq_ctx* ctx, const uint8_t* d_a_codes, const float* d_sa, const int8_t* d_a_operand,
                  const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
                  void* d_z, int64_t M, int64_t N, int64_t K, void* stream);
+
+/* luq_quant_int4 of the activations followed by luq_gemm_fwd, as ONE kernel (Eq. Forward on
+ * Q_INT(A), Sec. 3.3; Sec. 7 "Reducing the data movement": the passes over the tensors, not the
+ * MACs, are the cost).  For a layer with one column of output tiles (N <= 256) every row block
+ * of A is read by exactly one tile, so the GEMM takes the HIGH-PRECISION activations d_a
+ * [M x K, fp32 or bf16], quantizes them on the way in with the clip *d_clip (usually the max from
+ * luq_amax), and writes their packed codes d_a_codes [M x K/2] and scale *d_sa as by-products
+ * (the update GEMM reads them).  A is streamed once at memory speed and the tensor-core work
+ * hides under that stream.  Codes, scale, status bits and Z are exactly those of the two
+ * separate calls.  d_w_operand (optional): W's operand bytes from luq_quant_int4; without them
+ * W's codes are widened once into the context workspace.  K must be a multiple of 32.  Where
+ * the fusion does not apply (N > 256, bf16 output, unsigned activations, e4m3 operands forced)
+ * the call runs the two separate kernels. */
+int luq_quant_int4_gemm_fwd(luq_ctx* ctx, const void* d_a, int dtype, const float* d_clip,
+                            uint8_t* d_a_codes, float* d_sa,
+                            const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
+                            void* d_z, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* Backward GEMM (Eq. Backward), SMP average fused (Sec. 5.1):
  *   dA[m,k] = (alpha*sw/n_samples) * sum_s sum_n qG_s[m,n] * qW[n,k].

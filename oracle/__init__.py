@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
             L.oracle_gemm_fwd.argtypes = [u8p, dbl, u8p, dbl, i64, i64, i64, f64p]
             L.oracle_gemm_bwd.argtypes = [u8p, dbl, ctypes.c_int, u8p, dbl, i64, i64, i64, f64p]
             L.oracle_gemm_wgrad.argtypes = [u8p, dbl, ctypes.c_int, u8p, dbl, i64, i64, i64, f64p]
+            L.oracle_gemm_general.argtypes = [ctypes.c_int, u8p, ctypes.c_int, dbl, ctypes.c_int, u8p, ctypes.c_int, dbl,
+                                              i64, i64, i64, f64p]
             L.oracle_gemm_int64.argtypes = [ctypes.c_int, u8p, ctypes.c_int, u8p, i64, i64, i64, i64p]
             L.oracle_gemm_entries.argtypes = [ctypes.c_int, u8p, dbl, ctypes.c_int, u8p, dbl,
                                               i64, i64, i64, i64p, i64p, sz, f64p]
@@ -301,6 +303,22 @@ def gemm_wgrad(g_codes, alpha, n_samples, a_codes, sa, M, N, K) -> np.ndarray:
     lib().oracle_gemm_wgrad(_ptr(g_codes, ctypes.c_uint8), float(alpha), n_samples,
                             _ptr(a_codes, ctypes.c_uint8), float(sa), M, N, K, _ptr(dW, ctypes.c_double))
     return dW
+
+
+def gemm_general(which: str, x_codes, x_kind: str, sx, n_samples, y_codes, y_kind: str, sy, M, N, K) -> np.ndarray:
+    """The three products for operands of any code kind ('int4', 'luq', 'uint4'): `x` is the
+    activations (fwd) or the gradient planes (bwd, wgrad), `y` the weights (fwd, bwd) or the
+    activations (wgrad).  Same definition as gemm_fwd / gemm_bwd / gemm_wgrad."""
+    w = {"fwd": 0, "bwd": 1, "wgrad": 2}[which]
+    kinds = {"int4": 0, "luq": 1, "uint4": 2}
+    shape = {"fwd": (M, N), "bwd": (M, K), "wgrad": (N, K)}[which]
+    x_codes = np.ascontiguousarray(x_codes).reshape(-1)
+    y_codes = np.ascontiguousarray(y_codes).reshape(-1)
+    out = np.zeros(shape, dtype=np.float64)
+    lib().oracle_gemm_general(w, _ptr(x_codes, ctypes.c_uint8), kinds[x_kind], float(sx), n_samples,
+                              _ptr(y_codes, ctypes.c_uint8), kinds[y_kind], float(sy), M, N, K,
+                              _ptr(out, ctypes.c_double))
+    return out
 
 
 def gemm_int64(which: str, x_codes, n_samples, y_codes, M, N, K) -> np.ndarray:

@@ -403,8 +403,15 @@ double oracle_luq_value(uint8_t nibble) { /* in units of alpha */
 }
 
 /* ------------------------------------------------------------------------ */
-/* Dequantise and multiply: the plain definition (Appendix A.1: the scale is  */
-/* a single high-precision factor, all MACs act on the low-precision values). */
+/* Dequantise and multiply (Eqs. Forward / Backward / Update on quantized     */
+/* tensors).  Appendix A.1: a quantized tensor is ONE high-precision scale    */
+/* times low-precision values, and "all MACs act on the low-precision values": */
+/*   out = (s_x * s_y) * sum_k v_x[k] * v_y[k]                                 */
+/* with v the integer-valued codes (INT4: q; LUQ: +-2^(c-1); unsigned: nibble). */
+/* The sum is formed in double over those integers - exact below 2^53, so an   */
+/* output whose products cancel is exactly 0 - and the scale product is        */
+/* applied once.  SMP (Sec. 5.1) averages the RESULTS of the n_s samples: the   */
+/* samples' products are added and the sum is divided by n_s at the end.        */
 /* kind: 0 = INT4 codes (value q*scale), 1 = LUQ codes (value +-scale*2^(c-1)),  */
 /*       2 = unsigned INT4 codes (value nibble*scale)                            */
 /* ------------------------------------------------------------------------ */
@@ -418,77 +425,125 @@ void oracle_dequant(const uint8_t* codes, size_t n, double scale, int kind, doub
   for (size_t i = 0; i < n; ++i) out[i] = scale * code_value(codes, i, kind);
 }
 
-/* Z[M x N] = A_d . W_d^T with A_d = dequant(A codes [M x K]), W_d = dequant(W codes [N x K]) */
+/* the low-precision values of a packed tensor, as doubles (unit scale) */
+static double* code_values(const uint8_t* codes, size_t n, int kind) {
+  double* v = (double*)malloc(sizeof(double) * (n ? n : 1));
+  for (size_t i = 0; i < n; ++i) v[i] = code_value(codes, i, kind);
+  return v;
+}
+
+/* Z[M x N] = (sa*sw) * A_v . W_v^T, A_v / W_v the values of the A codes [M x K] / W codes [N x K] */
 void oracle_gemm_fwd(const uint8_t* a_codes, double sa, const uint8_t* w_codes, double sw,
                      int64_t M, int64_t N, int64_t K, double* Z) {
-  double* Ad = (double*)malloc(sizeof(double) * (size_t)(M * K));
-  double* Wd = (double*)malloc(sizeof(double) * (size_t)(N * K));
-  oracle_dequant(a_codes, (size_t)(M * K), sa, 0, Ad);
-  oracle_dequant(w_codes, (size_t)(N * K), sw, 0, Wd);
+  double* Av = code_values(a_codes, (size_t)(M * K), 0);
+  double* Wv = code_values(w_codes, (size_t)(N * K), 0);
+  const double scale = sa * sw;
 #pragma omp parallel for schedule(static)
   for (int64_t m = 0; m < M; ++m)
     for (int64_t n = 0; n < N; ++n) {
       double acc = 0.0;
-      for (int64_t k = 0; k < K; ++k) acc += Ad[m * K + k] * Wd[n * K + k];
-      Z[m * N + n] = acc;
+      for (int64_t k = 0; k < K; ++k) acc += Av[m * K + k] * Wv[n * K + k];
+      Z[m * N + n] = scale * acc;
     }
-  free(Ad); free(Wd);
+  free(Av); free(Wv);
 }
 
-/* Sample planes of the gradient, each dequantised on its own: Gs[s][M x N] */
-static double* gradient_samples(const uint8_t* g_codes, double alpha, int n_samples,
-                                int64_t M, int64_t N) {
-  size_t n = (size_t)(M * N), plane = (n + 1) / 2;
-  double* Gs = (double*)malloc(sizeof(double) * n * (size_t)n_samples);
-  for (int s = 0; s < n_samples; ++s)
-    oracle_dequant(g_codes + plane * (size_t)s, n, alpha, 1, Gs + n * (size_t)s);
-  return Gs;
-}
-
-/* dA[M x K] = (1/n_s) sum_s G_d,s . W_d.  SMP (Sec. 5.1) averages the RESULTS of the
- * n_s samples: every sample's product is formed, the products are added, and the
- * sum is divided by n_s once at the end. */
+/* dA[M x K] = (alpha*sw) * (sum_s G_v,s . W_v) / n_s */
 void oracle_gemm_bwd(const uint8_t* g_codes, double alpha, int n_samples,
                      const uint8_t* w_codes, double sw,
                      int64_t M, int64_t N, int64_t K, double* dA) {
-  double* Gs = gradient_samples(g_codes, alpha, n_samples, M, N);
-  double* Wd = (double*)malloc(sizeof(double) * (size_t)(N * K));
-  oracle_dequant(w_codes, (size_t)(N * K), sw, 0, Wd);
+  size_t gn = (size_t)(M * N), plane = (gn + 1) / 2;
+  double** Gv = (double**)malloc(sizeof(double*) * (size_t)n_samples);
+  for (int s = 0; s < n_samples; ++s) Gv[s] = code_values(g_codes + plane * (size_t)s, gn, 1);
+  double* Wv = code_values(w_codes, (size_t)(N * K), 0);
+  const double scale = alpha * sw;
 #pragma omp parallel for schedule(static)
   for (int64_t m = 0; m < M; ++m)
     for (int64_t k = 0; k < K; ++k) {
       double acc = 0.0;
-      for (int s = 0; s < n_samples; ++s) {
-        const double* Gd = Gs + (size_t)s * (size_t)(M * N);
-        for (int64_t n = 0; n < N; ++n) acc += Gd[m * N + n] * Wd[n * K + k];
-      }
-      dA[m * K + k] = acc / (double)n_samples;
+      for (int s = 0; s < n_samples; ++s)
+        for (int64_t n = 0; n < N; ++n) acc += Gv[s][m * N + n] * Wv[n * K + k];
+      dA[m * K + k] = scale * acc / (double)n_samples;
     }
-  free(Gs); free(Wd);
+  for (int s = 0; s < n_samples; ++s) free(Gv[s]);
+  free(Gv); free(Wv);
 }
 
-/* dW[N x K] = (1/n_s) sum_s G_d,s^T . A_d  (Sec. 5.1: the average of the samples' weight gradients) */
+/* dW[N x K] = (alpha*sa) * (sum_s G_v,s^T . A_v) / n_s  (Sec. 5.1: the average of the samples' weight gradients) */
 void oracle_gemm_wgrad(const uint8_t* g_codes, double alpha, int n_samples,
                        const uint8_t* a_codes, double sa,
                        int64_t M, int64_t N, int64_t K, double* dW) {
-  double* Gs = gradient_samples(g_codes, alpha, n_samples, M, N);
-  double* Ad = (double*)malloc(sizeof(double) * (size_t)(M * K));
-  oracle_dequant(a_codes, (size_t)(M * K), sa, 0, Ad);
+  size_t gn = (size_t)(M * N), plane = (gn + 1) / 2;
+  double** Gv = (double**)malloc(sizeof(double*) * (size_t)n_samples);
+  for (int s = 0; s < n_samples; ++s) Gv[s] = code_values(g_codes + plane * (size_t)s, gn, 1);
+  double* Av = code_values(a_codes, (size_t)(M * K), 0);
+  const double scale = alpha * sa;
 #pragma omp parallel for schedule(static)
   for (int64_t n = 0; n < N; ++n)
     for (int64_t k = 0; k < K; ++k) {
       double acc = 0.0;
-      for (int s = 0; s < n_samples; ++s) {
-        const double* Gd = Gs + (size_t)s * (size_t)(M * N);
-        for (int64_t m = 0; m < M; ++m) acc += Gd[m * N + n] * Ad[m * K + k];
-      }
-      dW[n * K + k] = acc / (double)n_samples;
+      for (int s = 0; s < n_samples; ++s)
+        for (int64_t m = 0; m < M; ++m) acc += Gv[s][m * N + n] * Av[m * K + k];
+      dW[n * K + k] = scale * acc / (double)n_samples;
     }
-  free(Gs); free(Ad);
+  for (int s = 0; s < n_samples; ++s) free(Gv[s]);
+  free(Gv); free(Av);
 }
 
-/* Second, independent form (Appendix A.1 scale factoring): integer codes are
- * multiplied and summed in int64, the scale product is applied once.
+/* The same three products for operands of any code kind (the unsigned INT4 activations of
+ * Appendix "Quantization formats", the INT4 gradient codes of the ablation's uniform arm):
+ * which 0 fwd  out[M x N] = (sx*sy)   sum_k   x[m,k] y[n,k]        x = activations, y = weights
+ *       1 bwd  out[M x K] = (sx*sy)/ns sum_s,n x_s[m,n] y[n,k]     x = gradient planes, y = weights
+ *       2 wgrad out[N x K] = (sx*sy)/ns sum_s,m x_s[m,n] y[m,k]    x = gradient planes, y = activations */
+void oracle_gemm_general(int which, const uint8_t* x_codes, int x_kind, double sx, int n_samples,
+                         const uint8_t* y_codes, int y_kind, double sy,
+                         int64_t M, int64_t N, int64_t K, double* out) {
+  const double scale = sx * sy;
+  if (which == 0) {
+    double* Xv = code_values(x_codes, (size_t)(M * K), x_kind);
+    double* Yv = code_values(y_codes, (size_t)(N * K), y_kind);
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+      for (int64_t n = 0; n < N; ++n) {
+        double acc = 0.0;
+        for (int64_t k = 0; k < K; ++k) acc += Xv[m * K + k] * Yv[n * K + k];
+        out[m * N + n] = scale * acc;
+      }
+    free(Xv); free(Yv);
+    return;
+  }
+  size_t gn = (size_t)(M * N), plane = (gn + 1) / 2;
+  double** Gv = (double**)malloc(sizeof(double*) * (size_t)n_samples);
+  for (int s = 0; s < n_samples; ++s) Gv[s] = code_values(x_codes + plane * (size_t)s, gn, x_kind);
+  if (which == 1) {
+    double* Wv = code_values(y_codes, (size_t)(N * K), y_kind);
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+      for (int64_t k = 0; k < K; ++k) {
+        double acc = 0.0;
+        for (int s = 0; s < n_samples; ++s)
+          for (int64_t n = 0; n < N; ++n) acc += Gv[s][m * N + n] * Wv[n * K + k];
+        out[m * K + k] = scale * acc / (double)n_samples;
+      }
+    free(Wv);
+  } else {
+    double* Av = code_values(y_codes, (size_t)(M * K), y_kind);
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+      for (int64_t k = 0; k < K; ++k) {
+        double acc = 0.0;
+        for (int s = 0; s < n_samples; ++s)
+          for (int64_t m = 0; m < M; ++m) acc += Gv[s][m * N + n] * Av[m * K + k];
+        out[n * K + k] = scale * acc / (double)n_samples;
+      }
+    free(Av);
+  }
+  for (int s = 0; s < n_samples; ++s) free(Gv[s]);
+  free(Gv);
+}
+
+/* The same sums in integer arithmetic (a cross-check of the double sums above):
+ * the values are multiplied and summed in int64.
  * which: 0 fwd, 1 bwd, 2 wgrad.  out gets the integer sums (not yet scaled,
  * summed over the n_samples planes). */
 void oracle_gemm_int64(int which, const uint8_t* x_codes, int n_samples, const uint8_t* y_codes,
@@ -529,8 +584,8 @@ void oracle_gemm_int64(int which, const uint8_t* x_codes, int n_samples, const u
 }
 
 /* Selected output entries of the three products at any size, computed one by
- * one from the codes (same definition as above: dequantise, multiply, add in
- * double, the samples' products added and divided by n_s at the end).  which: 0 fwd (r=m, c=n), 1 bwd (r=m, c=k), 2 wgrad (r=n, c=k). */
+ * one from the codes (same definition as above: the values' products added in
+ * double, one scale product, the samples' sum divided by n_s at the end).  which: 0 fwd (r=m, c=n), 1 bwd (r=m, c=k), 2 wgrad (r=n, c=k). */
 void oracle_gemm_entries(int which, const uint8_t* x_codes, double sx, int n_samples,
                          const uint8_t* y_codes, double sy,
                          int64_t M, int64_t N, int64_t K,
@@ -542,21 +597,19 @@ void oracle_gemm_entries(int which, const uint8_t* x_codes, double sx, int n_sam
     double acc = 0.0;
     if (which == 0) {
       for (int64_t k = 0; k < K; ++k)
-        acc += (sx * code_value(x_codes, (size_t)(r * K + k), 0)) *
-               (sy * code_value(y_codes, (size_t)(c * K + k), 0));
+        acc += code_value(x_codes, (size_t)(r * K + k), 0) * code_value(y_codes, (size_t)(c * K + k), 0);
     } else if (which == 1) {
       for (int s = 0; s < n_samples; ++s)
         for (int64_t n = 0; n < N; ++n)
-          acc += (sx * code_value(x_codes + plane * (size_t)s, (size_t)(r * N + n), 1)) *
-                 (sy * code_value(y_codes, (size_t)(n * K + c), 0));
-      acc /= (double)n_samples;
+          acc += code_value(x_codes + plane * (size_t)s, (size_t)(r * N + n), 1) *
+                 code_value(y_codes, (size_t)(n * K + c), 0);
     } else {
       for (int s = 0; s < n_samples; ++s)
         for (int64_t m = 0; m < M; ++m)
-          acc += (sx * code_value(x_codes + plane * (size_t)s, (size_t)(m * N + r), 1)) *
-                 (sy * code_value(y_codes, (size_t)(m * K + c), 0));
-      acc /= (double)n_samples;
+          acc += code_value(x_codes + plane * (size_t)s, (size_t)(m * N + r), 1) *
+                 code_value(y_codes, (size_t)(m * K + c), 0);
     }
+    acc = (sx * sy) * acc / (double)n_samples;
     out[e] = acc;
   }
 }

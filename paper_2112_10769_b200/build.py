@@ -48,7 +48,7 @@ def _stamp(target: str, digest: str) -> None:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "nvcc")
-    headers = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "luq.h")]
+    headers = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "int4_math.cuh"), os.path.join(ROOT, "include", "luq.h")]
     objs, digests, running = [], [], []
     for name, extra in UNITS.items():
         src = os.path.join(CSRC, name)

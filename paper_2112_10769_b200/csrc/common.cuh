@@ -22,6 +22,7 @@ struct luq_ctx {
   int out_bf16;             // the GEMMs write bf16 outputs
   int unsigned_act;         // activation codes handed to the forward / update GEMMs are unsigned INT4
   int grad_int4;            // gradient codes handed to the backward / update GEMMs are INT4 (the ablation's uniform arm)
+  int sm_limit;             // GEMM grids use at most this many SMs (0 = all)
   int kmax;                 // LUQ levels alpha * 2^0 .. alpha * 2^kmax (1..6, default LUQ_KMAX)
   int64_t launches;
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved at create
@@ -83,6 +84,13 @@ struct luq_gemm_args {
 };
 int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st);
 int luq_launch_expire_wait(luq_ctx* ctx, cudaStream_t st);
+// Forward product that quantizes its activations itself (one column of output tiles): writes the INT4
+// codes of A, its scale and Z = Q(A) . Q(W)^T.  d_w_operand may be null (W's codes are then widened
+// into the workspace).  Call only when luq_quant_fwd_fusable() says yes.
+bool luq_quant_fwd_fusable(const luq_ctx* ctx, int64_t M, int64_t N, int64_t K, bool have_w_bytes);
+int luq_launch_quant_fwd(luq_ctx* ctx, const void* d_a, int dtype, const float* d_clip, uint8_t* d_a_codes,
+                         float* d_sa, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
+                         float* d_z, int64_t M, int64_t N, int64_t K, cudaStream_t st);
 
 #ifdef __CUDACC__
 

@@ -46,6 +46,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "int4_math.cuh"
 
 namespace {
 
@@ -210,7 +211,8 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       mbar_init(ex_full(s), (kAnyPacked ? kConvWarps : 0) + (kAnyPlane ? 1 : 0));
       mbar_init(ex_empty(s), 1);
     }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
+    // whole-row staging has two epilogue warps per quarter of the accumulator's rows
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), ROWS ? 8 : 4); }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -370,12 +372,16 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (ok) tc_commit(acc_full(buf));
       }
     }
-  } else if (warp < kPlaneWarp) {
+  } else if (warp < kPlaneWarp || (ROWS && warp >= kFirstConvWarp && warp < kFirstConvWarp + 4)) {
     // ---------------------------------------------------------------- epilogue
+    // (whole-row staging: the kernel has no converters, and four of their warps form a second
+    // epilogue group - a warp may only read the quarter of tensor memory given by its index mod 4,
+    // so the two warps of a quarter share its rows and take four 32-column chunks each)
     const int quarter = warp & 3;  // tensor-memory lanes this warp may read
+    const int half = warp >= kFirstConvWarp ? 1 : 0;
     const float scale = p.splits == 1 ? (__ldg(p.scale_a) * __ldg(p.scale_b)) * p.post_scale : 1.0f;
-    const uint32_t stage0 = base + C::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
-    uint8_t* const stage0_gen = gen + C::staging + (warp - kFirstEpiWarp) * 2 * kStageBox;
+    const uint32_t stage0 = base + C::staging + ((warp - kFirstEpiWarp) & 3) * 2 * kStageBox;
+    uint8_t* const stage0_gen = gen + C::staging + ((warp - kFirstEpiWarp) & 3) * 2 * kStageBox;
     const int sw = lane & 7;
     const bool out_bf16 = p.out_bf16 && p.splits == 1;   // partial tiles of a split stay fp32
     uint32_t tile_it = 0, box_it = 0;
@@ -440,9 +446,14 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // threads to write unit s at step s they would hit one bank.  So thread `lane` writes unit
         // s ^ (lane & 7) at step s: its units are first permuted by that XOR (three rounds of
         // conditional swaps), and eight consecutive lanes then cover the eight slots of a 128-byte line.
-        const uint32_t strip = base + C::staging + (warp - kFirstEpiWarp) * kStripBytes;
-        uint8_t* const rowp = gen + C::staging + (warp - kFirstEpiWarp) * kStripBytes + lane * (BN * 4);
+        // The two warps of a quarter fill the same strip (chunks 0-3 and 4-7) and meet at a
+        // named barrier of 64 threads before and after: the first warp waits for the previous
+        // store to have read the strip, and issues this tile's store.
+        const int slot = (warp - kFirstEpiWarp) & 3;
+        const uint32_t strip = base + C::staging + slot * kStripBytes;
+        uint8_t* const rowp = gen + C::staging + slot * kStripBytes + lane * (BN * 4);
         const bool in_range = row0 < row_limit;       // warp-uniform
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + slot) : "memory"); };
         auto emit_rows = [&](uint32_t (&r)[32], int c) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
@@ -463,31 +474,32 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               }
             }
           }
-          if (c == 0) {   // first write of this tile: the previous tile's store must have read the strip
-            if (lane == 0) bulk_wait_read<0>();
-            __syncwarp();
-          }
           uint8_t* const line = rowp + c * 128;
           const int key = sw ^ (c & 7);
 #pragma unroll
           for (int s = 0; s < 8; ++s)   // position s holds unit s ^ sw, whose slot is (s ^ sw) ^ c
             *reinterpret_cast<uint4*>(line + ((s ^ key) << 4)) = make_uint4(r[4 * s], r[4 * s + 1], r[4 * s + 2], r[4 * s + 3]);
         };
+        constexpr int kChunks = BN / 32 / 2;          // chunks per warp
+        const int c_first = half * kChunks;
         uint32_t r0[32], r1[32];
-        tmem_ld_32x32(taddr, r0);
+        tmem_ld_32x32(taddr + c_first * 32, r0);
+        // first write of this tile: the previous tile's store must have read the strip
+        if (half == 0 && lane == 0) bulk_wait_read<0>();
+        pair_sync();
         tmem_ld_wait();
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; c += 2) {
+        for (int c = c_first; c < c_first + kChunks; c += 2) {
           tmem_ld_32x32(taddr + (c + 1) * 32, r1);
           emit_rows(r0, c);
           tmem_ld_wait();
-          if (c + 2 < BN / 32) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
+          if (c + 2 < c_first + kChunks) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
           emit_rows(r1, c + 1);
           tmem_ld_wait();
         }
         fence_proxy_async();
-        __syncwarp();
-        if (lane == 0 && in_range) {   // chunks and rows beyond the tensor are clipped by the copy
+        pair_sync();
+        if (half == 0 && lane == 0 && in_range) {   // chunks and rows beyond the tensor are clipped by the copy
           tma_store_3d(&tm_out, strip, 0, static_cast<int>(col_base / 32), static_cast<int>(row0));
           bulk_commit();
         }
@@ -784,6 +796,345 @@ luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   }
 }
 
+// ---------------------------------------------------------------------------
+// Activation quantizer fused into the forward GEMM (Eq. Forward with Q_INT of
+// Sec. 3.3 applied on the way in), for layers with one column of output tiles
+// (N <= 256): every 128-row block of A is then read by exactly one tile, so the
+// GEMM can take the HIGH-PRECISION activations, quantize them itself and write
+// the packed codes (the update GEMM needs them) as a by-product.  The kernel
+// streams A once at HBM speed and the tensor-core work hides under that stream.
+//   warp 0       TMA producer of raw activations: boxes of 128 rows x 32 elements
+//                (128-byte swizzle for fp32, 64-byte for bf16), two boxes per raw stage
+//   warp 6       TMA producer of W's operand bytes (two 128 x 128 slabs per stage)
+//   warps 7-14   converters: one row of one box per thread -> 32 INT4 codes; the codes go
+//                packed into a staging box that one thread stores with TMA (32-byte
+//                swizzle), and widened (16 * q) into the A slab of the operand stage
+//   warp 1       tcgen05.mma issue, kind::i8, accumulators in tensor memory (2 x 256 columns)
+//   warps 2-5    epilogue (one 32 x 32 staging box per warp)
+// An operand stage (128 deep) is made of two raw stages (64 deep).  Codes are
+// bit-identical to the streaming quantizer's: same arithmetic (int4_math.cuh).
+// ---------------------------------------------------------------------------
+template <bool BF16>
+struct FusedCfg {
+  static constexpr int box_bytes = 128 * 32 * (BF16 ? 2 : 4);   // one raw box
+  static constexpr int raw_stage = 2 * box_bytes;               // 64 contraction elements of 128 rows
+  static constexpr int RS = BF16 ? 6 : 3;                       // raw stages: 96 KB
+  static constexpr int ES = 2;                                  // operand stages
+  static constexpr int code_box = 128 * 32;                     // packed codes of one raw stage
+  static constexpr int threads = 32 * (kFirstConvWarp + 8);
+  static constexpr int expanded = 0;
+  static constexpr int raw = expanded + ES * kExpandedStage;
+  static constexpr int codes = raw + RS * raw_stage;            // two code boxes
+  static constexpr int staging = codes + 2 * code_box;          // 4 warps x 1 box
+  static constexpr int barriers = staging + 4 * kStageBox;
+  static constexpr int num_barriers = 2 * RS + 2 * ES + 4;
+  static constexpr int tmem_slot = barriers + 8 * num_barriers;
+  static constexpr int abort_flag = tmem_slot + 4;
+  static constexpr int total = abort_flag + 4;
+  static constexpr int smem_bytes = total + 1024;
+  static_assert(smem_bytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+};
+
+struct FusedParams {
+  const float* clip;      // max|A| (or a caller's clip)
+  const float* scale_b;   // weight scale
+  float* scale_a_out;     // receives clip / 7
+  unsigned int* status;
+  long long Mo, No, Kc;
+  int tiles_m, num_kb;
+};
+
+// all converter threads meet; returns true when every one of them passed `ok`
+__device__ __forceinline__ bool conv_barrier_all(bool ok) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred q, r;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred r, 5, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, r;\n\t}"
+      : "=r"(out) : "r"(static_cast<uint32_t>(ok)) : "memory");
+  return out != 0;
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__((FusedCfg<BF16>::threads), 1)
+luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_constant__ CUtensorMap tm_b,
+                     const __grid_constant__ CUtensorMap tm_codes, const __grid_constant__ CUtensorMap tm_out,
+                     const FusedParams p) {
+  using C = FusedCfg<BF16>;
+  constexpr int RS = C::RS, ES = C::ES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* const gen = smem_raw + (base - raw);
+
+  const uint32_t bar0 = base + C::barriers;
+  auto raw_full = [&](int s) { return bar0 + 8u * s; };
+  auto raw_empty = [&](int s) { return bar0 + 8u * (RS + s); };
+  auto ex_full = [&](int s) { return bar0 + 8u * (2 * RS + s); };
+  auto ex_empty = [&](int s) { return bar0 + 8u * (2 * RS + ES + s); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * RS + 2 * ES + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * RS + 2 * ES + 2 + b); };
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + C::tmem_slot);
+  volatile uint32_t* const abort_flag = reinterpret_cast<volatile uint32_t*>(gen + C::abort_flag);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < RS; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), 8); }
+    for (int s = 0; s < ES; ++s) {
+      mbar_init(ex_full(s), 2 * 8 + 1);   // eight converter warps for each half of the stage, and W's producer
+      mbar_init(ex_empty(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&tm_raw); tma_prefetch_desc(&tm_b); tma_prefetch_desc(&tm_codes); tma_prefetch_desc(&tm_out);
+  }
+  if (warp == 1) {
+    tmem_alloc(base + C::tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_trigger();
+
+  const int raw_iters = 2 * p.num_kb;   // raw stages per tile
+
+  if (warp == 0) {
+    // ------------------------------------------ producer of raw activations
+    if (lane == 0) {
+      uint32_t issued = 0, stage = 0, phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < p.tiles_m; t += gridDim.x) {
+        const int m0 = t * BM;
+        for (int it = 0; it < raw_iters; ++it) {
+          if (!mbar_wait(raw_empty(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t full = raw_full(stage);
+          const uint32_t dst = base + C::raw + stage * C::raw_stage;
+          mbar_arrive_expect_tx(full, C::raw_stage);
+          tma_load_2d(dst, &tm_raw, full, it * 64, m0);                      // columns beyond K read as zero
+          tma_load_2d(dst + C::box_bytes, &tm_raw, full, it * 64 + 32, m0);
+          ++issued;
+          if (++stage == static_cast<uint32_t>(RS)) { stage = 0; phase ^= 1u; }
+        }
+      }
+      for (int s = 0; s < RS; ++s) {   // drain: every copy issued here has landed before the CTA exits
+        if (issued > static_cast<uint32_t>(s)) {
+          const uint32_t last = (issued - 1 - s) / RS;
+          mbar_wait(raw_full(s), last & 1u, abort_flag);
+        }
+      }
+    }
+  } else if (warp == kPlaneWarp) {
+    // ------------------------------------------ producer of W's operand bytes
+    if (lane == 0) {
+      uint32_t issued = 0, stage = 0, phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < p.tiles_m; t += gridDim.x) {
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!mbar_wait(ex_empty(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t full = ex_full(stage);
+          const uint32_t dst = base + C::expanded + stage * kExpandedStage;
+          mbar_arrive_expect_tx(full, 2 * kExpandedSlab);
+          tma_load_2d(dst + kExpandedSlab, &tm_b, full, kb * BK, 0);
+          tma_load_2d(dst + 2 * kExpandedSlab, &tm_b, full, kb * BK, 128);
+          ++issued;
+          if (++stage == static_cast<uint32_t>(ES)) { stage = 0; phase ^= 1u; }
+        }
+      }
+      for (int s = 0; s < ES; ++s) {
+        if (issued > static_cast<uint32_t>(s)) {
+          const uint32_t last = (issued - 1 - s) / ES;
+          mbar_wait(ex_full(s), last & 1u, abort_flag);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10)      // S32 accumulator, signed 8-bit A and B
+                                 | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
+      const uint32_t a0 = base + C::expanded, b0 = a0 + kExpandedSlab;
+      const uint64_t da0 = umma_desc_sw128(a0, 16, 1024), db0 = umma_desc_sw128(b0, 16, 1024);
+      constexpr uint64_t kStep = 32 >> 4, kStageStep = kExpandedStage >> 4;
+      uint32_t stage = 0, phase = 0, tile_it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < p.tiles_m; t += gridDim.x, ++tile_it) {
+        const uint32_t buf = tile_it & 1u;
+        if (!mbar_wait(acc_empty(buf), ((tile_it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + buf * BN;
+        uint32_t accumulate = 0;
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!mbar_wait(ex_full(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t da = da0 + stage * kStageStep, db = db0 + stage * kStageStep;
+#pragma unroll
+          for (int kk = 0; kk < BK / 32; ++kk) {
+            tc_mma<1>(tmem_d, da + kk * kStep, db + kk * kStep, idesc, accumulate);
+            accumulate = 1;
+          }
+          tc_commit(ex_empty(stage));
+          if (++stage == static_cast<uint32_t>(ES)) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit(acc_full(buf));
+      }
+    }
+  } else if (warp < kPlaneWarp) {
+    // ---------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;
+    const float clip = __ldg(p.clip);
+    const float sa = scale_usable(clip, nullptr) ? clip / 7.0f : 0.0f;
+    const float scale = (sa * __ldg(p.scale_b)) * (1.0f / 256.0f);   // both operands carry 16 * q
+    const uint32_t box = base + C::staging + (warp - kFirstEpiWarp) * kStageBox;
+    uint8_t* const rowp = gen + C::staging + (warp - kFirstEpiWarp) * kStageBox + lane * 128;
+    const int sw = lane & 7;
+    uint32_t tile_it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < p.tiles_m; t += gridDim.x, ++tile_it) {
+      const long long row0 = static_cast<long long>(t) * BM + quarter * 32;
+      const uint32_t buf = tile_it & 1u;
+      if (!mbar_wait(acc_full(buf), (tile_it >> 1) & 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN;
+      auto emit = [&](const uint32_t (&r)[32], int c) {
+        const long long col0 = c * 32;
+        if (row0 < p.Mo && col0 < p.No) {   // warp-uniform
+          if (lane == 0) bulk_wait_read<0>();          // the store that last read this box is done
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            float4 v;
+            v.x = static_cast<float>(static_cast<int>(r[4 * j])) * scale;
+            v.y = static_cast<float>(static_cast<int>(r[4 * j + 1])) * scale;
+            v.z = static_cast<float>(static_cast<int>(r[4 * j + 2])) * scale;
+            v.w = static_cast<float>(static_cast<int>(r[4 * j + 3])) * scale;
+            *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tm_out, box, static_cast<int>(col0), static_cast<int>(row0));
+            bulk_commit();
+          }
+        }
+      };
+      uint32_t r0[32], r1[32];
+      tmem_ld_32x32(taddr, r0);
+      tmem_ld_wait();
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; c += 2) {
+        tmem_ld_32x32(taddr + (c + 1) * 32, r1);
+        emit(r0, c);
+        tmem_ld_wait();
+        if (c + 2 < BN / 32) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
+        emit(r1, c + 1);
+        tmem_ld_wait();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(buf));
+    }
+    if (lane == 0) bulk_wait<0>();
+  } else if (warp >= kFirstConvWarp) {
+    // -------------------------------------------------------------- converters
+    const int cw = warp - kFirstConvWarp;          // 0..7
+    const int ctid = threadIdx.x - kFirstConvWarp * 32;
+    const int boxi = cw >> 2;                      // which box of the raw stage
+    const int row = (cw & 3) * 32 + lane;          // row of the tile
+    const float clip = __ldg(p.clip);
+    const bool first = blockIdx.x == 0 && ctid == 0;
+    const bool usable = scale_usable(clip, first ? p.status : nullptr);
+    const float inv = usable ? 7.0f / clip : 0.0f;   // an unusable clip gives zero codes and a zero scale
+    if (first) *p.scale_a_out = usable ? clip / 7.0f : 0.0f;
+    constexpr int kUnits = BF16 ? 4 : 8;           // 16-byte units of a box row
+    // position of unit u of this row inside the swizzled box image
+    const int rkey = BF16 ? ((row >> 1) & 3) : (row & 7);
+    const uint32_t row_off = row * (BF16 ? 64 : 128);
+    uint32_t rs = 0, rphase = 0, es = 0, ephase = 0, stored = 0;
+    bool alive = true;
+    for (int t = blockIdx.x; alive && t < p.tiles_m; t += gridDim.x) {
+      const int m0 = t * BM;
+      for (int it = 0; it < raw_iters; ++it) {
+        const int second = it & 1;                 // which half of the operand stage
+        bool ok = mbar_wait(raw_full(rs), rphase, abort_flag);
+        if (ok && !second) ok = mbar_wait(ex_empty(es), ephase ^ 1u, abort_flag);
+        if (ok) {
+          const uint8_t* src = gen + C::raw + rs * C::raw_stage + boxi * C::box_bytes + row_off;
+          uint4 u[kUnits];
+#pragma unroll
+          for (int j = 0; j < kUnits; ++j) u[j] = *reinterpret_cast<const uint4*>(src + ((j ^ rkey) << 4));
+          // 32 elements -> 32 codes, element e in nibble e % 8 of word e / 8
+          uint32_t w[4] = {0u, 0u, 0u, 0u};
+          if constexpr (BF16) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t h[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                w[j] |= int4_code(__uint_as_float(h[i] << 16), inv) << (8 * i);
+                w[j] |= int4_code(__uint_as_float(h[i] & 0xFFFF0000u), inv) << (8 * i + 4);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t sh = 16 * (j & 1);
+              w[j >> 1] |= int4_code(__uint_as_float(u[j].x), inv) << sh;
+              w[j >> 1] |= int4_code(__uint_as_float(u[j].y), inv) << (sh + 4);
+              w[j >> 1] |= int4_code(__uint_as_float(u[j].z), inv) << (sh + 8);
+              w[j >> 1] |= int4_code(__uint_as_float(u[j].w), inv) << (sh + 12);
+            }
+          }
+          const uint4 packed = make_uint4(w[0], w[1], w[2], w[3]);
+          // operand bytes 16 * q, element order, into this row of the A slab (128-byte swizzle)
+          uint4 o0, o1;
+          expand32<1, false, false>(packed, make_uint4(0u, 0u, 0u, 0u), o0, o1);
+          uint8_t* drow = gen + C::expanded + es * kExpandedStage + row * 128;
+          const int unit = second * 4 + boxi * 2;
+          *reinterpret_cast<uint4*>(drow + ((unit ^ (row & 7)) << 4)) = o0;
+          *reinterpret_cast<uint4*>(drow + (((unit + 1) ^ (row & 7)) << 4)) = o1;
+          // packed codes into the staging box of this raw stage: 128 rows x 32 bytes, 32-byte swizzle
+          uint8_t* cbox = gen + C::codes + (stored & 1u) * C::code_box;
+          *reinterpret_cast<uint4*>(cbox + row * 32 + ((boxi ^ ((row >> 2) & 1)) << 4)) = packed;
+          fence_proxy_async();   // both writes are read by the async proxy (tensor core, TMA store)
+        }
+        // the store that read the other code box two raw stages ago has long finished; the one
+        // issued a stage ago must have read its box before that box is written again next time
+        if (ctid == 0) bulk_wait_read<0>();
+        alive = conv_barrier_all(ok);
+        if (!alive) break;
+        if (ctid == 0 && it * 64 < p.Kc) {
+          tma_store_2d(&tm_codes, base + C::codes + (stored & 1u) * C::code_box, it * 32, m0);
+          bulk_commit();
+        }
+        ++stored;
+        if (lane == 0) { mbar_arrive(raw_empty(rs)); mbar_arrive(ex_full(es)); }
+        if (++rs == static_cast<uint32_t>(RS)) { rs = 0; rphase ^= 1u; }
+        if (second) { if (++es == static_cast<uint32_t>(ES)) { es = 0; ephase ^= 1u; } }
+      }
+    }
+    if (ctid == 0) bulk_wait<0>();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, LUQ_STATUS_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
 // Sums the partial tiles of a split contraction in a fixed order, applies the
 // scales and writes the output.  One thread per float4 of a tile.
 __global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restrict__ ws, void* __restrict__ out_any,
@@ -978,10 +1329,12 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   p.num_kb = static_cast<int>((a.Kc + BK - 1) / BK);
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const int total_iters = p.n_samples * p.num_kb;
+  // the SMs this product may occupy (LUQ_OPT_SM_LIMIT): one persistent CTA each
+  const int sms = (ctx->sm_limit > 0 && ctx->sm_limit < ctx->sm_count) ? ctx->sm_limit : ctx->sm_count;
   int splits = 1;
   if (a.allow_split) {
     if (ctx->forced_splits > 0) splits = ctx->forced_splits;
-    else if (tiles * 2 <= ctx->sm_count) splits = static_cast<int>(ctx->sm_count / tiles);
+    else if (tiles * 2 <= sms) splits = static_cast<int>(sms / tiles);
     if (splits > total_iters / 4 && ctx->forced_splits <= 0) splits = total_iters / 4;
     if (splits > total_iters) splits = total_iters;
     if (splits < 1) splits = 1;
@@ -1103,7 +1456,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   // is not split: option LUQ_OPT_PAIRS (off unless set)
   if (ctx->use_pairs && a_plane && b_plane && p.splits == 1 && p.tiles_m >= 2 && !a.out_bf16) {
     const long long pair_tiles = static_cast<long long>((p.tiles_m + 1) / 2) * p.tiles_n;
-    const int max_pairs = ctx->sm_count / 2;
+    const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;
     const int pairs = static_cast<int>(pair_tiles < max_pairs ? pair_tiles : max_pairs);
     const int sel2 = (ctx->mma_kind ? 4 : 0) | (a.a_mn ? 2 : 0) | (a.b_mn ? 1 : 0);
     switch (sel2) {
@@ -1119,7 +1472,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
     return rc;
   }
 
-  const int grid = static_cast<int>(units < ctx->sm_count ? units : ctx->sm_count);
+  const int grid = static_cast<int>(units < sms ? units : sms);
   const int sel = (ctx->mma_kind ? 4 : 0) | (a.a_mn ? 2 : 0) | (a.b_mn ? 1 : 0);
   // the kernels expand signed INT4 codes in B, and in A signed INT4 (forward) or LUQ codes (backward,
   // update); any other kind of operand must have arrived as bytes
@@ -1158,6 +1511,92 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
     if (rc == 0) ctx->launches += 1;
   }
   return rc;
+}
+
+// ---------------------------------------------------------------------------
+// Forward product that quantizes its activations on the way in (luq_quant_int4_gemm_fwd).
+// ---------------------------------------------------------------------------
+namespace {
+
+// high-precision activations [rows x cols]: box of 128 rows x 32 elements, swizzled like the box's row width
+int encode_raw_map(void* fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, bool bf16) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * (bf16 ? 2 : 4)};
+  const cuuint32_t box[2] = {32, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+      map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims,
+      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : 1;
+}
+// packed codes [rows x cols/2 bytes] as the destination of 128-row x 32-byte boxes (32-byte swizzle in shared memory)
+int encode_codes_store_map(void* fn, CUtensorMap* map, uint8_t* ptr, uint64_t rows, uint64_t pitch) {
+  const cuuint64_t dims[2] = {pitch, rows};
+  const cuuint64_t strides[1] = {pitch};
+  const cuuint32_t box[2] = {32, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+      map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : 1;
+}
+
+}  // namespace
+
+// The fused kernel serves one column of output tiles with int8 operands and an fp32 output.
+bool luq_quant_fwd_fusable(const luq_ctx* ctx, int64_t M, int64_t N, int64_t K, bool have_w_bytes) {
+  if (M <= 0 || N <= 0 || K <= 0 || N > BN) return false;
+  if (ctx->mma_kind == 0 || ctx->out_bf16 || ctx->unsigned_act) return false;
+  if (112ll * 112ll * K >= (1ll << 31)) return false;                       // int32 accumulator
+  if (!have_w_bytes) {
+    const size_t bytes = static_cast<size_t>(N) * K;
+    if (bytes % 32 != 0 || ctx->d_workspace == nullptr || ctx->workspace_bytes < kSplitRegionBytes + bytes) return false;
+  }
+  return true;
+}
+
+int luq_launch_quant_fwd(luq_ctx* ctx, const void* d_a, int dtype, const float* d_clip, uint8_t* d_a_codes,
+                         float* d_sa, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
+                         float* d_z, int64_t M, int64_t N, int64_t K, cudaStream_t st) {
+  const bool bf16 = dtype == LUQ_BF16;
+  const uint8_t* w_plane = reinterpret_cast<const uint8_t*>(d_w_operand);
+  if (w_plane == nullptr) {   // widen W's codes once into the workspace (behind the split region)
+    uint8_t* dst = reinterpret_cast<uint8_t*>(ctx->d_workspace) + kSplitRegionBytes;
+    const int rc = launch_expand<1>(false, d_w_codes, dst, static_cast<size_t>(N) * K / 2, make_lut(1, 0), ctx->sm_count, st);
+    if (rc != 0) return rc;
+    ctx->launches += 1;
+    w_plane = dst;
+  }
+  FusedParams p{};
+  p.clip = d_clip; p.scale_b = d_sw; p.scale_a_out = d_sa; p.status = ctx->d_status;
+  p.Mo = M; p.No = N; p.Kc = K;
+  p.tiles_m = static_cast<int>((M + BM - 1) / BM);
+  p.num_kb = static_cast<int>((K + BK - 1) / BK);
+  CUtensorMap t_raw, t_b, t_codes, t_out;
+  int bad = encode_raw_map(ctx->encode_tiled, &t_raw, d_a, M, K, bf16);
+  bad |= encode_bytes_map(ctx->encode_tiled, &t_b, w_plane, K, N, 1, false, true);
+  bad |= encode_codes_store_map(ctx->encode_tiled, &t_codes, d_a_codes, M, K / 2);
+  bad |= encode_out_map(ctx->encode_tiled, &t_out, d_z, M, N, false);
+  if (bad) return LUQ_ERR_CUDA;
+  const int sms = (ctx->sm_limit > 0 && ctx->sm_limit < ctx->sm_count) ? ctx->sm_limit : ctx->sm_count;
+  const int grid = p.tiles_m < sms ? p.tiles_m : sms;
+  cudaError_t e;
+  if (bf16) {
+    auto kernel = luq_quant_fwd_kernel<true>;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<true>::smem_bytes);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = luq_launch_kernel(kernel, grid, FusedCfg<true>::threads, FusedCfg<true>::smem_bytes, st, LUQ_LAUNCH_EARLY, 1,
+                          t_raw, t_b, t_codes, t_out, p);
+  } else {
+    auto kernel = luq_quant_fwd_kernel<false>;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<false>::smem_bytes);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = luq_launch_kernel(kernel, grid, FusedCfg<false>::threads, FusedCfg<false>::smem_bytes, st, LUQ_LAUNCH_EARLY, 1,
+                          t_raw, t_b, t_codes, t_out, p);
+  }
+  if (e == cudaSuccess) ctx->launches += 1;
+  return static_cast<int>(e);
 }
 
 int luq_launch_expire_wait(luq_ctx* ctx, cudaStream_t st) {
@@ -1267,6 +1706,8 @@ extern "C" int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_al
   local.mma_kind = LUQ_DEFAULT_MMA_KIND;
   local.forced_splits = 0;
   local.use_pairs = 0;
+  local.sm_limit = 0;
+  local.grad_int4 = 0;
   local.kmax = LUQ_KMAX;
   local.unsigned_act = 0;
   local.out_bf16 = 0;

@@ -18,6 +18,7 @@
 // Compile this file without FMA contraction and with IEEE division: code
 // decisions must be bit-identical to a scalar IEEE implementation.
 #include "common.cuh"
+#include "int4_math.cuh"
 
 namespace {
 
@@ -27,20 +28,9 @@ constexpr int kUnroll = 4;  // independent 16-byte loads in flight per thread
 // the loads a thread has in flight are 4 KB apart, inside one DRAM page neighbourhood.
 constexpr int kTileItems = kThreads * kUnroll;
 
-// zero, non-finite or far-out-of-range max: every code is zero, the scale is zero
-__device__ __forceinline__ bool scale_usable(float c, unsigned int* status) {
-  const uint32_t b = __float_as_uint(c);
-  if (c == 0.0f) return false;
-  if ((b & 0x7FFFFFFFu) >= 0x7F800000u || (b >> 31)) {
-    if (status) atomicOr(status, LUQ_STATUS_NONFINITE);
-    return false;
-  }
-  if (c < 0x1p-100f || c > 0x1p100f) {
-    if (status) atomicOr(status, LUQ_STATUS_RANGE);
-    return false;
-  }
-  return true;
-}
+using luqdev::scale_usable;
+using luqdev::int4_code;
+using luqdev::uint4_code;
 
 template <bool BF16> struct Item {
   static constexpr int kElems = BF16 ? 8 : 4;  // elements per 16-byte piece
@@ -306,24 +296,6 @@ __device__ __forceinline__ bool fused_grid_max(const void* __restrict__ x, size_
 }
 
 // ------------------------------------------------------------------ INT4 ----
-// clamp, then add 1.5 * 2^23: the sum's low mantissa bits hold the integer rounded to
-// nearest-even, already in two's complement (clamping before rounding equals clamping
-// after it: the bounds are integers and rounding is monotone)
-__device__ __forceinline__ uint32_t int4_code(float x, float inv) {
-  const float y = x * inv;
-  const float c = fminf(fmaxf(y, -7.0f), 7.0f);
-  const uint32_t code = __float_as_uint(c + 12582912.0f) & 0xFu;
-  return (y == y) ? code : 0u;        // NaN element -> 0
-}
-
-// the same for the unsigned grid 0..15 (the clamp keeps negative inputs at 0)
-__device__ __forceinline__ uint32_t uint4_code(float x, float inv) {
-  const float y = x * inv;
-  const float c = fminf(fmaxf(y, 0.0f), 15.0f);
-  const uint32_t code = __float_as_uint(c + 12582912.0f) & 0xFu;
-  return (y == y) ? code : 0u;
-}
-
 // PLANE: the tensor-core operand bytes (int8, 16 * q: the code nibble in the high half of the
 // byte) are written next to the packed codes, one byte per element in element order.
 // UNSIGNED: the grid 0..15 with scale clip / 15 (non-negative tensors); operand byte = q.

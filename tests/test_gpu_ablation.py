@@ -195,11 +195,10 @@ def test_backward_and_update_products_on_int4_gradient_codes(ctx, M, K, N, ns, w
     finally:
         ctx.set_option(binding.OPT_MMA_KIND, 2)
         ctx.set_option(binding.OPT_GRADIENT_INT4, 0)
-    Gq = sum(oracle.dequant(og[s], M * N, float(osg), "int4").reshape(M, N) for s in range(ns)) / ns
-    Aq = oracle.dequant(ca.cpu().numpy(), M * K, sa.item(), "int4").reshape(M, K)
-    Wq = oracle.dequant(cw.cpu().numpy(), N * K, sw.item(), "int4").reshape(N, K)
-    assert_gemm_close(dA.cpu().numpy(), Gq @ Wq)
-    assert_gemm_close(dW.cpu().numpy(), Gq.T @ Aq)
+    assert_gemm_close(dA.cpu().numpy(), oracle.gemm_general("bwd", og, "int4", float(osg), ns, cw.cpu().numpy(), "int4",
+                                                            sw.item(), M, N, K))
+    assert_gemm_close(dW.cpu().numpy(), oracle.gemm_general("wgrad", og, "int4", float(osg), ns, ca.cpu().numpy(), "int4",
+                                                            sa.item(), M, N, K))
     # the option matters: read as LUQ codes the same nibbles give another product
     dA_luq = ctx.gemm_bwd(cg, sg, ns, cw, sw, M, N, K)
     assert not torch.equal(dA_luq, dA)

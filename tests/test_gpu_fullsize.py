@@ -115,10 +115,11 @@ def test_quantizer_sweep_sizes(ctx, exponent, ns):
     assert ctx.status() == 0
 
 
-def test_quantizer_sweep_largest_size_windows(ctx):
-    """2^30 elements (4 GiB of input): the maximum is checked against numpy, codes
-    on windows at the start, across the 2^32-byte boundary and at the end."""
-    e = inputs.SWEEP_EXPONENTS[-1]
+@pytest.mark.parametrize("e", [28, 30])
+def test_quantizer_sweep_largest_sizes_windows(ctx, e):
+    """2^28 and 2^30 elements (1 and 4 GiB of input): the maximum is checked against numpy, codes
+    on windows at the start, in the middle (for 2^30: across the 2^32-byte boundary) and at the end."""
+    assert e in inputs.SWEEP_EXPONENTS
     n = 1 << e
     x = inputs.sweep_tensor(e)
     xd = to_dev(x)

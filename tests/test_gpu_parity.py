@@ -292,6 +292,28 @@ def test_config1_whole_step(ctx):
     assert ctx.status() == 0
 
 
+def test_empty_contraction_gives_zeros(ctx):
+    """K = 0 in the forward product, an empty batch in the update product: the sum over nothing is 0
+    in every entry of a non-empty output (not stale memory)."""
+    one = scalar(1.0)
+    e = torch.zeros(0, dtype=torch.uint8, device="cuda")
+    Z = torch.full((64, 32), float("nan"), device="cuda")
+    ctx.gemm_fwd(e, one, e, one, 64, 32, 0, out=Z)
+    dW = torch.full((32, 64), float("nan"), device="cuda")
+    ctx.gemm_wgrad(e, one, 2, e, one, 0, 32, 64, out=dW)
+    dA = torch.full((64, 96), float("nan"), device="cuda")
+    ctx.gemm_bwd(e, one, 1, e, one, 64, 0, 96, out=dA)
+    assert not Z.any().item() and not dW.any().item() and not dA.any().item()
+    ctx.set_option(binding.OPT_OUTPUT_BF16, 1)
+    try:
+        Zh = torch.full((64, 32), float("nan"), dtype=torch.bfloat16, device="cuda")
+        ctx.gemm_fwd(e, one, e, one, 64, 32, 0, out=Zh)
+        assert not Zh.any().item()
+    finally:
+        ctx.set_option(binding.OPT_OUTPUT_BF16, 0)
+    assert ctx.status() == 0
+
+
 def test_gemm_large_integer_sums_are_exact(ctx):
     """Worst-case operands (every code at its extreme) over a long contraction:
     the accumulator must hold every integer partial sum exactly."""

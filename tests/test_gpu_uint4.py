@@ -56,10 +56,8 @@ def test_quant_uint4_caller_clip_and_specials(ctx):
 def reference_products(A, W, G, ca, sa, cw, sw, cg, al, ns):
     M, K = A.shape
     N = W.shape[0]
-    Ad = oracle.dequant(ca, M * K, sa, "uint4").reshape(M, K)
-    Wd = oracle.dequant(cw, N * K, sw, "int4").reshape(N, K)
-    Gd = sum(oracle.dequant(cg[s], M * N, al, "luq").reshape(M, N) for s in range(ns)) / ns
-    return Ad @ Wd.T, Gd.T @ Ad
+    return (oracle.gemm_general("fwd", ca, "uint4", sa, 1, cw, "int4", sw, M, N, K),
+            oracle.gemm_general("wgrad", cg, "luq", al, ns, ca, "uint4", sa, M, N, K))
 
 
 @pytest.mark.parametrize("mma_kind", [0, 2])

@@ -472,6 +472,30 @@ def test_gemms_against_numpy_and_int64(M, K, N, ns):
                                dW[rows, cols], rtol=1e-13)
 
 
+def test_general_kind_products_against_numpy_and_the_named_products():
+    """oracle.gemm_general (operands of any code kind) against numpy on the dequantized values, and equal
+    to gemm_fwd / gemm_bwd / gemm_wgrad for the kinds those take."""
+    M, K, N, ns = 10, 12, 8, 3
+    (A, W, G), (ca, sa), (cw, sw), (cg, al) = small_codes(M, K, N, 321, ns)
+    np.testing.assert_array_equal(oracle.gemm_general("fwd", ca, "int4", sa, 1, cw, "int4", sw, M, N, K),
+                                  oracle.gemm_fwd(ca, sa, cw, sw, M, N, K))
+    np.testing.assert_array_equal(oracle.gemm_general("bwd", cg, "luq", al, ns, cw, "int4", sw, M, N, K),
+                                  oracle.gemm_bwd(cg, al, ns, cw, sw, M, N, K))
+    np.testing.assert_array_equal(oracle.gemm_general("wgrad", cg, "luq", al, ns, ca, "int4", sa, M, N, K),
+                                  oracle.gemm_wgrad(cg, al, ns, ca, sa, M, N, K))
+    cu, su, _ = oracle.quant_uint4(np.maximum(A, 0), oracle.amax(A)[0])
+    gi, sg, _ = oracle.quant_int4_sr(G, oracle.amax(G)[0], 5, n_samples=ns)
+    Au = oracle.dequant(cu, M * K, su, "uint4").reshape(M, K)
+    Wd = oracle.dequant(cw, N * K, sw, "int4").reshape(N, K)
+    Gi = np.mean([oracle.dequant(gi[s], M * N, sg, "int4").reshape(M, N) for s in range(ns)], axis=0)
+    np.testing.assert_allclose(oracle.gemm_general("fwd", cu, "uint4", su, 1, cw, "int4", sw, M, N, K), Au @ Wd.T,
+                               rtol=1e-13, atol=1e-300)
+    np.testing.assert_allclose(oracle.gemm_general("bwd", gi, "int4", sg, ns, cw, "int4", sw, M, N, K), Gi @ Wd,
+                               rtol=1e-13, atol=1e-18)
+    np.testing.assert_allclose(oracle.gemm_general("wgrad", gi, "int4", sg, ns, cu, "uint4", su, M, N, K), Gi.T @ Au,
+                               rtol=1e-13, atol=1e-18)
+
+
 def test_gemm_orientation_with_unit_vectors():
     """One non-zero per operand: the product lands where the definition puts it
     (catches transposed operands and swapped index roles)."""
