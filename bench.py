@@ -304,22 +304,29 @@ class LayerBench:
     def step(self):
         """The gradient's max and LUQ pass depend on nothing the forward half of the step produces.  With
         two streams they run on a second stream, through a second context (a context's scratch and
-        workspace serve one stream at a time), beside the activation/weight passes and the forward
-        product; the backward and update products wait for both."""
+        workspace serve one stream at a time), beside the activations' and weights' passes; the backward
+        and update products wait for both.  The maxima of A and W come from one launch (luq_amax_multi):
+        the small tensor's launch and reduction latency hides behind the large one's stream."""
         torch = self.torch
         if self.stream_g is None:
             return self.step_one_stream()
+        s, c = self, self.ctx
         main = torch.cuda.current_stream()
         fork = torch.cuda.Event(); fork.record(main)
         self.stream_g.wait_event(fork)
         with torch.cuda.stream(self.stream_g):
-            self.ctx_g.amax(self.G, self.mG)
-            self.ctx_g.quant_grad(self.G, self.mG, self.seed, self.ns, self.cG, self.aG, self.oG)
+            self.ctx_g.amax(s.G, s.mG)
+            self.ctx_g.quant_grad(s.G, s.mG, s.seed, s.ns, s.cG, s.aG, s.oG)
             join = torch.cuda.Event(); join.record(self.stream_g)
-        for name in self.kernels:
-            if name in ("amax_G", "quant_grad_G", "gemm_bwd", "gemm_wgrad"):
-                continue
-            self.calls[name]()
+        if self.args.multi_amax:
+            c.amax_multi([s.A, s.W], [s.mA, s.mW])
+        else:
+            self.calls["amax_A"](); self.calls["amax_W"]()
+        self.calls["quant_int4_W"]()
+        if self.fused:
+            self.calls["quant_int4_A+gemm_fwd"]()
+        else:
+            self.calls["quant_int4_A"](); self.calls["gemm_fwd"]()
         main.wait_event(join)
         self.calls["gemm_bwd"](); self.calls["gemm_wgrad"]()
 
@@ -833,8 +840,9 @@ def run_ours(args):
                        "fused_forward": "quant_int4(A) + gemm_fwd in one kernel (luq_quant_int4_gemm_fwd)" if lb.fused else "no",
                        "operand_bytes": "W,G" + (",A" if lb.oA is not None else "") +
                                         ": the quantizers also write the codes' 8-bit form, the GEMMs are handed it",
-                       "streams": "2: gradient max + LUQ beside the activation/weight quantizers and the forward GEMM"
+                       "streams": "2: gradient max + LUQ beside the activation/weight passes and the forward product"
                                   if args.streams == 2 else "1",
+                       "amax_A_and_W": "one launch (luq_amax_multi)" if (args.multi_amax and args.streams == 2) else "two launches",
                        "l2": "inputs (%d MB of activations per step) against a 126 MB L2; no explicit flush" % (lb.A.numel() * lb.A.element_size() >> 20)},
             "timing": {"blocks": stats["blocks"], "steps_per_block": args.steps, "ms_per_step": "median block",
                        "ms_min": stats["ms_min"], "ms_max": stats["ms_max"], "ms_spread": stats["ms_spread"],
@@ -870,6 +878,8 @@ def main():
                     help="2: the gradient's max and LUQ pass run on a second stream beside the forward half")
     ap.add_argument("--min-seconds", type=float, default=1.0, help="least duration of the timed region")
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of a replayed CUDA graph")
+    ap.add_argument("--multi-amax", type=int, default=1, choices=(0, 1),
+                    help="1: max|A| and max|W| from one launch (luq_amax_multi) in the timed step")
     ap.add_argument("--no-fused", action="store_true", help="quant_int4(A) and gemm_fwd as two kernels")
     ap.add_argument("--no-peak", action="store_true", help="do not measure the 8-bit tensor peak with a library GEMM")
     ap.add_argument("--no-configs", action="store_true", help="skip the compact runs of the other configurations")

@@ -195,6 +195,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_test(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag);
 }
+// The same bounded wait for roles that wait by the dozen of warps (the converters of the fused forward
+// kernel): it sleeps between probes from the start, so that waiting warps leave the issue slots to the
+// working ones.
+static __device__ __noinline__ bool mbar_wait_idle_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+    if (mbar_test(bar, parity)) return true;
+    if ((spin & 255u) == 255u && *abort_flag) return false;
+    __nanosleep(spin > 4096 ? 512 : 48);
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_test(bar, parity)) return true;
+  return mbar_wait_idle_slow(bar, parity, abort_flag);
+}
 __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }

@@ -240,6 +240,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   // order of the reduction kernel, down the columns.
   auto tile_m = [&](int tile) { return p.splits == 1 ? tile / p.tiles_n : tile % p.tiles_m; };
   auto tile_n = [&](int tile) { return p.splits == 1 ? tile % p.tiles_n : tile / p.tiles_m; };
+  const int u_begin = static_cast<int>(blockIdx.x), u_end = units, u_step = static_cast<int>(gridDim.x);
   auto unit_range = [&](int u, int& tile, int& it_begin, int& it_end) {
     tile = u / p.splits;
     const int sp = u - tile * p.splits;
@@ -254,7 +255,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       // instruction stream and must stay well below the time of a stage
       uint32_t issued = 0, stage = 0, phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
+      for (int u = u_begin; ok && u < u_end; u += u_step) {
         int tile, it_begin, it_end;
         unit_range(u, tile, it_begin, it_end);
         const int m0 = tile_m(tile) * BM;
@@ -296,7 +297,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     if (kAnyPlane && lane == 0) {
       uint32_t issued = 0, stage = 0, phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
+      for (int u = u_begin; ok && u < u_end; u += u_step) {
         int tile, it_begin, it_end;
         unit_range(u, tile, it_begin, it_end);
         const int m0 = tile_m(tile) * BM;
@@ -349,7 +350,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       constexpr uint64_t kStageStep = kExpandedStage >> 4;
       uint32_t stage = 0, phase = 0, tile_it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < units; u += gridDim.x, ++tile_it) {
+      for (int u = u_begin; ok && u < u_end; u += u_step, ++tile_it) {
         int tile, it_begin, it_end;
         unit_range(u, tile, it_begin, it_end);
         const uint32_t buf = tile_it & 1u;
@@ -386,7 +387,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const bool out_bf16 = p.out_bf16 && p.splits == 1;   // partial tiles of a split stay fp32
     uint32_t tile_it = 0, box_it = 0;
     bool ok = true;
-    for (int u = blockIdx.x; ok && u < units; u += gridDim.x, ++tile_it) {
+    for (int u = u_begin; ok && u < u_end; u += u_step, ++tile_it) {
       int tile, it_begin, it_end;
       unit_range(u, tile, it_begin, it_end);
       // a split stores its whole partial tile at row u*128 of the workspace
@@ -536,7 +537,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int ctid = threadIdx.x - kFirstConvWarp * 32;
     uint32_t ps = 0, pphase = 0, es = 0, ephase = 0;
     bool ok = true;
-    for (int u = blockIdx.x; ok && u < units; u += gridDim.x) {
+    for (int u = u_begin; ok && u < u_end; u += u_step) {
       int tile, it_begin, it_end;
       unit_range(u, tile, it_begin, it_end);
       for (int k_it = it_begin; k_it < it_end; ++k_it) {
@@ -806,9 +807,11 @@ luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 //   warp 0       TMA producer of raw activations: boxes of 128 rows x 32 elements
 //                (128-byte swizzle for fp32, 64-byte for bf16), two boxes per raw stage
 //   warp 6       TMA producer of W's operand bytes (two 128 x 128 slabs per stage)
-//   warps 7-14   converters: one row of one box per thread -> 32 INT4 codes; the codes go
-//                packed into a staging box that one thread stores with TMA (32-byte
-//                swizzle), and widened (16 * q) into the A slab of the operand stage
+//   warps 7-22   converters, two groups of eight warps that take the raw stages in turn (one
+//                group computes while the other waits at its barrier): one row of one box
+//                per thread -> 32 INT4 codes; the codes go packed into a staging box that
+//                one thread of the group stores with TMA (32-byte swizzle), and widened
+//                (16 * q) into the A slab of the operand stage
 //   warp 1       tcgen05.mma issue, kind::i8, accumulators in tensor memory (2 x 256 columns)
 //   warps 2-5    epilogue (one 32 x 32 staging box per warp)
 // An operand stage (128 deep) is made of two raw stages (64 deep).  Codes are
@@ -819,13 +822,14 @@ struct FusedCfg {
   static constexpr int box_bytes = 128 * 32 * (BF16 ? 2 : 4);   // one raw box
   static constexpr int raw_stage = 2 * box_bytes;               // 64 contraction elements of 128 rows
   static constexpr int RS = BF16 ? 6 : 3;                       // raw stages: 96 KB
-  static constexpr int ES = 2;                                  // operand stages
+  static constexpr int ES = 2;                                  // operand stages (A slab + W's two slabs, 48 KB)
   static constexpr int code_box = 128 * 32;                     // packed codes of one raw stage
-  static constexpr int threads = 32 * (kFirstConvWarp + 8);
+  static constexpr int conv_groups = 2;                         // converter groups, eight warps each
+  static constexpr int threads = 32 * (kFirstConvWarp + 8 * conv_groups);
   static constexpr int expanded = 0;
   static constexpr int raw = expanded + ES * kExpandedStage;
-  static constexpr int codes = raw + RS * raw_stage;            // two code boxes
-  static constexpr int staging = codes + 2 * code_box;          // 4 warps x 1 box
+  static constexpr int codes = raw + RS * raw_stage;            // two code boxes per converter group
+  static constexpr int staging = codes + 2 * conv_groups * code_box;   // 4 warps x 1 box
   static constexpr int barriers = staging + 4 * kStageBox;
   static constexpr int num_barriers = 2 * RS + 2 * ES + 4;
   static constexpr int tmem_slot = barriers + 8 * num_barriers;
@@ -836,6 +840,7 @@ struct FusedCfg {
 };
 
 struct FusedParams {
+
   const float* clip;      // max|A| (or a caller's clip)
   const float* scale_b;   // weight scale
   float* scale_a_out;     // receives clip / 7
@@ -844,15 +849,15 @@ struct FusedParams {
   int tiles_m, num_kb;
 };
 
-// all converter threads meet; returns true when every one of them passed `ok`
-__device__ __forceinline__ bool conv_barrier_all(bool ok) {
+// the 256 threads of a converter group meet at named barrier `id`; returns true when every one of them passed `ok`
+__device__ __forceinline__ bool conv_barrier_all(bool ok, uint32_t id) {
   uint32_t out;
   asm volatile(
       "{\n\t.reg .pred q, r;\n\t"
       "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.and.pred r, 5, 256, q;\n\t"
+      "bar.red.and.pred r, %2, 256, q;\n\t"
       "selp.u32 %0, 1, 0, r;\n\t}"
-      : "=r"(out) : "r"(static_cast<uint32_t>(ok)) : "memory");
+      : "=r"(out) : "r"(static_cast<uint32_t>(ok)), "r"(id) : "memory");
   return out != 0;
 }
 
@@ -882,9 +887,9 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < RS; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), 8); }
+    for (int s = 0; s < RS; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), 16); }   // all converter warps release a stage
     for (int s = 0; s < ES; ++s) {
-      mbar_init(ex_full(s), 2 * 8 + 1);   // eight converter warps for each half of the stage, and W's producer
+      mbar_init(ex_full(s), 2 * 8 + 1);   // eight converter warps for each half of the A slab, and W's producer
       mbar_init(ex_empty(s), 1);
     }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
@@ -1027,17 +1032,14 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           }
         }
       };
-      uint32_t r0[32], r1[32];
-      tmem_ld_32x32(taddr, r0);
-      tmem_ld_wait();
+      // one register set: with 23 warps in the CTA a thread has 88 registers, and this epilogue has
+      // the whole main loop of the next tile (tens of microseconds) to finish in
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; c += 2) {
-        tmem_ld_32x32(taddr + (c + 1) * 32, r1);
-        emit(r0, c);
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + c * 32, r);
         tmem_ld_wait();
-        if (c + 2 < BN / 32) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
-        emit(r1, c + 1);
-        tmem_ld_wait();
+        emit(r, c);
       }
       tc_fence_before();
       __syncwarp();
@@ -1046,12 +1048,13 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
     if (lane == 0) bulk_wait<0>();
   } else if (warp >= kFirstConvWarp) {
     // -------------------------------------------------------------- converters
-    const int cw = warp - kFirstConvWarp;          // 0..7
-    const int ctid = threadIdx.x - kFirstConvWarp * 32;
+    const int group = (warp - kFirstConvWarp) >> 3;   // takes the raw stages of this parity
+    const int cw = (warp - kFirstConvWarp) & 7;
+    const int ctid = threadIdx.x - (kFirstConvWarp + 8 * group) * 32;   // 0..255 inside the group
     const int boxi = cw >> 2;                      // which box of the raw stage
     const int row = (cw & 3) * 32 + lane;          // row of the tile
     const float clip = __ldg(p.clip);
-    const bool first = blockIdx.x == 0 && ctid == 0;
+    const bool first = blockIdx.x == 0 && group == 0 && ctid == 0;
     const bool usable = scale_usable(clip, first ? p.status : nullptr);
     const float inv = usable ? 7.0f / clip : 0.0f;   // an unusable clip gives zero codes and a zero scale
     if (first) *p.scale_a_out = usable ? clip / 7.0f : 0.0f;
@@ -1059,67 +1062,91 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
     // position of unit u of this row inside the swizzled box image
     const int rkey = BF16 ? ((row >> 1) & 3) : (row & 7);
     const uint32_t row_off = row * (BF16 ? 64 : 128);
-    uint32_t rs = 0, rphase = 0, es = 0, ephase = 0, stored = 0;
-    bool alive = true;
+    // raw stage number q (over the whole CTA): ring slot q % RS; operand stage q / 2, half q % 2.
+    // raw_iters is even, so a group always fills the same half.  Both groups follow EVERY raw stage
+    // (wait for it, release it) although each converts only its own: a waiter that skipped phases of
+    // a barrier could no longer tell them apart by their parity, and a slot must not be refilled
+    // before both groups have seen it filled.
+    uint32_t q = 0, stored = 0;
+    bool alive = true, ok = true;
     for (int t = blockIdx.x; alive && t < p.tiles_m; t += gridDim.x) {
       const int m0 = t * BM;
-      for (int it = 0; it < raw_iters; ++it) {
-        const int second = it & 1;                 // which half of the operand stage
-        bool ok = mbar_wait(raw_full(rs), rphase, abort_flag);
-        if (ok && !second) ok = mbar_wait(ex_empty(es), ephase ^ 1u, abort_flag);
+      for (int it = 0; it < raw_iters; ++it, ++q) {
+        const uint32_t rs = q % RS, rphase = (q / RS) & 1u;
+        const uint32_t es = (q >> 1) % ES, ephase = ((q >> 1) / ES) & 1u;
+        ok = ok && mbar_wait_idle(raw_full(rs), rphase, abort_flag);
+        if ((it & 1) != group) {          // the other group's stage
+          __syncwarp();
+          if (ok && lane == 0) mbar_arrive(raw_empty(rs));
+          continue;
+        }
+        if (ok) ok = mbar_wait_idle(ex_empty(es), ephase ^ 1u, abort_flag);
+        const uint32_t cbox_off = C::codes + (2 * group + (stored & 1u)) * C::code_box;
         if (ok) {
           const uint8_t* src = gen + C::raw + rs * C::raw_stage + boxi * C::box_bytes + row_off;
           uint4 u[kUnits];
 #pragma unroll
           for (int j = 0; j < kUnits; ++j) u[j] = *reinterpret_cast<const uint4*>(src + ((j ^ rkey) << 4));
-          // 32 elements -> 32 codes, element e in nibble e % 8 of word e / 8
-          uint32_t w[4] = {0u, 0u, 0u, 0u};
+          // 32 elements -> 32 codes (element e in nibble e % 8 of word e / 8) and 32 operand bytes 16 * q
+          float v[32];
           if constexpr (BF16) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const uint32_t h[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                w[j] |= int4_code(__uint_as_float(h[i] << 16), inv) << (8 * i);
-                w[j] |= int4_code(__uint_as_float(h[i] & 0xFFFF0000u), inv) << (8 * i + 4);
+                v[8 * j + 2 * i] = __uint_as_float(h[i] << 16);
+                v[8 * j + 2 * i + 1] = __uint_as_float(h[i] & 0xFFFF0000u);
               }
             }
           } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              const uint32_t sh = 16 * (j & 1);
-              w[j >> 1] |= int4_code(__uint_as_float(u[j].x), inv) << sh;
-              w[j >> 1] |= int4_code(__uint_as_float(u[j].y), inv) << (sh + 4);
-              w[j >> 1] |= int4_code(__uint_as_float(u[j].z), inv) << (sh + 8);
-              w[j >> 1] |= int4_code(__uint_as_float(u[j].w), inv) << (sh + 12);
+              v[4 * j] = __uint_as_float(u[j].x); v[4 * j + 1] = __uint_as_float(u[j].y);
+              v[4 * j + 2] = __uint_as_float(u[j].z); v[4 * j + 3] = __uint_as_float(u[j].w);
             }
           }
-          const uint4 packed = make_uint4(w[0], w[1], w[2], w[3]);
-          // operand bytes 16 * q, element order, into this row of the A slab (128-byte swizzle)
-          uint4 o0, o1;
-          expand32<1, false, false>(packed, make_uint4(0u, 0u, 0u, 0u), o0, o1);
+          uint32_t lowb[8], any = 0u;
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const uint32_t t0 = int4_round_bits(v[4 * g], inv), t1 = int4_round_bits(v[4 * g + 1], inv);
+            const uint32_t t2 = int4_round_bits(v[4 * g + 2], inv), t3 = int4_round_bits(v[4 * g + 3], inv);
+            any |= t0 | t1 | t2 | t3;
+            lowb[g] = int4_low_bytes(t0, t1, t2, t3);
+          }
+          uint4 packed = make_uint4(int4_pack8(lowb[0], lowb[1]), int4_pack8(lowb[2], lowb[3]),
+                                    int4_pack8(lowb[4], lowb[5]), int4_pack8(lowb[6], lowb[7]));
+          uint4 o0 = make_uint4(int4_operand_bytes(lowb[0]), int4_operand_bytes(lowb[1]),
+                                int4_operand_bytes(lowb[2]), int4_operand_bytes(lowb[3]));
+          uint4 o1 = make_uint4(int4_operand_bytes(lowb[4]), int4_operand_bytes(lowb[5]),
+                                int4_operand_bytes(lowb[6]), int4_operand_bytes(lowb[7]));
+          if (any & 0x20000000u) {   // a NaN among the 32 products (rare): the element-wise rule, NaN -> 0
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int e = 0; e < 32; ++e) w[e >> 3] |= int4_code(v[e], inv) << (4 * (e & 7));
+            packed = make_uint4(w[0], w[1], w[2], w[3]);
+            expand32<1, false, false>(packed, make_uint4(0u, 0u, 0u, 0u), o0, o1);
+          }
+          // operand bytes, element order, into this row of the A slab (128-byte swizzle)
           uint8_t* drow = gen + C::expanded + es * kExpandedStage + row * 128;
-          const int unit = second * 4 + boxi * 2;
+          const int unit = group * 4 + boxi * 2;
           *reinterpret_cast<uint4*>(drow + ((unit ^ (row & 7)) << 4)) = o0;
           *reinterpret_cast<uint4*>(drow + (((unit + 1) ^ (row & 7)) << 4)) = o1;
           // packed codes into the staging box of this raw stage: 128 rows x 32 bytes, 32-byte swizzle
-          uint8_t* cbox = gen + C::codes + (stored & 1u) * C::code_box;
-          *reinterpret_cast<uint4*>(cbox + row * 32 + ((boxi ^ ((row >> 2) & 1)) << 4)) = packed;
+          *reinterpret_cast<uint4*>(gen + cbox_off + row * 32 + ((boxi ^ ((row >> 2) & 1)) << 4)) = packed;
           fence_proxy_async();   // both writes are read by the async proxy (tensor core, TMA store)
         }
-        // the store that read the other code box two raw stages ago has long finished; the one
-        // issued a stage ago must have read its box before that box is written again next time
+        // The group's two code boxes alternate.  Here the store issued one turn ago must have read its
+        // box: after the barrier below every thread may go on to the next turn and write that box again.
         if (ctid == 0) bulk_wait_read<0>();
-        alive = conv_barrier_all(ok);
+        alive = conv_barrier_all(ok, 5 + group);
         if (!alive) break;
         if (ctid == 0 && it * 64 < p.Kc) {
-          tma_store_2d(&tm_codes, base + C::codes + (stored & 1u) * C::code_box, it * 32, m0);
+          tma_store_2d(&tm_codes, base + cbox_off, it * 32, m0);
           bulk_commit();
         }
         ++stored;
         if (lane == 0) { mbar_arrive(raw_empty(rs)); mbar_arrive(ex_full(es)); }
-        if (++rs == static_cast<uint32_t>(RS)) { rs = 0; rphase ^= 1u; }
-        if (second) { if (++es == static_cast<uint32_t>(ES)) { es = 0; ephase ^= 1u; } }
       }
     }
     if (ctid == 0) bulk_wait<0>();

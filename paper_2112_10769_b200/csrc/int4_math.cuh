@@ -42,5 +42,30 @@ __device__ __forceinline__ uint32_t uint4_code(float x, float inv) {
   return (y == y) ? code : 0u;
 }
 
+// ---- four elements at a time (the GEMM that quantizes its activations on the way in) ----------
+// int4_round_bits: the bit pattern of clamp(x * inv) + 1.5 * 2^23, whose low nibble is the code.
+// The clamp propagates NaN (the sum is then a NaN pattern, bit 29 set; every valid sum is
+// 0x4B3FFFF9 .. 0x4B400007, bit 29 clear): OR the results together and test bit 29 to find out
+// whether any element needs int4_code()'s "NaN -> 0" rule.
+__device__ __forceinline__ uint32_t int4_round_bits(float x, float inv) {
+  const float y = __fmul_rn(x, inv);
+  float c;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(c) : "f"(y), "f"(-7.0f));
+  asm("min.NaN.f32 %0, %1, %2;" : "=f"(c) : "f"(c), "f"(7.0f));
+  return __float_as_uint(__fadd_rn(c, 12582912.0f));
+}
+// the low bytes of four such sums, element 0 in byte 0 (the low nibble of a byte is the element's code)
+__device__ __forceinline__ uint32_t int4_low_bytes(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3) {
+  return __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+}
+// those four bytes -> the four int8 operand bytes 16 * q
+__device__ __forceinline__ uint32_t int4_operand_bytes(uint32_t low_bytes) { return (low_bytes << 4) & 0xF0F0F0F0u; }
+// two such byte quadruples (elements 0-3 and 4-7) -> one word of eight packed codes
+__device__ __forceinline__ uint32_t int4_pack8(uint32_t low_bytes_a, uint32_t low_bytes_b) {
+  const uint32_t xa = low_bytes_a & 0x0F0F0F0Fu, xb = low_bytes_b & 0x0F0F0F0Fu;
+  const uint32_t ya = xa | (xa >> 4), yb = xb | (xb >> 4);   // bytes 0 and 2 hold two codes each
+  return __byte_perm(ya, yb, 0x6420);
+}
+
 }  // namespace luqdev
 #endif
