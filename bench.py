@@ -42,12 +42,13 @@ WORKLOAD = "cfg2"
 KERNELS = ("amax_A", "amax_W", "quant_int4_A", "quant_int4_W", "gemm_fwd",
            "amax_G", "quant_grad_G", "gemm_bwd", "gemm_wgrad")
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the cfg2 kernels.  NOT measured by this
-# run: copied from the ncu capture summarised in the file named by TRAFFIC_SOURCE (other workloads: None).
-TRAFFIC_SOURCE = "profiles/kernels_cfg2_full_size.md (an earlier ncu capture, not this run)"
-NCU_TRAFFIC_BYTES = {"amax_A": 469.0e6, "quant_int4_A": 511.6e6, "gemm_fwd": 64.1e6, "amax_G": 51.4e6,
-                     "quant_grad_G": 52.3e6, "gemm_bwd": 416.4e6, "gemm_wgrad": 74.3e6, "amax_W": 2.4e6,
-                     "quant_int4_W": 2.4e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the cfg2 kernels.  NOT measured by this run:
+# copied from the committed single-pass ncu capture of the same step (other workloads: None).
+TRAFFIC_SOURCE = "profiles/launch_list_and_dram_traffic_cfg2_step.md (committed ncu capture of this step, not this run)"
+TRAFFIC_SOURCE_UNFUSED = "profiles/kernels_cfg2_full_size.md (committed ncu capture, not this run)"
+NCU_TRAFFIC_BYTES = {"amax_A": 463.4e6, "amax_W": 2.4e6, "quant_int4_W": 2.4e6, "quant_int4_A+gemm_fwd": 550.1e6,
+                     "amax_G": 51.4e6, "quant_grad_G": 51.4e6, "gemm_bwd": 413.0e6, "gemm_wgrad": 89.8e6}
+NCU_TRAFFIC_BYTES_UNFUSED = {"quant_int4_A": 511.6e6, "gemm_fwd": 64.1e6}
 
 
 def load_peaks():
@@ -568,7 +569,8 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     if args.workload == "cfg4":
-        run_sweep(args, binding, inputs, torch, local)
+        exps = tuple(int(e) for e in args.sweep_exponents.split(",")) if args.sweep_exponents else None
+        run_sweep(args, binding, inputs, torch, local, exponents=exps, extras=not args.sweep_quick)
         return
 
     cfg = inputs.CONFIGS[args.workload]
@@ -661,8 +663,9 @@ def run_ours(args):
     full_cfg2 = args.workload == "cfg2" and not args.rows
     roofline = {"kernel": dominant, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
                 "frac": d["frac"],
-                "traffic": NCU_TRAFFIC_BYTES.get(dominant) if full_cfg2 else None,
-                "traffic_source": TRAFFIC_SOURCE if (full_cfg2 and dominant in NCU_TRAFFIC_BYTES) else None,
+                "traffic": (NCU_TRAFFIC_BYTES.get(dominant) or NCU_TRAFFIC_BYTES_UNFUSED.get(dominant)) if full_cfg2 else None,
+                "traffic_source": (TRAFFIC_SOURCE if dominant in NCU_TRAFFIC_BYTES else
+                                   TRAFFIC_SOURCE_UNFUSED if dominant in NCU_TRAFFIC_BYTES_UNFUSED else None) if full_cfg2 else None,
                 "algorithmic_bytes": alg[dominant][0], "algorithmic_flops": alg[dominant][1],
                 "peak_source": {"hbm": f"{peaks['source']} hbm copy", "tensor": tensor_peak_source}[d["bound"]]}
     # whole step against its own HBM ceiling: every tensor read twice (max, quantize), codes written and
@@ -680,7 +683,7 @@ def run_ours(args):
     # tensor instead of two.  Reported beside the headline, not as it: the codes differ (a lagging
     # estimate saturates / clips), the named path is max-then-quantize.
     hindsight = None
-    if not args.no_graph and not args.rows:
+    if not args.no_graph and not args.rows and not args.no_variants:
         try:
             eA, eW, eG = lb.mA.clone(), lb.mW.clone(), lb.mG.clone()      # estimates, initialised with the true maxima
             meas = torch.empty(3, device=dev)
@@ -713,7 +716,7 @@ def run_ours(args):
 
     # ---- the nine separate calls, for comparison, when the headline used the fused forward kernel
     named = None
-    if lb.fused and not args.rows:
+    if lb.fused and not args.rows and not args.no_variants:
         saved = lb.kernels, lb.fused
         lb.kernels, lb.fused = KERNELS, False
         try:
@@ -878,10 +881,15 @@ def main():
                     help="2: the gradient's max and LUQ pass run on a second stream beside the forward half")
     ap.add_argument("--min-seconds", type=float, default=1.0, help="least duration of the timed region")
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of a replayed CUDA graph")
+    ap.add_argument("--sweep-exponents", default=None,
+                    help="cfg4: comma-separated log2 sizes instead of the whole sweep (e.g. 26 for a profiling run)")
+    ap.add_argument("--sweep-quick", action="store_true", help="cfg4: max + LUQ only, without the variant quantizers")
     ap.add_argument("--multi-amax", type=int, default=1, choices=(0, 1),
                     help="1: max|A| and max|W| from one launch (luq_amax_multi) in the timed step")
     ap.add_argument("--no-fused", action="store_true", help="quant_int4(A) and gemm_fwd as two kernels")
     ap.add_argument("--no-peak", action="store_true", help="do not measure the 8-bit tensor peak with a library GEMM")
+    ap.add_argument("--no-variants", action="store_true",
+                    help="skip the in-hindsight and separate-forward-kernels variants (launch lists of the timed step alone)")
     ap.add_argument("--no-configs", action="store_true", help="skip the compact runs of the other configurations")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end, other-configuration and CPU-baseline legs")
     ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1, 2],

@@ -687,7 +687,17 @@ luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           if (++stage == static_cast<uint32_t>(ES)) { stage = 0; phase ^= 1u; }
         }
       }
-      (void)issued;
+      // drain: every copy of the pair counts its bytes on the leader's barriers, so the leader waits
+      // for the last fill of every stage (both CTAs' copies have then landed); its peer leaves only
+      // after the cluster barrier of the teardown, i.e. after this drain
+      if (leader) {
+        for (int s = 0; s < ES; ++s) {
+          if (issued > static_cast<uint32_t>(s)) {
+            const uint32_t last = (issued - 1 - s) / ES;
+            mbar_wait_cluster(full(s), last & 1u, abort_flag);
+          }
+        }
+      }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------- MMA issue (leader only)
