@@ -257,6 +257,8 @@ class LayerBench:
         for c in {id(self.ctx): self.ctx, id(self.ctx_g): self.ctx_g}.values():
             if args.mma_kind is not None:
                 c.set_option(binding.OPT_MMA_KIND, args.mma_kind)
+            if args.pairs is not None:
+                c.set_option(binding.OPT_PAIRS, args.pairs)
         self.stream_g = torch.cuda.Stream() if args.streams == 2 else None
         dev = self.A.device
         f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)  # noqa: E731
@@ -323,11 +325,15 @@ class LayerBench:
             c.amax_multi([s.A, s.W], [s.mA, s.mW])
         else:
             self.calls["amax_A"](); self.calls["amax_W"]()
-        self.calls["quant_int4_W"]()
         if self.fused:
+            self.calls["quant_int4_W"]()
             self.calls["quant_int4_A+gemm_fwd"]()
         else:
-            self.calls["quant_int4_A"](); self.calls["gemm_fwd"]()
+            if self.args.multi_amax:     # A and W through one quantizer launch as well
+                c.quant_int4_multi([s.A, s.W], [s.mA, s.mW], [s.cA, s.cW], [s.sA, s.sW], [s.oA, s.oW])
+            else:
+                self.calls["quant_int4_W"](); self.calls["quant_int4_A"]()
+            self.calls["gemm_fwd"]()
         main.wait_event(join)
         self.calls["gemm_bwd"](); self.calls["gemm_wgrad"]()
 
@@ -845,7 +851,8 @@ def run_ours(args):
                                         ": the quantizers also write the codes' 8-bit form, the GEMMs are handed it",
                        "streams": "2: gradient max + LUQ beside the activation/weight passes and the forward product"
                                   if args.streams == 2 else "1",
-                       "amax_A_and_W": "one launch (luq_amax_multi)" if (args.multi_amax and args.streams == 2) else "two launches",
+                       "amax_A_and_W": ("one launch (luq_amax_multi; without the fused forward kernel also luq_quant_int4_multi)"
+                                        if (args.multi_amax and args.streams == 2) else "two launches"),
                        "l2": "inputs (%d MB of activations per step) against a 126 MB L2; no explicit flush" % (lb.A.numel() * lb.A.element_size() >> 20)},
             "timing": {"blocks": stats["blocks"], "steps_per_block": args.steps, "ms_per_step": "median block",
                        "ms_min": stats["ms_min"], "ms_max": stats["ms_max"], "ms_spread": stats["ms_spread"],
@@ -892,6 +899,8 @@ def main():
                     help="skip the in-hindsight and separate-forward-kernels variants (launch lists of the timed step alone)")
     ap.add_argument("--no-configs", action="store_true", help="skip the compact runs of the other configurations")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end, other-configuration and CPU-baseline legs")
+    ap.add_argument("--pairs", type=int, default=None, choices=[0, 1, 2],
+                    help="CTA pairs (cta_group::2) for products whose operands both arrive as bytes; default: the library's choice")
     ap.add_argument("--mma-kind", type=int, default=None, choices=[0, 1, 2],
                     help="tensor-core operand type: 0 e4m3 (kind::f8f6f4), 1 int8 (kind::i8), 2 per product; default: the library's")
     args = ap.parse_args()

@@ -57,13 +57,20 @@ extern "C" {
 #define LUQ_STATUS_NONFINITE 1 /* a max / clip was Inf or NaN: zero codes, zero scale */
 #define LUQ_STATUS_RANGE 2     /* a non-zero max / clip outside [2^-100, 2^100]: zero codes, zero scale */
 #define LUQ_STATUS_TIMEOUT 4   /* a bounded wait inside a kernel expired; outputs unspecified */
+#define LUQ_STATUS_BOUNDS 8    /* only from the checking build of the library (compiled with -DLUQ_DEBUG, see
+                                  luq_debug_build): an address a kernel formed lay outside its region; that access
+                                  was skipped (never a trap), outputs unspecified */
 
 /* options for luq_set_option */
 #define LUQ_OPT_MMA_KIND 1 /* 0: tcgen05 kind::f8f6f4 on e4m3 operands (operand bytes passed to a GEMM are then
                               ignored); 1: kind::i8 on int8 operands; 2 (default): int8, except e4m3 where an
                               int32 accumulator could wrap (contractions beyond about 2^18 terms) */
 #define LUQ_OPT_SPLITS 2   /* 0: choose the contraction split automatically (default); n >= 1: force n */
-#define LUQ_OPT_PAIRS 3    /* 1: products whose operands are both 8-bit planes run on CTA pairs (cta_group::2) */
+#define LUQ_OPT_PAIRS 3    /* CTA pairs (tcgen05 cta_group::2: a 256-row tile on two SMs, each fetching half of B) for
+                              unsplit products whose operands both arrive as operand bytes.  0: never; 1: wherever
+                              possible; 2 (default): where measured faster - long contractions with B stored
+                              contraction-major (the backward and update products of a wide layer).  Results are
+                              bit-identical either way. */
 #define LUQ_OPT_UNSIGNED_ACTIVATIONS 5 /* 1: the activation codes given to luq_gemm_fwd and luq_gemm_wgrad are
                               unsigned INT4 (from luq_quant_uint4).  Such an operand is always fetched as bytes:
                               pass the operand bytes luq_quant_uint4 wrote, or the GEMM expands a plane into the
@@ -341,6 +348,17 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
 int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
                           const uint8_t* d_a_codes, const float* d_sa,
                           float* d_dw, int64_t M, int64_t N, int64_t K, void* stream);
+
+/* 1 if this library was compiled with -DLUQ_DEBUG: every shared-memory, tensor-memory and global
+ * address that the converters, epilogues and streaming loops form is checked against its region
+ * before use; a violation raises LUQ_STATUS_BOUNDS and skips the access.  (The pool this library
+ * was developed on offers no compute-sanitizer; this build stands in for it.)  0 otherwise. */
+int luq_debug_build(void);
+
+/* Diagnostic for the checking build (the paper has no counterpart): launches one thread that forms an
+ * address just beyond a small shared-memory region and puts it to the check WITHOUT accessing it.  In
+ * the checking build luq_status() then reports LUQ_STATUS_BOUNDS; in the normal build, nothing. */
+int luq_debug_bounds_probe(luq_ctx* ctx, void* stream);
 
 /* Synchronises `stream`, returns the device status bits in *host_flags and
  * clears them. */

@@ -13,19 +13,20 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libluq_b200.so")
+# LUQ_LIB selects another build of the same library, e.g. the bounds-checking one (libluq_b200_debug.so)
+LIB_PATH = os.environ.get("LUQ_LIB") or os.path.join(_HERE, "libluq_b200.so")
 
 LUQ_F32, LUQ_BF16 = 0, 1
-STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT = 1, 2, 4
+STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT, STATUS_BOUNDS = 1, 2, 4, 8
 OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS, OPT_UNSIGNED_ACTIVATIONS, OPT_OUTPUT_BF16 = 1, 2, 3, 4, 5, 6
 OPT_GRADIENT_INT4 = 7
 OPT_SM_LIMIT = 8
 SCHEME_FP4, SCHEME_FP4_SR, SCHEME_FP4_SU, SCHEME_LUQ, SCHEME_INT4_SR = 0, 1, 2, 3, 4
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
-SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_amax", "luq_quant_int4",
+SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_debug_build", "luq_amax", "luq_quant_int4",
            "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_int4_hindsight", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_ablation", "luq_quant_grad_pw2",
-           "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_debug_expire_wait", "luq_gemm_fwd", "luq_quant_int4_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
+           "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_debug_expire_wait", "luq_debug_bounds_probe", "luq_gemm_fwd", "luq_quant_int4_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
 _lib = None
@@ -49,6 +50,7 @@ def load() -> ctypes.CDLL:
         L.luq_destroy.argtypes = [vp]
         L.luq_set_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
         L.luq_kmax.argtypes = []
+        L.luq_debug_build.argtypes = []
         L.luq_amax.argtypes = [vp, vp, ctypes.c_int, sz, vp, vp]
         L.luq_quant_int4.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, vp, vp, vp, vp]
         L.luq_amax_multi.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int, vp, vp, vp]
@@ -64,6 +66,7 @@ def load() -> ctypes.CDLL:
         L.luq_quant_grad_hindsight.argtypes = [vp, vp, ctypes.c_int, sz, sz, vp, ctypes.c_float, ctypes.c_int, u64,
                                                ctypes.c_int, vp, vp, vp, vp, vp]
         L.luq_debug_expire_wait.argtypes = [vp, vp]
+        L.luq_debug_bounds_probe.argtypes = [vp, vp]
         L.luq_debug_quotient.argtypes = [vp, vp, sz, vp, vp, vp]
         L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_quant_int4_gemm_fwd.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
@@ -314,6 +317,10 @@ class Context:
         """Launches a kernel whose bounded wait runs out; status() then reports STATUS_TIMEOUT."""
         _check(load().luq_debug_expire_wait(self.handle, _stream()), "luq_debug_expire_wait")
 
+    def debug_bounds_probe(self):
+        """Puts an out-of-region address to the checking build's bounds check (nothing is accessed)."""
+        _check(load().luq_debug_bounds_probe(self.handle, _stream()), "luq_debug_bounds_probe")
+
     def debug_quotient(self, x: torch.Tensor, amax: torch.Tensor) -> torch.Tensor:
         out = torch.empty_like(x, dtype=torch.float32)
         _check(load().luq_debug_quotient(self.handle, x.data_ptr(), x.numel(), amax.data_ptr(), out.data_ptr(),
@@ -381,3 +388,8 @@ def gemm_wgrad_static(g_codes, alpha, n_samples: int, a_codes, sa, M: int, N: in
 
 def kmax() -> int:
     return int(load().luq_kmax())
+
+
+def debug_build() -> bool:
+    """True if the loaded library is the bounds-checking build (-DLUQ_DEBUG)."""
+    return bool(load().luq_debug_build())

@@ -16,6 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libluq_b200.so")
+LIB_DEBUG = os.path.join(HERE, "libluq_b200_debug.so")   # the same sources with -DLUQ_DEBUG (bounds-checking build)
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-std=c++17", "-O3", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
           "-I", CSRC, "--expt-relaxed-constexpr"]
@@ -46,14 +47,18 @@ def _stamp(target: str, digest: str) -> None:
         f.write(digest)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compiles the library; debug=True compiles the bounds-checking variant (-DLUQ_DEBUG) next to it."""
     nvcc = os.environ.get("NVCC", "nvcc")
+    lib = LIB_DEBUG if debug else LIB
+    suffix, define = (".dbg.o", ["-DLUQ_DEBUG"]) if debug else (".o", [])
     headers = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "int4_math.cuh"), os.path.join(ROOT, "include", "luq.h")]
     objs, digests, running = [], [], []
     for name, extra in UNITS.items():
         src = os.path.join(CSRC, name)
-        obj = os.path.join(CSRC, name.replace(".cu", ".o"))
+        obj = os.path.join(CSRC, name.replace(".cu", suffix))
         objs.append(obj)
+        extra = extra + define
         flags = ARCH + COMMON[:5] + extra        # the flags that change the code (not the include paths)
         digest = _digest([src] + headers, flags)
         digests.append(digest)
@@ -65,11 +70,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
             raise subprocess.CalledProcessError(proc.returncode, cmd)
         _stamp(obj, digest)
     link_digest = _digest([], digests)
-    if force or _stale(LIB, link_digest):
-        subprocess.run([nvcc] + ARCH + ["-shared", "-o", LIB] + objs, check=True)
-        _stamp(LIB, link_digest)
-    return LIB
+    if force or _stale(lib, link_digest):
+        subprocess.run([nvcc] + ARCH + ["-shared", "-o", lib] + objs, check=True)
+        _stamp(lib, link_digest)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

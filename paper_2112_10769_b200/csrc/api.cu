@@ -27,6 +27,14 @@ extern "C" {
 
 int luq_kmax(void) { return LUQ_KMAX; }
 
+int luq_debug_build(void) {
+#ifdef LUQ_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 const char* luq_strerror(int code) {
   switch (code) {
     case LUQ_OK: return "ok";
@@ -54,7 +62,7 @@ int luq_create(luq_ctx** out, int device) {
   c->sm_count = prop.multiProcessorCount;
   c->mma_kind = LUQ_DEFAULT_MMA_KIND;
   c->forced_splits = 0;
-  c->use_pairs = 0;
+  c->use_pairs = 2;
   c->kmax = LUQ_KMAX;
   c->unsigned_act = 0;
   c->grad_int4 = 0;
@@ -120,7 +128,7 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
       ctx->sm_limit = value;
       return LUQ_OK;
     case LUQ_OPT_PAIRS:
-      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      if (value < 0 || value > 2) return LUQ_ERR_ARG;
       ctx->use_pairs = value;
       return LUQ_OK;
     default:
@@ -321,6 +329,13 @@ int luq_debug_expire_wait(luq_ctx* ctx, void* stream) {
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_expire_wait(ctx, as_stream(stream)));
+}
+
+int luq_debug_bounds_probe(luq_ctx* ctx, void* stream) {
+  if (!ctx) return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  return cuda_rc(luq_launch_bounds_probe(ctx, as_stream(stream)));
 }
 
 int luq_debug_quotient(luq_ctx* ctx, const float* d_x, size_t n, const float* d_amax, float* d_t, void* stream) {

@@ -84,6 +84,7 @@ struct luq_gemm_args {
 };
 int luq_launch_gemm(luq_ctx* ctx, const luq_gemm_args& a, cudaStream_t st);
 int luq_launch_expire_wait(luq_ctx* ctx, cudaStream_t st);
+int luq_launch_bounds_probe(luq_ctx* ctx, cudaStream_t st);
 // Forward product that quantizes its activations itself (one column of output tiles): writes the INT4
 // codes of A, its scale and Z = Q(A) . Q(W)^T.  d_w_operand may be null (W's codes are then widened
 // into the workspace).  Call only when luq_quant_fwd_fusable() says yes.
@@ -136,7 +137,31 @@ cudaError_t luq_launch_kernel(void (*kernel)(KArgs...), int grid, int block, siz
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Checking build (-DLUQ_DEBUG): LUQ_IN_BOUNDS(cond, status) is `cond`, and a false one raises
+// LUQ_STATUS_BOUNDS in the status word; callers skip the access.  In the normal build it is `true`
+// and costs nothing.
+#ifdef LUQ_DEBUG
+#define LUQ_IN_BOUNDS(cond, status) ((cond) ? true : (atomicOr((status), LUQ_STATUS_BOUNDS), false))
+#else
+#define LUQ_IN_BOUNDS(cond, status) (true)
+#endif
+
 namespace luqdev {
+
+// is [p, p + bytes) inside the region [lo, hi) of the CTA's shared-memory block starting at `base`?
+// (always true, and free, outside the checking build)
+__device__ __forceinline__ bool smem_in(const void* p, const void* base, int lo, int hi, int bytes, unsigned int* status) {
+  const long long off = static_cast<const unsigned char*>(p) - static_cast<const unsigned char*>(base);
+  (void)off; (void)lo; (void)hi; (void)bytes; (void)status;
+  return LUQ_IN_BOUNDS(off >= lo && off + bytes <= hi, status);
+}
+// do the 32 accumulator columns read at `taddr` lie inside the `cols` columns allocated at `tmem_base`?
+__device__ __forceinline__ bool tmem_in(unsigned int taddr, unsigned int tmem_base, int cols, unsigned int* status) {
+  const int col = static_cast<int>(taddr & 0xFFFFu) - static_cast<int>(tmem_base & 0xFFFFu);
+  const int lane = static_cast<int>(taddr >> 16) - static_cast<int>(tmem_base >> 16);
+  (void)col; (void)lane; (void)cols; (void)status;
+  return LUQ_IN_BOUNDS(col >= 0 && col + 32 <= cols && lane >= 0 && lane + 32 <= 128, status);
+}
 
 // waits until the preceding kernel of the stream has completed and its memory is visible
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

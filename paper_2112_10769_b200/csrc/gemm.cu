@@ -117,6 +117,17 @@ struct GemmParams {
   uint4 lut_a, lut_b;  // nibble -> operand byte
 };
 
+// tcgen05.ld of 32 accumulator columns, checked against the allocation in the checking build
+// (the condition is the same in every lane of the warp; a violation reads zeros instead)
+__device__ __forceinline__ void tmem_ld_32x32_chk(uint32_t tmem_base, unsigned int* status, uint32_t taddr, uint32_t (&r)[32]) {
+  if (tmem_in(taddr, tmem_base, 512, status)) {
+    tmem_ld_32x32(taddr, r);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = 0u;
+  }
+}
+
 // eight nibbles of `w` -> eight operand bytes through a 16-entry table
 __device__ __forceinline__ void expand8_lut(uint32_t w, const uint4& lut, uint32_t& lo, uint32_t& hi) {
   const uint32_t sel0 = w & 0x7777u;
@@ -423,14 +434,16 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               v.y = pack_bf16x2(value(8 * j + 2), value(8 * j + 3));
               v.z = pack_bf16x2(value(8 * j + 4), value(8 * j + 5));
               v.w = pack_bf16x2(value(8 * j + 6), value(8 * j + 7));
-              *reinterpret_cast<uint4*>(rowp + ((j ^ sw64) << 4)) = v;
+              if (smem_in(rowp + ((j ^ sw64) << 4), gen, C::staging, C::barriers, 16, p.status))
+                *reinterpret_cast<uint4*>(rowp + ((j ^ sw64) << 4)) = v;
             }
           } else {
             uint8_t* const rowp = stage0_gen + b * kStageBox + lane * 128;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) =
-                  make_float4(value(4 * j), value(4 * j + 1), value(4 * j + 2), value(4 * j + 3));
+              if (smem_in(rowp + ((j ^ sw) << 4), gen, C::staging, C::barriers, 16, p.status))
+                *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) =
+                    make_float4(value(4 * j), value(4 * j + 1), value(4 * j + 2), value(4 * j + 3));
           }
           fence_proxy_async();
           __syncwarp();
@@ -479,22 +492,23 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           const int key = sw ^ (c & 7);
 #pragma unroll
           for (int s = 0; s < 8; ++s)   // position s holds unit s ^ sw, whose slot is (s ^ sw) ^ c
-            *reinterpret_cast<uint4*>(line + ((s ^ key) << 4)) = make_uint4(r[4 * s], r[4 * s + 1], r[4 * s + 2], r[4 * s + 3]);
+            if (smem_in(line + ((s ^ key) << 4), gen, C::staging, C::barriers, 16, p.status))
+              *reinterpret_cast<uint4*>(line + ((s ^ key) << 4)) = make_uint4(r[4 * s], r[4 * s + 1], r[4 * s + 2], r[4 * s + 3]);
         };
         constexpr int kChunks = BN / 32 / 2;          // chunks per warp
         const int c_first = half * kChunks;
         uint32_t r0[32], r1[32];
-        tmem_ld_32x32(taddr + c_first * 32, r0);
+        tmem_ld_32x32_chk(tmem_base, p.status, taddr + c_first * 32, r0);
         // first write of this tile: the previous tile's store must have read the strip
         if (half == 0 && lane == 0) bulk_wait_read<0>();
         pair_sync();
         tmem_ld_wait();
 #pragma unroll 1
         for (int c = c_first; c < c_first + kChunks; c += 2) {
-          tmem_ld_32x32(taddr + (c + 1) * 32, r1);
+          tmem_ld_32x32_chk(tmem_base, p.status, taddr + (c + 1) * 32, r1);
           emit_rows(r0, c);
           tmem_ld_wait();
-          if (c + 2 < c_first + kChunks) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
+          if (c + 2 < c_first + kChunks) tmem_ld_32x32_chk(tmem_base, p.status, taddr + (c + 2) * 32, r0);
           emit_rows(r1, c + 1);
           tmem_ld_wait();
         }
@@ -507,14 +521,14 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       } else if constexpr (C::epi_double) {
         // two register sets: the tensor-memory load of the next block is in flight while this one is emitted
         uint32_t r0[32], r1[32];
-        tmem_ld_32x32(taddr, r0);
+        tmem_ld_32x32_chk(tmem_base, p.status, taddr, r0);
         tmem_ld_wait();
 #pragma unroll 1
         for (int c = 0; c < BN / 32; c += 2) {
-          tmem_ld_32x32(taddr + (c + 1) * 32, r1);
+          tmem_ld_32x32_chk(tmem_base, p.status, taddr + (c + 1) * 32, r1);
           emit(r0, c);
           tmem_ld_wait();
-          if (c + 2 < BN / 32) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
+          if (c + 2 < BN / 32) tmem_ld_32x32_chk(tmem_base, p.status, taddr + (c + 2) * 32, r0);
           emit(r1, c + 1);
           tmem_ld_wait();
         }
@@ -522,7 +536,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           uint32_t r[32];
-          tmem_ld_32x32(taddr + c * 32, r);
+          tmem_ld_32x32_chk(tmem_base, p.status, taddr + c * 32, r);
           tmem_ld_wait();
           emit(r, c);
         }
@@ -549,7 +563,8 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         uint4 w[kTasks];
 #pragma unroll
         for (int j = 0; j < C::tasks_per_thread; ++j)
-          w[j] = *reinterpret_cast<const uint4*>(src + (ctid + j * kConvThreads) * 16);
+          w[j] = smem_in(src + (ctid + j * kConvThreads) * 16, gen, C::packed, C::staging, 16, p.status)
+                     ? *reinterpret_cast<const uint4*>(src + (ctid + j * kConvThreads) * 16) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
         for (int j = 0; j < C::tasks_per_thread; ++j) {
           const int id = ctid + j * kConvThreads;
@@ -563,8 +578,10 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           else expand32<KIND, false, kPermuteK>(w[j], p.lut_b, o0, o1);
           uint8_t* drow = dst + slab * kExpandedSlab + row * 128;
           const int swz = row & 7;
-          *reinterpret_cast<uint4*>(drow + (((2 * q) ^ swz) << 4)) = o0;
-          *reinterpret_cast<uint4*>(drow + (((2 * q + 1) ^ swz) << 4)) = o1;
+          if (smem_in(drow + (((2 * q) ^ swz) << 4), gen, C::expanded, C::packed, 16, p.status))
+            *reinterpret_cast<uint4*>(drow + (((2 * q) ^ swz) << 4)) = o0;
+          if (smem_in(drow + (((2 * q + 1) ^ swz) << 4), gen, C::expanded, C::packed, 16, p.status))
+            *reinterpret_cast<uint4*>(drow + (((2 * q + 1) ^ swz) << 4)) = o1;
         }
         fence_proxy_async();   // make the generic-proxy writes visible to the tensor core
         __syncwarp();
@@ -768,7 +785,8 @@ luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                               static_cast<float>(static_cast<int>(r[4 * j + 2])), static_cast<float>(static_cast<int>(r[4 * j + 3])));
             }
             v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
-            *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
+            if (smem_in(rowp + ((j ^ sw) << 4), gen, PairSmem::staging, PairSmem::barriers, 16, p.status))
+              *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
           }
           fence_proxy_async();
           __syncwarp();
@@ -779,14 +797,14 @@ luq_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         }
       };
       uint32_t r0[32], r1[32];
-      tmem_ld_32x32(taddr, r0);
+      tmem_ld_32x32_chk(tmem_base, p.status, taddr, r0);
       tmem_ld_wait();
 #pragma unroll 1
       for (int c = 0; c < BN / 32; c += 2) {
-        tmem_ld_32x32(taddr + (c + 1) * 32, r1);
+        tmem_ld_32x32_chk(tmem_base, p.status, taddr + (c + 1) * 32, r1);
         emit(r0, c);
         tmem_ld_wait();
-        if (c + 2 < BN / 32) tmem_ld_32x32(taddr + (c + 2) * 32, r0);
+        if (c + 2 < BN / 32) tmem_ld_32x32_chk(tmem_base, p.status, taddr + (c + 2) * 32, r0);
         emit(r1, c + 1);
         tmem_ld_wait();
       }
@@ -922,6 +940,8 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
   pdl_trigger();
 
   const int raw_iters = 2 * p.num_kb;   // raw stages per tile
+  // Tiles are walked from the END of the tensor: the max reduction that precedes this kernel read
+  // A front to back, so A's tail is what the L2 still holds.
 
   if (warp == 0) {
     // ------------------------------------------ producer of raw activations
@@ -929,7 +949,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
       uint32_t issued = 0, stage = 0, phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; ok && t < p.tiles_m; t += gridDim.x) {
-        const int m0 = t * BM;
+        const int m0 = (p.tiles_m - 1 - t) * BM;   // back to front, see below
         for (int it = 0; it < raw_iters; ++it) {
           if (!mbar_wait(raw_empty(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = raw_full(stage);
@@ -1015,7 +1035,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
     uint32_t tile_it = 0;
     bool ok = true;
     for (int t = blockIdx.x; ok && t < p.tiles_m; t += gridDim.x, ++tile_it) {
-      const long long row0 = static_cast<long long>(t) * BM + quarter * 32;
+      const long long row0 = static_cast<long long>(p.tiles_m - 1 - t) * BM + quarter * 32;
       const uint32_t buf = tile_it & 1u;
       if (!mbar_wait(acc_full(buf), (tile_it >> 1) & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -1032,7 +1052,8 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
             v.y = static_cast<float>(static_cast<int>(r[4 * j + 1])) * scale;
             v.z = static_cast<float>(static_cast<int>(r[4 * j + 2])) * scale;
             v.w = static_cast<float>(static_cast<int>(r[4 * j + 3])) * scale;
-            *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
+            if (smem_in(rowp + ((j ^ sw) << 4), gen, C::staging, C::barriers, 16, p.status))
+              *reinterpret_cast<float4*>(rowp + ((j ^ sw) << 4)) = v;
           }
           fence_proxy_async();
           __syncwarp();
@@ -1047,7 +1068,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
-        tmem_ld_32x32(taddr + c * 32, r);
+        tmem_ld_32x32_chk(tmem_base, p.status, taddr + c * 32, r);
         tmem_ld_wait();
         emit(r, c);
       }
@@ -1080,7 +1101,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
     uint32_t q = 0, stored = 0;
     bool alive = true, ok = true;
     for (int t = blockIdx.x; alive && t < p.tiles_m; t += gridDim.x) {
-      const int m0 = t * BM;
+      const int m0 = (p.tiles_m - 1 - t) * BM;
       for (int it = 0; it < raw_iters; ++it, ++q) {
         const uint32_t rs = q % RS, rphase = (q / RS) & 1u;
         const uint32_t es = (q >> 1) % ES, ephase = ((q >> 1) / ES) & 1u;
@@ -1096,7 +1117,9 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           const uint8_t* src = gen + C::raw + rs * C::raw_stage + boxi * C::box_bytes + row_off;
           uint4 u[kUnits];
 #pragma unroll
-          for (int j = 0; j < kUnits; ++j) u[j] = *reinterpret_cast<const uint4*>(src + ((j ^ rkey) << 4));
+          for (int j = 0; j < kUnits; ++j)
+            u[j] = smem_in(src + ((j ^ rkey) << 4), gen, C::raw, C::codes, 16, p.status)
+                       ? *reinterpret_cast<const uint4*>(src + ((j ^ rkey) << 4)) : make_uint4(0u, 0u, 0u, 0u);
           // 32 elements -> 32 codes (element e in nibble e % 8 of word e / 8) and 32 operand bytes 16 * q
           float v[32];
           if constexpr (BF16) {
@@ -1140,10 +1163,13 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           // operand bytes, element order, into this row of the A slab (128-byte swizzle)
           uint8_t* drow = gen + C::expanded + es * kExpandedStage + row * 128;
           const int unit = group * 4 + boxi * 2;
-          *reinterpret_cast<uint4*>(drow + ((unit ^ (row & 7)) << 4)) = o0;
-          *reinterpret_cast<uint4*>(drow + (((unit + 1) ^ (row & 7)) << 4)) = o1;
+          if (smem_in(drow + ((unit ^ (row & 7)) << 4), gen, C::expanded, C::raw, 16, p.status))
+            *reinterpret_cast<uint4*>(drow + ((unit ^ (row & 7)) << 4)) = o0;
+          if (smem_in(drow + (((unit + 1) ^ (row & 7)) << 4), gen, C::expanded, C::raw, 16, p.status))
+            *reinterpret_cast<uint4*>(drow + (((unit + 1) ^ (row & 7)) << 4)) = o1;
           // packed codes into the staging box of this raw stage: 128 rows x 32 bytes, 32-byte swizzle
-          *reinterpret_cast<uint4*>(gen + cbox_off + row * 32 + ((boxi ^ ((row >> 2) & 1)) << 4)) = packed;
+          if (smem_in(gen + cbox_off + row * 32 + ((boxi ^ ((row >> 2) & 1)) << 4), gen, C::codes, C::staging, 16, p.status))
+            *reinterpret_cast<uint4*>(gen + cbox_off + row * 32 + ((boxi ^ ((row >> 2) & 1)) << 4)) = packed;
           fence_proxy_async();   // both writes are read by the async proxy (tensor core, TMA store)
         }
         // The group's two code boxes alternate.  Here the store issued one turn ago must have read its
@@ -1422,7 +1448,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   // A short contraction with fp32 output is bound by its output stream: with both operands' bytes at
   // hand it runs the whole-row epilogue (bare store kernels: 6.0 TB/s in 1 KB rows against 5.4 in boxes).
   const bool rows_epilogue = !a.out_bf16 && a_given && b_given && p.splits == 1 && total_iters <= 4 &&
-                             a.No % 32 == 0 && !ctx->use_pairs;
+                             a.No % 32 == 0 && ctx->use_pairs != 1;
   const bool use_given = a.out_bf16 != 0 || rows_epilogue;
   if (b_must || rows_epilogue || ((long_contraction || (use_given && b_given)) && p.tiles_m >= 2)) {
     if (b_given) {
@@ -1489,9 +1515,12 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   else bad |= encode_out_map(ctx->encode_tiled, &to, a.d_out, a.Mo, a.No, a.out_bf16 != 0);
   if (bad) return LUQ_ERR_CUDA;
 
-  // CTA pairs when both operands are planes (no expansion inside the kernel) and the contraction
-  // is not split: option LUQ_OPT_PAIRS (off unless set)
-  if (ctx->use_pairs && a_plane && b_plane && p.splits == 1 && p.tiles_m >= 2 && !a.out_bf16) {
+  // CTA pairs need both operands as planes (no expansion inside the kernel) and an unsplit contraction
+  // CTA pairs: forced (1), or chosen here (2, the default) for the products they were measured faster on -
+  // a long contraction with B stored contraction-major (backward and update products of a wide layer:
+  // 35.2 -> 31.5 us and 33.1 -> 30.6 us on the Transformer shape; the forward product is 4 % slower on pairs)
+  const bool pairs_wanted = ctx->use_pairs == 1 || (ctx->use_pairs == 2 && a.b_mn && total_iters >= 8);
+  if (pairs_wanted && !rows_epilogue && a_plane && b_plane && p.splits == 1 && p.tiles_m >= 2 && !a.out_bf16) {
     const long long pair_tiles = static_cast<long long>((p.tiles_m + 1) / 2) * p.tiles_n;
     const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;
     const int pairs = static_cast<int>(pair_tiles < max_pairs ? pair_tiles : max_pairs);
@@ -1636,6 +1665,28 @@ int luq_launch_quant_fwd(luq_ctx* ctx, const void* d_a, int dtype, const float* 
   return static_cast<int>(e);
 }
 
+namespace {
+// Diagnostic for the checking build: forms an address one byte beyond a 64-byte shared-memory region and
+// asks the check about it.  Nothing is accessed.  With -DLUQ_DEBUG the check raises LUQ_STATUS_BOUNDS;
+// in the normal build the check is compiled out and nothing happens.
+__global__ void bounds_probe_kernel(unsigned int* status) {
+  __shared__ __align__(16) uint8_t region[64];
+  pdl_wait();
+  pdl_trigger();
+  if (threadIdx.x == 0) {
+    const bool inside = smem_in(region + 16, region, 0, 64, 16, status);
+    const bool beyond = smem_in(region + 49, region, 0, 64, 16, status);
+    (void)inside; (void)beyond;
+  }
+}
+}  // namespace
+
+int luq_launch_bounds_probe(luq_ctx* ctx, cudaStream_t st) {
+  const cudaError_t e = luq_launch_kernel(bounds_probe_kernel, 1, 32, 0, st, LUQ_LAUNCH_EARLY, 1, ctx->d_status);
+  ctx->launches += 1;
+  return static_cast<int>(e);
+}
+
 int luq_launch_expire_wait(luq_ctx* ctx, cudaStream_t st) {
   const cudaError_t e = luq_launch_kernel(expire_wait_kernel, 1, 32, 0, st, LUQ_LAUNCH_EARLY, 1, ctx->d_status, 1u << 16);
   ctx->launches += 1;
@@ -1742,7 +1793,7 @@ extern "C" int luq_gemm_wgrad_static(const uint8_t* d_g_codes, const float* d_al
   local.workspace_bytes = kStaticScratchBytes;
   local.mma_kind = LUQ_DEFAULT_MMA_KIND;
   local.forced_splits = 0;
-  local.use_pairs = 0;
+  local.use_pairs = 2;
   local.sm_limit = 0;
   local.grad_int4 = 0;
   local.kmax = LUQ_KMAX;

@@ -32,6 +32,13 @@ using luqdev::scale_usable;
 using luqdev::int4_code;
 using luqdev::uint4_code;
 
+// checking build: is piece `idx` one of the tensor's `items` 16-byte pieces?  (a violation raises
+// LUQ_STATUS_BOUNDS and the caller skips the access; always true, and free, in the normal build)
+__device__ __forceinline__ bool piece_ok(size_t idx, size_t items, unsigned int* status) {
+  (void)idx; (void)items; (void)status;
+  return LUQ_IN_BOUNDS(idx < items, status);
+}
+
 template <bool BF16> struct Item {
   static constexpr int kElems = BF16 ? 8 : 4;  // elements per 16-byte piece
   // widen one piece to fp32 (bf16 -> fp32 is exact: bits << 16)
@@ -165,7 +172,8 @@ __device__ __forceinline__ void amax_body(const void* __restrict__ x, size_t n, 
     const uint4* q = p + t * kTileItems + threadIdx.x;
     uint4 u[kUnroll];
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(q + j * kThreads);
+    for (int j = 0; j < kUnroll; ++j)
+      u[j] = piece_ok(t * kTileItems + threadIdx.x + j * kThreads, items, status) ? __ldg(q + j * kThreads) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) fold(u[j]);
   }
@@ -344,9 +352,11 @@ __device__ __forceinline__ void quant_int4_body(const void* __restrict__ x, size
     const size_t i0 = (full_tiles - 1 - t) * kTileItems + threadIdx.x;
     uint4 u[kUnroll];
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i0 + j * kThreads);
+    for (int j = 0; j < kUnroll; ++j)
+      u[j] = piece_ok(i0 + j * kThreads, items, status) ? __ldg(p + i0 + j * kThreads) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) emit(i0 + j * kThreads, u[j]);
+    for (int j = 0; j < kUnroll; ++j)
+      if (piece_ok(i0 + j * kThreads, items, status)) emit(i0 + j * kThreads, u[j]);
   }
   if (rank == count - 1)
     for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) emit(i, __ldg(p + i));
@@ -668,9 +678,11 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
       const size_t i0 = (back_to_front ? full_tiles - 1 - t : t) * kTileItems + threadIdx.x;
       uint4 u[kUnroll];
 #pragma unroll
-      for (int j = 0; j < kUnroll; ++j) u[j] = __ldg(p + i0 + j * kThreads);
+      for (int j = 0; j < kUnroll; ++j)
+        u[j] = piece_ok(i0 + j * kThreads, items, status) ? __ldg(p + i0 + j * kThreads) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-      for (int j = 0; j < kUnroll; ++j) process(i0 + j * kThreads, u[j], true);
+      for (int j = 0; j < kUnroll; ++j)
+        if (piece_ok(i0 + j * kThreads, items, status)) process(i0 + j * kThreads, u[j], true);
     }
     if (blockIdx.x == gridDim.x - 1)
       for (size_t i = full_tiles * kTileItems + threadIdx.x; i < items; i += kThreads) process(i, __ldg(p + i), false);
@@ -909,8 +921,7 @@ __global__ void __launch_bounds__(kThreads) luq_quotient_kernel(const float* __r
 }
 
 // Grid for a kernel that walks `tiles` tiles: at most the CTAs the GPU holds at once
-// (optionally fewer per SM), and then the smallest grid with the same number of rounds,
-// so that every CTA gets the same share.
+// (optionally fewer per SM), a multiple of the SM count.
 template <typename K>
 int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 30) {
   int per_sm = 0;
@@ -925,8 +936,11 @@ int grid_for(const luq_ctx* ctx, K kernel, size_t tiles, int max_per_sm = 1 << 3
   if (cap > LUQ_SCRATCH_REGION - 2) cap = LUQ_SCRATCH_REGION - 2;   // one scratch word per block of a reducing kernel
   if (tiles < 1) tiles = 1;
   if (tiles <= cap) return static_cast<int>(tiles);
-  const size_t rounds = (tiles + cap - 1) / cap;
-  return static_cast<int>((tiles + rounds - 1) / rounds);
+  // More tiles than resident blocks: a whole number of blocks per SM, so that every SM carries the
+  // same load (a grid of, say, 5.8 blocks per SM leaves the SMs with five blocks idle while those
+  // with six finish); the tiles are dealt out round-robin and differ by at most one per block.
+  const size_t whole = cap / static_cast<size_t>(ctx->sm_count) * static_cast<size_t>(ctx->sm_count);
+  return static_cast<int>(whole > 0 ? whole : cap);
 }
 
 }  // namespace

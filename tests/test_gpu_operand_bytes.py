@@ -254,6 +254,7 @@ def test_cta_pair_kernel_matches_the_single_cta_kernel(ctx, mma_kind):
     A, W, G = inputs.small_layer(M, K, N, 123)
     (ca, sa, ba), (cw, sw, bw), (cg, al, bg) = layer_with_bytes(ctx, A, W, G, seed=5, ns=ns)
     ctx.set_option(binding.OPT_MMA_KIND, mma_kind)
+    ctx.set_option(binding.OPT_PAIRS, 0)
     try:
         single = (ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=ba, w_operand=bw),
                   ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bg, w_operand=bw),
@@ -263,12 +264,16 @@ def test_cta_pair_kernel_matches_the_single_cta_kernel(ctx, mma_kind):
         paired = (ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=ba, w_operand=bw),
                   ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bg, w_operand=bw),
                   ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K, g_operand=bg, a_operand=ba))
+        ctx.set_option(binding.OPT_PAIRS, 2)      # the default: pairs where measured faster (backward, update)
+        auto = (ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=ba, w_operand=bw),
+                ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bg, w_operand=bw),
+                ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K, g_operand=bg, a_operand=ba))
     finally:
-        ctx.set_option(binding.OPT_PAIRS, 0)
+        ctx.set_option(binding.OPT_PAIRS, 2)
         ctx.set_option(binding.OPT_MMA_KIND, 2)
     assert ctx.status() == 0
-    for s, p in zip(single, paired):
-        assert torch.equal(s, p)
+    for s, p, a in zip(single, paired, auto):
+        assert torch.equal(s, p) and torch.equal(s, a)
     oa, ow, og = ca.cpu().numpy(), cw.cpu().numpy(), cg.cpu().numpy().reshape(ns, -1)
     r = np.array([0, 127, 128, 255, 256, 1000, M - 1, M - 1, 0], dtype=np.int64)
     c = np.array([0, 255, 256, 1, N - 1, 777, N - 1, 0, N - 1], dtype=np.int64)
