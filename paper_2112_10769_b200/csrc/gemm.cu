@@ -1214,7 +1214,15 @@ __global__ void __launch_bounds__(256) split_reduce_kernel(const float* __restri
   const int r = rem / (BN / 4), c4 = rem % (BN / 4);
   const float4* src = reinterpret_cast<const float4*>(ws) + (static_cast<size_t>(tile) * splits) * (kTileFloats / 4) + rem;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < splits; ++s) {
+  int s = 0;
+  for (; s + 8 <= splits; s += 8) {   // eight loads in flight, added in split order
+    float4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __ldcg(src + static_cast<size_t>(s + j) * (kTileFloats / 4));
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
+  }
+  for (; s < splits; ++s) {
     const float4 v = __ldcg(src + static_cast<size_t>(s) * (kTileFloats / 4));
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
   }
