@@ -335,7 +335,10 @@ class LayerBench:
                 self.calls["quant_int4_W"](); self.calls["quant_int4_A"]()
             self.calls["gemm_fwd"]()
         main.wait_event(join)
-        self.calls["gemm_bwd"](); self.calls["gemm_wgrad"]()
+        if self.args.wgrad_first:
+            self.calls["gemm_wgrad"](); self.calls["gemm_bwd"]()
+        else:
+            self.calls["gemm_bwd"](); self.calls["gemm_wgrad"]()
 
     def launches(self):
         return self.ctx.launches + (self.ctx_g.launches if self.ctx_g is not self.ctx else 0)
@@ -891,6 +894,8 @@ def main():
     ap.add_argument("--sweep-exponents", default=None,
                     help="cfg4: comma-separated log2 sizes instead of the whole sweep (e.g. 26 for a profiling run)")
     ap.add_argument("--sweep-quick", action="store_true", help="cfg4: max + LUQ only, without the variant quantizers")
+    ap.add_argument("--wgrad-first", type=int, default=0, choices=(0, 1),
+                    help="1 = update product before the backward product")
     ap.add_argument("--multi-amax", type=int, default=1, choices=(0, 1),
                     help="1: max|A| and max|W| from one launch (luq_amax_multi) in the timed step")
     ap.add_argument("--no-fused", action="store_true", help="quant_int4(A) and gemm_fwd as two kernels")

@@ -1120,6 +1120,12 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           for (int j = 0; j < kUnits; ++j)
             u[j] = smem_in(src + ((j ^ rkey) << 4), gen, C::raw, C::codes, 16, p.status)
                        ? *reinterpret_cast<const uint4*>(src + ((j ^ rkey) << 4)) : make_uint4(0u, 0u, 0u, 0u);
+          // The raw slot is given back as soon as this warp has loaded its rows, not after the conversion:
+          // what one SM can stream is the bytes its three raw slots keep in flight, and a slot that waits
+          // for arithmetic, stores and a barrier is not in flight.  The arrival has release semantics, so
+          // the loads above (every lane's, through the warp barrier) are performed before it is seen.
+          __syncwarp();
+          if (lane == 0) mbar_arrive(raw_empty(rs));
           // 32 elements -> 32 codes (element e in nibble e % 8 of word e / 8) and 32 operand bytes 16 * q
           float v[32];
           if constexpr (BF16) {
@@ -1182,7 +1188,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           bulk_commit();
         }
         ++stored;
-        if (lane == 0) { mbar_arrive(raw_empty(rs)); mbar_arrive(ex_full(es)); }
+        if (lane == 0) mbar_arrive(ex_full(es));
       }
     }
     if (ctid == 0) bulk_wait<0>();
