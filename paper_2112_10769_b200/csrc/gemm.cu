@@ -556,7 +556,6 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       unit_range(u, tile, it_begin, it_end);
       for (int k_it = it_begin; k_it < it_end; ++k_it) {
         if (!mbar_wait(pk_full(ps), pphase, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(ex_empty(es), ephase ^ 1u, abort_flag)) { ok = false; break; }
         const uint8_t* src = gen + C::packed + ps * C::packed_stage;
         uint8_t* dst = gen + C::expanded + es * kExpandedStage;
         constexpr int kTasks = C::tasks_per_thread > 0 ? C::tasks_per_thread : 1;
@@ -565,6 +564,12 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         for (int j = 0; j < C::tasks_per_thread; ++j)
           w[j] = smem_in(src + (ctid + j * kConvThreads) * 16, gen, C::packed, C::staging, 16, p.status)
                      ? *reinterpret_cast<const uint4*>(src + (ctid + j * kConvThreads) * 16) : make_uint4(0u, 0u, 0u, 0u);
+        // The packed slot goes back to the producer as soon as this warp has loaded its words - before
+        // the operand stage is free and before the expansion - so that the next copy is in flight
+        // meanwhile.  (The arrival has release semantics: the loads above are performed before it is seen.)
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pk_empty(ps));
+        if (!mbar_wait(ex_empty(es), ephase ^ 1u, abort_flag)) { ok = false; break; }
 #pragma unroll
         for (int j = 0; j < C::tasks_per_thread; ++j) {
           const int id = ctid + j * kConvThreads;
@@ -585,7 +590,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
         fence_proxy_async();   // make the generic-proxy writes visible to the tensor core
         __syncwarp();
-        if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive(ex_full(es)); }
+        if (lane == 0) mbar_arrive(ex_full(es));
         if (++ps == static_cast<uint32_t>(PS > 0 ? PS : 1)) { ps = 0; pphase ^= 1u; }
         if (++es == static_cast<uint32_t>(ES)) { es = 0; ephase ^= 1u; }
       }
@@ -1111,21 +1116,24 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           if (ok && lane == 0) mbar_arrive(raw_empty(rs));
           continue;
         }
-        if (ok) ok = mbar_wait_idle(ex_empty(es), ephase ^ 1u, abort_flag);
         const uint32_t cbox_off = C::codes + (2 * group + (stored & 1u)) * C::code_box;
+        uint4 u[kUnits];
         if (ok) {
           const uint8_t* src = gen + C::raw + rs * C::raw_stage + boxi * C::box_bytes + row_off;
-          uint4 u[kUnits];
 #pragma unroll
           for (int j = 0; j < kUnits; ++j)
             u[j] = smem_in(src + ((j ^ rkey) << 4), gen, C::raw, C::codes, 16, p.status)
                        ? *reinterpret_cast<const uint4*>(src + ((j ^ rkey) << 4)) : make_uint4(0u, 0u, 0u, 0u);
-          // The raw slot is given back as soon as this warp has loaded its rows, not after the conversion:
-          // what one SM can stream is the bytes its three raw slots keep in flight, and a slot that waits
-          // for arithmetic, stores and a barrier is not in flight.  The arrival has release semantics, so
-          // the loads above (every lane's, through the warp barrier) are performed before it is seen.
+          // The raw slot is given back as soon as this warp has loaded its rows - before the operand stage
+          // is free, before the conversion: what one SM can stream is the bytes its three raw slots keep
+          // in flight, and a slot that waits for arithmetic, stores and a barrier is not in flight.  The
+          // arrival has release semantics, so the loads above (every lane's, through the warp barrier)
+          // are performed before it is seen.
           __syncwarp();
           if (lane == 0) mbar_arrive(raw_empty(rs));
+          ok = mbar_wait_idle(ex_empty(es), ephase ^ 1u, abort_flag);
+        }
+        if (ok) {
           // 32 elements -> 32 codes (element e in nibble e % 8 of word e / 8) and 32 operand bytes 16 * q
           float v[32];
           if constexpr (BF16) {
