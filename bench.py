@@ -259,6 +259,9 @@ class LayerBench:
                 c.set_option(binding.OPT_MMA_KIND, args.mma_kind)
             if args.pairs is not None:
                 c.set_option(binding.OPT_PAIRS, args.pairs)
+            if args.sum_samples and cfg.n_samples > 1:
+                c.set_option(binding.OPT_SUM_SAMPLES, 1)
+        self.sum_samples = bool(args.sum_samples and cfg.n_samples > 1)
         self.stream_g = torch.cuda.Stream() if args.streams == 2 else None
         dev = self.A.device
         f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)  # noqa: E731
@@ -270,7 +273,7 @@ class LayerBench:
         # Operand bytes (the 8-bit form of the codes, written by the quantizer in the same pass) for the
         # tensors that many GEMM tiles re-read: always W and G; A when the layer is wide enough that the
         # forward product reads each row block of A four times or more.
-        self.oW, self.oG = i8(N * K), i8(ns * M * N)
+        self.oW, self.oG = i8(N * K), i8((1 if self.sum_samples else ns) * M * N)
         self.oA = i8(M * K) if N >= 1024 else None
         self.Z, self.dA, self.dW = f32(M, N), f32(M, K), f32(N, K)
         # the forward half as one kernel where the layer has a single column of output tiles
@@ -478,6 +481,8 @@ def bench_layer_compact(torch, binding, inputs, local, args, name, barrier, host
            "ms_min": round(st["ms_min"], 5), "blocks": st["blocks"],
            "tflops": round(3 * 2.0 * M * N * K / (st["ms_median"] * 1e-3) / 1e12, 2),
            "launches_per_step": per_step, "launch": mode, "fused_forward": lb.fused}
+    if lb.ns > 1:
+        out["sample_planes"] = "summed into one (LUQ_OPT_SUM_SAMPLES)" if lb.sum_samples else "one per sample"
     lb.close()
     del lb
     torch.cuda.empty_cache()
@@ -852,6 +857,9 @@ def run_ours(args):
                        "fused_forward": "quant_int4(A) + gemm_fwd in one kernel (luq_quant_int4_gemm_fwd)" if lb.fused else "no",
                        "operand_bytes": "W,G" + (",A" if lb.oA is not None else "") +
                                         ": the quantizers also write the codes' 8-bit form, the GEMMs are handed it",
+                       "sample_planes": ("one operand plane = the sum of the samples' bytes (LUQ_OPT_SUM_SAMPLES); "
+                                         "the gradient products read it once and divide by the sample count")
+                                        if lb.sum_samples else "one per sample",
                        "streams": "2: gradient max + LUQ beside the activation/weight passes and the forward product"
                                   if args.streams == 2 else "1",
                        "amax_A_and_W": ("one launch (luq_amax_multi; without the fused forward kernel also luq_quant_int4_multi)"
@@ -894,6 +902,10 @@ def main():
     ap.add_argument("--sweep-exponents", default=None,
                     help="cfg4: comma-separated log2 sizes instead of the whole sweep (e.g. 26 for a profiling run)")
     ap.add_argument("--sweep-quick", action="store_true", help="cfg4: max + LUQ only, without the variant quantizers")
+    ap.add_argument("--sum-samples", type=int, default=1, choices=(0, 1),
+                    help="1 (default) = with several samples the quantizer writes one operand plane, the sum of the "
+                         "samples' bytes, and the backward / update products read it (LUQ_OPT_SUM_SAMPLES): same "
+                         "results bit for bit at one sample's product cost; 0 = one plane per sample")
     ap.add_argument("--wgrad-first", type=int, default=0, choices=(0, 1),
                     help="1 = update product before the backward product")
     ap.add_argument("--multi-amax", type=int, default=1, choices=(0, 1),

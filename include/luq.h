@@ -90,6 +90,20 @@ extern "C" {
                               leaves the tensor cores idle, and the update product, which is bound by the tensor
                               cores and moves little memory - can then run side by side on two streams (two
                               contexts), each on its share of the SMs.  Results do not depend on the limit. */
+#define LUQ_OPT_SUM_SAMPLES 9 /* 1: with n_samples >= 2 (SMP, Sec. 5.1) the operand bytes that luq_quant_grad,
+                              luq_amax_quant_grad, luq_quant_grad_pw2 and luq_quant_grad_hindsight write are ONE
+                              plane of rows * cols bytes: byte e = the sum over the samples of the int8 value
+                              +-2^(c-1) of element e (the packed codes stay one plane per sample), and luq_gemm_bwd /
+                              luq_gemm_wgrad given such bytes with that n_samples read one plane and divide by
+                              n_samples.  The mean over samples of the products is, by linearity, the product with
+                              the summed operand divided by n_samples, and both are exact in the int32
+                              accumulator: results equal those of the per-sample planes bit for bit, at the cost
+                              of one sample's product.  Needs n_samples * 2^kmax <= 127 (two samples at the
+                              default level count, up to three at kmax = 5) and int8 operands, otherwise the
+                              quantizer / the product returns LUQ_ERR_UNSUPPORTED; the ablation's quantizers
+                              return it too.  Set it on the quantizing and on the multiplying context alike.
+                              0 (default): one plane per sample.  The paper states SMP as repeated products;
+                              it has no counterpart of this shortcut. */
 #define LUQ_OPT_LEVELS 4   /* kmax of the gradient quantizers, 1..6 (default luq_kmax() = 4): levels
                               alpha * 2^0 .. alpha * 2^kmax with alpha = max / 2^kmax, codes 0..kmax+1.  The
                               other grids of the paper from the same kernels: kmax = 2 is the FP2 grid of

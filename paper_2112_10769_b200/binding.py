@@ -21,6 +21,7 @@ STATUS_NONFINITE, STATUS_RANGE, STATUS_TIMEOUT, STATUS_BOUNDS = 1, 2, 4, 8
 OPT_MMA_KIND, OPT_SPLITS, OPT_PAIRS, OPT_LEVELS, OPT_UNSIGNED_ACTIVATIONS, OPT_OUTPUT_BF16 = 1, 2, 3, 4, 5, 6
 OPT_GRADIENT_INT4 = 7
 OPT_SM_LIMIT = 8
+OPT_SUM_SAMPLES = 9
 SCHEME_FP4, SCHEME_FP4_SR, SCHEME_FP4_SU, SCHEME_LUQ, SCHEME_INT4_SR = 0, 1, 2, 3, 4
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
@@ -134,6 +135,12 @@ class Context:
         _check(load().luq_set_option(self.handle, option, value), "luq_set_option")
         if option == OPT_OUTPUT_BF16:
             self.out_dtype = torch.bfloat16 if value else torch.float32
+        if option == OPT_SUM_SAMPLES:
+            self.sum_samples = bool(value)
+
+    def _planes(self, n_samples: int) -> int:
+        """Operand planes the LUQ quantizers write / the gradient products read: one per sample, or one in all."""
+        return 1 if getattr(self, "sum_samples", False) else n_samples
 
     def _out(self, out, rows: int, cols: int, device):
         """Output tensor of a GEMM: the caller's (type checked) or a new one of the context's output type."""
@@ -241,7 +248,7 @@ class Context:
         alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
         _check(load().luq_amax_quant_grad(self.handle, g.data_ptr(), _dtype_code(g), rows, cols,
                                           seed & (2 ** 64 - 1), n_samples, amax.data_ptr(), codes.data_ptr(),
-                                          alpha.data_ptr(), _opt(operand, n_samples * g.numel()), _stream()),
+                                          alpha.data_ptr(), _opt(operand, self._planes(n_samples) * g.numel()), _stream()),
                "luq_amax_quant_grad")
         return amax, codes, alpha
 
@@ -254,7 +261,7 @@ class Context:
         alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
         _check(load().luq_quant_grad(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
                                      seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
-                                     _opt(operand, n_samples * g.numel()), _stream()), "luq_quant_grad")
+                                     _opt(operand, self._planes(n_samples) * g.numel()), _stream()), "luq_quant_grad")
         return codes, alpha
 
     def quant_grad_nearest(self, g: torch.Tensor, amax: torch.Tensor, codes: torch.Tensor | None = None,
@@ -292,7 +299,7 @@ class Context:
         alpha = torch.empty(1, dtype=torch.float32, device=g.device) if alpha is None else alpha
         _check(load().luq_quant_grad_pw2(self.handle, g.data_ptr(), _dtype_code(g), rows, cols, amax.data_ptr(),
                                          seed & (2 ** 64 - 1), n_samples, codes.data_ptr(), alpha.data_ptr(),
-                                         _opt(operand, n_samples * g.numel()), _stream()), "luq_quant_grad_pw2")
+                                         _opt(operand, self._planes(n_samples) * g.numel()), _stream()), "luq_quant_grad_pw2")
         return codes, alpha
 
     def quant_grad_hindsight(self, g: torch.Tensor, m_hat: torch.Tensor, eta: float, seed: int, n_samples: int = 1,
@@ -309,7 +316,7 @@ class Context:
         _check(load().luq_quant_grad_hindsight(self.handle, g.data_ptr(), _dtype_code(g), rows, cols,
                                                m_hat.data_ptr(), eta, int(pw2), seed & (2 ** 64 - 1), n_samples,
                                                codes.data_ptr(), alpha.data_ptr(), measured.data_ptr(),
-                                               _opt(operand, n_samples * g.numel()), _stream()),
+                                               _opt(operand, self._planes(n_samples) * g.numel()), _stream()),
                "luq_quant_grad_hindsight")
         return codes, alpha, measured
 
@@ -355,7 +362,7 @@ class Context:
                  w_operand: torch.Tensor | None = None):
         out = self._out(out, M, K, g_codes.device)
         _check(load().luq_gemm_bwd(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
-                                   _opt(g_operand, n_samples * M * N), w_codes.data_ptr(), sw.data_ptr(),
+                                   _opt(g_operand, self._planes(n_samples) * M * N), w_codes.data_ptr(), sw.data_ptr(),
                                    _opt(w_operand, N * K), out.data_ptr(), M, N, K, _stream()), "luq_gemm_bwd")
         return out
 
@@ -364,7 +371,7 @@ class Context:
                    a_operand: torch.Tensor | None = None):
         out = self._out(out, N, K, g_codes.device)
         _check(load().luq_gemm_wgrad(self.handle, g_codes.data_ptr(), alpha.data_ptr(), n_samples,
-                                     _opt(g_operand, n_samples * M * N), a_codes.data_ptr(), sa.data_ptr(),
+                                     _opt(g_operand, self._planes(n_samples) * M * N), a_codes.data_ptr(), sa.data_ptr(),
                                      _opt(a_operand, M * K), out.data_ptr(), M, N, K, _stream()), "luq_gemm_wgrad")
         return out
 

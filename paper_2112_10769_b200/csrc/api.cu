@@ -127,6 +127,10 @@ int luq_set_option(luq_ctx* ctx, int option, int value) {
       if (value < 0 || value > 4096) return LUQ_ERR_ARG;
       ctx->sm_limit = value;
       return LUQ_OK;
+    case LUQ_OPT_SUM_SAMPLES:
+      if (value != 0 && value != 1) return LUQ_ERR_ARG;
+      ctx->sum_samples = value;
+      return LUQ_OK;
     case LUQ_OPT_PAIRS:
       if (value < 0 || value > 2) return LUQ_ERR_ARG;
       ctx->use_pairs = value;
@@ -247,15 +251,24 @@ static int quant_grad_args(luq_ctx* ctx, const void* d_g, int dtype, size_t rows
   return LUQ_OK;
 }
 
+// LUQ_OPT_SUM_SAMPLES: flag bit for the LUQ launcher (0 when the option does not apply to this call), or
+// LUQ_ERR_UNSUPPORTED when the sum of n_samples operand bytes of magnitude 2^kmax could leave int8
+static int sum_flag(const luq_ctx* ctx, int n_samples, const int8_t* d_operand) {
+  if (!ctx->sum_samples || !d_operand || n_samples < 2) return 0;
+  return (n_samples << ctx->kmax) <= 127 ? 8 : LUQ_ERR_UNSUPPORTED;
+}
+
 int luq_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, size_t cols, const float* d_amax,
                    uint64_t seed, int n_samples, uint8_t* d_codes, float* d_alpha, int8_t* d_operand, void* stream) {
   size_t n = 0;
   const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, d_operand, &n);
   if (rc) return rc;
+  const int sum = sum_flag(ctx, n_samples, d_operand);
+  if (sum < 0) return sum;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, nullptr, 0.0f, nullptr,
+                                          n ? d_operand : nullptr, d_alpha, sum, nullptr, nullptr, 0.0f, nullptr,
                                           as_stream(stream)));
 }
 
@@ -265,10 +278,12 @@ int luq_amax_quant_grad(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, s
   size_t n = 0;
   const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, d_operand, &n);
   if (rc) return rc;
+  const int sum = sum_flag(ctx, n_samples, d_operand);
+  if (sum < 0) return sum;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, nullptr, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 0, nullptr, nullptr, 0.0f, d_amax,
+                                          n ? d_operand : nullptr, d_alpha, sum, nullptr, nullptr, 0.0f, d_amax,
                                           as_stream(stream)));
 }
 
@@ -290,6 +305,7 @@ int luq_quant_grad_ablation(luq_ctx* ctx, const void* d_g, int dtype, size_t row
   const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_scale, d_operand, &n);
   if (rc) return rc;
   if (scheme < 0 || scheme > LUQ_SCHEME_INT4_SR) return LUQ_ERR_ARG;
+  if (ctx->sum_samples && d_operand && n_samples > 1) return LUQ_ERR_UNSUPPORTED;   // these kernels write one plane per sample
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ablation(ctx, d_g, dtype, n, d_amax, seed, n_samples, scheme, d_codes,
@@ -302,10 +318,12 @@ int luq_quant_grad_pw2(luq_ctx* ctx, const void* d_g, int dtype, size_t rows, si
   size_t n = 0;
   const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_amax, n_samples, d_codes, d_alpha, d_operand, &n);
   if (rc) return rc;
+  const int sum = sum_flag(ctx, n_samples, d_operand);
+  if (sum < 0) return sum;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_amax, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 1, nullptr, nullptr, 0.0f, nullptr,
+                                          n ? d_operand : nullptr, d_alpha, 1 | sum, nullptr, nullptr, 0.0f, nullptr,
                                           as_stream(stream)));
 }
 
@@ -316,11 +334,13 @@ int luq_quant_grad_hindsight(luq_ctx* ctx, const void* d_g, int dtype, size_t ro
   const int rc = quant_grad_args(ctx, d_g, dtype, rows, cols, d_mhat, n_samples, d_codes, d_alpha, d_operand, &n);
   if (rc) return rc;
   if (!d_measured_max || !(eta >= 0.0f && eta <= 1.0f) || (pw2 != 0 && pw2 != 1)) return LUQ_ERR_ARG;
+  const int sum = sum_flag(ctx, n_samples, d_operand);
+  if (sum < 0) return sum;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return LUQ_ERR_CUDA;
   // one kernel: quantize with the estimate, measure, and let the last block replace the estimate
   return cuda_rc(luq_launch_quant_grad_ex(ctx, d_g, dtype, n, d_mhat, seed, n_samples, d_codes,
-                                          n ? d_operand : nullptr, d_alpha, 2 | pw2, d_measured_max, d_mhat, eta,
+                                          n ? d_operand : nullptr, d_alpha, 2 | pw2 | sum, d_measured_max, d_mhat, eta,
                                           nullptr, as_stream(stream)));
 }
 
@@ -416,6 +436,7 @@ int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, i
   a.a_codes = d_g_codes; a.a_kind = ctx->grad_int4 ? 0 : 1; a.a_mn = 0; a.n_samples = n_samples;   // G[M x N]: contraction n contiguous
   a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 1;                            // W[N x K]: rows are the contraction
   a.a_operand = d_g_operand; a.b_operand = d_w_operand;
+  a.a_summed = (ctx->sum_samples && !ctx->grad_int4 && d_g_operand && n_samples > 1) ? n_samples : 0;
   a.d_scale_a = d_alpha; a.d_scale_b = d_sw; a.d_out = d_da; a.out_bf16 = ctx->out_bf16; a.Mo = M; a.No = K; a.Kc = N;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;
@@ -434,6 +455,7 @@ int luq_gemm_wgrad(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha,
   a.a_codes = d_g_codes; a.a_kind = ctx->grad_int4 ? 0 : 1; a.a_mn = 1; a.n_samples = n_samples;   // G[M x N]: rows are the contraction
   a.b_codes = d_a_codes; a.b_kind = ctx->unsigned_act ? 2 : 0; a.b_mn = 1;    // A[M x K]: rows are the contraction
   a.a_operand = d_g_operand; a.b_operand = d_a_operand;
+  a.a_summed = (ctx->sum_samples && !ctx->grad_int4 && d_g_operand && n_samples > 1) ? n_samples : 0;
   a.d_scale_a = d_alpha; a.d_scale_b = d_sa; a.d_out = d_dw; a.out_bf16 = ctx->out_bf16; a.Mo = N; a.No = K; a.Kc = M;
   a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
   a.allow_split = 1;

@@ -23,6 +23,7 @@ struct luq_ctx {
   int unsigned_act;         // activation codes handed to the forward / update GEMMs are unsigned INT4
   int grad_int4;            // gradient codes handed to the backward / update GEMMs are INT4 (the ablation's uniform arm)
   int sm_limit;             // GEMM grids use at most this many SMs (0 = all)
+  int sum_samples;          // the LUQ quantizers' operand bytes are one plane: the sum over the samples
   int kmax;                 // LUQ levels alpha * 2^0 .. alpha * 2^kmax (1..6, default LUQ_KMAX)
   int64_t launches;
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved at create
@@ -43,7 +44,8 @@ int luq_launch_quant_int4_hindsight(luq_ctx* ctx, const void* d_x, int dtype, si
                                     uint8_t* d_codes, int8_t* d_operand, float* d_scale, float* d_measured,
                                     cudaStream_t st);
 // flags: bit 0 = power-of-two scale; bit 1 = in-hindsight (d_amax is the running estimate: the tensor's own
-// max|x| goes to d_measured and d_estimate (= d_amax) is replaced by (1 - eta) * measured + eta * estimate)
+// max|x| goes to d_measured and d_estimate (= d_amax) is replaced by (1 - eta) * measured + eta * estimate);
+// bit 2 = deterministic rounding; bit 3 = d_operand is one plane, the sum of the samples' bytes
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
                              float* d_measured, float* d_estimate, float eta, float* d_amax_out, cudaStream_t st);
@@ -76,6 +78,7 @@ struct luq_gemm_args {
   const uint8_t* a_codes; int a_kind; int a_mn; int n_samples;
   const uint8_t* b_codes; int b_kind; int b_mn;
   const int8_t* a_operand; const int8_t* b_operand;   // int8 operand bytes from the quantizer, or null
+  int a_summed;   // > 1: a_operand is ONE plane, the sum of that many samples' bytes (n_samples equals it)
   const float* d_scale_a; const float* d_scale_b;
   void* d_out; int out_bf16;   // fp32 [Mo x No], or bf16 when out_bf16
   int64_t Mo, No, Kc;

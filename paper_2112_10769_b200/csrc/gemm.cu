@@ -1406,7 +1406,11 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   GemmParams p{};
   p.scale_a = a.d_scale_a; p.scale_b = a.d_scale_b; p.status = ctx->d_status;
   p.Mo = a.Mo; p.No = a.No; p.Kc = a.Kc;
-  p.n_samples = a.n_samples;
+  // a summed plane (LUQ_OPT_SUM_SAMPLES) is one sample as far as the contraction goes; the division by
+  // the sample count and the accumulator's range still follow a.n_samples
+  const int ns = a.a_summed > 1 ? 1 : a.n_samples;
+  if (a.a_summed > 1 && (a.a_summed != a.n_samples || a.a_kind != 1 || !a.a_operand)) return LUQ_ERR_ARG;
+  p.n_samples = ns;
   p.out_bf16 = a.out_bf16;
   if (a.out_bf16 && a.No % 8 != 0) return LUQ_ERR_ARG;   // output rows must stay 16-byte aligned
   p.tiles_m = static_cast<int>((a.Mo + BM - 1) / BM);
@@ -1445,12 +1449,13 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   const bool int32_safe = worst_product * a.Kc * a.n_samples < (1ll << 31);
   if (ctx->mma_kind == 2) ctx->mma_kind = int32_safe ? 1 : 0;
   if (ctx->mma_kind == 1 && !int32_safe) return LUQ_ERR_ARG;
+  if (a.a_summed > 1 && ctx->mma_kind != 1) return LUQ_ERR_UNSUPPORTED;   // sums of levels are int8 values, not e4m3
   // Operand planes: an operand that at least two tiles re-read is fetched as bytes.  The caller's
   // bytes (written by the quantizer, int8) are taken as they are; otherwise the codes are expanded
   // once into the workspace behind the split region, if there is room.  A product with a short
   // contraction is bound by its output stream and hides the in-kernel expansion completely
   // (measured: the backward product of the ResNet shape, 2 blocks per tile), so it keeps the codes.
-  const size_t a_plane_bytes = static_cast<size_t>(a.Mo) * a.Kc * a.n_samples;
+  const size_t a_plane_bytes = static_cast<size_t>(a.Mo) * a.Kc * ns;
   const size_t b_plane_bytes = static_cast<size_t>(a.No) * a.Kc;
   size_t plane_room = (a.d_workspace && a.workspace_bytes > kSplitRegionBytes) ? a.workspace_bytes - kSplitRegionBytes : 0;
   uint8_t* plane_ptr = a.d_workspace ? reinterpret_cast<uint8_t*>(a.d_workspace) + kSplitRegionBytes : nullptr;
@@ -1464,7 +1469,7 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   // always fetched as bytes, the caller's or a plane expanded here.
   // The same holds for signed INT4 codes as the first operand of the backward / update products
   // (the uniform arm of the gradient ablation): those kernels expand LUQ codes there.
-  const bool b_must = a.b_kind == 2, a_must = a.a_kind == 2 || (a.a_kind == 0 && (a.a_mn || a.b_mn));
+  const bool b_must = a.b_kind == 2, a_must = a.a_kind == 2 || (a.a_kind == 0 && (a.a_mn || a.b_mn)) || a.a_summed > 1;
   // (With bf16 outputs the output stream no longer hides the expansion: the caller's bytes are then
   // used for short contractions too - backward product of the ResNet shape 82 -> 65 us.)
   // A short contraction with fp32 output is bound by its output stream: with both operands' bytes at
@@ -1523,8 +1528,8 @@ static int luq_launch_gemm_impl(luq_ctx* ctx, const luq_gemm_args& a, cudaStream
   {
     const uint8_t* ptr = a_plane ? a_plane_ptr : a.a_codes;
     const uint64_t div = a_plane ? 1 : 2;   // bytes per row: elements (plane) or elements / 2 (codes)
-    if (a.a_mn) bad |= encode_bytes_map(ctx->encode_tiled, &ta, ptr, a.Mo / div, a.Kc, a.n_samples, true, a_plane);
-    else bad |= encode_bytes_map(ctx->encode_tiled, &ta, ptr, a.Kc / div, a.Mo, a.n_samples, true, a_plane);
+    if (a.a_mn) bad |= encode_bytes_map(ctx->encode_tiled, &ta, ptr, a.Mo / div, a.Kc, ns, true, a_plane);
+    else bad |= encode_bytes_map(ctx->encode_tiled, &ta, ptr, a.Kc / div, a.Mo, ns, true, a_plane);
   }
   {
     const uint8_t* ptr = b_plane ? b_plane_ptr : a.b_codes;

@@ -552,12 +552,14 @@ __device__ __forceinline__ float pw2_ceil(float m) {
 // block that finishes last writes the measured maximum and replaces the estimate by
 // (1 - eta) * measured + eta * estimate, every operation rounded once in binary32.
 // PLANE: the tensor-core operand bytes (int8, +-2^(c-1)) of every sample are written next to
-// the packed codes, one byte per element, sample s at offset s * n.
+// the packed codes, one byte per element, sample s at offset s * n - or, with sum_planes, ONE plane
+// whose byte is the sum of the samples' bytes (the host checks that n_samples * 2^kmax fits int8):
+// the mean over samples of the products equals the product with the summed operand over n_samples.
 template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
 __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restrict__ x, size_t n,
                                                              const float* d_amax,
                                                              const __grid_constant__ PhiloxKeySet keys,
-                                                             int n_samples_rt,
+                                                             int n_samples_rt, int sum_planes,
                                                              uint8_t* __restrict__ codes,
                                                              int8_t* __restrict__ operand,
                                                              float* __restrict__ d_alpha,
@@ -568,6 +570,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
   luqdev::pdl_wait();
   luqdev::pdl_trigger();
   const int n_samples = NS > 0 ? NS : n_samples_rt;
+  const bool sum = PLANE && NS != 1 && sum_planes != 0;
   constexpr int kElems = Item<BF16>::kElems;
   float given;
   if (!TRACK && d_amax_out != nullptr) {   // fused: the maximum of this tensor, reduced here
@@ -624,6 +627,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
         sn[j] = ((bits >> (28 - at)) & (8u << at)) | (1u << at);
         if constexpr (PLANE) ob[j] = ((bits >> 31) ? 0xFFu : 0x01u) << (8 * (j % 4));
       }
+      uint32_t total[kElems / 4] = {};   // per-byte sums over the samples (sum_planes)
 #pragma unroll
       for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
         if (NS == 0 && s >= n_samples) break;
@@ -643,13 +647,22 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
           }
         }
         Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
-        if constexpr (PLANE) Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
+        if constexpr (PLANE) {
+          if (sum) {
+#pragma unroll
+            for (int b = 0; b < kElems / 4; ++b) total[b] = __vadd4(total[b], bytes[b]);
+          } else {
+            Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
+          }
+        }
       }
+      if constexpr (PLANE) if (sum) Item<BF16>::store_bytes(operand, item, total, true);
       return;
     }
     uint32_t lo_code[kElems], thr[kElems];
 #pragma unroll
     for (int j = 0; j < kElems; ++j) luq_bin(luq_quotient_clamped<PW2>(v[j], sc, keys.q_top), lo_code[j], thr[j]);
+    uint32_t total[kElems / 4] = {};
 #pragma unroll
     for (int s = 0; s < (NS > 0 ? NS : LUQ_MAX_SAMPLES); ++s) {
       if (NS == 0 && s >= n_samples) break;
@@ -668,8 +681,16 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
         }
       }
       Item<BF16>::store(codes + plane * s, item, word, aligned || s == 0);
-      if constexpr (PLANE) Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
+      if constexpr (PLANE) {
+        if (sum) {
+#pragma unroll
+          for (int b = 0; b < kElems / 4; ++b) total[b] = __vadd4(total[b], bytes[b]);
+        } else {
+          Item<BF16>::store_bytes(operand + n * s, item, bytes, aligned_op || s == 0);
+        }
+      }
     }
+    if constexpr (PLANE) if (sum) Item<BF16>::store_bytes(operand, item, total, true);
   };
 
   const size_t full_tiles = items / kTileItems;
@@ -693,7 +714,7 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
         Item<BF16>::store(codes + plane * s, i, 0u, aligned || s == 0);
         if constexpr (PLANE) {
           const uint32_t zero[kElems / 4] = {};
-          Item<BF16>::store_bytes(operand + n * s, i, zero, aligned_op || s == 0);
+          if (!sum || s == 0) Item<BF16>::store_bytes(operand + n * s, i, zero, aligned_op || s == 0);
         }
       }
       if constexpr (TRACK) {   // an unusable estimate still needs this tensor's maximum for the next step
@@ -724,8 +745,14 @@ __global__ void __launch_bounds__(kThreads) quant_luq_kernel(const void* __restr
         }
         codes[plane * s + (e >> 1)] = static_cast<uint8_t>(nib[0] | (nib[1] << 4));
         if constexpr (PLANE) {
-          operand[n * s + e] = static_cast<int8_t>(luq_operand_byte(nib[0]));
-          if (e + 1 < n) operand[n * s + e + 1] = static_cast<int8_t>(luq_operand_byte(nib[1]));
+          if (sum) {   // this thread wrote the earlier samples' sum itself
+            const int8_t b0 = static_cast<int8_t>(luq_operand_byte(nib[0])), b1 = static_cast<int8_t>(luq_operand_byte(nib[1]));
+            operand[e] = static_cast<int8_t>((s ? operand[e] : 0) + b0);
+            if (e + 1 < n) operand[e + 1] = static_cast<int8_t>((s ? operand[e + 1] : 0) + b1);
+          } else {
+            operand[n * s + e] = static_cast<int8_t>(luq_operand_byte(nib[0]));
+            if (e + 1 < n) operand[n * s + e + 1] = static_cast<int8_t>(luq_operand_byte(nib[1]));
+          }
         }
       }
     }
@@ -1100,6 +1127,7 @@ struct LuqLaunch {
   uint8_t* codes; int8_t* operand; float* alpha; unsigned int* measured; float* estimate; float eta;
   float* amax_out;   // non-null: fused, the maximum is reduced by the same kernel (cooperative launch)
   cudaStream_t st;
+  int sum_planes;    // one operand plane holding the sum over samples
 };
 
 template <bool BF16, int NS, bool PW2, bool TRACK, bool PLANE>
@@ -1108,8 +1136,8 @@ int launch_luq_ns(const LuqLaunch& a) {
   const int grid = grid_for(a.ctx, quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, tiles);
   const int mode = a.amax_out ? LUQ_LAUNCH_COOPERATIVE : LUQ_LAUNCH_EARLY;
   return static_cast<int>(luq_launch_kernel(quant_luq_kernel<BF16, NS, PW2, TRACK, PLANE>, grid, kThreads, 0, a.st, mode, 1,
-                                            a.g, a.n, a.amax, a.keys, a.n_samples, a.codes, a.operand, a.alpha,
-                                            a.measured, a.estimate, a.eta, a.amax_out, a.ctx->d_scratch,
+                                            a.g, a.n, a.amax, a.keys, a.n_samples, a.sum_planes, a.codes, a.operand,
+                                            a.alpha, a.measured, a.estimate, a.eta, a.amax_out, a.ctx->d_scratch,
                                             a.ctx->d_status));
 }
 template <bool BF16, bool PW2, bool TRACK, bool PLANE>
@@ -1126,13 +1154,15 @@ int launch_luq(const LuqLaunch& a) {
 
 // flags: bit 0 = power-of-two scale; bit 1 = in-hindsight: d_amax is the running estimate, the
 // tensor's own maximum goes to d_measured and the estimate is replaced (eta) by the same kernel;
-// bit 2 = deterministic round-to-nearest-power instead of the random words
+// bit 2 = deterministic round-to-nearest-power instead of the random words;
+// bit 3 = d_operand is ONE plane holding the sum of the samples' operand bytes
 int luq_launch_quant_grad_ex(luq_ctx* ctx, const void* d_g, int dtype, size_t n, const float* d_amax, uint64_t seed,
                              int n_samples, uint8_t* d_codes, int8_t* d_operand, float* d_alpha, int flags,
                              float* d_measured, float* d_estimate, float eta, float* d_amax_out, cudaStream_t st) {
   const LuqLaunch a{ctx, d_g, n, d_amax, expand_keys(seed, n_samples, ctx->kmax, (flags & 4) ? 0x7FFFFFFFu : 0u),
                     n_samples, d_codes, d_operand, d_alpha,
-                    reinterpret_cast<unsigned int*>(d_measured), d_estimate, eta, d_amax_out, st};
+                    reinterpret_cast<unsigned int*>(d_measured), d_estimate, eta, d_amax_out, st,
+                    (flags & 8) && d_operand && n_samples > 1 ? 1 : 0};
   int rc;
   switch ((flags & 3) | (dtype == LUQ_BF16 ? 4 : 0)) {
     case 0: rc = launch_luq<false, false, false>(a); break;
