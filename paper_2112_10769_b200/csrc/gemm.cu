@@ -65,6 +65,18 @@ constexpr int kPlaneWarp = 6;
 constexpr int kFirstConvWarp = 7;
 constexpr int kTmemCols = 2 * BN;
 constexpr int kTileFloats = BM * BN;
+// True (always) once every lane of the warp holds the words it loaded into w[0..count): the vote
+// consumes a value computed from all of them, so it cannot complete while a load is outstanding, and
+// it doubles as the warp barrier.  The side effect (an atomic OR with zero, taken when some lane's
+// words happen to OR to one particular pattern) only keeps the compiler from discarding the chain.
+__device__ __forceinline__ bool loads_landed(const uint4* w, int count, unsigned int* status) {
+  uint32_t seen = 0u;
+#pragma unroll
+  for (int j = 0; j < count; ++j) seen |= w[j].x | w[j].y | w[j].z | w[j].w;
+  if (__any_sync(0xFFFFFFFFu, seen == 0x9E3779B9u) && (threadIdx.x & 31) == 0) atomicOr(status, 0u);
+  return true;
+}
+
 constexpr int kStageBox = 32 * 32 * 4;           // one 32 x 32 fp32 store box
 constexpr int kMaxBarriers = 24;
 
@@ -556,6 +568,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       unit_range(u, tile, it_begin, it_end);
       for (int k_it = it_begin; k_it < it_end; ++k_it) {
         if (!mbar_wait(pk_full(ps), pphase, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(ex_empty(es), ephase ^ 1u, abort_flag)) { ok = false; break; }
         const uint8_t* src = gen + C::packed + ps * C::packed_stage;
         uint8_t* dst = gen + C::expanded + es * kExpandedStage;
         constexpr int kTasks = C::tasks_per_thread > 0 ? C::tasks_per_thread : 1;
@@ -564,12 +577,6 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         for (int j = 0; j < C::tasks_per_thread; ++j)
           w[j] = smem_in(src + (ctid + j * kConvThreads) * 16, gen, C::packed, C::staging, 16, p.status)
                      ? *reinterpret_cast<const uint4*>(src + (ctid + j * kConvThreads) * 16) : make_uint4(0u, 0u, 0u, 0u);
-        // The packed slot goes back to the producer as soon as this warp has loaded its words - before
-        // the operand stage is free and before the expansion - so that the next copy is in flight
-        // meanwhile.  (The arrival has release semantics: the loads above are performed before it is seen.)
-        __syncwarp();
-        if (lane == 0) mbar_arrive(pk_empty(ps));
-        if (!mbar_wait(ex_empty(es), ephase ^ 1u, abort_flag)) { ok = false; break; }
 #pragma unroll
         for (int j = 0; j < C::tasks_per_thread; ++j) {
           const int id = ctid + j * kConvThreads;
@@ -590,7 +597,7 @@ luq_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
         fence_proxy_async();   // make the generic-proxy writes visible to the tensor core
         __syncwarp();
-        if (lane == 0) mbar_arrive(ex_full(es));
+        if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive(ex_full(es)); }
         if (++ps == static_cast<uint32_t>(PS > 0 ? PS : 1)) { ps = 0; pphase ^= 1u; }
         if (++es == static_cast<uint32_t>(ES)) { es = 0; ephase ^= 1u; }
       }
@@ -1124,13 +1131,14 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           for (int j = 0; j < kUnits; ++j)
             u[j] = smem_in(src + ((j ^ rkey) << 4), gen, C::raw, C::codes, 16, p.status)
                        ? *reinterpret_cast<const uint4*>(src + ((j ^ rkey) << 4)) : make_uint4(0u, 0u, 0u, 0u);
-          // The raw slot is given back as soon as this warp has loaded its rows - before the operand stage
-          // is free, before the conversion: what one SM can stream is the bytes its three raw slots keep
-          // in flight, and a slot that waits for arithmetic, stores and a barrier is not in flight.  The
-          // arrival has release semantics, so the loads above (every lane's, through the warp barrier)
-          // are performed before it is seen.
-          __syncwarp();
-          if (lane == 0) mbar_arrive(raw_empty(rs));
+          // The raw slot is given back as soon as this warp HOLDS its rows - before the operand stage is
+          // free, before the conversion: what one SM can stream is the bytes its three raw slots keep in
+          // flight, and a slot that waits for arithmetic, stores and a barrier is not in flight.  "Holds"
+          // must be literal: the refill is a write of the async proxy, which the release semantics of an
+          // arrival do not order against this warp's reads (arriving straight after issuing the loads
+          // gave wrong codes about once in 150 calls).  loads_landed() returns only when every lane's
+          // words are in registers.
+          if (loads_landed(u, kUnits, p.status) && lane == 0) mbar_arrive(raw_empty(rs));
           ok = mbar_wait_idle(ex_empty(es), ephase ^ 1u, abort_flag);
         }
         if (ok) {
