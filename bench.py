@@ -46,7 +46,7 @@ KERNELS = ("amax_A", "amax_W", "quant_int4_A", "quant_int4_W", "gemm_fwd",
 # copied from the committed single-pass ncu capture of the same step (other workloads: None).
 TRAFFIC_SOURCE = "profiles/launch_list_and_dram_traffic_cfg2_step.md (committed ncu capture of this step, not this run)"
 TRAFFIC_SOURCE_UNFUSED = "profiles/kernels_cfg2_full_size.md (committed ncu capture, not this run)"
-NCU_TRAFFIC_BYTES = {"amax_A": 463.4e6, "amax_W": 2.4e6, "quant_int4_W": 2.4e6, "quant_int4_A+gemm_fwd": 550.1e6,
+NCU_TRAFFIC_BYTES = {"amax_A": 463.4e6, "amax_W": 2.4e6, "quant_int4_W": 2.4e6, "quant_int4_A+gemm_fwd": 546.3e6,
                      "amax_G": 51.4e6, "quant_grad_G": 51.4e6, "gemm_bwd": 413.0e6, "gemm_wgrad": 89.8e6}
 NCU_TRAFFIC_BYTES_UNFUSED = {"quant_int4_A": 511.6e6, "gemm_fwd": 64.1e6}
 
