@@ -45,24 +45,34 @@ def check_entries(got, ref):
     assert (np.abs(got - ref) <= RTOL * np.abs(ref)).all()
 
 
-@pytest.mark.parametrize("operand_bytes", [True, False])
+@pytest.mark.parametrize("operand_bytes", [True, False, "timed"])
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg5"])
 def test_layer_configs_full_size(ctx, name, operand_bytes):
-    """operand_bytes=True is the configuration bench.py times: the quantizers also write the 8-bit
-    operand form of W and G (and of A for wide layers) and the GEMMs are handed those bytes."""
+    """operand_bytes=True: the quantizers also write the 8-bit operand form of W and G (and of A for
+    wide layers) and the GEMMs are handed those bytes.  "timed" is the configuration bench.py times:
+    the same, and in addition the forward product quantizes A itself where one column of output tiles
+    allows it (luq_quant_int4_gemm_fwd) and several samples share one summed operand plane."""
     cfg = inputs.CONFIGS[name]
     M, K, N, ns, seed = cfg.M, cfg.K, cfg.N, cfg.n_samples, cfg.luq_seed
+    timed = operand_bytes == "timed"
+    fused = timed and N <= 256
+    if timed and not fused and ns == 1:
+        pytest.skip("the timed configuration of this layer is operand_bytes=True")
+    ctx.set_option(binding.OPT_SUM_SAMPLES, 1 if (timed and ns > 1) else 0)   # the context is shared by the module
     A, W, G = inputs.layer_inputs(cfg)
     Ad, Wd, Gd = to_dev(A), to_dev(W), to_dev(G)
     mA, mW, mG = ctx.amax(Ad), ctx.amax(Wd), ctx.amax(Gd)
     i8 = lambda n: torch.empty(n, dtype=torch.int8, device="cuda")  # noqa: E731
     bW = i8(N * K) if operand_bytes else None
-    bG = i8(ns * M * N) if operand_bytes else None
+    bG = i8((1 if timed else ns) * M * N) if operand_bytes else None
     bA = i8(M * K) if operand_bytes and N >= 1024 else None
-    ca, sa = ctx.quant_int4(Ad, mA, operand=bA)
     cw, sw = ctx.quant_int4(Wd, mW, operand=bW)
     cg, al = ctx.quant_grad(Gd, mG, seed, ns, operand=bG)
-    Z = ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=bA, w_operand=bW)
+    if fused:
+        ca, sa, Z = ctx.quant_int4_gemm_fwd(Ad, mA, cw, sw, M, N, K, w_operand=bW)
+    else:
+        ca, sa = ctx.quant_int4(Ad, mA, operand=bA)
+        Z = ctx.gemm_fwd(ca, sa, cw, sw, M, N, K, a_operand=bA, w_operand=bW)
     dA = ctx.gemm_bwd(cg, al, ns, cw, sw, M, N, K, g_operand=bG, w_operand=bW)
     dW = ctx.gemm_wgrad(cg, al, ns, ca, sa, M, N, K, g_operand=bG, a_operand=bA)
     assert ctx.status() == 0
