@@ -19,7 +19,8 @@ LIB = os.path.join(HERE, "libluq_b200.so")
 LIB_DEBUG = os.path.join(HERE, "libluq_b200_debug.so")   # the same sources with -DLUQ_DEBUG (bounds-checking build)
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-std=c++17", "-O3", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
-          "-I", CSRC, "--expt-relaxed-constexpr"]
+          "-I", CSRC, "--expt-relaxed-constexpr",
+          "-diag-suppress", "177"]   # 177: a static member that one instantiation of a configuration struct does not use
 UNITS = {"quant.cu": ["-fmad=false"], "gemm.cu": [], "api.cu": []}
 
 
