@@ -69,7 +69,10 @@ class LuqLinearFunction(torch.autograd.Function):
         ns = ctx.n_samples
         lib = context(grad_out.device)
         g2 = grad_out.reshape(M, N).contiguous()
-        g_bytes = torch.empty(ns * M * N, dtype=torch.int8, device=g2.device)
+        # several samples (Sec. 5.1): one operand plane holding their sum while that sum fits int8 - the two
+        # products then cost what one sample's cost, with the same result (LUQ_OPT_SUM_SAMPLES)
+        lib.set_option(binding.OPT_SUM_SAMPLES, int(ns > 1 and (ns << binding.kmax()) <= 127))
+        g_bytes = torch.empty(lib._planes(ns) * M * N, dtype=torch.int8, device=g2.device)
         if ctx.estimates is None:
             cg, alpha = lib.quant_grad(g2, lib.amax(g2), ctx.seed, ns, operand=g_bytes)
         else:
