@@ -711,9 +711,13 @@ def run_ours(args):
                 with torch.cuda.stream(side_stream):
                     ctx_g.quant_grad_hindsight(lb.G, eG, 0.1, seed, ns, False, lb.cG, lb.aG, meas[2:3], lb.oG)
                     join = torch.cuda.Event(); join.record(side_stream)
-                ctx.quant_int4_hindsight(lb.A, eA, 0.1, lb.cA, lb.sA, meas[0:1], lb.oA)
                 ctx.quant_int4_hindsight(lb.W, eW, 0.1, lb.cW, lb.sW, meas[1:2], lb.oW)
-                lb.calls["gemm_fwd"]()
+                if lb.fused:     # A: quantized, measured and multiplied by one kernel
+                    ctx.quant_int4_hindsight_gemm_fwd(lb.A, eA, 0.1, lb.cW, lb.sW, M, N, K, lb.cA, lb.sA, meas[0:1],
+                                                      lb.Z, lb.oW)
+                else:
+                    ctx.quant_int4_hindsight(lb.A, eA, 0.1, lb.cA, lb.sA, meas[0:1], lb.oA)
+                    lb.calls["gemm_fwd"]()
                 main.wait_event(join)
                 lb.calls["gemm_bwd"](); lb.calls["gemm_wgrad"]()
 
@@ -724,7 +728,8 @@ def run_ours(args):
             assert lb.status() == 0
             hindsight = {"ms_per_step": h_ms, "value": world * flops_step / (h_ms * 1e-3) / 1e12, "unit": UNIT,
                          "launches_per_step": h_launches,
-                         "what": "in-hindsight maxima for A, W and G (eta 0.1): no max pass, one kernel per tensor"}
+                         "what": "in-hindsight maxima for A, W and G (eta 0.1): no max pass, one kernel per tensor" +
+                                 (", A's inside the forward product (luq_quant_int4_hindsight_gemm_fwd)" if lb.fused else "")}
         except Exception as e:  # pragma: no cover
             hindsight = {"unavailable": repr(e)}
 

@@ -319,6 +319,19 @@ int luq_quant_int4_gemm_fwd(luq_ctx* ctx, const void* d_a, int dtype, const floa
                             const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
                             void* d_z, int64_t M, int64_t N, int64_t K, void* stream);
 
+/* The same kernel with the in-hindsight maximum of Sec. 7 / App. A.5.4 (luq_quant_int4_hindsight followed by
+ * luq_gemm_fwd, as ONE pass over the activations): A is quantized with the running estimate *d_chat, not
+ * with its own maximum - values beyond it saturate at +-7 - while max|A| is measured on the way; *d_sa
+ * receives chat / 7, *d_measured_max the measured maximum, and *d_chat is replaced by
+ * (1 - eta) * measured + eta * chat for the next step (a non-finite measurement keeps the estimate and
+ * raises LUQ_STATUS_NONFINITE; an unusable estimate gives zero codes, a zero scale and a zero Z, and is
+ * replaced by the measurement).  No max pass over A at all.  Results are those of the two separate calls
+ * bit for bit; where the fusion does not apply the call runs them.  0 <= eta <= 1. */
+int luq_quant_int4_hindsight_gemm_fwd(luq_ctx* ctx, const void* d_a, int dtype, float* d_chat, float eta,
+                                      uint8_t* d_a_codes, float* d_sa, float* d_measured_max,
+                                      const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
+                                      void* d_z, int64_t M, int64_t N, int64_t K, void* stream);
+
 /* Backward GEMM (Eq. Backward), SMP average fused (Sec. 5.1):
  *   dA[m,k] = (alpha*sw/n_samples) * sum_s sum_n qG_s[m,n] * qW[n,k].
  * g_codes: n_samples planes [M x N/2]; w_codes [N x K/2].

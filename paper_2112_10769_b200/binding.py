@@ -26,7 +26,7 @@ SCHEME_FP4, SCHEME_FP4_SR, SCHEME_FP4_SU, SCHEME_LUQ, SCHEME_INT4_SR = 0, 1, 2, 
 ERR_ARG, ERR_CUDA, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 
 SYMBOLS = ("luq_create", "luq_destroy", "luq_set_option", "luq_kmax", "luq_debug_build", "luq_amax", "luq_quant_int4",
-           "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_int4_hindsight", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_ablation", "luq_quant_grad_pw2",
+           "luq_amax_multi", "luq_quant_int4_multi", "luq_quant_int4_hindsight_gemm_fwd", "luq_quant_uint4", "luq_amax_quant_int4", "luq_quant_int4_hindsight", "luq_quant_grad", "luq_amax_quant_grad", "luq_quant_grad_nearest", "luq_quant_grad_ablation", "luq_quant_grad_pw2",
            "luq_quant_grad_hindsight", "luq_debug_quotient", "luq_debug_expire_wait", "luq_debug_bounds_probe", "luq_gemm_fwd", "luq_quant_int4_gemm_fwd", "luq_gemm_bwd", "luq_gemm_wgrad",
            "luq_gemm_wgrad_static", "luq_status", "luq_launch_count", "luq_strerror")
 
@@ -71,6 +71,8 @@ def load() -> ctypes.CDLL:
         L.luq_debug_quotient.argtypes = [vp, vp, sz, vp, vp, vp]
         L.luq_gemm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_quant_int4_gemm_fwd.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+        L.luq_quant_int4_hindsight_gemm_fwd.argtypes = [vp, vp, ctypes.c_int, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp,
+                                                        i64, i64, i64, vp]
         L.luq_gemm_bwd.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_wgrad.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.luq_gemm_wgrad_static.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, i64, i64, i64, vp]
@@ -356,6 +358,26 @@ class Context:
                                               _opt(w_operand, N * K), out.data_ptr(), M, N, K, _stream()),
                "luq_quant_int4_gemm_fwd")
         return a_codes, sa, out
+
+    def quant_int4_hindsight_gemm_fwd(self, a: torch.Tensor, c_hat: torch.Tensor, eta: float, w_codes, sw,
+                                      M: int, N: int, K: int, a_codes: torch.Tensor | None = None,
+                                      sa: torch.Tensor | None = None, measured: torch.Tensor | None = None,
+                                      out: torch.Tensor | None = None, w_operand: torch.Tensor | None = None):
+        """quant_int4_hindsight(a) and gemm_fwd in one kernel (layers with N <= 256): quantizes with the
+        estimate in `c_hat`, measures max|a| into `measured`, replaces `c_hat` by the estimate for the next
+        step; returns (a_codes, sa, measured, Z)."""
+        if a.numel() != M * K or not a.is_contiguous():
+            raise TypeError(f"activations: contiguous tensor of {M} x {K} expected")
+        a_codes = torch.empty(M * K // 2, dtype=torch.uint8, device=a.device) if a_codes is None else a_codes
+        sa = torch.empty(1, dtype=torch.float32, device=a.device) if sa is None else sa
+        measured = torch.empty(1, dtype=torch.float32, device=a.device) if measured is None else measured
+        out = self._out(out, M, N, a.device)
+        _check(load().luq_quant_int4_hindsight_gemm_fwd(self.handle, a.data_ptr(), _dtype_code(a), c_hat.data_ptr(), eta,
+                                                        a_codes.data_ptr(), sa.data_ptr(), measured.data_ptr(),
+                                                        w_codes.data_ptr(), sw.data_ptr(), _opt(w_operand, N * K),
+                                                        out.data_ptr(), M, N, K, _stream()),
+               "luq_quant_int4_hindsight_gemm_fwd")
+        return a_codes, sa, measured, out
 
     def gemm_bwd(self, g_codes, alpha, n_samples: int, w_codes, sw, M: int, N: int, K: int,
                  out: torch.Tensor | None = None, g_operand: torch.Tensor | None = None,

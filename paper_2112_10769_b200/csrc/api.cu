@@ -424,6 +424,38 @@ int luq_quant_int4_gemm_fwd(luq_ctx* ctx, const void* d_a, int dtype, const floa
   return cuda_rc(luq_launch_gemm(ctx, a, st));
 }
 
+int luq_quant_int4_hindsight_gemm_fwd(luq_ctx* ctx, const void* d_a, int dtype, float* d_chat, float eta,
+                                      uint8_t* d_a_codes, float* d_sa, float* d_measured_max, const uint8_t* d_w_codes,
+                                      const float* d_sw, const int8_t* d_w_operand, void* d_z, int64_t M, int64_t N,
+                                      int64_t K, void* stream) {
+  if (!ctx || !d_chat || !d_sa || !d_sw || !d_measured_max || (dtype != LUQ_F32 && dtype != LUQ_BF16)) return LUQ_ERR_ARG;
+  if (!(eta >= 0.0f && eta <= 1.0f)) return LUQ_ERR_ARG;
+  if (M < 0 || N < 0 || K < 0 || M > (1ll << 31) || N > (1ll << 31) || K > (1ll << 31)) return LUQ_ERR_ARG;
+  if (K % 32 || N % 4) return LUQ_ERR_ARG;
+  if (M && K && (!d_a || !d_a_codes)) return LUQ_ERR_ARG;
+  if (M && N && K && (!d_w_codes || !d_z)) return LUQ_ERR_ARG;
+  if (!aligned16(d_a) || !aligned16(d_a_codes) || !aligned16(d_w_codes) || !aligned16(d_w_operand) || !aligned16(d_z))
+    return LUQ_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return LUQ_ERR_CUDA;
+  cudaStream_t st = as_stream(stream);
+  if (luq_quant_fwd_fusable(ctx, M, N, K, d_w_operand != nullptr))
+    return cuda_rc(luq_launch_quant_fwd(ctx, d_a, dtype, nullptr, d_a_codes, d_sa, d_w_codes, d_sw, d_w_operand,
+                                        static_cast<float*>(d_z), M, N, K, st, d_chat, eta, d_measured_max));
+  // the two separate kernels
+  int rc = cuda_rc(luq_launch_quant_int4_hindsight(ctx, d_a, dtype, static_cast<size_t>(M) * static_cast<size_t>(K),
+                                                   d_chat, eta, d_a_codes, nullptr, d_sa, d_measured_max, st));
+  if (rc) return rc;
+  luq_gemm_args a{};
+  a.a_codes = d_a_codes; a.a_kind = 0; a.a_mn = 0; a.n_samples = 1;
+  a.b_codes = d_w_codes; a.b_kind = 0; a.b_mn = 0;
+  a.a_operand = nullptr; a.b_operand = d_w_operand;
+  a.d_scale_a = d_sa; a.d_scale_b = d_sw; a.d_out = d_z; a.out_bf16 = ctx->out_bf16; a.Mo = M; a.No = N; a.Kc = K;
+  a.d_workspace = ctx->d_workspace; a.workspace_bytes = ctx->workspace_bytes;
+  a.allow_split = 1;
+  return cuda_rc(luq_launch_gemm(ctx, a, st));
+}
+
 int luq_gemm_bwd(luq_ctx* ctx, const uint8_t* d_g_codes, const float* d_alpha, int n_samples,
                  const int8_t* d_g_operand, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
                  void* d_da, int64_t M, int64_t N, int64_t K, void* stream) {

@@ -92,9 +92,12 @@ int luq_launch_bounds_probe(luq_ctx* ctx, cudaStream_t st);
 // codes of A, its scale and Z = Q(A) . Q(W)^T.  d_w_operand may be null (W's codes are then widened
 // into the workspace).  Call only when luq_quant_fwd_fusable() says yes.
 bool luq_quant_fwd_fusable(const luq_ctx* ctx, int64_t M, int64_t N, int64_t K, bool have_w_bytes);
+// In-hindsight form (d_estimate != null; d_clip is then ignored): A is quantized with *d_estimate, its own
+// max|a| goes to *d_measured and *d_estimate is replaced by (1 - eta) * measured + eta * estimate.
 int luq_launch_quant_fwd(luq_ctx* ctx, const void* d_a, int dtype, const float* d_clip, uint8_t* d_a_codes,
                          float* d_sa, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
-                         float* d_z, int64_t M, int64_t N, int64_t K, cudaStream_t st);
+                         float* d_z, int64_t M, int64_t N, int64_t K, cudaStream_t st, float* d_estimate = nullptr,
+                         float eta = 0.0f, float* d_measured = nullptr);
 
 #ifdef __CUDACC__
 

@@ -874,7 +874,8 @@ struct FusedCfg {
   static constexpr int num_barriers = 2 * RS + 2 * ES + 4;
   static constexpr int tmem_slot = barriers + 8 * num_barriers;
   static constexpr int abort_flag = tmem_slot + 4;
-  static constexpr int total = abort_flag + 4;
+  static constexpr int cta_max = abort_flag + 4;     // largest |a| bit pattern this CTA has seen (in-hindsight form)
+  static constexpr int total = cta_max + 4;
   static constexpr int smem_bytes = total + 1024;
   static_assert(smem_bytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 };
@@ -884,6 +885,9 @@ struct FusedParams {
   const float* clip;      // max|A| (or a caller's clip)
   const float* scale_b;   // weight scale
   float* scale_a_out;     // receives clip / 7
+  // In-hindsight form (estimate != null, and clip == estimate): the kernel also measures max|A|, writes its
+  // bit pattern to `measured` and replaces the estimate - see luq_quant_int4_hindsight.
+  float* estimate; unsigned int* measured; unsigned int* scratch; float eta;
   unsigned int* status;
   long long Mo, No, Kc;
   int tiles_m, num_kb;
@@ -922,6 +926,8 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
   auto acc_empty = [&](int b) { return bar0 + 8u * (2 * RS + 2 * ES + 2 + b); };
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + C::tmem_slot);
   volatile uint32_t* const abort_flag = reinterpret_cast<volatile uint32_t*>(gen + C::abort_flag);
+  uint32_t* const cta_max = reinterpret_cast<uint32_t*>(gen + C::cta_max);
+  const bool track = p.estimate != nullptr;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -934,6 +940,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
     }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     *abort_flag = 0;
+    *cta_max = 0u;
     fence_barrier_init();
     fence_proxy_async();
   }
@@ -950,6 +957,9 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();
   pdl_trigger();
+  // in-hindsight form: the estimate every CTA quantizes with; its replacement is written by the CTA
+  // that finishes last, when no CTA can read it any more
+  const float given = (track && threadIdx.x == 0) ? *p.clip : 0.0f;
 
   const int raw_iters = 2 * p.num_kb;   // raw stages per tile
   // Tiles are walked from the END of the tensor: the max reduction that precedes this kernel read
@@ -1098,7 +1108,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
     const int ctid = threadIdx.x - (kFirstConvWarp + 8 * group) * 32;   // 0..255 inside the group
     const int boxi = cw >> 2;                      // which box of the raw stage
     const int row = (cw & 3) * 32 + lane;          // row of the tile
-    const float clip = __ldg(p.clip);
+    const float clip = track ? *p.clip : __ldg(p.clip);   // the in-hindsight form writes the estimate at its very end
     const bool first = blockIdx.x == 0 && group == 0 && ctid == 0;
     const bool usable = scale_usable(clip, first ? p.status : nullptr);
     const float inv = usable ? 7.0f / clip : 0.0f;   // an unusable clip gives zero codes and a zero scale
@@ -1113,6 +1123,7 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
     // a barrier could no longer tell them apart by their parity, and a slot must not be refilled
     // before both groups have seen it filled.
     uint32_t q = 0, stored = 0;
+    uint32_t seen = 0u;   // largest |a| bit pattern among this thread's elements (in-hindsight form)
     bool alive = true, ok = true;
     for (int t = blockIdx.x; alive && t < p.tiles_m; t += gridDim.x) {
       const int m0 = (p.tiles_m - 1 - t) * BM;
@@ -1163,6 +1174,10 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
               v[4 * j + 2] = __uint_as_float(u[j].z); v[4 * j + 3] = __uint_as_float(u[j].w);
             }
           }
+          if (track) {   // copied columns beyond K and rows beyond M arrive as zeros
+#pragma unroll
+            for (int e = 0; e < 32; ++e) seen = max(seen, __float_as_uint(v[e]) & 0x7FFFFFFFu);
+          }
           uint32_t lowb[8], any = 0u;
 #pragma unroll
           for (int g = 0; g < 8; ++g) {
@@ -1210,12 +1225,32 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
       }
     }
     if (ctid == 0) bulk_wait<0>();
+    if (track) {
+      seen = __reduce_max_sync(0xFFFFFFFFu, seen);
+      if (lane == 0) atomicMax(cta_max, seen);
+    }
   }
 
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, LUQ_STATUS_TIMEOUT);
+  if (track && threadIdx.x == 0) {
+    // grid-wide maximum without a second launch: every CTA leaves its maximum in the scratch array
+    // and takes a ticket; the one that draws the last ticket folds the array, writes the measured
+    // maximum and the next estimate, and puts the ticket counter back to zero.  Nobody waits.
+    __stcg(p.scratch + 2 + blockIdx.x, *cta_max);
+    __threadfence();
+    if (atomicAdd(p.scratch, 1u) == gridDim.x - 1) {
+      __threadfence();
+      uint32_t m = 0u;
+      for (unsigned int b = 0; b < gridDim.x; ++b) m = max(m, __ldcg(p.scratch + 2 + b));
+      *p.measured = m;   // Inf/NaN patterns win the maximum and raise the flag
+      if (m >= 0x7F800000u) atomicOr(p.status, LUQ_STATUS_NONFINITE);
+      *p.estimate = hindsight_next(m, given, p.eta);
+      *p.scratch = 0u;
+    }
+  }
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
@@ -1661,7 +1696,8 @@ bool luq_quant_fwd_fusable(const luq_ctx* ctx, int64_t M, int64_t N, int64_t K, 
 
 int luq_launch_quant_fwd(luq_ctx* ctx, const void* d_a, int dtype, const float* d_clip, uint8_t* d_a_codes,
                          float* d_sa, const uint8_t* d_w_codes, const float* d_sw, const int8_t* d_w_operand,
-                         float* d_z, int64_t M, int64_t N, int64_t K, cudaStream_t st) {
+                         float* d_z, int64_t M, int64_t N, int64_t K, cudaStream_t st, float* d_estimate, float eta,
+                         float* d_measured) {
   const bool bf16 = dtype == LUQ_BF16;
   const uint8_t* w_plane = reinterpret_cast<const uint8_t*>(d_w_operand);
   if (w_plane == nullptr) {   // widen W's codes once into the workspace (behind the split region)
@@ -1672,7 +1708,8 @@ int luq_launch_quant_fwd(luq_ctx* ctx, const void* d_a, int dtype, const float* 
     w_plane = dst;
   }
   FusedParams p{};
-  p.clip = d_clip; p.scale_b = d_sw; p.scale_a_out = d_sa; p.status = ctx->d_status;
+  p.clip = d_estimate ? d_estimate : d_clip; p.scale_b = d_sw; p.scale_a_out = d_sa; p.status = ctx->d_status;
+  p.estimate = d_estimate; p.measured = reinterpret_cast<unsigned int*>(d_measured); p.scratch = ctx->d_scratch; p.eta = eta;
   p.Mo = M; p.No = N; p.Kc = K;
   p.tiles_m = static_cast<int>((M + BM - 1) / BM);
   p.num_kb = static_cast<int>((K + BK - 1) / BK);

@@ -67,5 +67,17 @@ __device__ __forceinline__ uint32_t int4_pack8(uint32_t low_bytes_a, uint32_t lo
   return __byte_perm(ya, yb, 0x6420);
 }
 
+// In-hindsight update of a running maximum (Sec. 7, App. A.5.4): (1 - eta) * measured + eta * estimate,
+// one rounding per operation.  A measurement that is not finite (an Inf/NaN element) leaves the
+// estimate as it was - one overflowed element must not turn every later estimate into Inf; an
+// estimate that is not a positive finite number (0 before the first step) is replaced by the measurement.
+__device__ __forceinline__ float hindsight_next(uint32_t measured_bits, float estimate, float eta) {
+  if (measured_bits >= 0x7F800000u) return estimate;
+  const uint32_t eb = __float_as_uint(estimate);
+  if (eb == 0u || eb >= 0x7F800000u) return __uint_as_float(measured_bits);   // 0, negative, Inf, NaN
+  const float keep = __fsub_rn(1.0f, eta);
+  return __fadd_rn(__fmul_rn(keep, __uint_as_float(measured_bits)), __fmul_rn(eta, estimate));
+}
+
 }  // namespace luqdev
 #endif

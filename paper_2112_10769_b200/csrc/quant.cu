@@ -31,6 +31,7 @@ constexpr int kTileItems = kThreads * kUnroll;
 using luqdev::scale_usable;
 using luqdev::int4_code;
 using luqdev::uint4_code;
+using luqdev::hindsight_next;
 
 // checking build: is piece `idx` one of the tensor's `items` 16-byte pieces?  (a violation raises
 // LUQ_STATUS_BOUNDS and the caller skips the access; always true, and free, in the normal build)
@@ -124,17 +125,6 @@ __device__ __forceinline__ bool grid_max_last_block(uint32_t& m, unsigned int* s
   return false;
 }
 
-// In-hindsight update of a running maximum (Sec. 7, App. A.5.4): (1 - eta) * measured + eta * estimate,
-// one rounding per operation.  A measurement that is not finite (an Inf/NaN element) leaves the
-// estimate as it was - one overflowed element must not turn every later estimate into Inf; an
-// estimate that is not a positive finite number (0 before the first step) is replaced by the measurement.
-__device__ __forceinline__ float hindsight_next(uint32_t measured_bits, float estimate, float eta) {
-  if (measured_bits >= 0x7F800000u) return estimate;
-  const uint32_t eb = __float_as_uint(estimate);
-  if (eb == 0u || eb >= 0x7F800000u) return __uint_as_float(measured_bits);   // 0, negative, Inf, NaN
-  const float keep = __fsub_rn(1.0f, eta);
-  return __fadd_rn(__fmul_rn(keep, __uint_as_float(measured_bits)), __fmul_rn(eta, estimate));
-}
 
 // ------------------------------------------------------------------ amax ----
 // |x| as an unsigned bit pattern is monotone in |x| for finite values, and every

@@ -146,3 +146,85 @@ def test_shapes_outside_the_fusion_run_the_two_kernels(ctx):
     ca, sa, Z = ctx.quant_int4_gemm_fwd(torch.zeros(0, 64, device="cuda"), scalar(1.0),
                                         torch.zeros(32 * 32, dtype=torch.uint8, device="cuda"), scalar(1.0), 0, 32, 64)
     assert Z.numel() == 0
+
+
+HINDSIGHT_SHAPES = [(300, 160, 96), (1000, 32, 32), (257, 96, 132), (4224, 640, 256)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("M,K,N", HINDSIGHT_SHAPES)
+def test_in_hindsight_form_over_a_sequence_of_steps(ctx, M, K, N, dtype):
+    """The kernel that quantizes with a running estimate, measures max|A| itself and replaces the estimate:
+    codes, scale, measured maximum, next estimate against the oracle bit for bit over steps whose scale
+    jumps (the estimate lags: some steps saturate); Z within 1e-5 of the oracle's product."""
+    eta = 0.1
+    A0, W, _ = inputs.small_layer(M, K, N, 4000 + M + K)
+    if dtype == "bf16":
+        W = inputs.to_bf16_bits(W)
+    Wd = to_dev(W)
+    bw = torch.empty(N * K, dtype=torch.int8, device="cuda")
+    cw, sw = ctx.quant_int4(Wd, ctx.amax(Wd), operand=bw)
+    ow = cw.cpu().numpy()
+    first = inputs.to_bf16_bits(A0) if dtype == "bf16" else A0
+    est_o = oracle.amax(first)[0]
+    est_d = scalar(float(est_o))
+    saturated = 0
+    for step, sc in enumerate([1.0, 0.3, 6.0, 0.05, 2.0]):
+        A = (A0 * np.float32(sc)).astype(np.float32)
+        A[step % M, step % K] = np.float32(-0.0)
+        if dtype == "bf16":
+            A = inputs.to_bf16_bits(A)
+        want, s_want, fl, meas_want, next_want = oracle.quant_int4_hindsight(A, est_o, eta)
+        launches = ctx.launches
+        ca, sa, measured, Z = ctx.quant_int4_hindsight_gemm_fwd(to_dev(A), est_d, eta, cw, sw, M, N, K, w_operand=bw)
+        assert ctx.launches - launches == 1
+        assert fl == 0 and sa.item() == s_want and measured.item() == meas_want and est_d.item() == next_want
+        np.testing.assert_array_equal(ca.cpu().numpy(), want)
+        assert_gemm_close(Z.cpu().numpy(), oracle.gemm_fwd(want, s_want, ow, sw.item(), M, N, K))
+        saturated += int(meas_want > est_o)
+        est_o = next_want
+    assert saturated >= 1
+    # the same step through the two separate kernels: identical results
+    e1, e2 = scalar(float(est_o)), scalar(float(est_o))
+    Ad = to_dev(A)
+    ca1, sa1, m1, Z1 = ctx.quant_int4_hindsight_gemm_fwd(Ad, e1, eta, cw, sw, M, N, K, w_operand=bw)
+    ca2, sa2, m2 = ctx.quant_int4_hindsight(Ad, e2, eta)
+    Z2 = ctx.gemm_fwd(ca2, sa2, cw, sw, M, N, K, w_operand=bw)
+    assert torch.equal(ca1, ca2) and torch.equal(Z1, Z2)
+    assert (sa1.item(), m1.item(), e1.item()) == (sa2.item(), m2.item(), e2.item())
+
+
+def test_in_hindsight_form_specials(ctx):
+    M, K, N = 384, 128, 64
+    A, W, _ = inputs.small_layer(M, K, N, 5)
+    Wd = to_dev(W)
+    cw, sw = ctx.quant_int4(Wd, ctx.amax(Wd))
+    # an estimate of zero quantizes everything to zero and is replaced by the measurement
+    est = scalar(0.0)
+    ca, sa, measured, Z = ctx.quant_int4_hindsight_gemm_fwd(to_dev(A), est, 0.1, cw, sw, M, N, K)
+    assert not ca.any().item() and sa.item() == 0 and not Z.any().item()
+    assert measured.item() == oracle.amax(A)[0] == est.item()
+    assert ctx.status() == 0
+    # an Inf among the activations: the measurement is Inf, the flag is raised, the estimate stays
+    B = A.copy(); B[17, 3] = np.inf; B[200, 100] = np.nan
+    est = scalar(1.5)
+    ca, sa, measured, Z = ctx.quant_int4_hindsight_gemm_fwd(to_dev(B), est, 0.1, cw, sw, M, N, K)
+    want, s_want, fl, meas_want, next_want = oracle.quant_int4_hindsight(B, np.float32(1.5), 0.1)
+    np.testing.assert_array_equal(ca.cpu().numpy(), want)
+    assert est.item() == 1.5 == next_want and not np.isfinite(measured.item())
+    assert ctx.status() == binding.STATUS_NONFINITE
+    # a layer too wide for the fusion runs the two kernels, with the same results
+    M2, K2, N2 = 256, 64, 512
+    A2, W2, _ = inputs.small_layer(M2, K2, N2, 9)
+    W2d = to_dev(W2)
+    cw2, sw2 = ctx.quant_int4(W2d, ctx.amax(W2d))
+    est = scalar(0.8)
+    launches = ctx.launches
+    ca, sa, measured, Z = ctx.quant_int4_hindsight_gemm_fwd(to_dev(A2), est, 0.25, cw2, sw2, M2, N2, K2)
+    assert ctx.launches - launches >= 2
+    want, s_want, fl, meas_want, next_want = oracle.quant_int4_hindsight(A2, np.float32(0.8), 0.25)
+    np.testing.assert_array_equal(ca.cpu().numpy(), want)
+    assert (sa.item(), measured.item(), est.item()) == (s_want, meas_want, next_want)
+    assert_gemm_close(Z.cpu().numpy(), oracle.gemm_fwd(want, s_want, cw2.cpu().numpy(), sw2.item(), M2, N2, K2))
+    with pytest.raises(binding.LuqError):
+        ctx.quant_int4_hindsight_gemm_fwd(to_dev(A), scalar(1.0), 1.5, cw, sw, M, N, K)
