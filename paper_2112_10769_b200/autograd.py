@@ -43,9 +43,11 @@ class LuqLinearFunction(torch.autograd.Function):
         M, K = a2.shape
         N = w2.shape[0]
         w_bytes = torch.empty(N * K, dtype=torch.int8, device=a.device)
+        # A is quantized inside the forward product where the layer allows it (one column of output tiles,
+        # N <= 256); elsewhere the same calls run the quantizer and the product one after the other
         if estimates is None:
-            ca, sa = lib.quant_int4(a2, lib.amax(a2))
             cw, sw = lib.quant_int4(w2, lib.amax(w2), operand=w_bytes)
+            ca, sa, z = lib.quant_int4_gemm_fwd(a2, lib.amax(a2), cw, sw, M, N, K, w_operand=w_bytes)
         else:
             if primed is not None:
                 # a tensor seen for the first time has no history: its estimate starts as its own maximum
@@ -53,9 +55,8 @@ class LuqLinearFunction(torch.autograd.Function):
                     lib.amax(a2, estimates[0:1]); primed[0] = True
                 if not primed[1]:
                     lib.amax(w2, estimates[1:2]); primed[1] = True
-            ca, sa, _ = lib.quant_int4_hindsight(a2, estimates[0:1], eta)
             cw, sw, _ = lib.quant_int4_hindsight(w2, estimates[1:2], eta, operand=w_bytes)
-        z = lib.gemm_fwd(ca, sa, cw, sw, M, N, K, w_operand=w_bytes)
+            ca, sa, _, z = lib.quant_int4_hindsight_gemm_fwd(a2, estimates[0:1], eta, cw, sw, M, N, K, w_operand=w_bytes)
         ctx.save_for_backward(ca, sa, cw, sw, w_bytes)
         ctx.dims = (M, N, K, a.shape, a.dtype, w.dtype)
         ctx.seed, ctx.n_samples = int(seed), int(n_samples)

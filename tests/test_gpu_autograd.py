@@ -12,9 +12,10 @@ from test_gpu_parity import assert_gemm_close
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("N", [288, 224])    # two columns of output tiles / one (A quantized inside the forward product)
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-def test_function_matches_the_oracle(dtype):
-    M, K, N, ns, seed = 384, 256, 288, 2, 17
+def test_function_matches_the_oracle(dtype, N):
+    M, K, ns, seed = 384, 256, 2, 17
     A, W, G = inputs.small_layer(M, K, N, 4)
     a = torch.from_numpy(A).cuda().to(dtype).requires_grad_(True)
     w = torch.from_numpy(W).cuda().to(dtype).requires_grad_(True)
@@ -58,8 +59,9 @@ def test_module_trains_a_small_regression():
     assert autograd.context(torch.device("cuda", 0)).status() == 0
 
 
-def test_function_with_in_hindsight_estimates_matches_the_oracle():
-    M, K, N, ns, seed, eta = 384, 256, 288, 2, 23, 0.1
+@pytest.mark.parametrize("N", [288, 224])
+def test_function_with_in_hindsight_estimates_matches_the_oracle(N):
+    M, K, ns, seed, eta = 384, 256, 2, 23, 0.1
     A, W, G = inputs.small_layer(M, K, N, 6)
     a = torch.from_numpy(A).cuda().requires_grad_(True)
     w = torch.from_numpy(W).cuda().requires_grad_(True)
