@@ -65,16 +65,21 @@ constexpr int kPlaneWarp = 6;
 constexpr int kFirstConvWarp = 7;
 constexpr int kTmemCols = 2 * BN;
 constexpr int kTileFloats = BM * BN;
-// True (always) once every lane of the warp holds the words it loaded into w[0..count): the vote
+// Returns once every lane of the warp holds the words it loaded into w[0..count): the vote
 // consumes a value computed from all of them, so it cannot complete while a load is outstanding, and
 // it doubles as the warp barrier.  The side effect (an atomic OR with zero, taken when some lane's
 // words happen to OR to one particular pattern) only keeps the compiler from discarding the chain.
-__device__ __forceinline__ bool loads_landed(const uint4* w, int count, unsigned int* status) {
+__device__ __forceinline__ uint32_t loads_landed(const uint4* w, int count, unsigned int* status) {
   uint32_t seen = 0u;
 #pragma unroll
   for (int j = 0; j < count; ++j) seen |= w[j].x | w[j].y | w[j].z | w[j].w;
-  if (__any_sync(0xFFFFFFFFu, seen == 0x9E3779B9u) && (threadIdx.x & 31) == 0) atomicOr(status, 0u);
-  return true;
+  const uint32_t rare = __any_sync(0xFFFFFFFFu, seen == 0x9E3779B9u);
+  if (rare && (threadIdx.x & 31) == 0) atomicOr(status, 0u);
+  return rare;
+}
+// an arrival that carries the value returned above as an operand, so that it cannot be issued before the vote
+__device__ __forceinline__ void mbar_arrive_after(uint32_t bar, uint32_t token) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];   // after %1" ::"r"(bar), "r"(token) : "memory");
 }
 
 constexpr int kStageBox = 32 * 32 * 4;           // one 32 x 32 fp32 store box
@@ -1151,7 +1156,10 @@ luq_quant_fwd_kernel(const __grid_constant__ CUtensorMap tm_raw, const __grid_co
           // arrival do not order against this warp's reads (arriving straight after issuing the loads
           // gave wrong codes about once in 150 calls).  loads_landed() returns only when every lane's
           // words are in registers.
-          if (loads_landed(u, kUnits, p.status) && lane == 0) mbar_arrive(raw_empty(rs));
+          {
+            const uint32_t token = loads_landed(u, kUnits, p.status);
+            if (lane == 0) mbar_arrive_after(raw_empty(rs), token);
+          }
           ok = mbar_wait_idle(ex_empty(es), ephase ^ 1u, abort_flag);
         }
         if (ok) {
