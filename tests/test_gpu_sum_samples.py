@@ -77,7 +77,7 @@ def test_unusable_scale_and_limits(ctx):
     ob = fresh_bytes(n + 8)
     codes, alpha = ctx.quant_grad(xd, ctx.amax(xd), 1, ns, operand=ob)
     assert not codes.any().item() and alpha.item() == 0 and not ob[:n].any().item() and (ob[n:] == 0x5A).all().item()
-    # three samples of magnitude 2^6 would leave int8; the ablation's kernels write one plane per sample
+    # two samples of magnitude 2^6 could sum to 128 and leave int8; the ablation's kernels write one plane per sample
     ctx.set_option(binding.OPT_LEVELS, 6)
     x = to_dev(luq_inputs(n, 3))
     with pytest.raises(binding.LuqError):
