@@ -349,13 +349,20 @@ class LayerBench:
     def status(self):
         return self.ctx.status() | (self.ctx_g.status() if self.ctx_g is not self.ctx else 0)
 
-    def capture(self, fn=None):
-        """No call of the path allocates or synchronises with the host, so one step is captured in a
-        CUDA graph and replayed: the small configurations are bound by launch rate otherwise."""
+    def capture(self, fn=None, steps=1):
+        """No call of the path allocates or synchronises with the host, so the steps are captured in a
+        CUDA graph and replayed: the small configurations are bound by launch rate otherwise.  A graph
+        holds as many consecutive steps (each complete, in stream order) as divide `steps` evenly, up to
+        `--steps-per-graph`: between two graph launches the GPU idles for about 4 us, inside a graph
+        the next step's first kernel is launched like any other.  The returned callable runs
+        `.steps` steps per call."""
         torch = self.torch
         fn = self.step if fn is None else fn
         if self.args.no_graph:
-            return fn, "direct calls"
+            fn_direct = lambda: fn()  # noqa: E731
+            fn_direct.steps = 1
+            return fn_direct, "direct calls"
+        per_graph = max(d for d in range(1, max(1, self.args.steps_per_graph) + 1) if steps % d == 0)
         try:
             side = torch.cuda.Stream()
             side.wait_stream(torch.cuda.current_stream())
@@ -364,25 +371,35 @@ class LayerBench:
                 torch.cuda.synchronize()
                 graph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(graph, stream=side):
-                    fn()
+                    for _ in range(per_graph):
+                        fn()
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
             graph.replay()
             torch.cuda.synchronize()
             self._graphs = getattr(self, "_graphs", []) + [graph]
-            return graph.replay, "CUDA graph of the step's calls, replayed"
+            replay = lambda: graph.replay()  # noqa: E731
+            replay.steps = per_graph
+            what = "CUDA graph of the step's calls, replayed" if per_graph == 1 else \
+                f"CUDA graph of {per_graph} consecutive steps, replayed"
+            return replay, what
         except Exception as e:  # pragma: no cover
-            return fn, f"direct calls (graph capture failed: {e!r})"
+            fn_direct = lambda: fn()  # noqa: E731
+            fn_direct.steps = 1
+            return fn_direct, f"direct calls (graph capture failed: {e!r})"
 
     def time_blocks(self, run_step, steps, min_seconds, barrier, max_blocks=400):
         """R blocks of `steps` replays, one event pair per block, no host synchronisation inside the
         region; R is chosen from a trial block so that the region lasts at least `min_seconds`.
         Returns the per-step milliseconds of every block."""
         torch = self.torch
+        per_call = getattr(run_step, "steps", 1)
+        assert steps % per_call == 0, "a block is a whole number of graph replays"
+        calls = steps // per_call
         ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
         e0, e1 = ev(), ev()
         e0.record()
-        for _ in range(steps):
+        for _ in range(calls):
             run_step()
         e1.record(); torch.cuda.synchronize()
         trial_ms = max(e0.elapsed_time(e1), 1e-3)
@@ -391,7 +408,7 @@ class LayerBench:
         marks = [ev() for _ in range(blocks + 1)]
         marks[0].record()
         for b in range(blocks):
-            for _ in range(steps):
+            for _ in range(calls):
                 run_step()
             marks[b + 1].record()
         barrier()
@@ -473,7 +490,7 @@ def bench_layer_compact(torch, binding, inputs, local, args, name, barrier, host
         lb.step()
     assert lb.status() == 0
     n0 = lb.launches(); lb.step(); per_step = lb.launches() - n0
-    run_step, mode = lb.capture()
+    run_step, mode = lb.capture(steps=20)
     st = block_stats(lb.time_blocks(run_step, 20, min_seconds, barrier))
     assert lb.status() == 0
     M, K, N = cfg.M, cfg.K, cfg.N
@@ -607,7 +624,7 @@ def run_ours(args):
     launches0 = lb.launches()
     lb.step()
     launches_per_step = lb.launches() - launches0
-    run_step, launch_mode = lb.capture()
+    run_step, launch_mode = lb.capture(steps=args.steps)
     # The timed region: blocks of K replays, an event pair around each, at least a second in total.
     t_region = time.perf_counter()
     per_block = lb.time_blocks(run_step, args.steps, args.min_seconds, barrier)
@@ -722,7 +739,7 @@ def run_ours(args):
                 lb.calls["gemm_bwd"](); lb.calls["gemm_wgrad"]()
 
             n0 = lb.launches(); hindsight_step(); h_launches = lb.launches() - n0
-            h_run, _ = lb.capture(hindsight_step)
+            h_run, _ = lb.capture(hindsight_step, steps=args.steps)
             hs = block_stats(lb.time_blocks(h_run, args.steps, 0.3, barrier))
             h_ms = replicas.max_over_ranks(hs["ms_median"], dev)
             assert lb.status() == 0
@@ -739,7 +756,7 @@ def run_ours(args):
         saved = lb.kernels, lb.fused
         lb.kernels, lb.fused = KERNELS, False
         try:
-            n_run, _ = lb.capture()
+            n_run, _ = lb.capture(steps=args.steps)
             nst = block_stats(lb.time_blocks(n_run, args.steps, 0.3, barrier))
             named = {"ms_per_step": nst["ms_median"], "value": world * flops_step / (nst["ms_median"] * 1e-3) / 1e12,
                      "what": "quant_int4(A) and gemm_fwd as two kernels (nine calls per step)"}
@@ -911,6 +928,9 @@ def main():
                     help="1 (default) = with several samples the quantizer writes one operand plane, the sum of the "
                          "samples' bytes, and the backward / update products read it (LUQ_OPT_SUM_SAMPLES): same "
                          "results bit for bit at one sample's product cost; 0 = one plane per sample")
+    ap.add_argument("--steps-per-graph", type=int, default=10,
+                    help="a replayed CUDA graph holds up to this many consecutive steps (the largest divisor of --steps "
+                         "not above it); 1 = one step per graph launch")
     ap.add_argument("--wgrad-first", type=int, default=0, choices=(0, 1),
                     help="1 = update product before the backward product")
     ap.add_argument("--multi-amax", type=int, default=1, choices=(0, 1),
