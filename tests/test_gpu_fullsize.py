@@ -150,3 +150,28 @@ def test_quantizer_sweep_largest_sizes_windows(ctx, e):
     assert ctx.status() == 0
     del xd, codes
     torch.cuda.empty_cache()
+
+
+def test_in_hindsight_forward_kernel_full_size(ctx):
+    """Config 2's forward half as bench.py's in-hindsight variant runs it: A quantized with a lagging estimate
+    inside the forward product, its maximum measured by the same kernel."""
+    ctx.set_option(binding.OPT_SUM_SAMPLES, 0)
+    cfg = inputs.CONFIGS["cfg2"]
+    M, K, N = cfg.M, cfg.K, cfg.N
+    A, W, _ = inputs.layer_inputs(cfg)
+    Ad, Wd = to_dev(A), to_dev(W)
+    bW = torch.empty(N * K, dtype=torch.int8, device="cuda")
+    cw, sw = ctx.quant_int4(Wd, ctx.amax(Wd), operand=bW)
+    true_max = oracle.amax(A)[0]
+    start = np.float32(true_max * np.float32(0.8))          # the estimate lags: the largest values saturate
+    est = torch.tensor([start], dtype=torch.float32, device="cuda")
+    ca, sa, measured, Z = ctx.quant_int4_hindsight_gemm_fwd(Ad, est, 0.1, cw, sw, M, N, K, w_operand=bW)
+    want, s_want, fl, meas_want, next_want = oracle.quant_int4_hindsight(A, start, 0.1)
+    assert fl == 0 and meas_want == true_max
+    assert (sa.item(), measured.item(), est.item()) == (s_want, meas_want, next_want)
+    assert np.array_equal(ca.cpu().numpy(), want)
+    ow = cw.cpu().numpy()
+    r, c = sample_entries(M, N, 300, 4)
+    check_entries(Z[torch.from_numpy(r).cuda(), torch.from_numpy(c).cuda()].cpu().numpy(),
+                  oracle.gemm_entries("fwd", want, s_want, 1, ow, sw.item(), M, N, K, r, c))
+    assert ctx.status() == 0
